@@ -1,0 +1,195 @@
+"""ctypes front end of the CPU oracle (oracle/rmm_oracle.c).
+
+TEST INFRASTRUCTURE.  Only tests/, the smoke check and the benchmark's cpu_baseline /
+reference arm may import this package.  It never touches the CUDA library and the CUDA
+library never touches it.
+
+Arrays are numpy: dtype uint16 carries raw bf16 bit patterns, float32 and float64 are
+themselves.  torch tensors are accepted and viewed without value change (bf16 -> uint16 bits).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rmm_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+_lib = None
+
+BF16, F32, F64 = 0, 1, 2
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, OpenMP).  Building the checker is not using it."""
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if force or stale:
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
+               "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    build()
+    L = ctypes.CDLL(_LIB)
+    i64, dbl, vp, i32 = ctypes.c_int64, ctypes.c_double, ctypes.c_void_p, ctypes.c_int
+    L.orc_keep_count.restype = i64
+    L.orc_keep_count.argtypes = [dbl, i64]
+    L.orc_num_threads.restype = i32
+    L.orc_set_threads.argtypes = [i32]
+    L.orc_score.restype = None
+    L.orc_score.argtypes = [vp, i32, i64, i64, i64, i64, vp, vp]
+    L.orc_select.restype = dbl
+    L.orc_select.argtypes = [vp, i64, i64, vp]
+    L.orc_reduced_gemm_rows.restype = None
+    L.orc_reduced_gemm_rows.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, i64, i64, i64,
+                                        vp, i64, vp, i64, i64]
+    L.orc_dense_gemm.restype = None
+    L.orc_dense_gemm.argtypes = [vp, i32, i64, i64, i64, i64, vp, i32, i64, i64, i64, vp]
+    L.orc_round_bf16.restype = dbl
+    L.orc_round_bf16.argtypes = [dbl]
+    L.orc_attn.restype = None
+    L.orc_attn.argtypes = [vp, vp, vp, i32, i64, i64, i64, i64, i64, i64, vp, vp, vp,
+                           i32, dbl, dbl, i32, vp, vp, vp, vp]
+    _lib = L
+    return L
+
+
+def as_np(x) -> np.ndarray:
+    """numpy view of a numpy array or CPU torch tensor; bf16 becomes uint16 bit patterns."""
+    if isinstance(x, np.ndarray):
+        return x
+    import torch  # only to recognise tensors handed in by the tests
+
+    if isinstance(x, torch.Tensor):
+        x = x.detach().cpu()
+        if x.dtype == torch.bfloat16:
+            return x.view(torch.int16).numpy().view(np.uint16)
+        return x.numpy()
+    return np.asarray(x)
+
+
+def _dt(a: np.ndarray) -> int:
+    if a.dtype == np.uint16:
+        return BF16
+    if a.dtype == np.float32:
+        return F32
+    if a.dtype == np.float64:
+        return F64
+    raise TypeError(f"oracle: unsupported dtype {a.dtype}")
+
+
+def _estr(a: np.ndarray) -> Tuple[int, ...]:
+    return tuple(s // a.itemsize for s in a.strides)
+
+
+def num_threads() -> int:
+    return int(_load().orc_num_threads())
+
+
+def set_threads(n: int) -> None:
+    _load().orc_set_threads(int(n))
+
+
+def keep_count(rho: float, K: int) -> int:
+    """|I| = ceil(rho K) (Sec. 3.2); -1 when rho is outside (0, 1] or K < 1."""
+    return int(_load().orc_keep_count(float(rho), int(K)))
+
+
+def score(A) -> Tuple[np.ndarray, np.ndarray]:
+    """(energy, score) of the columns of a 2-D matrix: sum of squares and its square root."""
+    A = as_np(A)
+    assert A.ndim == 2
+    M, K = A.shape
+    sr, sc = _estr(A)
+    e = np.empty(K, np.float64)
+    s = np.empty(K, np.float64)
+    _load().orc_score(A.ctypes.data, _dt(A), M, K, sr, sc, e.ctypes.data, s.ctypes.data)
+    return e, s
+
+
+def select(key, k: int) -> Tuple[np.ndarray, float]:
+    """(ascending index set of the k largest keys with ties to the lower index, kept key mass)."""
+    key = np.ascontiguousarray(as_np(key), dtype=np.float64)
+    K = key.shape[0]
+    assert 1 <= k <= K
+    idx = np.empty(k, np.int32)
+    kept = _load().orc_select(key.ctypes.data, K, int(k), idx.ctypes.data)
+    return idx, float(kept)
+
+
+def reduced_gemm(A, B, idx, rows: Optional[Tuple[int, int]] = None) -> np.ndarray:
+    """Y = A[:, idx] @ B[idx, :] in fp64.  rows=(r0, r1) computes only those rows (others 0)."""
+    A, B = as_np(A), as_np(B)
+    idx = np.ascontiguousarray(as_np(idx), dtype=np.int32)
+    M, K = A.shape
+    K2, N = B.shape
+    assert K == K2
+    assert idx.size == 0 or (idx.min() >= 0 and idx.max() < K)
+    Y = np.zeros((M, N), np.float64)
+    r0, r1 = rows if rows is not None else (0, M)
+    sra, sca = _estr(A)
+    srb, scb = _estr(B)
+    _load().orc_reduced_gemm_rows(A.ctypes.data, _dt(A), M, K, sra, sca, B.ctypes.data, _dt(B),
+                                  N, srb, scb, idx.ctypes.data, idx.size, Y.ctypes.data, r0, r1)
+    return Y
+
+
+def dense_gemm(A, B) -> np.ndarray:
+    """Y = A @ B in fp64 with no index indirection."""
+    A, B = as_np(A), as_np(B)
+    M, K = A.shape
+    K2, N = B.shape
+    assert K == K2
+    Y = np.zeros((M, N), np.float64)
+    sra, sca = _estr(A)
+    srb, scb = _estr(B)
+    _load().orc_dense_gemm(A.ctypes.data, _dt(A), M, K, sra, sca, B.ctypes.data, _dt(B), N, srb, scb,
+                           Y.ctypes.data)
+    return Y
+
+
+def round_bf16(x: float) -> float:
+    return float(_load().orc_round_bf16(float(x)))
+
+
+def rmm(A, B, rho: float):
+    """The whole operation of Sec. 3.2 on one product: returns (Y, idx, energy)."""
+    A = as_np(A)
+    e, _ = score(A)
+    k = keep_count(rho, A.shape[1])
+    idx, _ = select(e, k)
+    return reduced_gemm(A, B, idx), idx, e
+
+
+def attn(Q, K, V, causal: bool, rho_d: float, rho_t: float, round_p: bool = True, want_p: bool = False):
+    """Reduced attention of Sec. 3.3.  Q [B,Hq,Lq,Dh]; K, V [B,Hkv,Lk,Dh] (same dtype).
+
+    Returns (O [B,Hq,Lq,Dh] fp64, idx_feat [B,Hq,kd], idx_tok [B,Hq,kt] or None, P or None).
+    """
+    Q, K, V = as_np(Q), as_np(K), as_np(V)
+    assert Q.ndim == 4 and K.ndim == 4 and V.ndim == 4 and Q.dtype == K.dtype == V.dtype
+    B, Hq, Lq, Dh = Q.shape
+    _, Hkv, Lk, _ = K.shape
+    assert Hq % Hkv == 0
+    kd = keep_count(rho_d, Dh)
+    kt = keep_count(rho_t, Lk)
+    O = np.zeros((B, Hq, Lq, Dh), np.float64)
+    idx_feat = np.zeros((B, Hq, kd), np.int32)
+    idx_tok = np.zeros((B, Hq, kt), np.int32) if rho_t < 1.0 else None
+    P = np.zeros((B, Hq, Lq, Lk), np.float64) if want_p else None
+    s3 = [(ctypes.c_int64 * 4)(*_estr(x)) for x in (Q, K, V)]
+    _load().orc_attn(Q.ctypes.data, K.ctypes.data, V.ctypes.data, _dt(Q), B, Hq, Hkv, Lq, Lk, Dh,
+                     s3[0], s3[1], s3[2], int(bool(causal)), float(rho_d), float(rho_t),
+                     int(bool(round_p)), O.ctypes.data, idx_feat.ctypes.data,
+                     idx_tok.ctypes.data if idx_tok is not None else None,
+                     P.ctypes.data if P is not None else None)
+    return O, idx_feat, idx_tok, P
