@@ -1,0 +1,147 @@
+/*
+ * rmm.h — C ABI of the B200 (sm_100a) library for Reduced Matrix Multiplication (RMM).
+ *
+ * RMM replaces a matrix product Y = A B (A: M x K activations, B: K x N weight or intermediate)
+ * by Y~ = A[:, I] B[I, :], where I holds the ceil(rho K) indices of the contraction axis whose
+ * activation columns have the largest Euclidean norm (paper Sec. 3.2).  Sec. 3.3 applies the same
+ * rule to attention: feature dims of Q K^T chosen per query head from Q, token positions of P V
+ * chosen from the columns of P.
+ *
+ * General rules for every entry point
+ *   - every data pointer is a DEVICE pointer owned by the caller, unless a comment says "host";
+ *   - the library never allocates, frees or synchronises (rmm_status_read and rmm_product_host excepted,
+ *     see there); every launch is asynchronous on `stream` (a cudaStream_t passed as void*, NULL =
+ *     legacy default stream);
+ *   - scratch memory comes from the caller: `ws` must hold at least the matching
+ *     *_workspace_bytes(); it must be 256-byte aligned and its first RMM_WS_HEADER_BYTES must be zero
+ *     the first time it is handed to the library (the library leaves them reusable afterwards,
+ *     unless a call reported a device-side error); calls that share one workspace must be ordered on one stream;
+ *   - the return value is an rmm_status_t; on a host-side error nothing was launched and outputs
+ *     are untouched; rmm_last_error() then gives a thread-local message;
+ *   - device-side waits are bounded: a kernel that gives up writes RMM_ERR_TIMEOUT to the status
+ *     word at the start of the workspace, releases what it holds and returns; read it with
+ *     rmm_status_read() after synchronising the stream;
+ *   - inputs must be finite; there is no CPU fallback: a shape, stride or dtype the kernels do not
+ *     cover is refused with RMM_ERR_UNSUPPORTED.
+ */
+#ifndef RMM_B200_H
+#define RMM_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RMM_OK = 0,
+    RMM_ERR_INVALID_ARG = 1, /* null pointer, dimension <= 0, rho outside (0,1], k outside [1,K], index out of range */
+    RMM_ERR_UNSUPPORTED = 2, /* dtype / stride / alignment / size the kernels do not cover */
+    RMM_ERR_WORKSPACE = 3,   /* ws is NULL, misaligned or smaller than *_workspace_bytes() */
+    RMM_ERR_CUDA = 4,        /* a CUDA call failed; text kept for rmm_last_error() */
+    RMM_ERR_TIMEOUT = 5,     /* device status word: a bounded wait inside a kernel gave up */
+    RMM_ERR_BOUNDS = 6       /* device status word: an index outside [0, K) was met and skipped */
+} rmm_status_t;
+
+typedef enum { RMM_BF16 = 0, RMM_F32 = 1 } rmm_dtype_t;
+
+/* A batch of matrices in device memory.  Element (b, r, c) lives at
+ * ptr + (b*stride_batch + r*stride_row + c*stride_col) elements.  stride_batch may be 0 (one matrix
+ * shared by every batch element, e.g. a weight).  Strides are in elements and non-negative. */
+typedef struct {
+    void *ptr;
+    int32_t dtype; /* rmm_dtype_t */
+    int64_t batch, rows, cols;
+    int64_t stride_batch, stride_row, stride_col;
+} rmm_mat_t;
+
+#define RMM_WS_HEADER_BYTES 4096
+
+/* |I| = ceil(rho K) (Sec. 3.2), host only.  rho is taken as a double; the product rho*K is snapped
+ * to the nearest integer when it lies within 1e-9*K of it (so 0.07*100 gives 7, not 8), then
+ * rounded up and clamped to [1, K].  RMM_ERR_INVALID_ARG if rho is not in (0, 1], K < 1 or k is NULL. */
+int rmm_keep_count(double rho, int64_t K, int64_t *k);
+
+/* Importance scores s_j = ||A[:, j]||_2 (Sec. 3.2 "Activation-aware dimension selection"; in
+ * attention s_j = ||Q[:, j]||_2 and a_t = ||P[:, t]||_2, Sec. 3.3).  Only A is read.
+ *   axis   1: one score per column (the contraction axis of A B); 0: one score per row.
+ *   scores fp32 [batch, n] with n = cols (axis 1) or rows (axis 0), or NULL
+ *   energy fp32 [batch, n]: the squared scores sum_i A[i,j]^2, which are the selection keys, or NULL
+ * Squares of bf16 values are exact in fp32; sums run in short fp32 chains combined in fp64 in a fixed
+ * order, so results are deterministic and accurate to about 1e-7 relative. */
+size_t rmm_score_workspace_bytes(const rmm_mat_t *A, int axis);
+int rmm_score(const rmm_mat_t *A, int axis, float *scores, float *energy, void *ws, size_t ws_bytes, void *stream);
+
+/* I = TopK(keys, k) (Sec. 3.2; Theorem 1 shows it minimises the discarded energy).  One index set per
+ * batch element.  k > 0 is used as given, otherwise k = rmm_keep_count(rho, K).
+ *   keys     fp32 [batch, K], non-negative
+ *   idx      int32 [batch, k], ASCENDING; among equal keys the lower index is kept
+ *   retained fp32 [batch] or NULL: sum of the kept keys / sum of all keys (1 - eps_A(rho) of Eq. 5
+ *            when the keys are energies) */
+size_t rmm_select_workspace_bytes(int64_t batch, int64_t K);
+int rmm_select(const float *keys, int64_t batch, int64_t K, double rho, int64_t k, int32_t *idx, float *retained,
+               void *ws, size_t ws_bytes, void *stream);
+
+/* rmm_score followed by rmm_select on the energies, in ONE launch (the last thread block to finish
+ * a batch element's scores selects its index set).  scores / energy / retained may be NULL. */
+size_t rmm_score_select_workspace_bytes(const rmm_mat_t *A, int axis);
+int rmm_score_select(const rmm_mat_t *A, int axis, double rho, int64_t k, int32_t *idx, float *scores, float *energy,
+                     float *retained, void *ws, size_t ws_bytes, void *stream);
+
+/* Y = scale * A[:, I] B[I, :] (Sec. 3.2, RMM_rho(A,B); no rescaling: pass scale = 1).
+ *   A    [b, M, K]; B [b or shared, K, N] (stride_batch 0 = shared); Y [b, M, N] (written in full)
+ *   idx  int32 [b, k], each entry in [0, K); any set is accepted (so a cached or random set gives
+ *        the paper's static / random controls); order fixes the summation order
+ *   bf16 operands run on the tensor cores (fp32 accumulation) when A has stride_col 1, B has
+ *   stride_col 1 (slices of the contraction axis contiguous) or stride_row 1, Y has stride_col 1, and
+ *   pointers / leading strides are 16-byte aligned; Y may be bf16 or fp32.  Every other layout, and
+ *   fp32 operands, run on a plain FMA kernel (fp32 accumulation).  A and B must share a dtype. */
+size_t rmm_reduced_gemm_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y);
+int rmm_reduced_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
+                     const rmm_mat_t *Y, void *ws, size_t ws_bytes, void *stream);
+
+/* Reduced attention of Sec. 3.3 for B sequences, Hq query heads, Hkv key/value heads (Hq % Hkv == 0,
+ * query head h reads kv head h / (Hq/Hkv)).  Per (sequence, query head):
+ *   I  = TopK of ||Q[:, j]||_2, |I| = ceil(rho_d Dh);  S~ = Q[:, I] K[:, I]^T / sqrt(Dh)  (full Dh in the scale)
+ *   P  = softmax(S~ + M), M = causal mask aligned to the end (query i sees keys t <= i + Lk - Lq) or none;
+ *        P is rounded once to bf16 and that rounded P is what is scored and multiplied
+ *   rho_t < 1:  T = TopK of ||P[:, t]||_2, |T| = ceil(rho_t Lk);  O = P[:, T] V[T, :]  (no renormalisation)
+ *   rho_t == 1: O = P V
+ * Q [B,Hq,Lq,Dh], K,V [B,Hkv,Lk,Dh], O [B,Hq,Lq,Dh] are bf16 with explicit element strides
+ * (batch, head, row, 1).  idx_feat int32 [B,Hq,kd] and idx_tok int32 [B,Hq,kt] receive the index sets
+ * (either may be NULL).  S~ and P are materialised in the workspace one group of heads at a time. */
+typedef struct {
+    int64_t B, Hq, Hkv, Lq, Lk, Dh;
+    int32_t causal;
+    double rho_d; /* feature retention of Q K^T */
+    double rho_t; /* token retention of P V; 1.0 switches token reduction off */
+    int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3]; /* batch, head, row (elements); last dim contiguous */
+} rmm_attn_desc_t;
+size_t rmm_reduced_attn_workspace_bytes(const rmm_attn_desc_t *desc);
+int rmm_reduced_attn(const rmm_attn_desc_t *desc, const void *Q, const void *K, const void *V, void *O,
+                     int32_t *idx_feat, int32_t *idx_tok, void *ws, size_t ws_bytes, void *stream);
+
+/* The whole operation of Sec. 3.2 on one bf16 product held in HOST memory (pinned for speed):
+ * copies A [M,K] and B [K,N] (row-major, contiguous) to the device staging area inside ws, runs
+ * rmm_score_select and rmm_reduced_gemm, and copies Y [M,N] bf16 and idx [k] back, all asynchronously on
+ * `stream`; the caller synchronises the stream before reading Y_host / idx_host.  copy_B = 0 reuses the
+ * B already staged by an earlier call on the same workspace (a resident weight). */
+size_t rmm_product_host_workspace_bytes(int64_t M, int64_t K, int64_t N);
+int rmm_product_host(const void *A_host, const void *B_host, int64_t M, int64_t K, int64_t N, double rho, int copy_B,
+                     void *Y_host, int32_t *idx_host, void *ws, size_t ws_bytes, void *stream);
+
+/* Copy the device status word of a workspace to *device_status (an rmm_status_t) and clear it.
+ * Synchronous: call it after the stream the workspace was used on has been synchronised. */
+int rmm_status_read(void *ws, int *device_status);
+
+/* Thread-local text of the last error returned on this thread ("" if none). */
+const char *rmm_last_error(void);
+
+/* Number of kernels the library has launched from this process (for launch accounting). */
+int64_t rmm_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RMM_B200_H */

@@ -1,0 +1,295 @@
+"""Thin ctypes binding of librmm_b200.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (include/rmm.h).  Tensors are torch CUDA
+tensors used as plain device memory; the current torch stream is the launch stream.  Workspaces are
+torch allocations made here (zero-filled once, then cached per device and reused), because the C
+library itself never allocates.  There is no fallback: if the shared library is missing or a call is
+refused, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librmm_b200.so")
+
+RMM_OK, RMM_ERR_INVALID_ARG, RMM_ERR_UNSUPPORTED, RMM_ERR_WORKSPACE, RMM_ERR_CUDA, RMM_ERR_TIMEOUT, RMM_ERR_BOUNDS = range(7)
+RMM_BF16, RMM_F32 = 0, 1
+RMM_WS_HEADER_BYTES = 4096
+_STATUS_NAMES = ["RMM_OK", "RMM_ERR_INVALID_ARG", "RMM_ERR_UNSUPPORTED", "RMM_ERR_WORKSPACE", "RMM_ERR_CUDA",
+                 "RMM_ERR_TIMEOUT", "RMM_ERR_BOUNDS"]
+
+
+class RmmError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        self.code = code
+        name = _STATUS_NAMES[code] if 0 <= code < len(_STATUS_NAMES) else str(code)
+        super().__init__(f"{name}: {text}")
+
+
+class rmm_mat_t(ctypes.Structure):
+    _fields_ = [("ptr", ctypes.c_void_p), ("dtype", ctypes.c_int32), ("batch", ctypes.c_int64),
+                ("rows", ctypes.c_int64), ("cols", ctypes.c_int64), ("stride_batch", ctypes.c_int64),
+                ("stride_row", ctypes.c_int64), ("stride_col", ctypes.c_int64)]
+
+
+class rmm_attn_desc_t(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int64), ("Hq", ctypes.c_int64), ("Hkv", ctypes.c_int64), ("Lq", ctypes.c_int64),
+                ("Lk", ctypes.c_int64), ("Dh", ctypes.c_int64), ("causal", ctypes.c_int32),
+                ("rho_d", ctypes.c_double), ("rho_t", ctypes.c_double),
+                ("q_stride", ctypes.c_int64 * 3), ("k_stride", ctypes.c_int64 * 3),
+                ("v_stride", ctypes.c_int64 * 3), ("o_stride", ctypes.c_int64 * 3)]
+
+
+EXPORTS = ["rmm_keep_count", "rmm_score_workspace_bytes", "rmm_score", "rmm_select_workspace_bytes", "rmm_select",
+           "rmm_score_select_workspace_bytes", "rmm_score_select", "rmm_reduced_gemm_workspace_bytes",
+           "rmm_reduced_gemm", "rmm_reduced_attn_workspace_bytes", "rmm_reduced_attn",
+           "rmm_product_host_workspace_bytes", "rmm_product_host", "rmm_status_read", "rmm_last_error",
+           "rmm_launch_count"]
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the shared library; raise if it has not been built (no CPU stand-in exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2608_13426_b200.build` "
+                           "(nvcc, sm_100a); this package has no CPU fallback")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i64, dbl, i32, sz, flt = ctypes.c_void_p, ctypes.c_int64, ctypes.c_double, ctypes.c_int, ctypes.c_size_t, ctypes.c_float
+    mp = ctypes.POINTER(rmm_mat_t)
+    L.rmm_keep_count.argtypes = [dbl, i64, ctypes.POINTER(i64)]
+    L.rmm_score_workspace_bytes.argtypes = [mp, i32]
+    L.rmm_score_workspace_bytes.restype = sz
+    L.rmm_score.argtypes = [mp, i32, vp, vp, vp, sz, vp]
+    L.rmm_select_workspace_bytes.argtypes = [i64, i64]
+    L.rmm_select_workspace_bytes.restype = sz
+    L.rmm_select.argtypes = [vp, i64, i64, dbl, i64, vp, vp, vp, sz, vp]
+    L.rmm_score_select_workspace_bytes.argtypes = [mp, i32]
+    L.rmm_score_select_workspace_bytes.restype = sz
+    L.rmm_score_select.argtypes = [mp, i32, dbl, i64, vp, vp, vp, vp, vp, sz, vp]
+    L.rmm_reduced_gemm_workspace_bytes.argtypes = [mp, mp, i64, mp]
+    L.rmm_reduced_gemm_workspace_bytes.restype = sz
+    L.rmm_reduced_gemm.argtypes = [mp, mp, vp, i64, flt, mp, vp, sz, vp]
+    L.rmm_reduced_attn_workspace_bytes.argtypes = [ctypes.POINTER(rmm_attn_desc_t)]
+    L.rmm_reduced_attn_workspace_bytes.restype = sz
+    L.rmm_reduced_attn.argtypes = [ctypes.POINTER(rmm_attn_desc_t), vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.rmm_product_host_workspace_bytes.argtypes = [i64, i64, i64]
+    L.rmm_product_host_workspace_bytes.restype = sz
+    L.rmm_product_host.argtypes = [vp, vp, i64, i64, i64, dbl, i32, vp, vp, vp, sz, vp]
+    L.rmm_status_read.argtypes = [vp, ctypes.POINTER(i32)]
+    L.rmm_last_error.restype = ctypes.c_char_p
+    L.rmm_launch_count.restype = i64
+    _lib = L
+    return L
+
+
+def _check(rc: int) -> None:
+    if rc != RMM_OK:
+        raise RmmError(rc, lib().rmm_last_error().decode())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return RMM_BF16
+    if t.dtype == torch.float32:
+        return RMM_F32
+    raise RmmError(RMM_ERR_UNSUPPORTED, f"dtype {t.dtype} (bf16 and fp32 only)")
+
+
+def as_mat(t: torch.Tensor) -> rmm_mat_t:
+    """Describe a 2-D [rows, cols] or 3-D [batch, rows, cols] CUDA tensor (any strides) as an rmm_mat_t."""
+    if not t.is_cuda:
+        raise RmmError(RMM_ERR_INVALID_ARG, "tensor is not on a CUDA device")
+    if t.dim() == 2:
+        b, (r, c), sb, (sr, sc) = 1, t.shape, 0, t.stride()
+    elif t.dim() == 3:
+        b, r, c = t.shape
+        sb, sr, sc = t.stride()
+    else:
+        raise RmmError(RMM_ERR_INVALID_ARG, "expected a 2-D or 3-D tensor")
+    return rmm_mat_t(t.data_ptr(), _dtype_code(t), b, r, c, sb, sr, sc)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+_ws_cache = {}
+
+
+def workspace(nbytes: int, device: torch.device) -> torch.Tensor:
+    """A zero-initialised, cached, growing workspace per device (torch owns the memory)."""
+    key = (device.type, device.index if device.index is not None else torch.cuda.current_device())
+    ws = _ws_cache.get(key)
+    nbytes = max(int(nbytes), RMM_WS_HEADER_BYTES)
+    if ws is None or ws.numel() < nbytes:
+        ws = torch.zeros(nbytes + 256, dtype=torch.uint8, device=device)
+        _ws_cache[key] = ws
+    return ws
+
+
+def _ws_ptr(ws: torch.Tensor) -> Tuple[int, int]:
+    p = ws.data_ptr()
+    a = (p + 255) // 256 * 256
+    return a, ws.numel() - (a - p)
+
+
+def rmm_keep_count(rho: float, K: int) -> int:
+    k = ctypes.c_int64(0)
+    _check(lib().rmm_keep_count(float(rho), int(K), ctypes.byref(k)))
+    return int(k.value)
+
+
+def rmm_launch_count() -> int:
+    return int(lib().rmm_launch_count())
+
+
+def rmm_status_read(ws: Optional[torch.Tensor] = None, device=None) -> int:
+    """Synchronise the current stream, then read and clear the workspace's device status word."""
+    torch.cuda.current_stream().synchronize()
+    if ws is None:
+        ws = workspace(0, torch.device("cuda", torch.cuda.current_device()) if device is None else device)
+    st = ctypes.c_int(0)
+    p, _ = _ws_ptr(ws)
+    _check(lib().rmm_status_read(p, ctypes.byref(st)))
+    return int(st.value)
+
+
+def rmm_score(A: torch.Tensor, axis: int = 1, want_scores: bool = True, want_energy: bool = True,
+              ws: Optional[torch.Tensor] = None):
+    """(scores, energy) fp32 [batch, n] (2-D input: [n]); either may be None if not requested."""
+    m = as_mat(A)
+    n = m.cols if axis == 1 else m.rows
+    need = lib().rmm_score_workspace_bytes(ctypes.byref(m), axis)
+    if need == 0:
+        _check(lib().rmm_score(ctypes.byref(m), axis, None, None, None, 0, None) or RMM_ERR_INVALID_ARG)
+    ws = workspace(need, A.device) if ws is None else ws
+    p, nb = _ws_ptr(ws)
+    shape = (m.batch, n) if A.dim() == 3 else (n,)
+    scores = torch.empty(shape, dtype=torch.float32, device=A.device) if want_scores else None
+    energy = torch.empty(shape, dtype=torch.float32, device=A.device) if want_energy else None
+    _check(lib().rmm_score(ctypes.byref(m), axis, scores.data_ptr() if want_scores else None,
+                           energy.data_ptr() if want_energy else None, p, nb, _stream()))
+    return scores, energy
+
+
+def rmm_select(keys: torch.Tensor, rho: float = 0.0, k: int = 0, want_retained: bool = False,
+               ws: Optional[torch.Tensor] = None):
+    """idx int32 [batch, k] ascending (1-D keys: [k]); with want_retained also the kept key fraction."""
+    if keys.dtype != torch.float32 or not keys.is_cuda or not keys.is_contiguous():
+        raise RmmError(RMM_ERR_INVALID_ARG, "keys must be a contiguous fp32 CUDA tensor")
+    batch, K = (1, keys.shape[0]) if keys.dim() == 1 else keys.shape
+    kk = int(k) if k > 0 else rmm_keep_count(rho, K)
+    ws = workspace(lib().rmm_select_workspace_bytes(batch, K), keys.device) if ws is None else ws
+    p, nb = _ws_ptr(ws)
+    idx = torch.empty((batch, kk) if keys.dim() == 2 else (kk,), dtype=torch.int32, device=keys.device)
+    ret = torch.empty((batch,), dtype=torch.float32, device=keys.device) if want_retained else None
+    _check(lib().rmm_select(keys.data_ptr(), batch, K, float(rho), int(k), idx.data_ptr(),
+                            ret.data_ptr() if want_retained else None, p, nb, _stream()))
+    return (idx, ret) if want_retained else idx
+
+
+def rmm_score_select(A: torch.Tensor, rho: float = 0.0, k: int = 0, axis: int = 1, want_scores: bool = False,
+                     want_energy: bool = False, want_retained: bool = False, idx: Optional[torch.Tensor] = None,
+                     ws: Optional[torch.Tensor] = None):
+    """Fused score + top-k.  Returns (idx, scores, energy, retained); unrequested outputs are None."""
+    m = as_mat(A)
+    n = m.cols if axis == 1 else m.rows
+    kk = int(k) if k > 0 else rmm_keep_count(rho, n)
+    need = lib().rmm_score_select_workspace_bytes(ctypes.byref(m), axis)
+    ws = workspace(need, A.device) if ws is None else ws
+    p, nb = _ws_ptr(ws)
+    three = A.dim() == 3
+    if idx is None:
+        idx = torch.empty((m.batch, kk) if three else (kk,), dtype=torch.int32, device=A.device)
+    shape = (m.batch, n) if three else (n,)
+    scores = torch.empty(shape, dtype=torch.float32, device=A.device) if want_scores else None
+    energy = torch.empty(shape, dtype=torch.float32, device=A.device) if want_energy else None
+    ret = torch.empty((m.batch,), dtype=torch.float32, device=A.device) if want_retained else None
+    _check(lib().rmm_score_select(ctypes.byref(m), axis, float(rho), int(k), idx.data_ptr(),
+                                  scores.data_ptr() if want_scores else None,
+                                  energy.data_ptr() if want_energy else None,
+                                  ret.data_ptr() if want_retained else None, p, nb, _stream()))
+    return idx, scores, energy, ret
+
+
+def rmm_reduced_gemm(A: torch.Tensor, B: torch.Tensor, idx: torch.Tensor, scale: float = 1.0,
+                     out: Optional[torch.Tensor] = None, out_dtype: Optional[torch.dtype] = None,
+                     ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Y = scale * A[:, idx] @ B[idx, :].  A [M,K] or [b,M,K]; B [K,N] or [b,K,N]; idx int32 [k] or [b,k]."""
+    ma, mb = as_mat(A), as_mat(B)
+    if idx.dtype != torch.int32 or not idx.is_cuda or not idx.is_contiguous():
+        raise RmmError(RMM_ERR_INVALID_ARG, "idx must be a contiguous int32 CUDA tensor")
+    k = idx.shape[-1]
+    if idx.numel() != ma.batch * k:
+        raise RmmError(RMM_ERR_INVALID_ARG, "idx must hold one index list per batch element of A")
+    if out is None:
+        dt = out_dtype if out_dtype is not None else A.dtype
+        shape = (ma.batch, ma.rows, mb.cols) if A.dim() == 3 else (ma.rows, mb.cols)
+        out = torch.empty(shape, dtype=dt, device=A.device)
+    my = as_mat(out)
+    need = lib().rmm_reduced_gemm_workspace_bytes(ctypes.byref(ma), ctypes.byref(mb), k, ctypes.byref(my))
+    ws = workspace(need, A.device) if ws is None else ws
+    p, nb = _ws_ptr(ws)
+    _check(lib().rmm_reduced_gemm(ctypes.byref(ma), ctypes.byref(mb), idx.data_ptr(), k, float(scale),
+                                  ctypes.byref(my), p, nb, _stream()))
+    return out
+
+
+def rmm_reduced_attn(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, causal: bool, rho_d: float, rho_t: float = 1.0,
+                     want_idx: bool = False, ws: Optional[torch.Tensor] = None):
+    """Reduced attention.  Q [B,Hq,Lq,Dh], K,V [B,Hkv,Lk,Dh] bf16 with contiguous last dim.
+    Returns O [B,Hq,Lq,Dh] bf16, or (O, idx_feat, idx_tok) with want_idx (idx_tok None when rho_t == 1)."""
+    for t in (Q, K, V):
+        if t.dim() != 4 or t.dtype != torch.bfloat16 or not t.is_cuda or t.stride(3) != 1:
+            raise RmmError(RMM_ERR_UNSUPPORTED, "Q, K, V must be 4-D bf16 CUDA tensors with a contiguous last dim")
+    B, Hq, Lq, Dh = Q.shape
+    _, Hkv, Lk, _ = K.shape
+    O = torch.empty((B, Hq, Lq, Dh), dtype=torch.bfloat16, device=Q.device)
+    d = rmm_attn_desc_t(B, Hq, Hkv, Lq, Lk, Dh, int(bool(causal)), float(rho_d), float(rho_t),
+                        (ctypes.c_int64 * 3)(*Q.stride()[:3]), (ctypes.c_int64 * 3)(*K.stride()[:3]),
+                        (ctypes.c_int64 * 3)(*V.stride()[:3]), (ctypes.c_int64 * 3)(*O.stride()[:3]))
+    need = lib().rmm_reduced_attn_workspace_bytes(ctypes.byref(d))
+    if need == 0:
+        raise RmmError(RMM_ERR_INVALID_ARG, "reduced_attn: invalid description (check shapes and retention ratios)")
+    ws = workspace(need, Q.device) if ws is None else ws
+    p, nb = _ws_ptr(ws)
+    idx_feat = idx_tok = None
+    if want_idx:
+        idx_feat = torch.empty((B, Hq, rmm_keep_count(rho_d, Dh)), dtype=torch.int32, device=Q.device)
+        if rho_t < 1.0:
+            idx_tok = torch.empty((B, Hq, rmm_keep_count(rho_t, Lk)), dtype=torch.int32, device=Q.device)
+    _check(lib().rmm_reduced_attn(ctypes.byref(d), Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(),
+                                  idx_feat.data_ptr() if idx_feat is not None else None,
+                                  idx_tok.data_ptr() if idx_tok is not None else None, p, nb, _stream()))
+    return (O, idx_feat, idx_tok) if want_idx else O
+
+
+def rmm_product_host(A_host: torch.Tensor, B_host: torch.Tensor, rho: float, Y_host: torch.Tensor,
+                     idx_host: Optional[torch.Tensor] = None, copy_B: bool = True,
+                     ws: Optional[torch.Tensor] = None, device: Optional[torch.device] = None) -> None:
+    """Whole operation on (pinned) host bf16 buffers; asynchronous: synchronise the stream before reading Y_host."""
+    M, K = A_host.shape
+    _, N = B_host.shape
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    need = lib().rmm_product_host_workspace_bytes(M, K, N)
+    ws = workspace(need, device) if ws is None else ws
+    p, nb = _ws_ptr(ws)
+    _check(lib().rmm_product_host(A_host.data_ptr(), B_host.data_ptr(), M, K, N, float(rho), int(bool(copy_B)),
+                                  Y_host.data_ptr(), idx_host.data_ptr() if idx_host is not None else None,
+                                  p, nb, _stream()))
+
+
+def rmm(A: torch.Tensor, B: torch.Tensor, rho: float, out: Optional[torch.Tensor] = None):
+    """RMM_rho(A, B) of Sec. 3.2 on device tensors: fused score + select, then the reduced product.
+    Returns (Y, idx)."""
+    idx, _, _, _ = rmm_score_select(A, rho=rho)
+    return rmm_reduced_gemm(A, B, idx, out=out), idx

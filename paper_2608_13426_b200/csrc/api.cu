@@ -1,0 +1,283 @@
+// C ABI of the RMM library: argument checks, workspace layout and kernel dispatch.  No entry point
+// allocates device memory or synchronises (rmm_status_read excepted, which is a blocking copy).
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace rmm {
+
+static thread_local char t_error[512] = "";
+std::atomic<int64_t> g_launches{0};
+
+int fail(int code, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(t_error, sizeof t_error, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int check_launch(const char *what)
+{
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "%s: launch failed: %s", what, cudaGetErrorString(e));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return RMM_OK;
+}
+
+static int check_ws(void *ws, size_t ws_bytes, size_t need, const char *who)
+{
+    if (ws == nullptr) return fail(RMM_ERR_WORKSPACE, "%s: workspace is NULL (need %zu bytes)", who, need);
+    if (reinterpret_cast<uintptr_t>(ws) % 256 != 0) return fail(RMM_ERR_WORKSPACE, "%s: workspace is not 256-byte aligned", who);
+    if (ws_bytes < need) return fail(RMM_ERR_WORKSPACE, "%s: workspace has %zu bytes, needs %zu", who, ws_bytes, need);
+    return RMM_OK;
+}
+
+static int check_mat(const rmm_mat_t *X, const char *who, const char *name)
+{
+    if (X == nullptr || X->ptr == nullptr) return fail(RMM_ERR_INVALID_ARG, "%s: %s is NULL", who, name);
+    if (X->batch < 1 || X->rows < 1 || X->cols < 1)
+        return fail(RMM_ERR_INVALID_ARG, "%s: %s has a non-positive dimension", who, name);
+    if (X->dtype != RMM_BF16 && X->dtype != RMM_F32) return fail(RMM_ERR_UNSUPPORTED, "%s: %s has an unknown dtype", who, name);
+    if (X->stride_batch < 0 || X->stride_row < 0 || X->stride_col < 0)
+        return fail(RMM_ERR_UNSUPPORTED, "%s: %s has a negative stride", who, name);
+    return RMM_OK;
+}
+
+static int resolve_k(double rho, int64_t k, int64_t K, int64_t *out, const char *who)
+{
+    if (k > 0) {
+        if (k > K) return fail(RMM_ERR_INVALID_ARG, "%s: k = %lld exceeds K = %lld", who, (long long)k, (long long)K);
+        *out = k;
+        return RMM_OK;
+    }
+    if (k < 0) return fail(RMM_ERR_INVALID_ARG, "%s: k is negative", who);
+    int rc = rmm_keep_count(rho, K, out);
+    if (rc != RMM_OK) return fail(rc, "%s: rho = %g is outside (0, 1]", who, rho);
+    return RMM_OK;
+}
+
+}  // namespace rmm
+
+using namespace rmm;
+
+extern "C" {
+
+int rmm_keep_count(double rho, int64_t K, int64_t *k)
+{
+    if (k == nullptr || K < 1 || !(rho > 0.0) || !(rho <= 1.0))
+        return fail(RMM_ERR_INVALID_ARG, "keep_count: need rho in (0, 1], K >= 1 and a non-NULL result");
+    const double x = rho * (double)K;
+    const double r = nearbyint(x);
+    int64_t v = fabs(x - r) <= 1e-9 * (double)K ? (int64_t)r : (int64_t)ceil(x);
+    if (v < 1) v = 1;
+    if (v > K) v = K;
+    *k = v;
+    return RMM_OK;
+}
+
+size_t rmm_score_workspace_bytes(const rmm_mat_t *A, int axis)
+{
+    ScorePlan p;
+    if (plan_score(A, axis, &p) != RMM_OK) return 0;
+    return p.total_bytes;
+}
+
+int rmm_score(const rmm_mat_t *A, int axis, float *scores, float *energy, void *ws, size_t ws_bytes, void *stream)
+{
+    ScorePlan p;
+    int rc = plan_score(A, axis, &p);
+    if (rc != RMM_OK) return rc;
+    if (scores == nullptr && energy == nullptr) return fail(RMM_ERR_INVALID_ARG, "score: both outputs are NULL");
+    rc = check_ws(ws, ws_bytes, p.total_bytes, "score");
+    if (rc != RMM_OK) return rc;
+    return launch_score_select(A, p, false, 0, nullptr, scores, energy, nullptr, ws, static_cast<cudaStream_t>(stream));
+}
+
+size_t rmm_select_workspace_bytes(int64_t batch, int64_t K)
+{
+    (void)batch;
+    (void)K;
+    return RMM_WS_HEADER_BYTES;
+}
+
+int rmm_select(const float *keys, int64_t batch, int64_t K, double rho, int64_t k, int32_t *idx, float *retained,
+               void *ws, size_t ws_bytes, void *stream)
+{
+    if (keys == nullptr || idx == nullptr) return fail(RMM_ERR_INVALID_ARG, "select: keys or idx is NULL");
+    if (batch < 1 || K < 1) return fail(RMM_ERR_INVALID_ARG, "select: non-positive dimension");
+    if (K > ((int64_t)1 << 30) || batch > INT32_MAX) return fail(RMM_ERR_UNSUPPORTED, "select: dimension too large");
+    int64_t kk;
+    int rc = resolve_k(rho, k, K, &kk, "select");
+    if (rc != RMM_OK) return rc;
+    rc = check_ws(ws, ws_bytes, RMM_WS_HEADER_BYTES, "select");
+    if (rc != RMM_OK) return rc;
+    return launch_select(keys, batch, K, kk, idx, retained, ws, static_cast<cudaStream_t>(stream));
+}
+
+size_t rmm_score_select_workspace_bytes(const rmm_mat_t *A, int axis) { return rmm_score_workspace_bytes(A, axis); }
+
+int rmm_score_select(const rmm_mat_t *A, int axis, double rho, int64_t k, int32_t *idx, float *scores, float *energy,
+                     float *retained, void *ws, size_t ws_bytes, void *stream)
+{
+    ScorePlan p;
+    int rc = plan_score(A, axis, &p);
+    if (rc != RMM_OK) return rc;
+    if (idx == nullptr) return fail(RMM_ERR_INVALID_ARG, "score_select: idx is NULL");
+    int64_t kk;
+    rc = resolve_k(rho, k, p.n, &kk, "score_select");
+    if (rc != RMM_OK) return rc;
+    rc = check_ws(ws, ws_bytes, p.total_bytes, "score_select");
+    if (rc != RMM_OK) return rc;
+    return launch_score_select(A, p, true, kk, idx, scores, energy, retained, ws, static_cast<cudaStream_t>(stream));
+}
+
+static int check_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, const rmm_mat_t *Y)
+{
+    int rc;
+    if ((rc = check_mat(A, "reduced_gemm", "A")) != RMM_OK) return rc;
+    if ((rc = check_mat(B, "reduced_gemm", "B")) != RMM_OK) return rc;
+    if ((rc = check_mat(Y, "reduced_gemm", "Y")) != RMM_OK) return rc;
+    if (idx == nullptr) return fail(RMM_ERR_INVALID_ARG, "reduced_gemm: idx is NULL");
+    if (A->cols != B->rows) return fail(RMM_ERR_INVALID_ARG, "reduced_gemm: A has %lld columns but B has %lld rows",
+                                        (long long)A->cols, (long long)B->rows);
+    if (Y->rows != A->rows || Y->cols != B->cols || Y->batch != A->batch)
+        return fail(RMM_ERR_INVALID_ARG, "reduced_gemm: Y must be [batch of A, rows of A, columns of B]");
+    if (B->batch != A->batch && !(B->batch == 1))
+        return fail(RMM_ERR_INVALID_ARG, "reduced_gemm: B must have A's batch or batch 1");
+    if (k < 1 || k > A->cols) return fail(RMM_ERR_INVALID_ARG, "reduced_gemm: k = %lld is outside [1, K]", (long long)k);
+    if (A->dtype != B->dtype) return fail(RMM_ERR_UNSUPPORTED, "reduced_gemm: A and B must share a dtype");
+    if (Y->stride_batch == 0 && Y->batch > 1) return fail(RMM_ERR_INVALID_ARG, "reduced_gemm: Y batches overlap");
+    return RMM_OK;
+}
+
+// B with batch 1 is shared by every batch element of A: normalise its batch stride to 0.
+static rmm_mat_t shared_b(const rmm_mat_t *A, const rmm_mat_t *B)
+{
+    rmm_mat_t b = *B;
+    if (B->batch == 1 && A->batch >= 1) b.stride_batch = 0;
+    b.batch = A->batch;
+    return b;
+}
+
+size_t rmm_reduced_gemm_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y)
+{
+    if (A == nullptr || B == nullptr || Y == nullptr) return 0;
+    rmm_mat_t b = shared_b(A, B);
+    TcPlan plan;
+    if (tc_eligible(A, &b, k, Y, &plan)) return plan.total_bytes;
+    return RMM_WS_HEADER_BYTES;
+}
+
+int rmm_reduced_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
+                     const rmm_mat_t *Y, void *ws, size_t ws_bytes, void *stream)
+{
+    int rc = check_gemm(A, B, idx, k, Y);
+    if (rc != RMM_OK) return rc;
+    rmm_mat_t b = shared_b(A, B);
+    TcPlan plan;
+    if (tc_eligible(A, &b, k, Y, &plan)) {
+        rc = check_ws(ws, ws_bytes, plan.total_bytes, "reduced_gemm");
+        if (rc != RMM_OK) return rc;
+        return launch_gemm_tc(A, &b, idx, k, scale, Y, plan, ws, static_cast<cudaStream_t>(stream));
+    }
+    rc = check_ws(ws, ws_bytes, RMM_WS_HEADER_BYTES, "reduced_gemm");
+    if (rc != RMM_OK) return rc;
+    return launch_gemm_simt(A, &b, idx, k, scale, Y, ws, static_cast<cudaStream_t>(stream));
+}
+
+// ---- whole operation on host buffers -------------------------------------------------------------
+struct HostPlan {
+    size_t off_a, off_b, off_y, off_idx, off_inner, inner_bytes, total;
+    rmm_mat_t A, B, Y;
+};
+
+static int plan_host(int64_t M, int64_t K, int64_t N, void *ws, HostPlan *h)
+{
+    if (M < 1 || K < 1 || N < 1) return fail(RMM_ERR_INVALID_ARG, "product_host: non-positive dimension");
+    size_t off = 0;
+    h->off_inner = off;  // the inner calls' workspace comes first so that its header is the status word
+    char *w = static_cast<char *>(ws);
+    rmm_mat_t A = {nullptr, RMM_BF16, 1, M, K, M * K, K, 1};
+    rmm_mat_t B = {nullptr, RMM_BF16, 1, K, N, K * N, N, 1};
+    rmm_mat_t Y = {nullptr, RMM_BF16, 1, M, N, M * N, N, 1};
+    // sizes that do not depend on the pointers: use aligned dummies for the planners
+    A.ptr = B.ptr = Y.ptr = reinterpret_cast<void *>(uintptr_t(256));
+    size_t s1 = rmm_score_select_workspace_bytes(&A, 1);
+    size_t s2 = rmm_reduced_gemm_workspace_bytes(&A, &B, K, &Y);  // k = K bounds every k
+    if (s1 == 0 || s2 == 0) return RMM_ERR_UNSUPPORTED;
+    h->inner_bytes = align_up(s1 > s2 ? s1 : s2, 256);
+    off += h->inner_bytes;
+    h->off_a = off; off += align_up((size_t)M * K * 2, 256);
+    h->off_b = off; off += align_up((size_t)K * N * 2, 256);
+    h->off_y = off; off += align_up((size_t)M * N * 2, 256);
+    h->off_idx = off; off += align_up((size_t)K * 4, 256);
+    h->total = off;
+    A.ptr = w ? w + h->off_a : nullptr;
+    B.ptr = w ? w + h->off_b : nullptr;
+    Y.ptr = w ? w + h->off_y : nullptr;
+    h->A = A; h->B = B; h->Y = Y;
+    return RMM_OK;
+}
+
+size_t rmm_product_host_workspace_bytes(int64_t M, int64_t K, int64_t N)
+{
+    HostPlan h;
+    if (plan_host(M, K, N, nullptr, &h) != RMM_OK) return 0;
+    return h.total;
+}
+
+int rmm_product_host(const void *A_host, const void *B_host, int64_t M, int64_t K, int64_t N, double rho, int copy_B,
+                     void *Y_host, int32_t *idx_host, void *ws, size_t ws_bytes, void *stream)
+{
+    if (A_host == nullptr || Y_host == nullptr || (copy_B && B_host == nullptr))
+        return fail(RMM_ERR_INVALID_ARG, "product_host: NULL host buffer");
+    HostPlan h;
+    int rc = plan_host(M, K, N, ws, &h);
+    if (rc != RMM_OK) return rc;
+    rc = check_ws(ws, ws_bytes, h.total, "product_host");
+    if (rc != RMM_OK) return rc;
+    int64_t k;
+    rc = resolve_k(rho, 0, K, &k, "product_host");
+    if (rc != RMM_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *w = static_cast<char *>(ws);
+    int32_t *idx = reinterpret_cast<int32_t *>(w + h.off_idx);
+    cudaError_t e = cudaMemcpyAsync(h.A.ptr, A_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && copy_B) e = cudaMemcpyAsync(h.B.ptr, B_host, (size_t)K * N * 2, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "product_host: host-to-device copy: %s", cudaGetErrorString(e));
+    rc = rmm_score_select(&h.A, 1, rho, k, idx, nullptr, nullptr, nullptr, w + h.off_inner, h.inner_bytes, stream);
+    if (rc != RMM_OK) return rc;
+    rc = rmm_reduced_gemm(&h.A, &h.B, idx, k, 1.0f, &h.Y, w + h.off_inner, h.inner_bytes, stream);
+    if (rc != RMM_OK) return rc;
+    e = cudaMemcpyAsync(Y_host, h.Y.ptr, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && idx_host != nullptr)
+        e = cudaMemcpyAsync(idx_host, idx, (size_t)k * 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "product_host: device-to-host copy: %s", cudaGetErrorString(e));
+    return RMM_OK;
+}
+
+int rmm_status_read(void *ws, int *device_status)
+{
+    if (ws == nullptr || device_status == nullptr) return fail(RMM_ERR_INVALID_ARG, "status_read: NULL argument");
+    int v = 0;
+    cudaError_t e = cudaMemcpy(&v, ws, sizeof v, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "status_read: %s", cudaGetErrorString(e));
+    if (v != 0) {
+        int zero = 0;
+        e = cudaMemcpy(ws, &zero, sizeof zero, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "status_read: %s", cudaGetErrorString(e));
+    }
+    *device_status = v;
+    return RMM_OK;
+}
+
+const char *rmm_last_error(void) { return t_error; }
+
+int64_t rmm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,230 @@
+// Reduced attention (paper Sec. 3.3) composed from the library's own kernels, one group of query heads
+// at a time:
+//   score + select on Q          -> I per query head              (score_select_kernel)
+//   pack Q[:, I], K_g[:, I]      -> K-major operands              (pack_cols_kernel)
+//   S~ = Q[:, I] K[:, I]^T / sqrt(Dh), fp32                        (reduced_gemm_tc_kernel, K-major B)
+//   P  = bf16(softmax(S~ + causal mask))                            (softmax_rows_kernel)
+//   rho_t < 1: score + select on P -> T; pack P[:, T]; O = P[:, T] V_g[T, :] with V rows fetched by TMA gather4
+//   rho_t = 1: O = P V_g (same kernel, P loaded in place, rows 0 .. Lk-1 of V)
+// S~ and P live in the workspace (materialised), so this form is bound by HBM traffic, not by the tensor cores.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace rmm {
+namespace {
+
+constexpr int kSoftmaxThreads = 256;
+
+__device__ __forceinline__ float block_reduce(float v, bool is_max, float *sh)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        float o = __shfl_xor_sync(0xffffffffu, v, d);
+        v = is_max ? fmaxf(v, o) : v + o;
+    }
+    __syncthreads();
+    if (lane == 0) sh[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        float w = lane < (blockDim.x >> 5) ? sh[lane] : (is_max ? -INFINITY : 0.f);
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            float o = __shfl_xor_sync(0xffffffffu, w, d);
+            w = is_max ? fmaxf(w, o) : w + o;
+        }
+        if (lane == 0) sh[0] = w;
+    }
+    __syncthreads();
+    return sh[0];
+}
+
+// One block per row: max, sum of exp, normalise, round to bf16 (RNE).  Keys t > i + (Lk - Lq) are masked
+// when causal; a row with no visible key is all zeros.
+__global__ void __launch_bounds__(kSoftmaxThreads) softmax_rows_kernel(const float *__restrict__ S, int64_t ld_s,
+                                                                       int64_t Lq, int64_t Lk, int causal,
+                                                                       __nv_bfloat16 *__restrict__ P, int64_t ld_p)
+{
+    __shared__ float sh[32];
+    const int64_t i = blockIdx.x, h = blockIdx.y;
+    const float *s = S + (h * Lq + i) * ld_s;
+    __nv_bfloat16 *p = P + (h * Lq + i) * ld_p;
+    int64_t visible = causal ? i + (Lk - Lq) + 1 : Lk;
+    if (visible > Lk) visible = Lk;
+    if (visible < 0) visible = 0;
+
+    float mx = -INFINITY;
+    for (int64_t t = threadIdx.x; t < visible; t += kSoftmaxThreads) mx = fmaxf(mx, s[t]);
+    mx = block_reduce(mx, true, sh);
+    float sum = 0.f;
+    for (int64_t t = threadIdx.x; t < visible; t += kSoftmaxThreads) sum += expf(s[t] - mx);
+    sum = block_reduce(sum, false, sh);
+    const float inv = sum > 0.f ? 1.0f / sum : 0.f;
+    for (int64_t t = threadIdx.x; t < ld_p; t += kSoftmaxThreads) {
+        float v = t < visible ? expf(s[t] - mx) * inv : 0.f;
+        p[t] = __float2bfloat16_rn(v);
+    }
+}
+
+struct AttnPlan {
+    int64_t kd, kt, ldd, ldt, ld_s, ld_p, hg;
+    size_t inner_bytes, off_idxf, off_idxt, off_qp, off_kp, off_s, off_p, off_pp, total;
+};
+
+int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
+{
+    if (d == nullptr) return fail(RMM_ERR_INVALID_ARG, "reduced_attn: NULL description");
+    if (d->B < 1 || d->Hq < 1 || d->Hkv < 1 || d->Lq < 1 || d->Lk < 1 || d->Dh < 1)
+        return fail(RMM_ERR_INVALID_ARG, "reduced_attn: non-positive dimension");
+    if (d->Hq % d->Hkv != 0) return fail(RMM_ERR_INVALID_ARG, "reduced_attn: Hq must be a multiple of Hkv");
+    if (rmm_keep_count(d->rho_d, d->Dh, &p->kd) != RMM_OK || rmm_keep_count(d->rho_t, d->Lk, &p->kt) != RMM_OK)
+        return fail(RMM_ERR_INVALID_ARG, "reduced_attn: rho_d and rho_t must lie in (0, 1]");
+    if (d->Dh % 8 != 0) return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: Dh must be a multiple of 8");
+    if (d->Lq > INT32_MAX || d->Lk > INT32_MAX || d->Hq > 65535) return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: too large");
+    for (int i = 0; i < 3; ++i)
+        if (d->q_stride[i] % 8 || d->k_stride[i] % 8 || d->v_stride[i] % 8 || d->o_stride[i] % 8)
+            return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: strides must be multiples of 8 elements");
+    // V must flatten to one 2-D [B*Hkv*Lk, Dh] tensor for the row gather
+    if (d->v_stride[2] < d->Dh || d->v_stride[1] != d->Lk * d->v_stride[2] || d->v_stride[0] != d->Hkv * d->v_stride[1])
+        return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: V must be contiguous over (batch, head, token)");
+    if (d->B * d->Hkv * d->Lk > INT32_MAX) return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: B*Hkv*Lk exceeds 2^31");
+    p->ldd = (p->kd + 7) / 8 * 8;
+    p->ldt = (p->kt + 7) / 8 * 8;
+    p->ld_p = (d->Lk + 7) / 8 * 8;
+    p->ld_s = (d->Lk + 3) / 4 * 4;
+    // heads per group: keep S~ (fp32) + P (bf16) + P[:, T] within about 6 GiB
+    const double per_head = (double)d->Lq * ((double)p->ld_s * 4 + (double)p->ld_p * 2 + (double)p->ldt * 2);
+    int64_t hg = (int64_t)(6.0 * 1073741824.0 / per_head);
+    if (hg < 1) hg = 1;
+    if (hg > d->Hq) hg = d->Hq;
+    p->hg = hg;
+
+    // workspace of the inner score/select calls (the larger of the Q pass and the P pass)
+    rmm_mat_t qm = {reinterpret_cast<void *>(uintptr_t(256)), RMM_BF16, hg, d->Lq, d->Dh, d->q_stride[1], d->q_stride[2], 1};
+    rmm_mat_t pm = {reinterpret_cast<void *>(uintptr_t(256)), RMM_BF16, hg, d->Lq, d->Lk, d->Lq * p->ld_p, p->ld_p, 1};
+    ScorePlan sq, sp;
+    int rc = plan_score(&qm, 1, &sq);
+    if (rc != RMM_OK) return rc;
+    rc = plan_score(&pm, 1, &sp);
+    if (rc != RMM_OK) return rc;
+    p->inner_bytes = align_up(sq.total_bytes > sp.total_bytes ? sq.total_bytes : sp.total_bytes, 256);
+    size_t off = p->inner_bytes;
+    p->off_idxf = off; off += align_up((size_t)hg * p->kd * 4, 256);
+    p->off_idxt = off; off += align_up((size_t)hg * p->kt * 4, 256);
+    p->off_qp = off; off += align_up((size_t)hg * d->Lq * p->ldd * 2, 256);
+    p->off_kp = off; off += align_up((size_t)hg * d->Lk * p->ldd * 2, 256);
+    p->off_s = off; off += align_up((size_t)hg * d->Lq * p->ld_s * 4, 256);
+    p->off_p = off; off += align_up((size_t)hg * d->Lq * p->ld_p * 2, 256);
+    p->off_pp = off; off += align_up((size_t)hg * d->Lq * p->ldt * 2, 256);
+    p->total = off;
+    return RMM_OK;
+}
+
+}  // namespace
+
+int launch_softmax_rows(const float *S, int64_t ld_s, int64_t heads, int64_t Lq, int64_t Lk, int causal,
+                        __nv_bfloat16 *P, int64_t ld_p, cudaStream_t stream)
+{
+    dim3 grid((unsigned)Lq, (unsigned)heads);
+    softmax_rows_kernel<<<grid, kSoftmaxThreads, 0, stream>>>(S, ld_s, Lq, Lk, causal, P, ld_p);
+    return check_launch("softmax_rows_kernel");
+}
+
+}  // namespace rmm
+
+using namespace rmm;
+
+extern "C" {
+
+size_t rmm_reduced_attn_workspace_bytes(const rmm_attn_desc_t *desc)
+{
+    AttnPlan p;
+    if (plan_attn(desc, &p) != RMM_OK) return 0;
+    return p.total;
+}
+
+int rmm_reduced_attn(const rmm_attn_desc_t *d, const void *Q, const void *K, const void *V, void *O, int32_t *idx_feat,
+                     int32_t *idx_tok, void *ws, size_t ws_bytes, void *stream)
+{
+    AttnPlan p;
+    int rc = plan_attn(d, &p);
+    if (rc != RMM_OK) return rc;
+    if (Q == nullptr || K == nullptr || V == nullptr || O == nullptr) return fail(RMM_ERR_INVALID_ARG, "reduced_attn: NULL tensor");
+    for (const void *ptr : {Q, K, V, (const void *)O})
+        if (reinterpret_cast<uintptr_t>(ptr) % 16 != 0) return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: tensors must be 16-byte aligned");
+    if (ws == nullptr || reinterpret_cast<uintptr_t>(ws) % 256 != 0 || ws_bytes < p.total)
+        return fail(RMM_ERR_WORKSPACE, "reduced_attn: workspace must be 256-byte aligned and hold %zu bytes", p.total);
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *w = static_cast<char *>(ws);
+    int *status = &reinterpret_cast<WsHeader *>(w)->status;
+    const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(Q), *kk = static_cast<const __nv_bfloat16 *>(K),
+                        *v = static_cast<const __nv_bfloat16 *>(V);
+    __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(O);
+    __nv_bfloat16 *Qp = reinterpret_cast<__nv_bfloat16 *>(w + p.off_qp), *Kp = reinterpret_cast<__nv_bfloat16 *>(w + p.off_kp);
+    __nv_bfloat16 *P = reinterpret_cast<__nv_bfloat16 *>(w + p.off_p), *Pp = reinterpret_cast<__nv_bfloat16 *>(w + p.off_pp);
+    float *S = reinterpret_cast<float *>(w + p.off_s);
+    const int64_t group = d->Hq / d->Hkv;
+    const float scale = (float)(1.0 / sqrt((double)d->Dh));
+    const bool tok = d->rho_t < 1.0;
+
+    for (int64_t b = 0; b < d->B; ++b) {
+        for (int64_t h0 = 0; h0 < d->Hq; h0 += p.hg) {
+            const int64_t hg = d->Hq - h0 < p.hg ? d->Hq - h0 : p.hg;
+            int32_t *If = idx_feat ? idx_feat + (b * d->Hq + h0) * p.kd : reinterpret_cast<int32_t *>(w + p.off_idxf);
+            int32_t *It = idx_tok ? idx_tok + (b * d->Hq + h0) * p.kt : reinterpret_cast<int32_t *>(w + p.off_idxt);
+
+            // feature scores on Q only, one index set per query head
+            rmm_mat_t qm = {const_cast<__nv_bfloat16 *>(q + b * d->q_stride[0] + h0 * d->q_stride[1]), RMM_BF16, hg, d->Lq, d->Dh,
+                            d->q_stride[1], d->q_stride[2], 1};
+            ScorePlan sq;
+            if ((rc = plan_score(&qm, 1, &sq)) != RMM_OK) return rc;
+            if ((rc = launch_score_select(&qm, sq, true, p.kd, If, nullptr, nullptr, nullptr, w, st)) != RMM_OK) return rc;
+
+            // Q[:, I_h] and K_{g(h)}[:, I_h]
+            rc = launch_pack_cols(static_cast<const __nv_bfloat16 *>(qm.ptr), hg, d->Lq, d->Dh, d->q_stride[1], d->q_stride[2], 0, 1,
+                                  If, p.kd, p.kd, Qp, p.ldd, status, st);
+            if (rc != RMM_OK) return rc;
+            rc = launch_pack_cols(kk + b * d->k_stride[0], hg, d->Lk, d->Dh, d->k_stride[1], d->k_stride[2], h0, group, If, p.kd,
+                                  p.kd, Kp, p.ldd, status, st);
+            if (rc != RMM_OK) return rc;
+
+            // S~ = Q[:, I] K[:, I]^T / sqrt(Dh)  (the scale keeps the full head dimension)
+            TcProblem g1 = {};
+            g1.batch = hg; g1.M = d->Lq; g1.N = d->Lk; g1.k = p.kd;
+            g1.a = Qp; g1.a_ld = p.ldd; g1.a_sb = d->Lq * p.ldd;
+            g1.b_kmajor = 1; g1.b = Kp; g1.b_ld = p.ldd; g1.b_sb = d->Lk * p.ldd;
+            g1.y = S; g1.y_bf16 = 0; g1.y_sb = d->Lq * p.ld_s; g1.y_sr = p.ld_s;
+            g1.scale = scale; g1.status = status;
+            if ((rc = launch_gemm_tc_problem(g1, st)) != RMM_OK) return rc;
+
+            if ((rc = launch_softmax_rows(S, p.ld_s, hg, d->Lq, d->Lk, d->causal, P, p.ld_p, st)) != RMM_OK) return rc;
+
+            TcProblem g2 = {};
+            g2.batch = hg; g2.M = d->Lq; g2.N = d->Dh;
+            g2.b_kmajor = 0; g2.b = v; g2.b_ld = d->v_stride[2]; g2.b_rows_total = d->B * d->Hkv * d->Lk;
+            g2.b_batch_rows = d->Lk; g2.b_batch_off = b * d->Hq + h0; g2.b_batch_div = group;
+            g2.y = o + b * d->o_stride[0] + h0 * d->o_stride[1]; g2.y_bf16 = 1; g2.y_sb = d->o_stride[1]; g2.y_sr = d->o_stride[2];
+            g2.scale = 1.0f; g2.status = status;
+            if (tok) {
+                // token scores on the rounded P, one token set per query head, then O = P[:, T] V[T, :]
+                rmm_mat_t pm = {P, RMM_BF16, hg, d->Lq, d->Lk, d->Lq * p.ld_p, p.ld_p, 1};
+                ScorePlan sp;
+                if ((rc = plan_score(&pm, 1, &sp)) != RMM_OK) return rc;
+                if ((rc = launch_score_select(&pm, sp, true, p.kt, It, nullptr, nullptr, nullptr, w, st)) != RMM_OK) return rc;
+                rc = launch_pack_cols(P, hg, d->Lq, d->Lk, d->Lq * p.ld_p, p.ld_p, 0, 1, It, p.kt, p.kt, Pp, p.ldt, status, st);
+                if (rc != RMM_OK) return rc;
+                g2.k = p.kt; g2.a = Pp; g2.a_ld = p.ldt; g2.a_sb = d->Lq * p.ldt;
+                g2.idx = It; g2.idx_stride = p.kt;
+            } else {
+                g2.k = d->Lk; g2.a = P; g2.a_ld = p.ld_p; g2.a_sb = d->Lq * p.ld_p;
+                g2.idx = nullptr; g2.idx_stride = 0;
+            }
+            if ((rc = launch_gemm_tc_problem(g2, st)) != RMM_OK) return rc;
+        }
+    }
+    return RMM_OK;
+}
+
+}  // extern "C"

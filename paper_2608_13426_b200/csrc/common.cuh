@@ -1,0 +1,96 @@
+// Shared declarations of the RMM library's translation units (internal; the public ABI is rmm.h).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "rmm.h"
+
+namespace rmm {
+
+// ---- error text (thread-local) and launch accounting -------------------------------------------
+int fail(int code, const char *fmt, ...);
+extern std::atomic<int64_t> g_launches;
+int check_launch(const char *what);  // cudaGetLastError -> RMM_OK / RMM_ERR_CUDA, counts the launch
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+static inline size_t dtype_size(int dt) { return dt == RMM_BF16 ? 2 : 4; }
+
+// ---- workspace header: status word, then self-resetting arrival counters --------------------------
+struct WsHeader {
+    int status;  // rmm_status_t written by kernels (0 = ok)
+    int pad[15];
+    unsigned counters[(RMM_WS_HEADER_BYTES - 64) / 4];
+};
+static_assert(sizeof(WsHeader) == RMM_WS_HEADER_BYTES, "header size");
+constexpr int64_t kHeaderCounters = (RMM_WS_HEADER_BYTES - 64) / 4;
+
+// ---- score + select ---------------------------------------------------------------------------------
+struct ScorePlan {
+    int vec;         // elements per load: 8 (bf16, 16 B), 4 (fp32, 16 B) or 1 (generic strides)
+    int tx, ty;      // thread layout: tx column groups x ty row lanes, tx * ty = 256
+    int col_blocks;  // ceil(n / (tx * vec))
+    int row_splits;  // row ranges summed by separate blocks
+    int64_t rows_per_split;
+    int64_t n, m;    // scored axis length, reduced axis length
+    int64_t s_batch, s_red, s_n;  // element strides: batch, reduced axis, scored axis
+    size_t off_counters, off_partials, off_energy, total_bytes;
+    bool counters_in_header;
+};
+int plan_score(const rmm_mat_t *A, int axis, ScorePlan *plan);
+int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, int64_t k, int32_t *idx,
+                        float *scores, float *energy, float *retained, void *ws, cudaStream_t stream);
+int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_t *idx, float *retained, void *ws,
+                  cudaStream_t stream);
+
+// ---- reduced GEMM ------------------------------------------------------------------------------------
+// Plain FMA kernel: any strides, bf16 or fp32 operands, fp32 accumulation, bf16 or fp32 output.
+int launch_gemm_simt(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
+                     const rmm_mat_t *Y, void *ws, cudaStream_t stream);
+
+// Tensor-core path (tcgen05, TMEM accumulators).  Operands must satisfy tc_eligible().
+struct TcPlan {
+    int b_kmajor;       // 0: B rows (contraction slices) contiguous, gathered by TMA; 1: B is K-contiguous, packed first
+    int64_t ldp;        // leading dimension of the packed operands (multiple of 8)
+    size_t off_ap, off_bp, total_bytes;
+};
+bool tc_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y, TcPlan *plan);
+int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
+                   const rmm_mat_t *Y, const TcPlan &plan, void *ws, cudaStream_t stream);
+
+// A tensor-core problem on operands that are already in TMA-loadable form.
+struct TcProblem {
+    int64_t batch, M, N, k;
+    const __nv_bfloat16 *a;  // K-major A [batch, M, a_ld]: the kept columns are its first k columns
+    int64_t a_ld, a_sb;      // row pitch and batch stride in elements (multiples of 8)
+    int b_kmajor;
+    const __nv_bfloat16 *b;  // K-major: [batch, N, b_ld] (kept columns first); MN-major: 2-D [b_rows_total, N], pitch b_ld
+    int64_t b_ld, b_sb, b_rows_total;
+    const int32_t *idx;      // MN-major B: kept rows per batch entry (NULL = rows 0 .. k-1), lists idx_stride apart
+    int64_t idx_stride;
+    int64_t b_batch_rows, b_batch_off, b_batch_div;  // MN-major B: first row of entry i = ((i + off) / div) * rows
+    void *y;
+    int y_bf16;
+    int64_t y_sb, y_sr;
+    float scale;
+    int *status;
+};
+int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream);
+
+// Gather columns: dst[b, r, j] = src[sb, r, idx[b, j]] for j < k with source batch sb = (b + b_off) / b_div
+// (dst row pitch ld_dst >= k; columns k..ld_dst are zeroed).  bf16 only.  idx_stride = elements between the
+// index lists of two batch entries.
+int launch_pack_cols(const __nv_bfloat16 *src, int64_t batch, int64_t rows, int64_t K, int64_t s_batch, int64_t s_row,
+                     int64_t b_off, int64_t b_div, const int32_t *idx, int64_t idx_stride, int64_t k,
+                     __nv_bfloat16 *dst, int64_t ld_dst, int *status, cudaStream_t stream);
+
+// ---- attention helpers --------------------------------------------------------------------------------
+// Row softmax of fp32 logits S [heads, Lq, ld_s] with optional end-aligned causal mask; writes bf16
+// P [heads, Lq, ld_p] (columns Lk .. ld_p zeroed).
+int launch_softmax_rows(const float *S, int64_t ld_s, int64_t heads, int64_t Lq, int64_t Lk, int causal,
+                        __nv_bfloat16 *P, int64_t ld_p, cudaStream_t stream);
+
+}  // namespace rmm

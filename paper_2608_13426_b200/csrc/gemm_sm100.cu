@@ -1,0 +1,565 @@
+// Reduced product Y = scale * A[:, I] B[I, :] (paper Sec. 3.2) on the sm_100a tensor cores.
+//
+// Data path per 128 x BN output tile (persistent blocks, one per SM, static round-robin tiles):
+//   A[:, I]   packed once by pack_cols_kernel into Ap [b, M, ldp] (K-major); TMA 2-D/3-D tile loads
+//             of 128 rows x 64 kept columns into 128-byte-swizzled shared memory.  Columns beyond k
+//             are outside the tensor map and arrive as zeros, so k needs no padding.
+//   B[I, :]   never packed when B's contraction slices (rows) are contiguous: the producer warp reads
+//             the index list and fetches the kept rows straight from B with TMA gather4 (4 arbitrary rows
+//             x 64 columns per instruction), giving an MN-major swizzled operand.
+//             When B is K-contiguous (K^T in attention) it is packed like A and loaded as K-major tiles.
+//   MMA       one elected thread issues tcgen05.mma (bf16 x bf16 -> fp32, M=128, N=BN, K=16 per instruction);
+//             accumulators live in TMEM, double buffered (2 x BN columns) so that the epilogue of one tile
+//             overlaps the main loop of the next.
+//   epilogue  4 warps read TMEM with tcgen05.ld (one accumulator row per thread), scale, round to bf16
+//             (or keep fp32) and store 64 contiguous bytes per thread.
+// Every mbarrier wait is bounded: on expiry the block records RMM_ERR_TIMEOUT in the workspace status
+// word, stops issuing work, lets copies in flight land, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace rmm {
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;           // contraction indices per pipeline stage (128 bytes of bf16)
+constexpr int UMMA_K = 16;
+constexpr int kThreadsTc = 192;  // warp 0 producer, warp 1 MMA + TMEM owner, warps 2-5 epilogue
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+// ----------------------------------------------------------------------------------------------
+// PTX wrappers
+// ----------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false when the block is aborting (this or another thread ran out of time).
+__device__ __forceinline__ bool mbar_wait_lane(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+{
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 127u) == 127u) {
+            if (*abort_flag) return false;
+            unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicExch(status, (int)RMM_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+// Whole-warp form: every lane waits, and the warp takes one common decision.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+{
+    bool ok = mbar_wait_lane(bar, parity, abort_flag, status);
+    return __all_sync(0xffffffffu, ok);
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
+// Four rows (y0..y3) of a 2-D tensor, columns x .. x+box-1, land as four consecutive shared-memory rows.
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap *map, int x, int y0, int y1, int y2, int y3,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive on an mbarrier once every tcgen05 operation issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory operand descriptor (tcgen05 format): 128-byte swizzle, addresses and offsets in 16-byte units.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;  // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;  // swizzle mode: 128 bytes
+    return d;
+}
+
+struct TcArgs {
+    int64_t M, N, k, batch;
+    // MN-major B: first row of batch entry i in the flattened 2-D tensor = ((i + b_batch_off) / b_batch_div) * b_batch_rows
+    int64_t b_batch_rows, b_batch_off, b_batch_div;
+    const int32_t *idx;     // kept rows, one list per batch entry idx_stride apart; NULL = rows 0 .. k-1
+    int64_t idx_stride;
+    void *Y;
+    int64_t y_sb, y_sr;     // element strides of Y (column stride 1)
+    float scale;
+    int tiles_m, tiles_n;
+    int *status;
+};
+
+template <int BN>
+struct SmemLayout {
+    static constexpr int kStages = BN == 256 ? 4 : 6;
+    static constexpr int kABytes = BM * BK * 2;
+    static constexpr int kBBytes = BN * BK * 2;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kBarOffset = kStages * kStageBytes;
+    static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack to align the base to 1024 B
+};
+
+template <int BN, bool B_KMAJOR, bool OUT_BF16>
+__global__ void __launch_bounds__(kThreadsTc, 1)
+reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcArgs a)
+{
+    using L = SmemLayout<BN>;
+    constexpr int kStages = L::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bar_base = base + L::kBarOffset;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+    auto tfull_bar = [&](int i) { return bar_base + 8u * (2 * kStages + i); };
+    auto tempty_bar = [&](int i) { return bar_base + 8u * (2 * kStages + 2 + i); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + L::kBarOffset + 8 * (2 * kStages + 4));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + L::kBarOffset + 8 * (2 * kStages + 4) + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t num_tiles = a.batch * a.tiles_m * a.tiles_n;
+    const int num_kb = (int)((a.k + BK - 1) / BK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(tfull_bar(i), 1);
+            mbar_init(tempty_bar(i), 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), 2 * BN);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- producer
+        uint32_t it = 0;
+        for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+            const int tn = (int)(tile % a.tiles_n);
+            const int tm = (int)((tile / a.tiles_n) % a.tiles_m);
+            const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
+            const int32_t *ix = a.idx != nullptr ? a.idx + b * a.idx_stride : nullptr;
+            const int row_base = (int)(((b + a.b_batch_off) / a.b_batch_div) * a.b_batch_rows);
+            auto kept_row = [&](int64_t j) -> int {
+                if (j >= a.k) j = a.k - 1;  // positions past k repeat the last kept row; A supplies zeros there
+                return ix != nullptr ? __ldg(ix + j) : (int)j;
+            };
+            // kept rows of B this lane fetches in each stage: row group g = lane % 16, i.e. positions 4g .. 4g+3
+            const int g = lane & 15;
+            int rows_next[4];
+            bool ok = true;
+            if constexpr (!B_KMAJOR) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) rows_next[i] = kept_row(4 * g + i);
+            }
+            for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const int s = it % kStages;
+                const uint32_t ph = (it / kStages) & 1u;
+                int rows[4];
+                if constexpr (!B_KMAJOR) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) rows[i] = rows_next[i];
+                    if (kb + 1 < num_kb) {  // prefetch the next stage's indices before blocking on the ring
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) rows_next[i] = kept_row((int64_t)(kb + 1) * BK + 4 * g + i);
+                    }
+                }
+                if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status)) { ok = false; break; }
+                const uint32_t sa = base + s * L::kStageBytes;
+                const uint32_t sb = sa + L::kABytes;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(full_bar(s), L::kStageBytes);
+                    tma_load_3d(sa, &map_a, kb * BK, tm * BM, (int)b, full_bar(s));
+                    if constexpr (B_KMAJOR) tma_load_3d(sb, &map_b, kb * BK, tn * BN, (int)b, full_bar(s));
+                }
+                __syncwarp();
+                if constexpr (!B_KMAJOR) {
+                    // BN/64 column chunks x 16 row groups = BN/4 gathers per stage, BN/128 per lane
+#pragma unroll
+                    for (int c = lane >> 4; c < BN / 64; c += 2) {
+                        const uint32_t dst = sb + c * (BK * 128) + g * 512;
+                        tma_gather4(dst, &map_b, tn * BN + c * 64, row_base + rows[0], row_base + rows[1],
+                                    row_base + rows[2], row_base + rows[3], full_bar(s));
+                    }
+                }
+            }
+            if (!ok) break;
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B K- or MN-major, N = BN, M = 128
+        constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((B_KMAJOR ? 0u : 1u) << 16) |
+                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        uint32_t it = 0, tcount = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+            const uint32_t acc = tcount & 1u, acc_ph = (tcount >> 1) & 1u;
+            if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, a.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * BN;
+            for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const int s = it % kStages;
+                const uint32_t ph = (it / kStages) & 1u;
+                if (!mbar_wait(full_bar(s), ph, abort_flag, a.status)) { ok = false; break; }
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t sa = base + s * L::kStageBytes;
+                    const uint32_t sb = sa + L::kABytes;
+                    const int64_t left = a.k - (int64_t)kb * BK;
+                    const int steps = left >= BK ? BK / UMMA_K : (int)((left + UMMA_K - 1) / UMMA_K);
+                    for (int ks = 0; ks < steps; ++ks) {
+                        // A, and a K-major B: 128-byte rows, 8-row groups 1024 B apart; 16 indices = 32 B along the row
+                        const uint64_t da = smem_desc(sa + ks * 32, 16, 1024);
+                        // MN-major B: 64-column chunks BK*128 B apart, 8-index groups 1024 B apart; 16 indices = 2048 B
+                        const uint64_t db = B_KMAJOR ? smem_desc(sb + ks * 32, 16, 1024)
+                                                     : smem_desc(sb + ks * 2048, BK * 128, 1024);
+                        umma_bf16(d_tmem, da, db, idesc, (kb | ks) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(s));
+                }
+                __syncwarp();
+            }
+            if (ok && lane == 0) umma_commit(tfull_bar(acc));
+            __syncwarp();
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (warps 2..5)
+        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        uint32_t tcount = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+            const int tn = (int)(tile % a.tiles_n);
+            const int tm = (int)((tile / a.tiles_n) % a.tiles_m);
+            const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
+            const uint32_t acc = tcount & 1u, acc_ph = (tcount >> 1) & 1u;
+            if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, a.status)) { ok = false; break; }
+            tc_fence_after();
+            const int64_t m = (int64_t)tm * BM + q * 32 + lane;
+            const int64_t n0 = (int64_t)tn * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c * 32, r);
+                const int64_t n = n0 + c * 32;
+                if (m < a.M && n < a.N) {
+                    if constexpr (OUT_BF16) {
+                        __nv_bfloat16 *y = reinterpret_cast<__nv_bfloat16 *>(a.Y) + b * a.y_sb + m * a.y_sr + n;
+                        if (n + 32 <= a.N) {
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) {
+                                uint32_t w[4];
+#pragma unroll
+                                for (int p = 0; p < 4; ++p) {
+                                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * v + 2 * p]) * a.scale,
+                                                                             __uint_as_float(r[8 * v + 2 * p + 1]) * a.scale);
+                                    w[p] = *reinterpret_cast<uint32_t *>(&h);
+                                }
+                                reinterpret_cast<uint4 *>(y)[v] = make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                        } else {
+                            for (int e = 0; e < 32 && n + e < a.N; ++e)
+                                y[e] = __float2bfloat16_rn(__uint_as_float(r[e]) * a.scale);
+                        }
+                    } else {
+                        float *y = reinterpret_cast<float *>(a.Y) + b * a.y_sb + m * a.y_sr + n;
+                        if (n + 32 <= a.N) {
+#pragma unroll
+                            for (int v = 0; v < 8; ++v)
+                                reinterpret_cast<float4 *>(y)[v] =
+                                    make_float4(__uint_as_float(r[4 * v]) * a.scale, __uint_as_float(r[4 * v + 1]) * a.scale,
+                                                __uint_as_float(r[4 * v + 2]) * a.scale, __uint_as_float(r[4 * v + 3]) * a.scale);
+                        } else {
+                            for (int e = 0; e < 32 && n + e < a.N; ++e) y[e] = __uint_as_float(r[e]) * a.scale;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    __syncthreads();
+    if (*abort_flag) {
+        // give copies and MMAs still in flight time to land before shared memory and TMEM are released
+        unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    tc_fence_after();
+    if (warp == 1) tmem_dealloc(tmem_base, 2 * BN);
+}
+
+// ----------------------------------------------------------------------------------------------
+// host side
+// ----------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 tensor map with 128-byte swizzle; dims / strides innermost first, strides in bytes for dims 1..rank-1
+int make_map(CUtensorMap *map, void *ptr, int rank, const uint64_t *dims, const uint64_t *strides_bytes,
+             const uint32_t *box)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return fail(RMM_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    cuuint64_t d[5], st[4];
+    cuuint32_t bx[5], es[5];
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) st[i] = strides_bytes[i];
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, ptr, d, st, bx, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(RMM_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return RMM_OK;
+}
+
+int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    }
+    return n;
+}
+
+template <int BN, bool B_KMAJOR, bool OUT_BF16>
+int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const TcArgs &a, cudaStream_t stream)
+{
+    auto kern = reduced_gemm_tc_kernel<BN, B_KMAJOR, OUT_BF16>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout<BN>::kTotal);
+        if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+        configured = true;
+    }
+    int64_t tiles = a.batch * a.tiles_m * a.tiles_n;
+    int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+    kern<<<grid, kThreadsTc, SmemLayout<BN>::kTotal, stream>>>(ma, mb, a);
+    return check_launch("reduced_gemm_tc_kernel");
+}
+
+}  // namespace
+
+bool tc_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y, TcPlan *plan)
+{
+    if (A->dtype != RMM_BF16 || B->dtype != RMM_BF16) return false;
+    const int64_t M = A->rows, K = A->cols, N = B->cols, batch = A->batch;
+    auto al16 = [](const void *p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; };
+    if (A->stride_col != 1) return false;
+    if (Y->stride_col != 1 || !al16(Y->ptr)) return false;
+    const int64_t yq = Y->dtype == RMM_BF16 ? 8 : 4;
+    if (Y->stride_row % yq != 0 || Y->stride_batch % yq != 0) return false;
+    if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX || batch > INT32_MAX) return false;
+    int b_kmajor;
+    if (B->stride_col == 1 && B->rows > 0) {
+        // rows of B contiguous: gathered by TMA straight from B, which must flatten to one 2-D tensor
+        b_kmajor = 0;
+        if (!al16(B->ptr) || B->stride_row % 8 != 0 || B->stride_row < N) return false;
+        if (B->stride_batch != 0 && B->stride_batch != K * B->stride_row) return false;
+        if ((B->stride_batch == 0 ? K : batch * K) > INT32_MAX) return false;
+    } else if (B->stride_row == 1) {
+        b_kmajor = 1;  // K-contiguous: packed like A
+    } else {
+        return false;
+    }
+    if (plan != nullptr) {
+        plan->b_kmajor = b_kmajor;
+        plan->ldp = (k + 7) / 8 * 8;
+        size_t off = RMM_WS_HEADER_BYTES;
+        plan->off_ap = off;
+        off += align_up((size_t)batch * M * plan->ldp * 2, 256);
+        plan->off_bp = off;
+        if (b_kmajor) off += align_up((size_t)batch * N * plan->ldp * 2, 256);
+        plan->total_bytes = off;
+    }
+    return true;
+}
+
+int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
+{
+    CUtensorMap ma, mb;
+    int rc;
+    {
+        uint64_t dims[3] = {(uint64_t)p.k, (uint64_t)p.M, (uint64_t)p.batch};
+        uint64_t st[2] = {(uint64_t)p.a_ld * 2, (uint64_t)p.a_sb * 2};
+        uint32_t box[3] = {BK, BM, 1};
+        rc = make_map(&ma, const_cast<__nv_bfloat16 *>(p.a), 3, dims, st, box);
+        if (rc != RMM_OK) return rc;
+    }
+    const int BN = p.N <= 128 ? 128 : 256;
+    TcArgs a;
+    a.M = p.M; a.N = p.N; a.k = p.k; a.batch = p.batch;
+    a.idx = p.idx; a.idx_stride = p.idx_stride;
+    a.b_batch_rows = p.b_batch_rows; a.b_batch_off = p.b_batch_off; a.b_batch_div = p.b_batch_div > 0 ? p.b_batch_div : 1;
+    a.Y = p.y; a.y_sb = p.y_sb; a.y_sr = p.y_sr;
+    a.scale = p.scale;
+    a.tiles_m = (int)ceil_div(p.M, BM);
+    a.tiles_n = (int)ceil_div(p.N, BN);
+    a.status = p.status;
+    if (p.b_kmajor) {
+        uint64_t dims[3] = {(uint64_t)p.k, (uint64_t)p.N, (uint64_t)p.batch};
+        uint64_t st[2] = {(uint64_t)p.b_ld * 2, (uint64_t)p.b_sb * 2};
+        uint32_t box[3] = {BK, (uint32_t)BN, 1};
+        rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 3, dims, st, box);
+    } else {
+        uint64_t dims[2] = {(uint64_t)p.N, (uint64_t)p.b_rows_total};
+        uint64_t st[1] = {(uint64_t)p.b_ld * 2};
+        uint32_t box[2] = {64, 1};
+        rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 2, dims, st, box);
+    }
+    if (rc != RMM_OK) return rc;
+    const bool out_bf16 = p.y_bf16 != 0;
+    if (BN == 256) {
+        if (p.b_kmajor) return out_bf16 ? launch_variant<256, true, true>(ma, mb, a, stream) : launch_variant<256, true, false>(ma, mb, a, stream);
+        return out_bf16 ? launch_variant<256, false, true>(ma, mb, a, stream) : launch_variant<256, false, false>(ma, mb, a, stream);
+    }
+    if (p.b_kmajor) return out_bf16 ? launch_variant<128, true, true>(ma, mb, a, stream) : launch_variant<128, true, false>(ma, mb, a, stream);
+    return out_bf16 ? launch_variant<128, false, true>(ma, mb, a, stream) : launch_variant<128, false, false>(ma, mb, a, stream);
+}
+
+int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
+                   const rmm_mat_t *Y, const TcPlan &plan, void *ws, cudaStream_t stream)
+{
+    char *w = static_cast<char *>(ws);
+    int *status = &reinterpret_cast<WsHeader *>(w)->status;
+    const int64_t M = A->rows, K = A->cols, N = B->cols, batch = A->batch;
+    __nv_bfloat16 *Ap = reinterpret_cast<__nv_bfloat16 *>(w + plan.off_ap);
+    int rc = launch_pack_cols(static_cast<const __nv_bfloat16 *>(A->ptr), batch, M, K, A->stride_batch, A->stride_row, 0, 1,
+                              idx, k, k, Ap, plan.ldp, status, stream);
+    if (rc != RMM_OK) return rc;
+    TcProblem p = {};
+    p.batch = batch; p.M = M; p.N = N; p.k = k;
+    p.a = Ap; p.a_ld = plan.ldp; p.a_sb = M * plan.ldp;
+    p.b_kmajor = plan.b_kmajor;
+    p.y = Y->ptr; p.y_bf16 = Y->dtype == RMM_BF16; p.y_sb = Y->stride_batch; p.y_sr = Y->stride_row;
+    p.scale = scale; p.status = status;
+    if (plan.b_kmajor) {
+        // B is K-contiguous ([N, K] in memory): pack B[idx, :]^T into Bp [batch, N, ldp]; a shared B
+        // (stride_batch 0) is packed once per index set
+        __nv_bfloat16 *Bp = reinterpret_cast<__nv_bfloat16 *>(w + plan.off_bp);
+        rc = launch_pack_cols(static_cast<const __nv_bfloat16 *>(B->ptr), batch, N, K, B->stride_batch, B->stride_col, 0, 1,
+                              idx, k, k, Bp, plan.ldp, status, stream);
+        if (rc != RMM_OK) return rc;
+        p.b = Bp; p.b_ld = plan.ldp; p.b_sb = N * plan.ldp;
+    } else {
+        const int64_t b_batches = B->stride_batch == 0 ? 1 : batch;
+        p.b = static_cast<const __nv_bfloat16 *>(B->ptr); p.b_ld = B->stride_row;
+        p.b_rows_total = b_batches * K;
+        p.idx = idx; p.idx_stride = k;
+        p.b_batch_rows = B->stride_batch == 0 ? 0 : K; p.b_batch_off = 0; p.b_batch_div = 1;
+    }
+    return launch_gemm_tc_problem(p, stream);
+}
+
+}  // namespace rmm

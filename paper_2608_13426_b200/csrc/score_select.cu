@@ -1,0 +1,435 @@
+// Importance scores and top-k index selection (paper Sec. 3.2: s_j = ||A[:, j]||_2,
+// I = TopK({s_j}, ceil(rho d))), as one streaming pass over A whose last-arriving thread block
+// selects the index set.
+//
+// Score pass: HBM-bound.  Each thread owns VEC adjacent columns (one 16-byte load per row) and a
+// strided subset of the block's rows; squares of bf16 values are exact in fp32, sums run in fp32
+// chains of at most 16 terms that are flushed into fp64, row lanes are combined in fp64 through
+// shared memory, row splits through an fp64 partial array combined in split order by the last
+// block to arrive (self-resetting atomicInc counter).  Results are therefore run-to-run identical.
+//
+// Select: radix select on the order-preserving integer image of the fp32 keys (4 passes of 8 bits,
+// warp-aggregated shared-memory histograms), then one ordered compaction pass that emits the kept
+// indices ascending; among keys equal to the threshold the lowest indices are kept.
+#include "common.cuh"
+
+namespace rmm {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kUnroll = 4;       // rows in flight per thread
+constexpr int kFlushEvery = 4;   // loop trips between fp32 -> fp64 flushes (kUnroll * kFlushEvery = 16 terms)
+
+struct SelectSmem {
+    unsigned hist[256];
+    unsigned long long warp_tot[32];
+    unsigned long long carry;
+    unsigned long long round_total;
+    unsigned bin;
+    unsigned remaining;
+    double red[64];
+};
+
+__device__ __forceinline__ unsigned key_image(float f)
+{
+    unsigned u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // total order: larger float <=> larger image
+}
+
+// Block-wide top-k of keys[0..K): writes idx[0..k) ascending, optional retained fraction.
+// Every thread of the block must call it; keys are read through L2 (they may have just been
+// written by other blocks).
+__device__ void block_select(const float *keys, int K, int k, int32_t *idx, float *retained, SelectSmem &sm)
+{
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    unsigned prefix = 0, mask = 0, remaining = (unsigned)k;
+
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = tid; i < 256; i += nthr) sm.hist[i] = 0;
+        __syncthreads();
+        for (int j0 = 0; j0 < K; j0 += nthr) {
+            int j = j0 + tid;
+            bool live = false;
+            unsigned bin = 0;
+            if (j < K) {
+                unsigned u = key_image(__ldcg(keys + j));
+                live = (u & mask) == prefix;
+                bin = (u >> shift) & 255u;
+            }
+            // one shared-memory atomic per distinct bin per warp
+            unsigned act = __ballot_sync(0xffffffffu, live);
+            if (live) {
+                unsigned peers = __match_any_sync(act, bin);
+                if (lane == __ffs(peers) - 1) atomicAdd(&sm.hist[bin], (unsigned)__popc(peers));
+            }
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane l owns bins 255-8l .. 248-8l (descending); find where the count from the top crosses `remaining`
+            unsigned mine = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) mine += sm.hist[255 - 8 * lane - i];
+            unsigned incl = mine;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                unsigned v = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += v;
+            }
+            unsigned excl = incl - mine;
+            if (excl < remaining && remaining <= incl) {
+                unsigned above = excl;
+                for (int i = 0; i < 8; ++i) {
+                    unsigned h = sm.hist[255 - 8 * lane - i];
+                    if (remaining <= above + h) {
+                        sm.bin = 255 - 8 * lane - i;
+                        sm.remaining = remaining - above;
+                        break;
+                    }
+                    above += h;
+                }
+            }
+        }
+        __syncthreads();
+        prefix |= sm.bin << shift;
+        mask |= 255u << shift;
+        remaining = sm.remaining;
+        __syncthreads();
+    }
+    const unsigned tau = prefix;          // image of the k-th largest key
+    const unsigned need_eq = remaining;   // how many keys equal to tau are kept (lowest indices first)
+
+    // ordered compaction, 4 consecutive indices per thread per round
+    if (tid == 0) sm.carry = 0ull;
+    __syncthreads();
+    double sum_kept = 0.0, sum_all = 0.0;
+    const int per_round = nthr * 4;
+    for (int base = 0; base < K; base += per_round) {
+        int j = base + tid * 4;
+        unsigned u[4];
+        float f[4];
+        unsigned long long mine = 0ull;  // (count > tau) << 32 | (count == tau)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (j + i < K) {
+                f[i] = __ldcg(keys + j + i);
+                u[i] = key_image(f[i]);
+                mine += (u[i] > tau) ? (1ull << 32) : 0ull;
+                mine += (u[i] == tau) ? 1ull : 0ull;
+            } else {
+                f[i] = 0.f;
+                u[i] = 0u;
+            }
+        }
+        unsigned long long incl = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            unsigned long long v = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += v;
+        }
+        if (lane == 31) sm.warp_tot[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            unsigned long long w = (lane < (nthr >> 5)) ? sm.warp_tot[lane] : 0ull;
+            unsigned long long wi = w;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                unsigned long long v = __shfl_up_sync(0xffffffffu, wi, d);
+                if (lane >= d) wi += v;
+            }
+            sm.warp_tot[lane] = wi - w;  // exclusive prefix of warp totals
+            if (lane == 31) sm.round_total = wi;
+        }
+        __syncthreads();
+        unsigned long long before = sm.carry + sm.warp_tot[warp] + (incl - mine);
+        unsigned gt_before = (unsigned)(before >> 32), eq_before = (unsigned)(before & 0xffffffffu);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (j + i < K) {
+                sum_all += (double)f[i];
+                bool gt = u[i] > tau, eq = u[i] == tau;
+                if (gt || (eq && eq_before < need_eq)) {
+                    unsigned pos = gt_before + (eq_before < need_eq ? eq_before : need_eq);
+                    idx[pos] = j + i;
+                    sum_kept += (double)f[i];
+                }
+                gt_before += gt;
+                eq_before += eq;
+            }
+        }
+        __syncthreads();
+        if (tid == 0) sm.carry += sm.round_total;
+        __syncthreads();
+    }
+
+    if (retained != nullptr) {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            sum_kept += __shfl_down_sync(0xffffffffu, sum_kept, d);
+            sum_all += __shfl_down_sync(0xffffffffu, sum_all, d);
+        }
+        if (lane == 0) {
+            sm.red[warp] = sum_kept;
+            sm.red[32 + warp] = sum_all;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            double a = 0.0, b = 0.0;
+            for (int w = 0; w < (nthr >> 5); ++w) {
+                a += sm.red[w];
+                b += sm.red[32 + w];
+            }
+            *retained = (b > 0.0) ? (float)(a / b) : 1.0f;
+        }
+    }
+    __syncthreads();
+}
+
+struct ScoreArgs {
+    const void *A;
+    int64_t s_batch, s_red, s_n;  // element strides: batch, reduced axis (rows), scored axis (columns)
+    int64_t n, m, rows_per_split;
+    int row_splits, col_blocks, tx, ty;
+    double *partials;    // [batch, row_splits, n]   (unused when row_splits == 1)
+    unsigned *counters;  // [batch, col_blocks + 1]
+    float *energy;       // [batch, n]  always written (caller's array or workspace)
+    float *scores;       // [batch, n]  or null
+    int do_select;
+    int k;
+    int32_t *idx;        // [batch, k]
+    float *retained;     // [batch] or null
+};
+
+template <int VEC, bool BF16>
+__device__ __forceinline__ void load_vec(const void *A, int64_t off, int64_t s_n, float (&v)[VEC])
+{
+    if constexpr (BF16 && VEC == 8) {
+        uint4 q = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(A) + off));
+        unsigned w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    } else if constexpr (!BF16 && VEC == 4) {
+        float4 q = __ldg(reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(A) + off));
+        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+    } else {
+        static_assert(VEC == 1 || VEC == 4 || VEC == 8, "vector width");
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            if constexpr (BF16)
+                v[i] = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(A)[off + i * s_n]);
+            else
+                v[i] = reinterpret_cast<const float *>(A)[off + i * s_n];
+        }
+    }
+}
+
+template <int VEC, bool BF16>
+__global__ void __launch_bounds__(kThreads) score_select_kernel(ScoreArgs a)
+{
+    __shared__ double s_part[kThreads * VEC];
+    __shared__ SelectSmem s_sel;
+    __shared__ int s_flag;
+
+    const int tid = threadIdx.x;
+    const int tx = tid % a.tx, ty = tid / a.tx;
+    const int64_t b = blockIdx.z;
+    const int split = blockIdx.y;
+    const int width = a.tx * VEC;  // columns per block
+    const int64_t col0 = (int64_t)blockIdx.x * width;
+    const int64_t col = col0 + (int64_t)tx * VEC;
+    const int64_t r_begin = (int64_t)split * a.rows_per_split;
+    const int64_t r_end = min(a.m, r_begin + a.rows_per_split);
+
+    double dacc[VEC];
+    float facc[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) { dacc[e] = 0.0; facc[e] = 0.f; }
+
+    if (col < a.n) {
+        const int64_t base = b * a.s_batch + col * a.s_n;
+        int trips = 0;
+        for (int64_t r = r_begin + ty; r < r_end; r += (int64_t)a.ty * kUnroll) {
+            float v[kUnroll][VEC];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                int64_t rr = r + (int64_t)u * a.ty;
+                if (rr < r_end) {
+                    load_vec<VEC, BF16>(a.A, base + rr * a.s_red, a.s_n, v[u]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) v[u][e] = 0.f;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) facc[e] = fmaf(v[u][e], v[u][e], facc[e]);
+            if (++trips == kFlushEvery) {
+                trips = 0;
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) { dacc[e] += (double)facc[e]; facc[e] = 0.f; }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) dacc[e] += (double)facc[e];
+    }
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) s_part[ty * width + tx * VEC + e] = dacc[e];
+    __syncthreads();
+
+    // combine the row lanes in lane order: thread t < width owns column col0 + t
+    double colsum = 0.0;
+    const int64_t mycol = col0 + tid;
+    const bool owner = tid < width && mycol < a.n;
+    if (owner)
+        for (int y = 0; y < a.ty; ++y) colsum += s_part[y * width + tid];
+
+    bool finalize = true;
+    if (a.row_splits > 1) {
+        if (owner) a.partials[(b * a.row_splits + split) * a.n + mycol] = colsum;
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            unsigned old = atomicInc(&a.counters[b * (a.col_blocks + 1) + blockIdx.x], (unsigned)a.row_splits - 1u);
+            s_flag = (old == (unsigned)a.row_splits - 1u);
+        }
+        __syncthreads();
+        finalize = s_flag != 0;
+        if (finalize) {
+            __threadfence();
+            if (owner) {
+                colsum = 0.0;
+                for (int s = 0; s < a.row_splits; ++s) colsum += __ldcg(&a.partials[(b * a.row_splits + s) * a.n + mycol]);
+            }
+        }
+    }
+    if (!finalize) return;
+
+    if (owner) {
+        a.energy[b * a.n + mycol] = (float)colsum;
+        if (a.scores != nullptr) a.scores[b * a.n + mycol] = (float)sqrt(colsum);
+    }
+    if (!a.do_select) return;
+
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        unsigned old = atomicInc(&a.counters[b * (a.col_blocks + 1) + a.col_blocks], (unsigned)a.col_blocks - 1u);
+        s_flag = (old == (unsigned)a.col_blocks - 1u);
+    }
+    __syncthreads();
+    if (!s_flag) return;
+    __threadfence();
+    block_select(a.energy + b * a.n, (int)a.n, a.k, a.idx + b * (int64_t)a.k,
+                 a.retained ? a.retained + b : nullptr, s_sel);
+}
+
+__global__ void __launch_bounds__(1024) select_kernel(const float *keys, int K, int k, int32_t *idx, float *retained)
+{
+    __shared__ SelectSmem s_sel;
+    const int64_t b = blockIdx.x;
+    block_select(keys + b * K, K, k, idx + b * (int64_t)k, retained ? retained + b : nullptr, s_sel);
+}
+
+}  // namespace
+
+int plan_score(const rmm_mat_t *A, int axis, ScorePlan *p)
+{
+    if (A == nullptr || A->ptr == nullptr) return fail(RMM_ERR_INVALID_ARG, "score: null matrix");
+    if (A->batch < 1 || A->rows < 1 || A->cols < 1) return fail(RMM_ERR_INVALID_ARG, "score: non-positive dimension");
+    if (axis != 0 && axis != 1) return fail(RMM_ERR_INVALID_ARG, "score: axis must be 0 or 1");
+    if (A->dtype != RMM_BF16 && A->dtype != RMM_F32) return fail(RMM_ERR_UNSUPPORTED, "score: dtype");
+    if (A->stride_batch < 0 || A->stride_row < 0 || A->stride_col < 0)
+        return fail(RMM_ERR_UNSUPPORTED, "score: negative stride");
+    p->n = axis == 1 ? A->cols : A->rows;
+    p->m = axis == 1 ? A->rows : A->cols;
+    p->s_n = axis == 1 ? A->stride_col : A->stride_row;
+    p->s_red = axis == 1 ? A->stride_row : A->stride_col;
+    p->s_batch = A->stride_batch;
+    if (p->n > (int64_t)1 << 30 || p->m > (int64_t)1 << 40 || A->batch > 65535)
+        return fail(RMM_ERR_UNSUPPORTED, "score: dimension too large (n <= 2^30, batch <= 65535)");
+
+    const size_t es = dtype_size(A->dtype);
+    const int full = A->dtype == RMM_BF16 ? 8 : 4;
+    const bool vec_ok = p->s_n == 1 && p->n % full == 0 && (reinterpret_cast<uintptr_t>(A->ptr) % 16 == 0) &&
+                        (p->s_red * es) % 16 == 0 && (p->s_batch * es) % 16 == 0;
+    p->vec = vec_ok ? full : 1;
+    int64_t groups = ceil_div(p->n, p->vec);
+    int tx = 32;
+    while (tx > 1 && tx / 2 >= groups) tx /= 2;
+    p->tx = tx;
+    p->ty = kThreads / tx;
+    p->col_blocks = (int)ceil_div(p->n, (int64_t)tx * p->vec);
+
+    // enough blocks to fill the machine several times over, but at least 4 loop trips of rows each
+    const int64_t want_blocks = 148 * 8;
+    int64_t splits = ceil_div(want_blocks, (int64_t)p->col_blocks * A->batch);
+    int64_t min_rows = (int64_t)p->ty * kUnroll * 2;
+    int64_t max_splits = p->m / min_rows;
+    if (max_splits < 1) max_splits = 1;
+    if (splits > max_splits) splits = max_splits;
+    if (splits > 64) splits = 64;
+    if (splits < 1) splits = 1;
+    p->rows_per_split = ceil_div(p->m, splits);
+    p->row_splits = (int)ceil_div(p->m, p->rows_per_split);
+
+    int64_t n_counters = A->batch * (p->col_blocks + 1);
+    p->counters_in_header = n_counters <= kHeaderCounters;
+    size_t off = RMM_WS_HEADER_BYTES;
+    p->off_counters = off;
+    if (!p->counters_in_header) off += align_up((size_t)n_counters * 4, 256);
+    p->off_partials = off;
+    if (p->row_splits > 1) off += align_up((size_t)A->batch * p->row_splits * p->n * 8, 256);
+    p->off_energy = off;
+    off += align_up((size_t)A->batch * p->n * 4, 256);
+    p->total_bytes = off;
+    return RMM_OK;
+}
+
+int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, int64_t k, int32_t *idx,
+                        float *scores, float *energy, float *retained, void *ws, cudaStream_t stream)
+{
+    char *w = static_cast<char *>(ws);
+    WsHeader *hdr = reinterpret_cast<WsHeader *>(w);
+    ScoreArgs a;
+    a.A = A->ptr;
+    a.s_batch = p.s_batch; a.s_red = p.s_red; a.s_n = p.s_n;
+    a.n = p.n; a.m = p.m; a.rows_per_split = p.rows_per_split;
+    a.row_splits = p.row_splits; a.col_blocks = p.col_blocks; a.tx = p.tx; a.ty = p.ty;
+    a.partials = reinterpret_cast<double *>(w + p.off_partials);
+    if (p.counters_in_header) {
+        a.counters = hdr->counters;
+    } else {
+        a.counters = reinterpret_cast<unsigned *>(w + p.off_counters);
+        cudaError_t e = cudaMemsetAsync(a.counters, 0, (size_t)A->batch * (p.col_blocks + 1) * 4, stream);
+        if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "score: memset: %s", cudaGetErrorString(e));
+    }
+    a.energy = energy ? energy : reinterpret_cast<float *>(w + p.off_energy);
+    a.scores = scores;
+    a.do_select = do_select ? 1 : 0;
+    a.k = (int)k;
+    a.idx = idx;
+    a.retained = retained;
+
+    dim3 grid((unsigned)p.col_blocks, (unsigned)p.row_splits, (unsigned)A->batch);
+    const bool bf16 = A->dtype == RMM_BF16;
+    if (bf16 && p.vec == 8) score_select_kernel<8, true><<<grid, kThreads, 0, stream>>>(a);
+    else if (bf16) score_select_kernel<1, true><<<grid, kThreads, 0, stream>>>(a);
+    else if (p.vec == 4) score_select_kernel<4, false><<<grid, kThreads, 0, stream>>>(a);
+    else score_select_kernel<1, false><<<grid, kThreads, 0, stream>>>(a);
+    return check_launch("score_select_kernel");
+}
+
+int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_t *idx, float *retained, void *ws,
+                  cudaStream_t stream)
+{
+    (void)ws;
+    int threads = K >= 4096 ? 1024 : (K >= 1024 ? 512 : 256);
+    select_kernel<<<(unsigned)batch, threads, 0, stream>>>(keys, (int)K, (int)k, idx, retained);
+    return check_launch("select_kernel");
+}
+
+}  // namespace rmm

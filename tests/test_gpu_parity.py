@@ -1,0 +1,356 @@
+"""Parity of the CUDA path against the CPU oracle, element by element, through the C ABI (GPU only).
+
+Bars (from the benchmark spec of this library):
+  - index sets: bit-exact outside the tie band |score - threshold| <= 1e-6 * max score;
+  - products: relative Frobenius error <= 1e-2 (bf16 operands) / 1e-5 (fp32 operands) against the
+    oracle evaluated on the GPU's own index set.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_13426_b200 as rmm
+from paper_2608_13426_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 1e-2
+TOL_F32 = 1e-5
+TIE_BAND = 1e-6
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _device():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    torch.cuda.set_device(0)
+    yield
+    assert rmm.rmm_status_read() == 0, "a kernel left an error in the workspace status word"
+
+
+def dev(t):
+    return t.cuda()
+
+
+def rel_fro(got, want):
+    got = np.asarray(got, dtype=np.float64)
+    return float(np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-300))
+
+
+def check_index_set(idx_gpu, energy64, k):
+    """The GPU set must equal the oracle set outside the tie band around the threshold score, have k
+    distinct ascending members, and every difference must lie inside the band."""
+    import oracle
+
+    idx_gpu = np.asarray(idx_gpu, dtype=np.int64)
+    assert idx_gpu.shape == (k,)
+    assert np.all(np.diff(idx_gpu) > 0), "indices must be strictly ascending"
+    assert idx_gpu.min() >= 0 and idx_gpu.max() < len(energy64)
+    want, _ = oracle.select(energy64, k)
+    s = np.sqrt(energy64)
+    tau = np.sort(s)[::-1][k - 1]
+    band = TIE_BAND * s.max()
+    diff = np.setxor1d(idx_gpu, want)
+    assert np.all(np.abs(s[diff] - tau) <= band), f"{len(diff)} indices differ outside the tie band"
+    return len(diff)
+
+
+# ------------------------------------------------------------------------------------------------
+# score
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("M,K", [(1, 1), (2, 7), (63, 8), (64, 9), (65, 15), (127, 16), (128, 17), (129, 63), (300, 64),
+                                 (64, 512), (257, 1000), (2048, 4096), (33, 129)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_score_matches_oracle(oracle, M, K, dtype):
+    A = synth.heavy_tailed_activations(M, K, seed=M * 7 + K, dtype=dtype)
+    e64, s64 = oracle.score(A)
+    s, e = rmm.rmm_score(dev(A))
+    assert np.allclose(e.cpu().numpy(), e64, rtol=3e-7, atol=0)
+    assert np.allclose(s.cpu().numpy(), s64, rtol=3e-7, atol=0)
+
+
+def test_score_batched_strided_and_rows(oracle):
+    A = synth.gaussian((3, 70, 96), 1.0, seed=5)
+    Ad = dev(A)
+    s, e = rmm.rmm_score(Ad)
+    for b in range(3):
+        e64, _ = oracle.score(A[b])
+        assert np.allclose(e[b].cpu().numpy(), e64, rtol=3e-7)
+    view = Ad[:, 3:50, 8:72]                     # non-contiguous rows and batch, still 16-byte aligned columns
+    s2, e2 = rmm.rmm_score(view)
+    for b in range(3):
+        e64, _ = oracle.score(A[b, 3:50, 8:72])
+        assert np.allclose(e2[b].cpu().numpy(), e64, rtol=3e-7)
+    odd = Ad[:, :, 1:66]                         # misaligned start: scalar path
+    _, e3 = rmm.rmm_score(odd)
+    e64, _ = oracle.score(A[1, :, 1:66])
+    assert np.allclose(e3[1].cpu().numpy(), e64, rtol=3e-7)
+    # axis 0 scores rows
+    _, e4 = rmm.rmm_score(Ad[0], axis=0)
+    e64, _ = oracle.score(A[0].T)
+    assert np.allclose(e4.cpu().numpy(), e64, rtol=3e-7)
+
+
+def test_score_is_deterministic():
+    A = dev(synth.heavy_tailed_activations(1024, 2048, seed=1))
+    _, e1 = rmm.rmm_score(A)
+    _, e2 = rmm.rmm_score(A)
+    assert torch.equal(e1, e2)
+
+
+# ------------------------------------------------------------------------------------------------
+# select
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("K", [1, 2, 7, 31, 32, 33, 255, 256, 1000, 1024, 4097, 8192, 28672, 32768])
+@pytest.mark.parametrize("rho", [0.25, 0.5, 0.75, 1.0])
+def test_select_matches_oracle_bit_exact(oracle, K, rho):
+    g = torch.Generator().manual_seed(K)
+    keys = (torch.randn(K, generator=g).abs() * 50 + 2000).float()      # narrow range: shared exponent bits
+    k = rmm.rmm_keep_count(rho, K)
+    idx, ret = rmm.rmm_select(dev(keys), rho=rho, want_retained=True)
+    want, kept = oracle.select(keys.double().numpy(), k)
+    assert np.array_equal(idx.cpu().numpy(), want)
+    assert float(ret[0]) == pytest.approx(kept / float(keys.double().sum()), rel=1e-6)
+
+
+def test_select_ties_and_extremes(oracle):
+    keys = torch.tensor([1.0, 5.0, 5.0, 5.0, 0.5, 5.0, 9.0], dtype=torch.float32)
+    assert rmm.rmm_select(dev(keys), k=3).cpu().tolist() == [1, 2, 6]
+    assert rmm.rmm_select(dev(torch.full((1000,), 2.5)), k=333).cpu().tolist() == list(range(333))
+    assert rmm.rmm_select(dev(torch.zeros(77)), k=5).cpu().tolist() == [0, 1, 2, 3, 4]
+    keys = torch.zeros(5000)
+    keys[[4999, 17, 2500]] = torch.tensor([3.0, 1e30, 7.0])
+    assert rmm.rmm_select(dev(keys), k=3).cpu().tolist() == [17, 2500, 4999]
+    assert rmm.rmm_select(dev(keys), k=5).cpu().tolist() == [0, 1, 17, 2500, 4999]
+    # k = 1 / K, k = K
+    g = torch.Generator().manual_seed(3)
+    keys = torch.rand(513, generator=g)
+    assert rmm.rmm_select(dev(keys), k=1).cpu().tolist() == [int(keys.argmax())]
+    assert rmm.rmm_select(dev(keys), k=513).cpu().tolist() == list(range(513))
+    # batched: one set per row
+    kb = torch.rand(5, 300, generator=g)
+    idx = rmm.rmm_select(dev(kb), rho=0.3).cpu().numpy()
+    for b in range(5):
+        want, _ = oracle.select(kb[b].double().numpy(), 90)
+        assert np.array_equal(idx[b], want)
+
+
+# ------------------------------------------------------------------------------------------------
+# fused score + select
+# ------------------------------------------------------------------------------------------------
+def test_outlier_product_config_whole_path(oracle):
+    """Smallest benchmark configuration: A 64x512 with 8 outlier channels x20, B 512x256, rho = 0.5, seed 0."""
+    A, B, cols = synth.outlier_product(seed=0)
+    e64, _ = oracle.score(A)
+    idx, s, e, ret = rmm.rmm_score_select(dev(A), rho=0.5, want_scores=True, want_energy=True, want_retained=True)
+    assert check_index_set(idx.cpu().numpy(), e64, 256) <= 1
+    assert set(cols.tolist()) <= set(idx.cpu().tolist())
+    want_idx, kept = oracle.select(e64, 256)
+    assert float(ret[0]) == pytest.approx(kept / e64.sum(), rel=1e-5)
+    Y = rmm.rmm_reduced_gemm(dev(A), dev(B), idx)
+    want = oracle.reduced_gemm(A, B, idx.cpu().numpy())
+    assert rel_fro(Y.float().cpu().numpy(), want) <= TOL_BF16
+    # run to run bitwise identical
+    Y2, idx2 = rmm.rmm(dev(A), dev(B), 0.5)
+    assert torch.equal(idx2, idx) and torch.equal(Y2, Y)
+
+
+@pytest.mark.parametrize("M,K,rho", [(2048, 8192, 0.25), (2048, 8192, 0.5), (2048, 8192, 0.75), (2048, 8192, 1.0),
+                                     (300, 1000, 0.5), (4096, 28672, 0.5), (17, 40, 0.3)])
+def test_score_select_sets(oracle, M, K, rho):
+    A = synth.heavy_tailed_activations(M, K, seed=0)
+    e64, _ = oracle.score(A)
+    k = oracle.keep_count(rho, K)
+    idx, _, _, _ = rmm.rmm_score_select(dev(A), rho=rho)
+    n_diff = check_index_set(idx.cpu().numpy(), e64, k)
+    assert n_diff <= 40
+
+
+def test_duplicate_columns_keep_the_lower_index(oracle):
+    A = synth.gaussian((256, 64), 1.0, seed=9).clone()
+    e64, _ = oracle.score(A)
+    order = np.argsort(-e64, kind="stable")
+    k = 20
+    a, b = int(order[k - 1]), int(order[k])
+    lo, hi = min(a, b), max(a, b)
+    A[:, hi] = A[:, lo]
+    idx, _, _, _ = rmm.rmm_score_select(dev(A), k=k)
+    got = idx.cpu().tolist()
+    assert lo in got and hi not in got
+    e2, _ = oracle.score(A)
+    assert np.array_equal(got, oracle.select(e2, k)[0])
+    # every column identical: the first k indices
+    A[:] = A[:, :1]
+    idx, _, _, _ = rmm.rmm_score_select(dev(A), k=k)
+    assert idx.cpu().tolist() == list(range(k))
+
+
+def test_batched_score_select_per_head(oracle):
+    Q, _, _ = synth.attention_qkv(1, 6, 6, 200, 8, 128, seed=4)
+    idx, _, _, _ = rmm.rmm_score_select(dev(Q[0]), rho=0.5)
+    for h in range(6):
+        e64, _ = oracle.score(Q[0, h])
+        check_index_set(idx[h].cpu().numpy(), e64, 64)
+
+
+# ------------------------------------------------------------------------------------------------
+# reduced product
+# ------------------------------------------------------------------------------------------------
+def oracle_set(oracle, A, rho):
+    e, _ = oracle.score(A)
+    return oracle.select(e, oracle.keep_count(rho, A.shape[1]))[0]
+
+
+@pytest.mark.parametrize("M,K,N,rho", [
+    (128, 64, 256, 1.0), (128, 128, 256, 0.5), (64, 512, 256, 0.5), (129, 1000, 264, 0.75), (300, 4096, 136, 0.25),
+    (1, 64, 8, 1.0), (63, 129 * 8, 120, 0.5), (257, 1024, 128, 0.5), (512, 2048, 1024, 0.6), (384, 8192, 512, 0.3),
+    (2, 16, 16, 0.07), (200, 136, 1032, 0.9)])
+def test_reduced_gemm_tensor_core_path(oracle, M, K, N, rho):
+    A, B = synth.mlp_product(M, K, N, seed=M + N)
+    idx = oracle_set(oracle, A, rho)
+    want = oracle.reduced_gemm(A, B, idx)
+    idx_d = dev(torch.from_numpy(idx))
+    Y = rmm.rmm_reduced_gemm(dev(A), dev(B), idx_d)
+    assert Y.dtype == torch.bfloat16
+    assert rel_fro(Y.float().cpu().numpy(), want) <= TOL_BF16
+    Yf = rmm.rmm_reduced_gemm(dev(A), dev(B), idx_d, out_dtype=torch.float32)
+    assert rel_fro(Yf.cpu().numpy(), want) <= 1e-5          # fp32 accumulation of exact bf16 products
+    assert np.abs(Yf.cpu().numpy() - want).max() <= 1e-4 * max(1.0, np.abs(want).max())
+
+
+def test_reduced_gemm_k_contiguous_b_and_batch(oracle):
+    """B given K-contiguous (as K^T in attention) and a batch with one index set per entry."""
+    b, M, K, N = 3, 150, 128, 200
+    A = synth.gaussian((b, M, K), 1.0, seed=1)
+    Bt = synth.gaussian((b, N, K), 1.0, seed=2)           # B[b] = Bt[b].T
+    idx = np.stack([np.sort(np.random.default_rng(s).choice(K, 77, replace=False)).astype(np.int32) for s in range(b)])
+    Y = rmm.rmm_reduced_gemm(dev(A), dev(Bt).transpose(1, 2), dev(torch.from_numpy(idx)), scale=0.125, out_dtype=torch.float32)
+    for i in range(b):
+        want = 0.125 * oracle.reduced_gemm(A[i], Bt[i].T, idx[i])
+        assert rel_fro(Y[i].cpu().numpy(), want) <= 1e-5
+    # batched row-contiguous B, and a shared B
+    Bb = synth.gaussian((b, K, N), 0.05, seed=3)
+    Y2 = rmm.rmm_reduced_gemm(dev(A), dev(Bb), dev(torch.from_numpy(idx)))
+    Y3 = rmm.rmm_reduced_gemm(dev(A), dev(Bb[1]), dev(torch.from_numpy(idx)))
+    for i in range(b):
+        assert rel_fro(Y2[i].float().cpu().numpy(), oracle.reduced_gemm(A[i], Bb[i], idx[i])) <= TOL_BF16
+        assert rel_fro(Y3[i].float().cpu().numpy(), oracle.reduced_gemm(A[i], Bb[1], idx[i])) <= TOL_BF16
+
+
+@pytest.mark.parametrize("M,K,N,rho", [(1, 1, 1, 1.0), (2, 7, 1, 0.5), (63, 9, 8, 0.75), (65, 17, 120, 0.25), (129, 65, 136, 0.5),
+                                       (300, 1000, 264, 0.5)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_reduced_gemm_fma_path(oracle, M, K, N, rho, dtype):
+    """fp32 operands (1e-5 bar) and bf16 operands whose shapes break the TMA alignment rules."""
+    A = synth.heavy_tailed_activations(M, K, seed=3, dtype=dtype)
+    B = synth.weight(K, N + 1, seed=4, std=0.05, dtype=dtype)[:, :N]       # row pitch N+1: never 16-byte aligned rows
+    idx = oracle_set(oracle, A, rho)
+    want = oracle.reduced_gemm(A, B, idx)
+    Y = rmm.rmm_reduced_gemm(dev(A), dev(B), dev(torch.from_numpy(idx)), out_dtype=torch.float32)
+    assert rel_fro(Y.cpu().numpy(), want) <= TOL_F32
+    Yb = rmm.rmm_reduced_gemm(dev(A), dev(B), dev(torch.from_numpy(idx)), out_dtype=torch.bfloat16)
+    assert rel_fro(Yb.float().cpu().numpy(), want) <= TOL_BF16
+
+
+def test_reduced_gemm_any_index_set_and_bad_index(oracle):
+    """A cached or random set is accepted (static / random controls); an out-of-range index is skipped and reported."""
+    A, B = synth.mlp_product(256, 512, 256, seed=11)
+    g = torch.Generator().manual_seed(0)
+    idx = torch.randperm(512, generator=g)[:200].int()                      # unsorted on purpose
+    Y = rmm.rmm_reduced_gemm(dev(A), dev(B), dev(idx), out_dtype=torch.float32)
+    assert rel_fro(Y.cpu().numpy(), oracle.reduced_gemm(A, B, idx.numpy())) <= 1e-5
+    bad = idx.clone()
+    bad[5] = 512
+    Yb = rmm.rmm_reduced_gemm(dev(A), dev(B), dev(bad), out_dtype=torch.float32)
+    assert rmm.rmm_status_read() == 6                                       # RMM_ERR_BOUNDS, and cleared by the read
+    keep = torch.cat([idx[:5], idx[6:]])
+    assert rel_fro(Yb.cpu().numpy(), oracle.reduced_gemm(A, B, keep.numpy())) <= 1e-5
+    assert rmm.rmm_status_read() == 0
+
+
+def test_rho_one_equals_dense_product(oracle):
+    A, B = synth.mlp_product(256, 1024, 384, seed=2)
+    Y, idx = rmm.rmm(dev(A), dev(B), 1.0)
+    assert idx.cpu().tolist() == list(range(1024))
+    ref = (A.double() @ B.double()).numpy()
+    assert rel_fro(Y.float().cpu().numpy(), ref) <= TOL_BF16
+
+
+def test_mlp_config_full_size_sampled_rows(oracle):
+    """1B-class down projection at full size (2048 x 8192 x 2048), in the launch configuration the benchmark times:
+    index sets checked in full, products on sampled rows including tile edges."""
+    A, B = synth.mlp_product(2048, 8192, 2048, seed=0)
+    Ad, Bd = dev(A), dev(B)
+    e64, _ = oracle.score(A)
+    rows = [0, 1, 127, 128, 129, 1023, 1024, 2046, 2047] + list(np.random.default_rng(0).choice(2048, 8, replace=False))
+    for rho in (0.25, 0.5, 0.75, 1.0):
+        k = oracle.keep_count(rho, 8192)
+        Y, idx = rmm.rmm(Ad, Bd, rho)
+        check_index_set(idx.cpu().numpy(), e64, k)
+        idx_np = idx.cpu().numpy()
+        Yc = Y.float().cpu().numpy()
+        for r in rows:
+            want = oracle.reduced_gemm(A, B, idx_np, rows=(int(r), int(r) + 1))[int(r)]
+            assert rel_fro(Yc[int(r)], want) <= TOL_BF16
+    assert rmm.rmm_status_read() == 0
+
+
+def test_host_buffer_entry_point(oracle):
+    A, B = synth.mlp_product(384, 1024, 512, seed=6)
+    Ah, Bh = A.pin_memory(), B.pin_memory()
+    Yh = torch.empty(384, 512, dtype=torch.bfloat16).pin_memory()
+    ih = torch.empty(512, dtype=torch.int32).pin_memory()
+    rmm.rmm_product_host(Ah, Bh, 0.5, Yh, ih)
+    torch.cuda.synchronize()
+    e64, _ = oracle.score(A)
+    check_index_set(ih.numpy(), e64, 512)
+    assert rel_fro(Yh.float().numpy(), oracle.reduced_gemm(A, B, ih.numpy())) <= TOL_BF16
+
+
+# ------------------------------------------------------------------------------------------------
+# attention
+# ------------------------------------------------------------------------------------------------
+def check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t, seed, n_outlier=4):
+    Q, K, V = synth.attention_qkv(B, Hq, Hkv, Lq, Lk, Dh, seed=seed, n_outlier=n_outlier)
+    O, idx_feat, idx_tok = rmm.rmm_reduced_attn(dev(Q), dev(K), dev(V), causal, rho_d, rho_t, want_idx=True)
+    Oo, If, It, P = oracle.attn(Q, K, V, causal, rho_d, rho_t, round_p=True, want_p=True)
+    kd = oracle.keep_count(rho_d, Dh)
+    for b in range(B):
+        for h in range(Hq):
+            e64, _ = oracle.score(Q[b, h])
+            check_index_set(idx_feat[b, h].cpu().numpy(), e64, kd)
+    same_feat = np.array_equal(idx_feat.cpu().numpy(), If)
+    if rho_t < 1.0:
+        kt = oracle.keep_count(rho_t, Lk)
+        got = idx_tok.cpu().numpy()
+        assert got.shape == (B, Hq, kt)
+        if same_feat:
+            for b in range(B):
+                for h in range(Hq):
+                    # token scores come from an fp32 softmax on the GPU: judge the criterion (Theorem 1) --
+                    # the oracle-evaluated retained energy of the GPU's set is within 1e-6 of the optimum --
+                    # and set equality outside a 1e-4 * max band
+                    a2 = (P[b, h] ** 2).sum(axis=0)
+                    assert np.all(np.diff(got[b, h]) > 0)
+                    assert a2[got[b, h]].sum() >= (1 - 1e-6) * a2[It[b, h]].sum()
+                    s = np.sqrt(a2)
+                    tau = np.sort(s)[::-1][kt - 1]
+                    diff = np.setxor1d(got[b, h], It[b, h])
+                    assert np.all(np.abs(s[diff] - tau) <= 1e-4 * s.max())
+    if same_feat and (rho_t == 1.0 or np.array_equal(idx_tok.cpu().numpy(), It)):
+        assert rel_fro(O.float().cpu().numpy(), Oo) <= TOL_BF16
+    return same_feat
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("rho_d,rho_t", [(1.0, 1.0), (0.5, 1.0), (0.75, 0.5), (0.5, 0.25)])
+def test_reduced_attention_small(oracle, causal, rho_d, rho_t):
+    assert check_attention(oracle, 1, 4, 4, 160, 160, 64, causal, rho_d, rho_t, seed=30)
+
+
+def test_reduced_attention_gqa_and_ragged(oracle):
+    assert check_attention(oracle, 2, 8, 2, 100, 173, 128, True, 0.5, 0.5, seed=31)
+    assert check_attention(oracle, 1, 4, 1, 257, 257, 128, False, 0.75, 0.3, seed=32)
+    assert check_attention(oracle, 1, 2, 2, 1, 300, 64, True, 0.5, 1.0, seed=33)      # a single query row (decode shape)
