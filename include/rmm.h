@@ -83,15 +83,16 @@ size_t rmm_select_workspace_bytes(int64_t batch, int64_t K);
 int rmm_select(const float *keys, int64_t batch, int64_t K, double rho, int64_t k, int32_t *idx, float *retained,
                void *ws, size_t ws_bytes, void *stream);
 
-/* rmm_score followed by rmm_select on the energies, in ONE launch (the last thread block to finish
- * a batch element's scores selects its index set).  scores / energy / retained may be NULL. */
+/* rmm_score followed by rmm_select on the energies, in ONE launch when n <= 8192 (the last thread block to finish
+ * a batch element's scores selects its index set; larger n: the select kernel follows as a second launch).
+ * scores / energy / retained may be NULL. */
 size_t rmm_score_select_workspace_bytes(const rmm_mat_t *A, int axis);
 int rmm_score_select(const rmm_mat_t *A, int axis, double rho, int64_t k, int32_t *idx, float *scores, float *energy,
                      float *retained, void *ws, size_t ws_bytes, void *stream);
 
 /* Y = scale * A[:, I] B[I, :] (Sec. 3.2, RMM_rho(A,B); no rescaling: pass scale = 1).
  *   A    [b, M, K]; B [b or shared, K, N] (stride_batch 0 = shared); Y [b, M, N] (written in full)
- *   idx  int32 [b, k], each entry in [0, K); any set is accepted (so a cached or random set gives
+ *   idx  int32 [b, k], each entry in [0, K) (NULL with k == K: the unreduced product, nothing is gathered); any set is accepted (so a cached or random set gives
  *        the paper's static / random controls); order fixes the summation order
  *   bf16 operands run on the tensor cores (fp32 accumulation) when A has stride_col 1, B has
  *   stride_col 1 (slices of the contraction axis contiguous) or stride_row 1, Y has stride_col 1, and

@@ -221,16 +221,20 @@ def rmm_score_select(A: torch.Tensor, rho: float = 0.0, k: int = 0, axis: int = 
     return idx, scores, energy, ret
 
 
-def rmm_reduced_gemm(A: torch.Tensor, B: torch.Tensor, idx: torch.Tensor, scale: float = 1.0,
+def rmm_reduced_gemm(A: torch.Tensor, B: torch.Tensor, idx: Optional[torch.Tensor], scale: float = 1.0,
                      out: Optional[torch.Tensor] = None, out_dtype: Optional[torch.dtype] = None,
                      ws: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """Y = scale * A[:, idx] @ B[idx, :].  A [M,K] or [b,M,K]; B [K,N] or [b,K,N]; idx int32 [k] or [b,k]."""
+    """Y = scale * A[:, idx] @ B[idx, :].  A [M,K] or [b,M,K]; B [K,N] or [b,K,N]; idx int32 [k] or [b,k]
+    (None: the unreduced product, k = K, nothing gathered)."""
     ma, mb = as_mat(A), as_mat(B)
-    if idx.dtype != torch.int32 or not idx.is_cuda or not idx.is_contiguous():
-        raise RmmError(RMM_ERR_INVALID_ARG, "idx must be a contiguous int32 CUDA tensor")
-    k = idx.shape[-1]
-    if idx.numel() != ma.batch * k:
-        raise RmmError(RMM_ERR_INVALID_ARG, "idx must hold one index list per batch element of A")
+    if idx is None:
+        k = ma.cols
+    else:
+        if idx.dtype != torch.int32 or not idx.is_cuda or not idx.is_contiguous():
+            raise RmmError(RMM_ERR_INVALID_ARG, "idx must be a contiguous int32 CUDA tensor")
+        k = idx.shape[-1]
+        if idx.numel() != ma.batch * k:
+            raise RmmError(RMM_ERR_INVALID_ARG, "idx must hold one index list per batch element of A")
     if out is None:
         dt = out_dtype if out_dtype is not None else A.dtype
         shape = (ma.batch, ma.rows, mb.cols) if A.dim() == 3 else (ma.rows, mb.cols)
@@ -239,7 +243,7 @@ def rmm_reduced_gemm(A: torch.Tensor, B: torch.Tensor, idx: torch.Tensor, scale:
     need = lib().rmm_reduced_gemm_workspace_bytes(ctypes.byref(ma), ctypes.byref(mb), k, ctypes.byref(my))
     ws = workspace(need, A.device) if ws is None else ws
     p, nb = _ws_ptr(ws)
-    _check(lib().rmm_reduced_gemm(ctypes.byref(ma), ctypes.byref(mb), idx.data_ptr(), k, float(scale),
+    _check(lib().rmm_reduced_gemm(ctypes.byref(ma), ctypes.byref(mb), idx.data_ptr() if idx is not None else None, k, float(scale),
                                   ctypes.byref(my), p, nb, _stream()))
     return out
 

@@ -142,7 +142,8 @@ static int check_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx
     if ((rc = check_mat(A, "reduced_gemm", "A")) != RMM_OK) return rc;
     if ((rc = check_mat(B, "reduced_gemm", "B")) != RMM_OK) return rc;
     if ((rc = check_mat(Y, "reduced_gemm", "Y")) != RMM_OK) return rc;
-    if (idx == nullptr) return fail(RMM_ERR_INVALID_ARG, "reduced_gemm: idx is NULL");
+    if (idx == nullptr && k != A->cols)
+        return fail(RMM_ERR_INVALID_ARG, "reduced_gemm: idx is NULL (allowed only with k == K, the unreduced product)");
     if (A->cols != B->rows) return fail(RMM_ERR_INVALID_ARG, "reduced_gemm: A has %lld columns but B has %lld rows",
                                         (long long)A->cols, (long long)B->rows);
     if (Y->rows != A->rows || Y->cols != B->cols || Y->batch != A->batch)

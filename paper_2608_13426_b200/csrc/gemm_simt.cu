@@ -42,7 +42,7 @@ __global__ void __launch_bounds__(THREADS) reduced_gemm_simt_kernel(SimtArgs a)
     const int64_t b = blockIdx.z;
     const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
     const int ty = tid / 16, tx = tid % 16;  // thread owns rows ty*4.., cols tx*4..
-    const int32_t *idx = a.idx + b * a.k;
+    const int32_t *idx = a.idx != nullptr ? a.idx + b * a.k : nullptr;
     const int64_t a0 = b * a.a_sb, b0 = b * a.b_sb;
 
     float acc[4][4];
@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(THREADS) reduced_gemm_simt_kernel(SimtArgs a)
         if (tid < BK) {
             int j = -1;
             if (kk + tid < a.k) {
-                j = idx[kk + tid];
+                j = idx != nullptr ? idx[kk + tid] : (int)(kk + tid);
                 if (j < 0 || j >= a.K) {  // skip a bad index and report it
                     atomicExch(a.status, (int)RMM_ERR_BOUNDS);
                     j = -1;

@@ -97,6 +97,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
 // Four rows (y0..y3) of a 2-D tensor, columns x .. x+box-1, land as four consecutive shared-memory rows.
 __device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap *map, int x, int y0, int y1, int y2, int y3,
                                             uint32_t bar)
@@ -267,6 +274,12 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 }
                 __syncwarp();
                 if constexpr (!B_KMAJOR) {
+                    if (ix == nullptr) {
+                        // rows 0 .. k-1 in order: plain tile loads of 64 rows x 64 columns (rows past the tensor read as zeros)
+                        if (lane < BN / 64)
+                            tma_load_2d(sb + lane * (BK * 128), &map_b, tn * BN + lane * 64, row_base + kb * BK, full_bar(s));
+                        continue;
+                    }
                     // BN/64 column chunks x 16 row groups = BN/4 gathers per stage, BN/128 per lane
 #pragma unroll
                     for (int c = lane >> 4; c < BN / 64; c += 2) {
@@ -515,7 +528,7 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     } else {
         uint64_t dims[2] = {(uint64_t)p.N, (uint64_t)p.b_rows_total};
         uint64_t st[1] = {(uint64_t)p.b_ld * 2};
-        uint32_t box[2] = {64, 1};
+        uint32_t box[2] = {64, p.idx != nullptr ? 1u : (uint32_t)BK};  // one row per gathered row, or a 64-row tile
         rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 2, dims, st, box);
     }
     if (rc != RMM_OK) return rc;
@@ -535,12 +548,20 @@ int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, i
     int *status = &reinterpret_cast<WsHeader *>(w)->status;
     const int64_t M = A->rows, K = A->cols, N = B->cols, batch = A->batch;
     __nv_bfloat16 *Ap = reinterpret_cast<__nv_bfloat16 *>(w + plan.off_ap);
-    int rc = launch_pack_cols(static_cast<const __nv_bfloat16 *>(A->ptr), batch, M, K, A->stride_batch, A->stride_row, 0, 1,
-                              idx, k, k, Ap, plan.ldp, status, stream);
-    if (rc != RMM_OK) return rc;
+    int rc;
     TcProblem p = {};
     p.batch = batch; p.M = M; p.N = N; p.k = k;
-    p.a = Ap; p.a_ld = plan.ldp; p.a_sb = M * plan.ldp;
+    // the unreduced product (idx NULL, k == K) on a TMA-loadable A needs no gather at all
+    const bool a_in_place = idx == nullptr && reinterpret_cast<uintptr_t>(A->ptr) % 16 == 0 && A->stride_row % 8 == 0 &&
+                            A->stride_batch % 8 == 0 && !plan.b_kmajor;
+    if (a_in_place) {
+        p.a = static_cast<const __nv_bfloat16 *>(A->ptr); p.a_ld = A->stride_row; p.a_sb = batch > 1 ? A->stride_batch : M * A->stride_row;
+    } else {
+        rc = launch_pack_cols(static_cast<const __nv_bfloat16 *>(A->ptr), batch, M, K, A->stride_batch, A->stride_row, 0, 1,
+                              idx, k, k, Ap, plan.ldp, status, stream);
+        if (rc != RMM_OK) return rc;
+        p.a = Ap; p.a_ld = plan.ldp; p.a_sb = M * plan.ldp;
+    }
     p.b_kmajor = plan.b_kmajor;
     p.y = Y->ptr; p.y_bf16 = Y->dtype == RMM_BF16; p.y_sb = Y->stride_batch; p.y_sr = Y->stride_row;
     p.scale = scale; p.status = status;

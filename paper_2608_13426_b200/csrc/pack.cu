@@ -25,7 +25,7 @@ __global__ void __launch_bounds__(kWarps * 32) pack_cols_kernel(const __nv_bfloa
     const int64_t b = blockIdx.z;
     const int64_t j0 = ((int64_t)blockIdx.x * kWarps + warp) * 256;  // first output column of this warp
     if (j0 >= ld_dst) return;
-    const int32_t *ix = idx + b * idx_stride;
+    const int32_t *ix = idx != nullptr ? idx + b * idx_stride : nullptr;  // NULL: columns 0 .. k-1 in order
 
     int c[8];  // source columns of this lane's 4 output pairs; -1 = write zero
 #pragma unroll
@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(kWarps * 32) pack_cols_kernel(const __nv_bfloa
             int64_t j = j0 + 64 * i + 2 * lane + h;
             int v = -1;
             if (j < k) {
-                v = __ldg(ix + j);
+                v = ix != nullptr ? __ldg(ix + j) : (int)j;
                 if (v < 0 || v >= K) {
                     atomicExch(status, (int)RMM_ERR_BOUNDS);
                     v = -1;

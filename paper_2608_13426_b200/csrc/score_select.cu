@@ -20,6 +20,8 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kUnroll = 4;       // rows in flight per thread
 constexpr int kFlushEvery = 4;   // loop trips between fp32 -> fp64 flushes (kUnroll * kFlushEvery = 16 terms)
+constexpr int kFusedSelectMax = 8192;    // largest K whose select runs in the score kernel's tail (32 KB key cache)
+constexpr int kCachedSelectMax = 49152;  // largest K the stand-alone select kernel caches in shared memory (192 KB)
 
 struct SelectSmem {
     unsigned hist[256];
@@ -40,10 +42,25 @@ __device__ __forceinline__ unsigned key_image(float f)
 // Block-wide top-k of keys[0..K): writes idx[0..k) ascending, optional retained fraction.
 // Every thread of the block must call it; keys are read through L2 (they may have just been
 // written by other blocks).
-__device__ void block_select(const float *keys, int K, int k, int32_t *idx, float *retained, SelectSmem &sm)
+//
+// kcache, if not NULL, is shared memory for K key images: the keys are then fetched once (independent
+// loads, so their latencies overlap) and every later pass runs out of shared memory.
+__device__ __forceinline__ float key_value(unsigned u)
+{
+    return __uint_as_float((u & 0x80000000u) ? (u ^ 0x80000000u) : ~u);
+}
+
+__device__ void block_select(const float *keys, int K, int k, int32_t *idx, float *retained, SelectSmem &sm,
+                             unsigned *kcache)
 {
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
     unsigned prefix = 0, mask = 0, remaining = (unsigned)k;
+    if (kcache != nullptr) {
+#pragma unroll 8
+        for (int j = tid; j < K; j += nthr) kcache[j] = key_image(__ldcg(keys + j));
+        __syncthreads();
+    }
+    auto image = [&](int j) -> unsigned { return kcache != nullptr ? kcache[j] : key_image(__ldcg(keys + j)); };
 
     for (int shift = 24; shift >= 0; shift -= 8) {
         for (int i = tid; i < 256; i += nthr) sm.hist[i] = 0;
@@ -53,7 +70,7 @@ __device__ void block_select(const float *keys, int K, int k, int32_t *idx, floa
             bool live = false;
             unsigned bin = 0;
             if (j < K) {
-                unsigned u = key_image(__ldcg(keys + j));
+                unsigned u = image(j);
                 live = (u & mask) == prefix;
                 bin = (u >> shift) & 255u;
             }
@@ -112,8 +129,8 @@ __device__ void block_select(const float *keys, int K, int k, int32_t *idx, floa
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             if (j + i < K) {
-                f[i] = __ldcg(keys + j + i);
-                u[i] = key_image(f[i]);
+                u[i] = image(j + i);
+                f[i] = key_value(u[i]);
                 mine += (u[i] > tau) ? (1ull << 32) : 0ull;
                 mine += (u[i] == tau) ? 1ull : 0ull;
             } else {
@@ -229,7 +246,8 @@ __device__ __forceinline__ void load_vec(const void *A, int64_t off, int64_t s_n
 template <int VEC, bool BF16>
 __global__ void __launch_bounds__(kThreads) score_select_kernel(ScoreArgs a)
 {
-    __shared__ double s_part[kThreads * VEC];
+    extern __shared__ __align__(16) unsigned char s_dyn[];  // row-lane partial sums, later the select's key cache
+    double *s_part = reinterpret_cast<double *>(s_dyn);
     __shared__ SelectSmem s_sel;
     __shared__ int s_flag;
 
@@ -324,14 +342,17 @@ __global__ void __launch_bounds__(kThreads) score_select_kernel(ScoreArgs a)
     if (!s_flag) return;
     __threadfence();
     block_select(a.energy + b * a.n, (int)a.n, a.k, a.idx + b * (int64_t)a.k,
-                 a.retained ? a.retained + b : nullptr, s_sel);
+                 a.retained ? a.retained + b : nullptr, s_sel, reinterpret_cast<unsigned *>(s_dyn));
 }
 
-__global__ void __launch_bounds__(1024) select_kernel(const float *keys, int K, int k, int32_t *idx, float *retained)
+__global__ void __launch_bounds__(1024) select_kernel(const float *keys, int K, int k, int32_t *idx, float *retained,
+                                                      int use_cache)
 {
+    extern __shared__ __align__(16) unsigned char s_dyn[];
     __shared__ SelectSmem s_sel;
     const int64_t b = blockIdx.x;
-    block_select(keys + b * K, K, k, idx + b * (int64_t)k, retained ? retained + b : nullptr, s_sel);
+    block_select(keys + b * K, K, k, idx + b * (int64_t)k, retained ? retained + b : nullptr, s_sel,
+                 use_cache ? reinterpret_cast<unsigned *>(s_dyn) : nullptr);
 }
 
 }  // namespace
@@ -409,18 +430,23 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
     }
     a.energy = energy ? energy : reinterpret_cast<float *>(w + p.off_energy);
     a.scores = scores;
-    a.do_select = do_select ? 1 : 0;
+    const bool fused = do_select && p.n <= kFusedSelectMax;
+    a.do_select = fused ? 1 : 0;
     a.k = (int)k;
     a.idx = idx;
     a.retained = retained;
 
     dim3 grid((unsigned)p.col_blocks, (unsigned)p.row_splits, (unsigned)A->batch);
     const bool bf16 = A->dtype == RMM_BF16;
-    if (bf16 && p.vec == 8) score_select_kernel<8, true><<<grid, kThreads, 0, stream>>>(a);
-    else if (bf16) score_select_kernel<1, true><<<grid, kThreads, 0, stream>>>(a);
-    else if (p.vec == 4) score_select_kernel<4, false><<<grid, kThreads, 0, stream>>>(a);
-    else score_select_kernel<1, false><<<grid, kThreads, 0, stream>>>(a);
-    return check_launch("score_select_kernel");
+    size_t smem = (size_t)kThreads * p.vec * sizeof(double);
+    if (fused && (size_t)p.n * 4 > smem) smem = (size_t)p.n * 4;
+    if (bf16 && p.vec == 8) score_select_kernel<8, true><<<grid, kThreads, smem, stream>>>(a);
+    else if (bf16) score_select_kernel<1, true><<<grid, kThreads, smem, stream>>>(a);
+    else if (p.vec == 4) score_select_kernel<4, false><<<grid, kThreads, smem, stream>>>(a);
+    else score_select_kernel<1, false><<<grid, kThreads, smem, stream>>>(a);
+    int rc = check_launch("score_select_kernel");
+    if (rc != RMM_OK || !do_select || fused) return rc;
+    return launch_select(a.energy, A->batch, p.n, k, idx, retained, ws, stream);
 }
 
 int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_t *idx, float *retained, void *ws,
@@ -428,7 +454,15 @@ int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_
 {
     (void)ws;
     int threads = K >= 4096 ? 1024 : (K >= 1024 ? 512 : 256);
-    select_kernel<<<(unsigned)batch, threads, 0, stream>>>(keys, (int)K, (int)k, idx, retained);
+    const int use_cache = K <= kCachedSelectMax;
+    const size_t smem = use_cache ? (size_t)K * 4 : 0;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCachedSelectMax * 4);
+        if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "select: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+        configured = true;
+    }
+    select_kernel<<<(unsigned)batch, threads, smem, stream>>>(keys, (int)K, (int)k, idx, retained, use_cache);
     return check_launch("select_kernel");
 }
 
