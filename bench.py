@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Benchmark of the RMM hot path on B200.
+
+A step is one pass of the whole hot path over one product: fused score + top-k select on A, then the
+reduced product Y = A[:, I] B[I, :] (gathers included).  Workload at N = 1: the 1B-class MLP down
+projection (A 2048 x 8192 activations with 1 % heavy-tailed channels, B 8192 x 2048 weight, bf16), headline
+retention ratio rho = 0.5; the other ratios are reported in `per_rho`.  With N > 1 every rank runs the
+same workload on its own GPU (independent replicas, no data-path collective).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+prints ONE JSON line.  `--impl reference` times the CPU oracle (the slow fp64 checker) on a bounded
+sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+M, K, N = 2048, 8192, 2048
+RHO = 0.5
+RHOS = (0.25, 0.5, 0.75, 1.0)
+METRIC = "reduced-GEMM retained TFLOP/s (whole RMM op: score + select + reduced product)"
+UNIT = "TFLOP/s"
+WORKLOAD = "1B-class MLP down-projection: A 2048x8192 bf16 N(0,1) with 1% Student-t(3) channels, B 8192x2048 bf16 N(0,0.02^2)"
+
+
+def retained_flops(rho: float) -> float:
+    import math
+    k = max(1, math.ceil(rho * K - 1e-9))
+    return 2.0 * M * k * N
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"bf16_burst": float(d["bf16_tflops"]), "bf16_sustained": float(d["bf16_tflops_sustained"]),
+                "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return {"bf16_burst": 1590.0, "bf16_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_setup(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    return rank, world, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def max_over_ranks(x: float, world: int) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def time_region(fn, steps: int, world: int) -> float:
+    """ms per step over exactly `steps` calls, device-timed, barrier + synchronize on both sides, max over ranks."""
+    barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        fn(i)
+    e1.record()
+    barrier(world)
+    return max_over_ranks(e0.elapsed_time(e1), world) / steps
+
+
+def cpu_oracle_sample(A, B, rho: float, target_s: float = 12.0):
+    """Time the oracle as it stands (score + select at full size, product on a sample of rows)."""
+    import oracle
+    oracle.build()
+    cores = oracle.num_threads()
+    t0 = time.perf_counter()
+    e, _ = oracle.score(A)
+    idx, _ = oracle.select(e, oracle.keep_count(rho, A.shape[1]))
+    t_sel = time.perf_counter() - t0
+    probe = min(M, 4 * cores)
+    t0 = time.perf_counter()
+    oracle.reduced_gemm(A, B, idx, rows=(0, probe))
+    t_probe = time.perf_counter() - t0
+    rows = int(max(probe, min(M, target_s / max(t_probe / probe, 1e-9))))
+    rows = max(cores, rows // cores * cores)
+    t0 = time.perf_counter()
+    oracle.reduced_gemm(A, B, idx, rows=(0, rows))
+    t_rows = time.perf_counter() - t0
+    # whole-op time for the sampled rows: the score/select pass is charged in proportion to the rows kept
+    t = t_rows + t_sel * rows / M
+    flops = 2.0 * rows * len(idx) * N
+    return {"value": flops / t / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"score+select on the full {M}x{K} A ({t_sel:.3f} s, charged pro rata), product on rows 0..{rows - 1} of {M} "
+                      f"at rho={rho} ({t_rows:.2f} s)", "seconds": t_rows + t_sel}
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle, timed on this machine's host cores; rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2608_13426_b200 import synth
+    A, B = synth.mlp_product(M, K, N, seed=0)
+    import oracle
+    oracle.build()
+    cores = oracle.num_threads()
+    e, _ = oracle.score(A)
+    idx, _ = oracle.select(e, oracle.keep_count(RHO, K))
+    rows = max(cores, 2 * cores)             # bounded sample per step
+    times = []
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        e, _ = oracle.score(A[: max(rows, 1)])          # score pass on the same row sample
+        oracle.select(e, len(idx))
+        oracle.reduced_gemm(A, B, idx, rows=(0, rows))
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    val = 2.0 * rows * len(idx) * N / (ms / 1e3) / 1e12
+    sample = f"rows 0..{rows - 1} of {M} per step (score, select and product on that sample), rho={RHO}"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD, "rho": RHO, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU oracle timing (quick runs, profiling)")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the per-rho sweep")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import paper_2608_13426_b200 as rmm
+    from paper_2608_13426_b200 import binding, synth
+
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local if world > 1 else 0)
+    peaks = measured_peaks()
+
+    # ---- inputs: several independent (A, B, Y) sets, together well above the 126 MB L2, rotated per step
+    n_sets = 5
+    sets = []
+    for s in range(n_sets):
+        A, B = synth.mlp_product(M, K, N, seed=100 * rank + s)
+        sets.append((A.to(dev), B.to(dev), torch.empty(M, N, dtype=torch.bfloat16, device=dev)))
+    A0_cpu, B0_cpu = synth.mlp_product(M, K, N, seed=0)
+    resident_bytes = n_sets * (M * K + K * N + M * N) * 2
+    k = rmm.rmm_keep_count(RHO, K)
+    idx_buf = torch.empty(k, dtype=torch.int32, device=dev)
+
+    def step(i, rho=RHO, idx=idx_buf):
+        A, B, Y = sets[i % n_sets]
+        rmm.rmm_score_select(A, rho=rho, idx=idx)
+        rmm.rmm_reduced_gemm(A, B, idx, out=Y)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    assert rmm.rmm_status_read() == 0
+
+    # ---- timed region: exactly K steps; the GEMM kernel of every step is bracketed by events on the same stream
+    sampler = ClockSampler(local if world > 1 else 0)
+    timer = binding.GemmTimer(args.steps)
+    launches0 = rmm.rmm_launch_count()
+    sampler.start()
+    with timer:
+        ms_step = time_region(step, args.steps, world)
+    clocks = sampler.stop()
+    launches = rmm.rmm_launch_count() - launches0
+    gemm_ms = timer.times_ms()
+    gemm_ms_avg = sum(gemm_ms) / len(gemm_ms)
+    assert rmm.rmm_status_read() == 0
+    value = world * retained_flops(RHO) / (ms_step * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel (the tensor-core GEMM): retained FLOPs of one launch / its mean duration
+    achieved = retained_flops(RHO) / (gemm_ms_avg * 1e-3) / 1e12
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "gemm_traffic.json")
+    if os.path.exists(tpath):
+        traffic = json.load(open(tpath)).get("dram_bytes_per_launch_rho0.5")
+    roofline = {"bound": "tensor", "kernel": "reduced_gemm_tc_kernel", "achieved": achieved, "peak": peaks["bf16_sustained"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": traffic,
+                "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step loop)",
+                "frac_of_burst_peak": achieved / peaks["bf16_burst"], "kernel_ms": gemm_ms_avg}
+
+    # ---- end to end: host buffers in, host buffer out, through the C-ABI host entry point
+    Ah, Bh = A0_cpu.pin_memory(), B0_cpu.pin_memory()
+    Yh = torch.empty(M, N, dtype=torch.bfloat16).pin_memory()
+    ih = torch.empty(K, dtype=torch.int32).pin_memory()
+
+    def step_e2e(i):
+        rmm.rmm_product_host(Ah, Bh, RHO, Yh, ih)
+        torch.cuda.current_stream().synchronize()      # the caller reads Y_host after every step
+
+    for i in range(3):
+        step_e2e(i)
+    e2e_steps = max(5, min(args.steps, 50))
+    ms_e2e = time_region(step_e2e, e2e_steps, world)
+    e2e = {"value": world * retained_flops(RHO) / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e, "steps": e2e_steps,
+           "h2d_bytes_per_step": (M * K + K * N) * 2, "d2h_bytes_per_step": M * N * 2 + k * 4}
+
+    # ---- per-rho sweep: whole op, its parts, dense cuBLAS at the same shape
+    per_rho = []
+    if not args.no_sweep and rank == 0:
+        reps = 40
+        dense_ms = time_region(lambda i: torch.matmul(sets[i % n_sets][0], sets[i % n_sets][1], out=sets[i % n_sets][2]), reps, 1)
+        for rho in RHOS:
+            kk = rmm.rmm_keep_count(rho, K)
+            idx_r = torch.empty(kk, dtype=torch.int32, device=dev)
+            for i in range(3):
+                step(i, rho, idx_r)
+            t = binding.GemmTimer(reps)
+            with t:
+                whole = time_region(lambda i: step(i, rho, idx_r), reps, 1)
+            g = sum(t.times_ms()) / reps
+            sel = time_region(lambda i: rmm.rmm_score_select(sets[i % n_sets][0], rho=rho, idx=idx_r), reps, 1)
+            fl = retained_flops(rho)
+            per_rho.append({"rho": rho, "k": kk, "whole_op_ms": whole, "whole_op_tflops": fl / whole / 1e9,
+                            "gemm_kernel_ms": g, "gemm_kernel_tflops": fl / g / 1e9,
+                            "gemm_frac_of_sustained_peak": fl / g / 1e9 / peaks["bf16_sustained"],
+                            "gemm_frac_of_burst_peak": fl / g / 1e9 / peaks["bf16_burst"],
+                            "score_select_ms": sel, "score_select_gbs": M * K * 2 / sel / 1e6,
+                            "score_select_frac_of_hbm": M * K * 2 / sel / 1e6 / peaks["hbm_gbs"],
+                            "dense_cublas_ms": dense_ms, "speedup_vs_dense_cublas": dense_ms / whole})
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_oracle_sample(A0_cpu, B0_cpu, RHO)
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "rho": RHO, "k": k, "M": M, "K": K, "N": N, "parallelism": f"replicas x{world}",
+                       "l2_policy": f"inputs larger than L2: {n_sets} rotating (A, B, Y) sets, {resident_bytes / 1e6:.0f} MB resident"},
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "per_rho": per_rho, "peaks": peaks,
+        }
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -136,6 +136,14 @@ int rmm_product_host(const void *A_host, const void *B_host, int64_t M, int64_t 
  * Synchronous: call it after the stream the workspace was used on has been synchronised. */
 int rmm_status_read(void *ws, int *device_status);
 
+/* Timing hook for benchmarks (the paper has no counterpart).  After rmm_profile_gemm(start, stop, n), the i-th
+ * launch of the tensor-core GEMM kernel (i < n) is bracketed by cudaEventRecord(start[i]) and
+ * cudaEventRecord(stop[i]) on its stream; the arrays hold cudaEvent_t handles created by the caller with timing
+ * enabled, and must stay alive until the hook is cleared with (NULL, NULL, 0).  Host arrays; not thread-safe.
+ * rmm_profile_gemm_count() tells how many pairs have been recorded since the hook was set. */
+int rmm_profile_gemm(void **start_events, void **stop_events, int n);
+int rmm_profile_gemm_count(void);
+
 /* Thread-local text of the last error returned on this thread ("" if none). */
 const char *rmm_last_error(void);
 

@@ -49,7 +49,7 @@ EXPORTS = ["rmm_keep_count", "rmm_score_workspace_bytes", "rmm_score", "rmm_sele
            "rmm_score_select_workspace_bytes", "rmm_score_select", "rmm_reduced_gemm_workspace_bytes",
            "rmm_reduced_gemm", "rmm_reduced_attn_workspace_bytes", "rmm_reduced_attn",
            "rmm_product_host_workspace_bytes", "rmm_product_host", "rmm_status_read", "rmm_last_error",
-           "rmm_launch_count"]
+           "rmm_launch_count", "rmm_profile_gemm", "rmm_profile_gemm_count"]
 
 _lib = None
 
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
     L.rmm_status_read.argtypes = [vp, ctypes.POINTER(i32)]
     L.rmm_last_error.restype = ctypes.c_char_p
     L.rmm_launch_count.restype = i64
+    L.rmm_profile_gemm.argtypes = [vp, vp, i32]
     _lib = L
     return L
 
@@ -150,6 +151,34 @@ def rmm_keep_count(rho: float, K: int) -> int:
 
 def rmm_launch_count() -> int:
     return int(lib().rmm_launch_count())
+
+
+class GemmTimer:
+    """Brackets the next n launches of the tensor-core GEMM kernel with CUDA events (rmm_profile_gemm)."""
+
+    def __init__(self, n: int):
+        self.n = n
+        self.start = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        self.stop = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for e in self.start + self.stop:      # torch creates the handle at the first record
+            e.record()
+        torch.cuda.synchronize()
+        self._s = (ctypes.c_void_p * n)(*[e.cuda_event for e in self.start])
+        self._e = (ctypes.c_void_p * n)(*[e.cuda_event for e in self.stop])
+
+    def __enter__(self):
+        _check(lib().rmm_profile_gemm(self._s, self._e, self.n))
+        return self
+
+    def __exit__(self, *exc):
+        self.count = int(lib().rmm_profile_gemm_count())
+        _check(lib().rmm_profile_gemm(None, None, 0))
+        return False
+
+    def times_ms(self):
+        """Durations of the recorded launches (synchronises)."""
+        torch.cuda.synchronize()
+        return [self.start[i].elapsed_time(self.stop[i]) for i in range(self.count)]
 
 
 def rmm_status_read(ws: Optional[torch.Tensor] = None, device=None) -> int:

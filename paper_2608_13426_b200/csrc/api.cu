@@ -277,6 +277,16 @@ int rmm_status_read(void *ws, int *device_status)
     return RMM_OK;
 }
 
+int rmm_profile_gemm(void **start_events, void **stop_events, int n)
+{
+    if (n < 0 || ((start_events == nullptr || stop_events == nullptr) && n != 0))
+        return fail(RMM_ERR_INVALID_ARG, "profile_gemm: need two event arrays, or NULL, NULL, 0");
+    set_gemm_profile(start_events, stop_events, n);
+    return RMM_OK;
+}
+
+int rmm_profile_gemm_count(void) { return gemm_profile_used(); }
+
 const char *rmm_last_error(void) { return t_error; }
 
 int64_t rmm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

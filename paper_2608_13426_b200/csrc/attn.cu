@@ -4,8 +4,8 @@
 //   pack Q[:, I], K_g[:, I]      -> K-major operands              (pack_cols_kernel)
 //   S~ = Q[:, I] K[:, I]^T / sqrt(Dh), fp32                        (reduced_gemm_tc_kernel, K-major B)
 //   P  = bf16(softmax(S~ + causal mask))                            (softmax_rows_kernel)
-//   rho_t < 1: score + select on P -> T; pack P[:, T]; O = P[:, T] V_g[T, :] with V rows fetched by TMA gather4
-//   rho_t = 1: O = P V_g (same kernel, P loaded in place, rows 0 .. Lk-1 of V)
+//   rho_t < 1: score + select on P -> T; pack P[:, T] and V_g[T, :]; O = P[:, T] V_g[T, :]
+//   rho_t = 1: O = P V_g (same kernel, P and V loaded in place)
 // S~ and P live in the workspace (materialised), so this form is bound by HBM traffic, not by the tensor cores.
 #include <math.h>
 
@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(kSoftmaxThreads) softmax_rows_kernel(const flo
 
 struct AttnPlan {
     int64_t kd, kt, ldd, ldt, ld_s, ld_p, hg;
-    size_t inner_bytes, off_idxf, off_idxt, off_qp, off_kp, off_s, off_p, off_pp, total;
+    size_t inner_bytes, off_idxf, off_idxt, off_qp, off_kp, off_s, off_p, off_pp, off_vp, total;
 };
 
 int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
@@ -85,10 +85,9 @@ int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
     for (int i = 0; i < 3; ++i)
         if (d->q_stride[i] % 8 || d->k_stride[i] % 8 || d->v_stride[i] % 8 || d->o_stride[i] % 8)
             return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: strides must be multiples of 8 elements");
-    // V must flatten to one 2-D [B*Hkv*Lk, Dh] tensor for the row gather
-    if (d->v_stride[2] < d->Dh || d->v_stride[1] != d->Lk * d->v_stride[2] || d->v_stride[0] != d->Hkv * d->v_stride[1])
-        return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: V must be contiguous over (batch, head, token)");
-    if (d->B * d->Hkv * d->Lk > INT32_MAX) return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: B*Hkv*Lk exceeds 2^31");
+    // V's (batch, head) pairs must form one batch axis of the tensor map used when V is read in place
+    if (d->v_stride[2] < d->Dh || d->v_stride[0] != d->Hkv * d->v_stride[1])
+        return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: V needs batch stride = Hkv * head stride");
     p->ldd = (p->kd + 7) / 8 * 8;
     p->ldt = (p->kt + 7) / 8 * 8;
     p->ld_p = (d->Lk + 7) / 8 * 8;
@@ -117,6 +116,7 @@ int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
     p->off_s = off; off += align_up((size_t)hg * d->Lq * p->ld_s * 4, 256);
     p->off_p = off; off += align_up((size_t)hg * d->Lq * p->ld_p * 2, 256);
     p->off_pp = off; off += align_up((size_t)hg * d->Lq * p->ldt * 2, 256);
+    p->off_vp = off; off += align_up((size_t)hg * p->kt * d->Dh * 2, 256);
     p->total = off;
     return RMM_OK;
 }
@@ -164,6 +164,7 @@ int rmm_reduced_attn(const rmm_attn_desc_t *d, const void *Q, const void *K, con
     __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(O);
     __nv_bfloat16 *Qp = reinterpret_cast<__nv_bfloat16 *>(w + p.off_qp), *Kp = reinterpret_cast<__nv_bfloat16 *>(w + p.off_kp);
     __nv_bfloat16 *P = reinterpret_cast<__nv_bfloat16 *>(w + p.off_p), *Pp = reinterpret_cast<__nv_bfloat16 *>(w + p.off_pp);
+    __nv_bfloat16 *Vp = reinterpret_cast<__nv_bfloat16 *>(w + p.off_vp);
     float *S = reinterpret_cast<float *>(w + p.off_s);
     const int64_t group = d->Hq / d->Hkv;
     const float scale = (float)(1.0 / sqrt((double)d->Dh));
@@ -195,6 +196,7 @@ int rmm_reduced_attn(const rmm_attn_desc_t *d, const void *Q, const void *K, con
             g1.batch = hg; g1.M = d->Lq; g1.N = d->Lk; g1.k = p.kd;
             g1.a = Qp; g1.a_ld = p.ldd; g1.a_sb = d->Lq * p.ldd;
             g1.b_kmajor = 1; g1.b = Kp; g1.b_ld = p.ldd; g1.b_sb = d->Lk * p.ldd;
+            g1.b_batches = hg; g1.b_batch_off = 0; g1.b_batch_div = 1;
             g1.y = S; g1.y_bf16 = 0; g1.y_sb = d->Lq * p.ld_s; g1.y_sr = p.ld_s;
             g1.scale = scale; g1.status = status;
             if ((rc = launch_gemm_tc_problem(g1, st)) != RMM_OK) return rc;
@@ -203,8 +205,7 @@ int rmm_reduced_attn(const rmm_attn_desc_t *d, const void *Q, const void *K, con
 
             TcProblem g2 = {};
             g2.batch = hg; g2.M = d->Lq; g2.N = d->Dh;
-            g2.b_kmajor = 0; g2.b = v; g2.b_ld = d->v_stride[2]; g2.b_rows_total = d->B * d->Hkv * d->Lk;
-            g2.b_batch_rows = d->Lk; g2.b_batch_off = b * d->Hq + h0; g2.b_batch_div = group;
+            g2.b_kmajor = 0;
             g2.y = o + b * d->o_stride[0] + h0 * d->o_stride[1]; g2.y_bf16 = 1; g2.y_sb = d->o_stride[1]; g2.y_sr = d->o_stride[2];
             g2.scale = 1.0f; g2.status = status;
             if (tok) {
@@ -215,11 +216,15 @@ int rmm_reduced_attn(const rmm_attn_desc_t *d, const void *Q, const void *K, con
                 if ((rc = launch_score_select(&pm, sp, true, p.kt, It, nullptr, nullptr, nullptr, w, st)) != RMM_OK) return rc;
                 rc = launch_pack_cols(P, hg, d->Lq, d->Lk, d->Lq * p.ld_p, p.ld_p, 0, 1, It, p.kt, p.kt, Pp, p.ldt, status, st);
                 if (rc != RMM_OK) return rc;
+                rc = launch_pack_rows(v + b * d->v_stride[0], hg, d->Lk, d->Dh, d->v_stride[1], d->v_stride[2], h0, group, It, p.kt,
+                                      p.kt, Vp, d->Dh, status, st);
+                if (rc != RMM_OK) return rc;
                 g2.k = p.kt; g2.a = Pp; g2.a_ld = p.ldt; g2.a_sb = d->Lq * p.ldt;
-                g2.idx = It; g2.idx_stride = p.kt;
+                g2.b = Vp; g2.b_ld = d->Dh; g2.b_sb = p.kt * d->Dh; g2.b_batches = hg; g2.b_batch_off = 0; g2.b_batch_div = 1;
             } else {
                 g2.k = d->Lk; g2.a = P; g2.a_ld = p.ld_p; g2.a_sb = d->Lq * p.ld_p;
-                g2.idx = nullptr; g2.idx_stride = 0;
+                g2.b = v; g2.b_ld = d->v_stride[2]; g2.b_sb = d->v_stride[1]; g2.b_batches = d->B * d->Hkv;
+                g2.b_batch_off = b * d->Hq + h0; g2.b_batch_div = group;
             }
             if ((rc = launch_gemm_tc_problem(g2, st)) != RMM_OK) return rc;
         }

@@ -53,7 +53,7 @@ int launch_gemm_simt(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx,
 
 // Tensor-core path (tcgen05, TMEM accumulators).  Operands must satisfy tc_eligible().
 struct TcPlan {
-    int b_kmajor;       // 0: B rows (contraction slices) contiguous, gathered by TMA; 1: B is K-contiguous, packed first
+    int b_kmajor;       // 0: B rows (contraction slices) contiguous, kept rows copied; 1: B is K-contiguous, packed like A
     int64_t ldp;        // leading dimension of the packed operands (multiple of 8)
     size_t off_ap, off_bp, total_bytes;
 };
@@ -67,11 +67,9 @@ struct TcProblem {
     const __nv_bfloat16 *a;  // K-major A [batch, M, a_ld]: the kept columns are its first k columns
     int64_t a_ld, a_sb;      // row pitch and batch stride in elements (multiples of 8)
     int b_kmajor;
-    const __nv_bfloat16 *b;  // K-major: [batch, N, b_ld] (kept columns first); MN-major: 2-D [b_rows_total, N], pitch b_ld
-    int64_t b_ld, b_sb, b_rows_total;
-    const int32_t *idx;      // MN-major B: kept rows per batch entry (NULL = rows 0 .. k-1), lists idx_stride apart
-    int64_t idx_stride;
-    int64_t b_batch_rows, b_batch_off, b_batch_div;  // MN-major B: first row of entry i = ((i + off) / div) * rows
+    const __nv_bfloat16 *b;  // K-major: [b_batches, N, b_ld] (kept columns first); MN-major: [b_batches, k, b_ld], rows = kept slices
+    int64_t b_ld, b_sb, b_batches;
+    int64_t b_batch_off, b_batch_div;  // B batch entry used by problem i = min((i + off) / div, b_batches - 1)
     void *y;
     int y_bf16;
     int64_t y_sb, y_sr;
@@ -79,11 +77,19 @@ struct TcProblem {
     int *status;
 };
 int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream);
+void set_gemm_profile(void **start, void **stop, int n);
+int gemm_profile_used();
 
 // Gather columns: dst[b, r, j] = src[sb, r, idx[b, j]] for j < k with source batch sb = (b + b_off) / b_div
 // (dst row pitch ld_dst >= k; columns k..ld_dst are zeroed).  bf16 only.  idx_stride = elements between the
 // index lists of two batch entries.
 int launch_pack_cols(const __nv_bfloat16 *src, int64_t batch, int64_t rows, int64_t K, int64_t s_batch, int64_t s_row,
+                     int64_t b_off, int64_t b_div, const int32_t *idx, int64_t idx_stride, int64_t k,
+                     __nv_bfloat16 *dst, int64_t ld_dst, int *status, cudaStream_t stream);
+
+// Gather rows: dst[b, j, 0:n] = src[sb, idx[b, j], 0:n] for j < k (NULL idx: rows 0 .. k-1), 16-byte vectors:
+// n, both pitches and both bases must be multiples of 8 elements.  Source batch sb = (b + b_off) / b_div.
+int launch_pack_rows(const __nv_bfloat16 *src, int64_t batch, int64_t K, int64_t n, int64_t s_batch, int64_t s_row,
                      int64_t b_off, int64_t b_div, const int32_t *idx, int64_t idx_stride, int64_t k,
                      __nv_bfloat16 *dst, int64_t ld_dst, int *status, cudaStream_t stream);
 

@@ -4,10 +4,11 @@
 //   A[:, I]   packed once by pack_cols_kernel into Ap [b, M, ldp] (K-major); TMA 2-D/3-D tile loads
 //             of 128 rows x 64 kept columns into 128-byte-swizzled shared memory.  Columns beyond k
 //             are outside the tensor map and arrive as zeros, so k needs no padding.
-//   B[I, :]   never packed when B's contraction slices (rows) are contiguous: the producer warp reads
-//             the index list and fetches the kept rows straight from B with TMA gather4 (4 arbitrary rows
-//             x 64 columns per instruction), giving an MN-major swizzled operand.
-//             When B is K-contiguous (K^T in attention) it is packed like A and loaded as K-major tiles.
+//   B[I, :]   when B's contraction slices (rows) are contiguous, pack_rows_kernel copies the kept rows into
+//             Bp [b, k, N] and 64 x 64 tiles of it are loaded as an MN-major swizzled operand; when B is
+//             K-contiguous (K^T in attention) it is packed like A and loaded as K-major tiles.  (Fetching the
+//             kept rows inside the producer with TMA gather4 was measured first: at 512 bytes per instruction
+//             the copy engine sustained about one instruction per 70 clocks, 2.5x slower than this form.)
 //   MMA       one elected thread issues tcgen05.mma (bf16 x bf16 -> fp32, M=128, N=BN, K=16 per instruction);
 //             accumulators live in TMEM, double buffered (2 x BN columns) so that the epilogue of one tile
 //             overlaps the main loop of the next.
@@ -97,23 +98,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
-        : "memory");
-}
-// Four rows (y0..y3) of a 2-D tensor, columns x .. x+box-1, land as four consecutive shared-memory rows.
-__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap *map, int x, int y0, int y1, int y2, int y3,
-                                            uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3), "r"(bar)
-        : "memory");
-}
-
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols)
 {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
@@ -170,10 +154,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 
 struct TcArgs {
     int64_t M, N, k, batch;
-    // MN-major B: first row of batch entry i in the flattened 2-D tensor = ((i + b_batch_off) / b_batch_div) * b_batch_rows
-    int64_t b_batch_rows, b_batch_off, b_batch_div;
-    const int32_t *idx;     // kept rows, one list per batch entry idx_stride apart; NULL = rows 0 .. k-1
-    int64_t idx_stride;
+    int64_t b_batch_off, b_batch_div, b_batches;  // B batch entry of problem i = min((i + off) / div, b_batches - 1)
     void *Y;
     int64_t y_sb, y_sr;     // element strides of Y (column stride 1)
     float scale;
@@ -234,62 +215,33 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     if (warp == 0) {
         // ---------------------------------------------------------------- producer
         uint32_t it = 0;
-        for (int64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
             const int tn = (int)(tile % a.tiles_n);
             const int tm = (int)((tile / a.tiles_n) % a.tiles_m);
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
-            const int32_t *ix = a.idx != nullptr ? a.idx + b * a.idx_stride : nullptr;
-            const int row_base = (int)(((b + a.b_batch_off) / a.b_batch_div) * a.b_batch_rows);
-            auto kept_row = [&](int64_t j) -> int {
-                if (j >= a.k) j = a.k - 1;  // positions past k repeat the last kept row; A supplies zeros there
-                return ix != nullptr ? __ldg(ix + j) : (int)j;
-            };
-            // kept rows of B this lane fetches in each stage: row group g = lane % 16, i.e. positions 4g .. 4g+3
-            const int g = lane & 15;
-            int rows_next[4];
-            bool ok = true;
-            if constexpr (!B_KMAJOR) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) rows_next[i] = kept_row(4 * g + i);
-            }
+            int64_t bb = (b + a.b_batch_off) / a.b_batch_div;
+            if (bb >= a.b_batches) bb = a.b_batches - 1;
             for (int kb = 0; kb < num_kb; ++kb, ++it) {
                 const int s = it % kStages;
                 const uint32_t ph = (it / kStages) & 1u;
-                int rows[4];
-                if constexpr (!B_KMAJOR) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) rows[i] = rows_next[i];
-                    if (kb + 1 < num_kb) {  // prefetch the next stage's indices before blocking on the ring
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) rows_next[i] = kept_row((int64_t)(kb + 1) * BK + 4 * g + i);
-                    }
-                }
                 if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status)) { ok = false; break; }
-                const uint32_t sa = base + s * L::kStageBytes;
-                const uint32_t sb = sa + L::kABytes;
                 if (lane == 0) {
+                    const uint32_t sa = base + s * L::kStageBytes;
+                    const uint32_t sb = sa + L::kABytes;
                     mbar_arrive_expect_tx(full_bar(s), L::kStageBytes);
                     tma_load_3d(sa, &map_a, kb * BK, tm * BM, (int)b, full_bar(s));
-                    if constexpr (B_KMAJOR) tma_load_3d(sb, &map_b, kb * BK, tn * BN, (int)b, full_bar(s));
+                    if constexpr (B_KMAJOR) {
+                        tma_load_3d(sb, &map_b, kb * BK, tn * BN, (int)bb, full_bar(s));
+                    } else {
+                        // 64 contraction rows x 64 columns per load; rows past k read as zeros
+#pragma unroll
+                        for (int c = 0; c < BN / 64; ++c)
+                            tma_load_3d(sb + c * (BK * 128), &map_b, tn * BN + c * 64, kb * BK, (int)bb, full_bar(s));
+                    }
                 }
                 __syncwarp();
-                if constexpr (!B_KMAJOR) {
-                    if (ix == nullptr) {
-                        // rows 0 .. k-1 in order: plain tile loads of 64 rows x 64 columns (rows past the tensor read as zeros)
-                        if (lane < BN / 64)
-                            tma_load_2d(sb + lane * (BK * 128), &map_b, tn * BN + lane * 64, row_base + kb * BK, full_bar(s));
-                        continue;
-                    }
-                    // BN/64 column chunks x 16 row groups = BN/4 gathers per stage, BN/128 per lane
-#pragma unroll
-                    for (int c = lane >> 4; c < BN / 64; c += 2) {
-                        const uint32_t dst = sb + c * (BK * 128) + g * 512;
-                        tma_gather4(dst, &map_b, tn * BN + c * 64, row_base + rows[0], row_base + rows[1],
-                                    row_base + rows[2], row_base + rows[3], full_bar(s));
-                    }
-                }
             }
-            if (!ok) break;
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
@@ -446,6 +398,12 @@ int sm_count()
     return n;
 }
 
+// Optional profiling hook (rmm_profile_gemm): events recorded around each launch of the GEMM kernel.
+struct GemmProfile {
+    cudaEvent_t *start = nullptr, *stop = nullptr;
+    int capacity = 0, used = 0;
+} g_profile;
+
 template <int BN, bool B_KMAJOR, bool OUT_BF16>
 int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const TcArgs &a, cudaStream_t stream)
 {
@@ -458,11 +416,23 @@ int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const TcArgs &a
     }
     int64_t tiles = a.batch * a.tiles_m * a.tiles_n;
     int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+    const bool prof = g_profile.used < g_profile.capacity;
+    if (prof) cudaEventRecord(g_profile.start[g_profile.used], stream);
     kern<<<grid, kThreadsTc, SmemLayout<BN>::kTotal, stream>>>(ma, mb, a);
+    if (prof) cudaEventRecord(g_profile.stop[g_profile.used++], stream);
     return check_launch("reduced_gemm_tc_kernel");
 }
 
 }  // namespace
+
+void set_gemm_profile(void **start, void **stop, int n)
+{
+    g_profile.start = reinterpret_cast<cudaEvent_t *>(start);
+    g_profile.stop = reinterpret_cast<cudaEvent_t *>(stop);
+    g_profile.capacity = (start != nullptr && stop != nullptr) ? n : 0;
+    g_profile.used = 0;
+}
+int gemm_profile_used() { return g_profile.used; }
 
 bool tc_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y, TcPlan *plan)
 {
@@ -473,14 +443,12 @@ bool tc_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_ma
     if (Y->stride_col != 1 || !al16(Y->ptr)) return false;
     const int64_t yq = Y->dtype == RMM_BF16 ? 8 : 4;
     if (Y->stride_row % yq != 0 || Y->stride_batch % yq != 0) return false;
-    if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX || batch > INT32_MAX) return false;
+    if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX || batch > 65535) return false;
     int b_kmajor;
-    if (B->stride_col == 1 && B->rows > 0) {
-        // rows of B contiguous: gathered by TMA straight from B, which must flatten to one 2-D tensor
+    if (B->stride_col == 1) {
+        // rows of B (contraction slices) contiguous: row copies of 16-byte vectors
         b_kmajor = 0;
-        if (!al16(B->ptr) || B->stride_row % 8 != 0 || B->stride_row < N) return false;
-        if (B->stride_batch != 0 && B->stride_batch != K * B->stride_row) return false;
-        if ((B->stride_batch == 0 ? K : batch * K) > INT32_MAX) return false;
+        if (!al16(B->ptr) || B->stride_row % 8 != 0 || B->stride_batch % 8 != 0 || N % 8 != 0) return false;
     } else if (B->stride_row == 1) {
         b_kmajor = 1;  // K-contiguous: packed like A
     } else {
@@ -493,7 +461,7 @@ bool tc_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_ma
         plan->off_ap = off;
         off += align_up((size_t)batch * M * plan->ldp * 2, 256);
         plan->off_bp = off;
-        if (b_kmajor) off += align_up((size_t)batch * N * plan->ldp * 2, 256);
+        off += align_up(b_kmajor ? (size_t)batch * N * plan->ldp * 2 : (size_t)batch * k * N * 2, 256);
         plan->total_bytes = off;
     }
     return true;
@@ -513,23 +481,23 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     const int BN = p.N <= 128 ? 128 : 256;
     TcArgs a;
     a.M = p.M; a.N = p.N; a.k = p.k; a.batch = p.batch;
-    a.idx = p.idx; a.idx_stride = p.idx_stride;
-    a.b_batch_rows = p.b_batch_rows; a.b_batch_off = p.b_batch_off; a.b_batch_div = p.b_batch_div > 0 ? p.b_batch_div : 1;
+    a.b_batch_off = p.b_batch_off; a.b_batch_div = p.b_batch_div > 0 ? p.b_batch_div : 1; a.b_batches = p.b_batches;
     a.Y = p.y; a.y_sb = p.y_sb; a.y_sr = p.y_sr;
     a.scale = p.scale;
     a.tiles_m = (int)ceil_div(p.M, BM);
     a.tiles_n = (int)ceil_div(p.N, BN);
     a.status = p.status;
+    const uint64_t b_sb = p.b_batches > 1 ? (uint64_t)p.b_sb * 2 : (uint64_t)p.b_ld * 2 * (uint64_t)(p.b_kmajor ? p.N : p.k);
     if (p.b_kmajor) {
-        uint64_t dims[3] = {(uint64_t)p.k, (uint64_t)p.N, (uint64_t)p.batch};
-        uint64_t st[2] = {(uint64_t)p.b_ld * 2, (uint64_t)p.b_sb * 2};
+        uint64_t dims[3] = {(uint64_t)p.k, (uint64_t)p.N, (uint64_t)p.b_batches};
+        uint64_t st[2] = {(uint64_t)p.b_ld * 2, b_sb};
         uint32_t box[3] = {BK, (uint32_t)BN, 1};
         rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 3, dims, st, box);
     } else {
-        uint64_t dims[2] = {(uint64_t)p.N, (uint64_t)p.b_rows_total};
-        uint64_t st[1] = {(uint64_t)p.b_ld * 2};
-        uint32_t box[2] = {64, p.idx != nullptr ? 1u : (uint32_t)BK};  // one row per gathered row, or a 64-row tile
-        rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 2, dims, st, box);
+        uint64_t dims[3] = {(uint64_t)p.N, (uint64_t)p.k, (uint64_t)p.b_batches};
+        uint64_t st[2] = {(uint64_t)p.b_ld * 2, b_sb};
+        uint32_t box[3] = {64, BK, 1};
+        rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 3, dims, st, box);
     }
     if (rc != RMM_OK) return rc;
     const bool out_bf16 = p.y_bf16 != 0;
@@ -547,38 +515,39 @@ int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, i
     char *w = static_cast<char *>(ws);
     int *status = &reinterpret_cast<WsHeader *>(w)->status;
     const int64_t M = A->rows, K = A->cols, N = B->cols, batch = A->batch;
-    __nv_bfloat16 *Ap = reinterpret_cast<__nv_bfloat16 *>(w + plan.off_ap);
+    const __nv_bfloat16 *a_src = static_cast<const __nv_bfloat16 *>(A->ptr), *b_src = static_cast<const __nv_bfloat16 *>(B->ptr);
+    __nv_bfloat16 *Ap = reinterpret_cast<__nv_bfloat16 *>(w + plan.off_ap), *Bp = reinterpret_cast<__nv_bfloat16 *>(w + plan.off_bp);
     int rc;
     TcProblem p = {};
     p.batch = batch; p.M = M; p.N = N; p.k = k;
-    // the unreduced product (idx NULL, k == K) on a TMA-loadable A needs no gather at all
-    const bool a_in_place = idx == nullptr && reinterpret_cast<uintptr_t>(A->ptr) % 16 == 0 && A->stride_row % 8 == 0 &&
-                            A->stride_batch % 8 == 0 && !plan.b_kmajor;
-    if (a_in_place) {
-        p.a = static_cast<const __nv_bfloat16 *>(A->ptr); p.a_ld = A->stride_row; p.a_sb = batch > 1 ? A->stride_batch : M * A->stride_row;
-    } else {
-        rc = launch_pack_cols(static_cast<const __nv_bfloat16 *>(A->ptr), batch, M, K, A->stride_batch, A->stride_row, 0, 1,
-                              idx, k, k, Ap, plan.ldp, status, stream);
-        if (rc != RMM_OK) return rc;
-        p.a = Ap; p.a_ld = plan.ldp; p.a_sb = M * plan.ldp;
-    }
     p.b_kmajor = plan.b_kmajor;
     p.y = Y->ptr; p.y_bf16 = Y->dtype == RMM_BF16; p.y_sb = Y->stride_batch; p.y_sr = Y->stride_row;
     p.scale = scale; p.status = status;
+    p.b_batch_off = 0; p.b_batch_div = 1; p.b_batches = batch;
+
+    // the unreduced product (idx NULL, k == K) on TMA-loadable operands needs no gather at all
+    const bool in_place = idx == nullptr && !plan.b_kmajor && reinterpret_cast<uintptr_t>(A->ptr) % 16 == 0 &&
+                          A->stride_row % 8 == 0 && A->stride_batch % 8 == 0;
+    if (in_place) {
+        p.a = a_src; p.a_ld = A->stride_row; p.a_sb = batch > 1 ? A->stride_batch : M * A->stride_row;
+        p.b = b_src; p.b_ld = B->stride_row;
+        if (B->stride_batch == 0) { p.b_batches = 1; p.b_sb = 0; }
+        else { p.b_sb = B->stride_batch; }
+        return launch_gemm_tc_problem(p, stream);
+    }
+    rc = launch_pack_cols(a_src, batch, M, K, A->stride_batch, A->stride_row, 0, 1, idx, k, k, Ap, plan.ldp, status, stream);
+    if (rc != RMM_OK) return rc;
+    p.a = Ap; p.a_ld = plan.ldp; p.a_sb = M * plan.ldp;
     if (plan.b_kmajor) {
         // B is K-contiguous ([N, K] in memory): pack B[idx, :]^T into Bp [batch, N, ldp]; a shared B
         // (stride_batch 0) is packed once per index set
-        __nv_bfloat16 *Bp = reinterpret_cast<__nv_bfloat16 *>(w + plan.off_bp);
-        rc = launch_pack_cols(static_cast<const __nv_bfloat16 *>(B->ptr), batch, N, K, B->stride_batch, B->stride_col, 0, 1,
-                              idx, k, k, Bp, plan.ldp, status, stream);
+        rc = launch_pack_cols(b_src, batch, N, K, B->stride_batch, B->stride_col, 0, 1, idx, k, k, Bp, plan.ldp, status, stream);
         if (rc != RMM_OK) return rc;
         p.b = Bp; p.b_ld = plan.ldp; p.b_sb = N * plan.ldp;
     } else {
-        const int64_t b_batches = B->stride_batch == 0 ? 1 : batch;
-        p.b = static_cast<const __nv_bfloat16 *>(B->ptr); p.b_ld = B->stride_row;
-        p.b_rows_total = b_batches * K;
-        p.idx = idx; p.idx_stride = k;
-        p.b_batch_rows = B->stride_batch == 0 ? 0 : K; p.b_batch_off = 0; p.b_batch_div = 1;
+        rc = launch_pack_rows(b_src, batch, K, N, B->stride_batch, B->stride_row, 0, 1, idx, k, k, Bp, N, status, stream);
+        if (rc != RMM_OK) return rc;
+        p.b = Bp; p.b_ld = N; p.b_sb = k * N;
     }
     return launch_gemm_tc_problem(p, stream);
 }

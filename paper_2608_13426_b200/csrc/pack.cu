@@ -12,7 +12,8 @@ namespace rmm {
 namespace {
 
 constexpr int kWarps = 8;
-constexpr int kRowsPerBlock = 32;
+constexpr int kRowsPerBlock = 8;   // rows per warp, all in flight at once (the pass is latency-bound otherwise)
+constexpr int kRowVecThreads = 256;
 
 __global__ void __launch_bounds__(kWarps * 32) pack_cols_kernel(const __nv_bfloat16 *__restrict__ src, int64_t rows,
                                                                 int64_t K, int64_t s_batch, int64_t s_row,
@@ -49,21 +50,61 @@ __global__ void __launch_bounds__(kWarps * 32) pack_cols_kernel(const __nv_bfloa
     unsigned *d32 = reinterpret_cast<unsigned *>(dst + b * rows * ld_dst);
     const int64_t r_begin = (int64_t)blockIdx.y * kRowsPerBlock;
     const int64_t r_end = min(rows, r_begin + kRowsPerBlock);
-#pragma unroll 2
-    for (int64_t r = r_begin; r < r_end; ++r) {
-        const unsigned short *row = s16 + r * s_row;
-        unsigned out[4];
+    unsigned out[kRowsPerBlock][4];
+#pragma unroll
+    for (int rr = 0; rr < kRowsPerBlock; ++rr) {
+        const int64_t r = r_begin + rr;
+        const unsigned short *row = s16 + (r < r_end ? r : r_begin) * s_row;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             unsigned lo = c[2 * i] >= 0 ? (unsigned)__ldg(row + c[2 * i]) : 0u;
             unsigned hi = c[2 * i + 1] >= 0 ? (unsigned)__ldg(row + c[2 * i + 1]) : 0u;
-            out[i] = lo | (hi << 16);
+            out[rr][i] = lo | (hi << 16);
         }
+    }
+#pragma unroll
+    for (int rr = 0; rr < kRowsPerBlock; ++rr) {
+        const int64_t r = r_begin + rr;
+        if (r >= r_end) break;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             int64_t j = j0 + 64 * i + 2 * lane;
-            if (j < ld_dst) d32[(r * ld_dst + j) >> 1] = out[i];
+            if (j < ld_dst) d32[(r * ld_dst + j) >> 1] = out[rr][i];
         }
+    }
+}
+
+// Row gather with 16-byte vectors: one block copies 4 kept rows.
+__global__ void __launch_bounds__(kRowVecThreads) pack_rows_kernel(const uint4 *__restrict__ src, int64_t K, int64_t nvec,
+                                                                   int64_t s_batch_v, int64_t s_row_v, int64_t b_off,
+                                                                   int64_t b_div, const int32_t *__restrict__ idx,
+                                                                   int64_t idx_stride, int64_t k, uint4 *__restrict__ dst,
+                                                                   int64_t ld_dst_v, int *status)
+{
+    const int64_t b = blockIdx.z;
+    const int64_t j0 = (int64_t)blockIdx.y * 4;
+    const uint4 *sbase = src + ((b + b_off) / b_div) * s_batch_v;
+    uint4 *dbase = dst + (b * k) * ld_dst_v;
+    int rows[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int v = -1;
+        if (j0 + i < k) {
+            v = idx != nullptr ? __ldg(idx + b * idx_stride + j0 + i) : (int)(j0 + i);
+            if (v < 0 || v >= K) {
+                if (threadIdx.x == 0) atomicExch(status, (int)RMM_ERR_BOUNDS);
+                v = -2;  // write zeros
+            }
+        }
+        rows[i] = v;
+    }
+    for (int64_t c = (int64_t)blockIdx.x * kRowVecThreads + threadIdx.x; c < nvec; c += (int64_t)gridDim.x * kRowVecThreads) {
+        uint4 v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] = rows[i] >= 0 ? __ldg(sbase + rows[i] * s_row_v + c) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (rows[i] != -1) dbase[(j0 + i) * ld_dst_v + c] = v[i];
     }
 }
 
@@ -79,6 +120,23 @@ int launch_pack_cols(const __nv_bfloat16 *src, int64_t batch, int64_t rows, int6
     pack_cols_kernel<<<grid, kWarps * 32, 0, stream>>>(src, rows, K, s_batch, s_row, b_off, b_div > 0 ? b_div : 1, idx, idx_stride, k, dst,
                                                                ld_dst, status);
     return check_launch("pack_cols_kernel");
+}
+
+int launch_pack_rows(const __nv_bfloat16 *src, int64_t batch, int64_t K, int64_t n, int64_t s_batch, int64_t s_row,
+                     int64_t b_off, int64_t b_div, const int32_t *idx, int64_t idx_stride, int64_t k,
+                     __nv_bfloat16 *dst, int64_t ld_dst, int *status, cudaStream_t stream)
+{
+    if (n % 8 || s_batch % 8 || s_row % 8 || ld_dst % 8 || reinterpret_cast<uintptr_t>(src) % 16 || reinterpret_cast<uintptr_t>(dst) % 16)
+        return fail(RMM_ERR_UNSUPPORTED, "pack_rows: operands must be 16-byte aligned with pitches that are multiples of 8");
+    const int64_t nvec = n / 8;
+    int64_t gx = ceil_div(nvec, kRowVecThreads);
+    if (gx > 8) gx = 8;
+    dim3 grid((unsigned)gx, (unsigned)ceil_div(k, 4), (unsigned)batch);
+    if (grid.y > 65535u || grid.z > 65535u) return fail(RMM_ERR_UNSUPPORTED, "pack_rows: k/4 or batch exceeds 65535");
+    pack_rows_kernel<<<grid, kRowVecThreads, 0, stream>>>(reinterpret_cast<const uint4 *>(src), K, nvec, s_batch / 8, s_row / 8, b_off,
+                                                         b_div > 0 ? b_div : 1, idx, idx_stride, k,
+                                                         reinterpret_cast<uint4 *>(dst), ld_dst / 8, status);
+    return check_launch("pack_rows_kernel");
 }
 
 }  // namespace rmm

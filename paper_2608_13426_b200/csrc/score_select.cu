@@ -18,8 +18,8 @@ namespace rmm {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kUnroll = 4;       // rows in flight per thread
-constexpr int kFlushEvery = 4;   // loop trips between fp32 -> fp64 flushes (kUnroll * kFlushEvery = 16 terms)
+constexpr int kUnroll = 8;       // rows in flight per thread
+constexpr int kFlushEvery = 2;   // loop trips between fp32 -> fp64 flushes (kUnroll * kFlushEvery = 16 terms)
 constexpr int kFusedSelectMax = 8192;    // largest K whose select runs in the score kernel's tail (32 KB key cache)
 constexpr int kCachedSelectMax = 49152;  // largest K the stand-alone select kernel caches in shared memory (192 KB)
 
@@ -53,65 +53,114 @@ __device__ __forceinline__ float key_value(unsigned u)
 __device__ void block_select(const float *keys, int K, int k, int32_t *idx, float *retained, SelectSmem &sm,
                              unsigned *kcache)
 {
-    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
-    unsigned prefix = 0, mask = 0, remaining = (unsigned)k;
-    if (kcache != nullptr) {
-#pragma unroll 8
-        for (int j = tid; j < K; j += nthr) kcache[j] = key_image(__ldcg(keys + j));
-        __syncthreads();
-    }
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     auto image = [&](int j) -> unsigned { return kcache != nullptr ? kcache[j] : key_image(__ldcg(keys + j)); };
 
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int i = tid; i < 256; i += nthr) sm.hist[i] = 0;
-        __syncthreads();
-        for (int j0 = 0; j0 < K; j0 += nthr) {
-            int j = j0 + tid;
-            bool live = false;
-            unsigned bin = 0;
+    // fetch the keys once, eight independent loads at a time so that their latencies overlap; find the
+    // bits all of them share, so that the first radix digit is well spread
+    unsigned lo = 0xffffffffu, hi = 0u;
+    for (int j0 = tid; j0 < K; j0 += 8 * nthr) {
+        unsigned u[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int j = j0 + i * nthr;
+            u[i] = j < K ? key_image(__ldcg(keys + j)) : 0u;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int j = j0 + i * nthr;
             if (j < K) {
-                unsigned u = image(j);
-                live = (u & mask) == prefix;
-                bin = (u >> shift) & 255u;
-            }
-            // one shared-memory atomic per distinct bin per warp
-            unsigned act = __ballot_sync(0xffffffffu, live);
-            if (live) {
-                unsigned peers = __match_any_sync(act, bin);
-                if (lane == __ffs(peers) - 1) atomicAdd(&sm.hist[bin], (unsigned)__popc(peers));
+                if (kcache != nullptr) kcache[j] = u[i];
+                lo = min(lo, u[i]);
+                hi = max(hi, u[i]);
             }
         }
-        __syncthreads();
-        if (warp == 0) {
-            // lane l owns bins 255-8l .. 248-8l (descending); find where the count from the top crosses `remaining`
-            unsigned mine = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) mine += sm.hist[255 - 8 * lane - i];
-            unsigned incl = mine;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                unsigned v = __shfl_up_sync(0xffffffffu, incl, d);
-                if (lane >= d) incl += v;
-            }
-            unsigned excl = incl - mine;
-            if (excl < remaining && remaining <= incl) {
-                unsigned above = excl;
-                for (int i = 0; i < 8; ++i) {
-                    unsigned h = sm.hist[255 - 8 * lane - i];
-                    if (remaining <= above + h) {
-                        sm.bin = 255 - 8 * lane - i;
-                        sm.remaining = remaining - above;
-                        break;
-                    }
-                    above += h;
+    }
+    lo = __reduce_min_sync(0xffffffffu, lo);
+    hi = __reduce_max_sync(0xffffffffu, hi);
+    if (lane == 0) {
+        sm.hist[warp] = lo;
+        sm.hist[32 + warp] = hi;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        unsigned l = lane < nwarp ? sm.hist[lane] : 0xffffffffu, h = lane < nwarp ? sm.hist[32 + lane] : 0u;
+        l = __reduce_min_sync(0xffffffffu, l);
+        h = __reduce_max_sync(0xffffffffu, h);
+        if (lane == 0) {
+            sm.bin = l;
+            sm.remaining = h;
+        }
+    }
+    __syncthreads();
+    lo = sm.bin;
+    hi = sm.remaining;
+    __syncthreads();
+
+    const int lcp = (lo ^ hi) ? __clz(lo ^ hi) : 32;  // leading bits common to every key
+    unsigned mask = lcp == 0 ? 0u : (lcp == 32 ? 0xffffffffu : ~(0xffffffffu >> lcp));
+    unsigned prefix = hi & mask;
+    unsigned remaining = (unsigned)k;
+
+    if (lcp < 32) {
+        int shift = 32 - lcp - 8;
+        if (shift < 0) shift = 0;
+        for (;;) {
+            for (int i = tid; i < 256; i += nthr) sm.hist[i] = 0;
+            __syncthreads();
+            for (int j0 = 0; j0 < K; j0 += nthr) {
+                int j = j0 + tid;
+                bool live = false;
+                unsigned bin = 0;
+                if (j < K) {
+                    unsigned u = image(j);
+                    live = (u & mask) == prefix;
+                    bin = (u >> shift) & 255u;
+                }
+                // lanes that agree with the first live lane are counted by it in one atomic; the others add their own
+                unsigned act = __ballot_sync(0xffffffffu, live);
+                if (act != 0u) {
+                    const int leader = __ffs(act) - 1;
+                    const unsigned lbin = __shfl_sync(0xffffffffu, bin, leader);
+                    const unsigned agree = __ballot_sync(0xffffffffu, live && bin == lbin);
+                    if (lane == leader) atomicAdd(&sm.hist[lbin], (unsigned)__popc(agree));
+                    else if (live && bin != lbin) atomicAdd(&sm.hist[bin], 1u);
                 }
             }
+            __syncthreads();
+            if (warp == 0) {
+                // lane l owns bins 255-8l .. 248-8l (descending); find where the count from the top crosses `remaining`
+                unsigned mine = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) mine += sm.hist[255 - 8 * lane - i];
+                unsigned incl = mine;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    unsigned v = __shfl_up_sync(0xffffffffu, incl, d);
+                    if (lane >= d) incl += v;
+                }
+                unsigned excl = incl - mine;
+                if (excl < remaining && remaining <= incl) {
+                    unsigned above = excl;
+                    for (int i = 0; i < 8; ++i) {
+                        unsigned h = sm.hist[255 - 8 * lane - i];
+                        if (remaining <= above + h) {
+                            sm.bin = 255 - 8 * lane - i;
+                            sm.remaining = remaining - above;
+                            break;
+                        }
+                        above += h;
+                    }
+                }
+            }
+            __syncthreads();
+            prefix = (prefix & ~(255u << shift)) | (sm.bin << shift);
+            mask |= 255u << shift;
+            remaining = sm.remaining;
+            __syncthreads();
+            if (shift == 0) break;
+            shift = shift >= 8 ? shift - 8 : 0;
         }
-        __syncthreads();
-        prefix |= sm.bin << shift;
-        mask |= 255u << shift;
-        remaining = sm.remaining;
-        __syncthreads();
     }
     const unsigned tau = prefix;          // image of the k-th largest key
     const unsigned need_eq = remaining;   // how many keys equal to tau are kept (lowest indices first)
@@ -320,7 +369,14 @@ __global__ void __launch_bounds__(kThreads) score_select_kernel(ScoreArgs a)
             __threadfence();
             if (owner) {
                 colsum = 0.0;
-                for (int s = 0; s < a.row_splits; ++s) colsum += __ldcg(&a.partials[(b * a.row_splits + s) * a.n + mycol]);
+                for (int s0 = 0; s0 < a.row_splits; s0 += 8) {  // eight independent loads at a time, summed in split order
+                    double v[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        v[i] = s0 + i < a.row_splits ? __ldcg(&a.partials[(b * a.row_splits + s0 + i) * a.n + mycol]) : 0.0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) colsum += v[i];
+                }
             }
         }
     }
