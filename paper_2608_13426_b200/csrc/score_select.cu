@@ -23,13 +23,14 @@ constexpr int kFlushEvery = 2;   // loop trips between fp32 -> fp64 flushes (kUn
 constexpr int kFusedSelectMax = 8192;    // largest K whose select runs in the score kernel's tail (32 KB key cache)
 constexpr int kCachedSelectMax = 49152;  // largest K the stand-alone select kernel caches in shared memory (192 KB)
 
+constexpr int kBins = 2048;      // first radix digit: up to 11 bits
+constexpr int kCandMax = 1024;   // keys that share the threshold's first digit are finished from this list
+
 struct SelectSmem {
-    unsigned hist[256];
-    unsigned long long warp_tot[32];
-    unsigned long long carry;
-    unsigned long long round_total;
-    unsigned bin;
-    unsigned remaining;
+    unsigned hist[kBins];
+    unsigned cand[kCandMax];
+    unsigned warp_a[32], warp_b[32];
+    unsigned bin, remaining, count;
     double red[64];
 };
 
@@ -38,26 +39,70 @@ __device__ __forceinline__ unsigned key_image(float f)
     unsigned u = __float_as_uint(f);
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // total order: larger float <=> larger image
 }
-
-// Block-wide top-k of keys[0..K): writes idx[0..k) ascending, optional retained fraction.
-// Every thread of the block must call it; keys are read through L2 (they may have just been
-// written by other blocks).
-//
-// kcache, if not NULL, is shared memory for K key images: the keys are then fetched once (independent
-// loads, so their latencies overlap) and every later pass runs out of shared memory.
 __device__ __forceinline__ float key_value(unsigned u)
 {
     return __uint_as_float((u & 0x80000000u) ? (u ^ 0x80000000u) : ~u);
 }
 
-__device__ void block_select(const float *keys, int K, int k, int32_t *idx, float *retained, SelectSmem &sm,
-                             unsigned *kcache)
+// Among hist[0..nbins) find the bin b such that (keys in bins above b) < remaining <= (keys in bins >= b); publish it
+// in sm.bin and the count still wanted inside that bin in sm.remaining.  Whole block; hist complete before the call.
+__device__ __forceinline__ void find_bin(SelectSmem &sm, int nbins, unsigned remaining)
+{
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+    const int per = nbins >= nthr ? nbins / nthr : 1;  // bins owned by a thread, taken from the top down
+    const int first = nbins - 1 - tid * per;             // highest bin of this thread (negative: owns none)
+    unsigned mine = 0;
+    if (first >= 0)
+        for (int i = 0; i < per; ++i) mine += sm.hist[first - i];
+    unsigned incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        unsigned v = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += v;
+    }
+    if (lane == 31) sm.warp_a[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned w = lane < nwarp ? sm.warp_a[lane] : 0u, wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            unsigned v = __shfl_up_sync(0xffffffffu, wi, d);
+            if (lane >= d) wi += v;
+        }
+        sm.warp_b[lane] = wi - w;
+    }
+    __syncthreads();
+    incl += sm.warp_b[warp];
+    unsigned above = incl - mine;
+    if (first >= 0 && above < remaining && remaining <= incl) {
+        for (int i = 0; i < per; ++i) {
+            unsigned h = sm.hist[first - i];
+            if (remaining <= above + h) {
+                sm.bin = (unsigned)(first - i);
+                sm.remaining = remaining - above;
+                break;
+            }
+            above += h;
+        }
+    }
+    __syncthreads();
+}
+
+// Block-wide top-k of keys[0..K): writes idx[0..k) ascending (ties at the threshold go to the lowest indices) and,
+// if asked, the kept fraction of the key mass.  Every thread of the block must call it.  Keys are read through L2
+// (other blocks may have just written them).  kcache, if not NULL, is shared memory for K key images: the keys
+// are then fetched once and every later pass runs out of shared memory.
+//
+// Radix select on the order-preserving integer image of the keys: the bits common to all keys are skipped, one
+// digit of up to 11 bits is histogrammed over all keys, the (few) keys that share the threshold's digit are copied
+// to a short list and finished there with 8-bit digits.  The kept indices are then emitted by warps that own
+// consecutive chunks of the index range, ranks coming from ballots.
+__device__ void block_select(const float *__restrict__ keys, int K, int k, int32_t *__restrict__ idx, float *retained,
+                             SelectSmem &sm, unsigned *kcache)
 {
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     auto image = [&](int j) -> unsigned { return kcache != nullptr ? kcache[j] : key_image(__ldcg(keys + j)); };
-
-    // fetch the keys once, eight independent loads at a time so that their latencies overlap; find the
-    // bits all of them share, so that the first radix digit is well spread
+    // ---- fetch the keys, eight independent loads at a time; min and max give the common leading bits
     unsigned lo = 0xffffffffu, hi = 0u;
     for (int j0 = tid; j0 < K; j0 += 8 * nthr) {
         unsigned u[8];
@@ -79,22 +124,17 @@ __device__ void block_select(const float *keys, int K, int k, int32_t *idx, floa
     lo = __reduce_min_sync(0xffffffffu, lo);
     hi = __reduce_max_sync(0xffffffffu, hi);
     if (lane == 0) {
-        sm.hist[warp] = lo;
-        sm.hist[32 + warp] = hi;
+        sm.warp_a[warp] = lo;
+        sm.warp_b[warp] = hi;
     }
+    for (int i = tid; i < kBins; i += nthr) sm.hist[i] = 0;
+    if (tid == 0) sm.count = 0;
     __syncthreads();
-    if (warp == 0) {
-        unsigned l = lane < nwarp ? sm.hist[lane] : 0xffffffffu, h = lane < nwarp ? sm.hist[32 + lane] : 0u;
-        l = __reduce_min_sync(0xffffffffu, l);
-        h = __reduce_max_sync(0xffffffffu, h);
-        if (lane == 0) {
-            sm.bin = l;
-            sm.remaining = h;
-        }
+    {
+        unsigned l = lane < nwarp ? sm.warp_a[lane] : 0xffffffffu, h = lane < nwarp ? sm.warp_b[lane] : 0u;
+        lo = __reduce_min_sync(0xffffffffu, l);
+        hi = __reduce_max_sync(0xffffffffu, h);
     }
-    __syncthreads();
-    lo = sm.bin;
-    hi = sm.remaining;
     __syncthreads();
 
     const int lcp = (lo ^ hi) ? __clz(lo ^ hi) : 32;  // leading bits common to every key
@@ -103,131 +143,99 @@ __device__ void block_select(const float *keys, int K, int k, int32_t *idx, floa
     unsigned remaining = (unsigned)k;
 
     if (lcp < 32) {
-        int shift = 32 - lcp - 8;
-        if (shift < 0) shift = 0;
-        for (;;) {
+        // ---- first digit over all keys
+        const int d1 = 32 - lcp < 11 ? 32 - lcp : 11;
+        int shift = 32 - lcp - d1;
+        const unsigned dmask = (1u << d1) - 1u;
+        for (int j = tid; j < K; j += nthr) atomicAdd(&sm.hist[(image(j) >> shift) & dmask], 1u);
+        __syncthreads();
+        find_bin(sm, 1 << d1, remaining);
+        prefix |= sm.bin << shift;
+        mask |= dmask << shift;
+        remaining = sm.remaining;
+        const unsigned n_cand = sm.hist[sm.bin];
+        __syncthreads();
+
+        // ---- the keys that share this digit: copy them to the short list if they fit
+        const bool listed = n_cand <= (unsigned)kCandMax;
+        if (listed && shift > 0) {
+            for (int j0 = 0; j0 < K; j0 += nthr) {
+                const int j = j0 + tid;
+                const unsigned u = j < K ? image(j) : 0u;
+                const bool live = j < K && (u & mask) == prefix;
+                const unsigned act = __ballot_sync(0xffffffffu, live);
+                if (act != 0u) {
+                    unsigned base = 0;
+                    if (lane == 0) base = atomicAdd(&sm.count, (unsigned)__popc(act));
+                    base = __shfl_sync(0xffffffffu, base, 0);
+                    if (live) sm.cand[base + __popc(act & ((1u << lane) - 1u))] = u;
+                }
+            }
+            __syncthreads();
+        }
+        // ---- remaining bits, 8 at a time, over the list (or over all keys if the list would not fit)
+        const int n_items = listed ? (int)n_cand : K;
+        while (shift > 0) {
+            const int d = shift < 8 ? shift : 8;
+            shift -= d;
+            const unsigned m = (1u << d) - 1u;
             for (int i = tid; i < 256; i += nthr) sm.hist[i] = 0;
             __syncthreads();
-            for (int j0 = 0; j0 < K; j0 += nthr) {
-                int j = j0 + tid;
-                bool live = false;
-                unsigned bin = 0;
-                if (j < K) {
-                    unsigned u = image(j);
-                    live = (u & mask) == prefix;
-                    bin = (u >> shift) & 255u;
-                }
-                // lanes that agree with the first live lane are counted by it in one atomic; the others add their own
-                unsigned act = __ballot_sync(0xffffffffu, live);
-                if (act != 0u) {
-                    const int leader = __ffs(act) - 1;
-                    const unsigned lbin = __shfl_sync(0xffffffffu, bin, leader);
-                    const unsigned agree = __ballot_sync(0xffffffffu, live && bin == lbin);
-                    if (lane == leader) atomicAdd(&sm.hist[lbin], (unsigned)__popc(agree));
-                    else if (live && bin != lbin) atomicAdd(&sm.hist[bin], 1u);
-                }
+            for (int i = tid; i < n_items; i += nthr) {
+                const unsigned u = listed ? sm.cand[i] : image(i);
+                if ((u & mask) == prefix) atomicAdd(&sm.hist[(u >> shift) & m], 1u);
             }
             __syncthreads();
-            if (warp == 0) {
-                // lane l owns bins 255-8l .. 248-8l (descending); find where the count from the top crosses `remaining`
-                unsigned mine = 0;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) mine += sm.hist[255 - 8 * lane - i];
-                unsigned incl = mine;
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    unsigned v = __shfl_up_sync(0xffffffffu, incl, d);
-                    if (lane >= d) incl += v;
-                }
-                unsigned excl = incl - mine;
-                if (excl < remaining && remaining <= incl) {
-                    unsigned above = excl;
-                    for (int i = 0; i < 8; ++i) {
-                        unsigned h = sm.hist[255 - 8 * lane - i];
-                        if (remaining <= above + h) {
-                            sm.bin = 255 - 8 * lane - i;
-                            sm.remaining = remaining - above;
-                            break;
-                        }
-                        above += h;
-                    }
-                }
-            }
-            __syncthreads();
-            prefix = (prefix & ~(255u << shift)) | (sm.bin << shift);
-            mask |= 255u << shift;
+            find_bin(sm, 1 << d, remaining);
+            prefix |= sm.bin << shift;
+            mask |= m << shift;
             remaining = sm.remaining;
             __syncthreads();
-            if (shift == 0) break;
-            shift = shift >= 8 ? shift - 8 : 0;
         }
     }
     const unsigned tau = prefix;          // image of the k-th largest key
     const unsigned need_eq = remaining;   // how many keys equal to tau are kept (lowest indices first)
 
-    // ordered compaction, 4 consecutive indices per thread per round
-    if (tid == 0) sm.carry = 0ull;
-    __syncthreads();
-    double sum_kept = 0.0, sum_all = 0.0;
-    const int per_round = nthr * 4;
-    for (int base = 0; base < K; base += per_round) {
-        int j = base + tid * 4;
-        unsigned u[4];
-        float f[4];
-        unsigned long long mine = 0ull;  // (count > tau) << 32 | (count == tau)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (j + i < K) {
-                u[i] = image(j + i);
-                f[i] = key_value(u[i]);
-                mine += (u[i] > tau) ? (1ull << 32) : 0ull;
-                mine += (u[i] == tau) ? 1ull : 0ull;
-            } else {
-                f[i] = 0.f;
-                u[i] = 0u;
-            }
-        }
-        unsigned long long incl = mine;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            unsigned long long v = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += v;
-        }
-        if (lane == 31) sm.warp_tot[warp] = incl;
-        __syncthreads();
-        if (warp == 0) {
-            unsigned long long w = (lane < (nthr >> 5)) ? sm.warp_tot[lane] : 0ull;
-            unsigned long long wi = w;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                unsigned long long v = __shfl_up_sync(0xffffffffu, wi, d);
-                if (lane >= d) wi += v;
-            }
-            sm.warp_tot[lane] = wi - w;  // exclusive prefix of warp totals
-            if (lane == 31) sm.round_total = wi;
-        }
-        __syncthreads();
-        unsigned long long before = sm.carry + sm.warp_tot[warp] + (incl - mine);
-        unsigned gt_before = (unsigned)(before >> 32), eq_before = (unsigned)(before & 0xffffffffu);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (j + i < K) {
-                sum_all += (double)f[i];
-                bool gt = u[i] > tau, eq = u[i] == tau;
-                if (gt || (eq && eq_before < need_eq)) {
-                    unsigned pos = gt_before + (eq_before < need_eq ? eq_before : need_eq);
-                    idx[pos] = j + i;
-                    sum_kept += (double)f[i];
-                }
-                gt_before += gt;
-                eq_before += eq;
-            }
-        }
-        __syncthreads();
-        if (tid == 0) sm.carry += sm.round_total;
-        __syncthreads();
+    // ---- ordered emission: warp w owns indices [w * chunk, (w + 1) * chunk)
+    const int chunk = ((K + nwarp - 1) / nwarp + 31) / 32 * 32;
+    const int c_begin = warp * chunk, c_end = min(K, c_begin + chunk);
+    unsigned n_gt = 0, n_eq = 0;
+    for (int j0 = c_begin; j0 < c_end; j0 += 32) {
+        const int j = j0 + lane;
+        const unsigned u = j < c_end ? image(j) : 0u;
+        n_gt += __popc(__ballot_sync(0xffffffffu, j < c_end && u > tau));
+        n_eq += __popc(__ballot_sync(0xffffffffu, j < c_end && u == tau));
     }
-
+    if (lane == 0) {
+        sm.warp_a[warp] = n_gt;
+        sm.warp_b[warp] = n_eq;
+    }
+    __syncthreads();
+    unsigned gt_base = 0, eq_base = 0;
+    for (int w = 0; w < warp; ++w) {
+        gt_base += sm.warp_a[w];
+        eq_base += sm.warp_b[w];
+    }
+    double sum_kept = 0.0, sum_all = 0.0;
+    const unsigned lt = (1u << lane) - 1u;
+    for (int j0 = c_begin; j0 < c_end; j0 += 32) {
+        const int j = j0 + lane;
+        const bool in = j < c_end;
+        const unsigned u = in ? image(j) : 0u;
+        const bool gt = in && u > tau, eq = in && u == tau;
+        const unsigned g = __ballot_sync(0xffffffffu, gt), e = __ballot_sync(0xffffffffu, eq);
+        const unsigned gt_before = gt_base + __popc(g & lt), eq_before = eq_base + __popc(e & lt);
+        if (in) {
+            const double f = (double)key_value(u);
+            sum_all += f;
+            if (gt || (eq && eq_before < need_eq)) {
+                idx[gt_before + (eq_before < need_eq ? eq_before : need_eq)] = j;
+                sum_kept += f;
+            }
+        }
+        gt_base += __popc(g);
+        eq_base += __popc(e);
+    }
     if (retained != nullptr) {
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) {
@@ -241,7 +249,7 @@ __device__ void block_select(const float *keys, int K, int k, int32_t *idx, floa
         __syncthreads();
         if (tid == 0) {
             double a = 0.0, b = 0.0;
-            for (int w = 0; w < (nthr >> 5); ++w) {
+            for (int w = 0; w < nwarp; ++w) {
                 a += sm.red[w];
                 b += sm.red[32 + w];
             }
