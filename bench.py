@@ -66,7 +66,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -183,7 +183,7 @@ def run_reference(args):
     cores = oracle.num_threads()
     e, _ = oracle.score(A)
     idx, _ = oracle.select(e, oracle.keep_count(RHO, K))
-    rows = max(cores, 2 * cores)             # bounded sample per step
+    rows = cores                             # bounded sample per step: one row per thread
     times = []
     for i in range(args.warmup + args.steps):
         t0 = time.perf_counter()
@@ -208,7 +208,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU oracle timing (quick runs, profiling)")
@@ -249,14 +249,14 @@ def main():
 
     # ---- timed region: exactly K steps; the GEMM kernel of every step is bracketed by events on the same stream
     sampler = ClockSampler(local if world > 1 else 0)
-    timer = binding.GemmTimer(args.steps)
+    timer = binding.KernelTimer(min(args.steps, 4096), "reduced_gemm_tc_kernel")
     launches0 = rmm.rmm_launch_count()
     sampler.start()
     with timer:
         ms_step = time_region(step, args.steps, world)
     clocks = sampler.stop()
     launches = rmm.rmm_launch_count() - launches0
-    gemm_ms = timer.times_ms()
+    gemm_ms = [t for _, t in timer.times_ms()]
     gemm_ms_avg = sum(gemm_ms) / len(gemm_ms)
     assert rmm.rmm_status_read() == 0
     value = world * retained_flops(RHO) / (ms_step * 1e-3) / 1e12
@@ -292,16 +292,18 @@ def main():
     per_rho = []
     if not args.no_sweep and rank == 0:
         reps = 40
+        for i in range(5):
+            torch.matmul(sets[i % n_sets][0], sets[i % n_sets][1], out=sets[i % n_sets][2])
         dense_ms = time_region(lambda i: torch.matmul(sets[i % n_sets][0], sets[i % n_sets][1], out=sets[i % n_sets][2]), reps, 1)
         for rho in RHOS:
             kk = rmm.rmm_keep_count(rho, K)
             idx_r = torch.empty(kk, dtype=torch.int32, device=dev)
             for i in range(3):
                 step(i, rho, idx_r)
-            t = binding.GemmTimer(reps)
+            t = binding.KernelTimer(reps, "reduced_gemm_tc_kernel")
             with t:
                 whole = time_region(lambda i: step(i, rho, idx_r), reps, 1)
-            g = sum(t.times_ms()) / reps
+            g = sum(x for _, x in t.times_ms()) / reps
             sel = time_region(lambda i: rmm.rmm_score_select(sets[i % n_sets][0], rho=rho, idx=idx_r), reps, 1)
             fl = retained_flops(rho)
             per_rho.append({"rho": rho, "k": kk, "whole_op_ms": whole, "whole_op_tflops": fl / whole / 1e9,
@@ -311,6 +313,18 @@ def main():
                             "score_select_ms": sel, "score_select_gbs": M * K * 2 / sel / 1e6,
                             "score_select_frac_of_hbm": M * K * 2 / sel / 1e6 / peaks["hbm_gbs"],
                             "dense_cublas_ms": dense_ms, "speedup_vs_dense_cublas": dense_ms / whole})
+
+    # ---- per-kernel breakdown of one step (a separate, untimed pass with every launch bracketed by events)
+    breakdown = {}
+    if rank == 0:
+        nb = 20
+        kt = binding.KernelTimer(nb * 8)
+        with kt:
+            for i in range(nb):
+                step(i)
+        for name, t in kt.times_ms():
+            breakdown.setdefault(name, []).append(t)
+        breakdown = {name: {"launches_per_step": len(v) / nb, "mean_us": 1e3 * sum(v) / len(v)} for name, v in breakdown.items()}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -324,7 +338,7 @@ def main():
             "config": {"workload": WORKLOAD, "rho": RHO, "k": k, "M": M, "K": K, "N": N, "parallelism": f"replicas x{world}",
                        "l2_policy": f"inputs larger than L2: {n_sets} rotating (A, B, Y) sets, {resident_bytes / 1e6:.0f} MB resident"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
-            "per_rho": per_rho, "peaks": peaks,
+            "kernel_breakdown": breakdown, "per_rho": per_rho, "peaks": peaks,
         }
         print(json.dumps(out))
     if world > 1:

@@ -49,7 +49,7 @@ EXPORTS = ["rmm_keep_count", "rmm_score_workspace_bytes", "rmm_score", "rmm_sele
            "rmm_score_select_workspace_bytes", "rmm_score_select", "rmm_reduced_gemm_workspace_bytes",
            "rmm_reduced_gemm", "rmm_reduced_attn_workspace_bytes", "rmm_reduced_attn",
            "rmm_product_host_workspace_bytes", "rmm_product_host", "rmm_status_read", "rmm_last_error",
-           "rmm_launch_count", "rmm_profile_gemm", "rmm_profile_gemm_count"]
+           "rmm_launch_count", "rmm_profile_kernels", "rmm_profile_count", "rmm_profile_name"]
 
 _lib = None
 
@@ -87,7 +87,9 @@ def lib() -> ctypes.CDLL:
     L.rmm_status_read.argtypes = [vp, ctypes.POINTER(i32)]
     L.rmm_last_error.restype = ctypes.c_char_p
     L.rmm_launch_count.restype = i64
-    L.rmm_profile_gemm.argtypes = [vp, vp, i32]
+    L.rmm_profile_kernels.argtypes = [vp, vp, i32, ctypes.c_char_p]
+    L.rmm_profile_name.argtypes = [i32]
+    L.rmm_profile_name.restype = ctypes.c_char_p
     _lib = L
     return L
 
@@ -153,11 +155,13 @@ def rmm_launch_count() -> int:
     return int(lib().rmm_launch_count())
 
 
-class GemmTimer:
-    """Brackets the next n launches of the tensor-core GEMM kernel with CUDA events (rmm_profile_gemm)."""
+class KernelTimer:
+    """Brackets the next n launches of library kernels whose name contains `name_filter` with CUDA events
+    (rmm_profile_kernels).  Use as a context manager; times_ms() then gives (kernel name, duration) pairs."""
 
-    def __init__(self, n: int):
+    def __init__(self, n: int, name_filter: str = ""):
         self.n = n
+        self.filter = name_filter.encode()
         self.start = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
         self.stop = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
         for e in self.start + self.stop:      # torch creates the handle at the first record
@@ -165,20 +169,23 @@ class GemmTimer:
         torch.cuda.synchronize()
         self._s = (ctypes.c_void_p * n)(*[e.cuda_event for e in self.start])
         self._e = (ctypes.c_void_p * n)(*[e.cuda_event for e in self.stop])
+        self.count = 0
+        self.names = []
 
     def __enter__(self):
-        _check(lib().rmm_profile_gemm(self._s, self._e, self.n))
+        _check(lib().rmm_profile_kernels(self._s, self._e, self.n, self.filter))
         return self
 
     def __exit__(self, *exc):
-        self.count = int(lib().rmm_profile_gemm_count())
-        _check(lib().rmm_profile_gemm(None, None, 0))
+        self.count = int(lib().rmm_profile_count())
+        self.names = [lib().rmm_profile_name(i).decode() for i in range(self.count)]
+        _check(lib().rmm_profile_kernels(None, None, 0, None))
         return False
 
     def times_ms(self):
-        """Durations of the recorded launches (synchronises)."""
+        """[(kernel name, milliseconds)] of the recorded launches (synchronises)."""
         torch.cuda.synchronize()
-        return [self.start[i].elapsed_time(self.stop[i]) for i in range(self.count)]
+        return [(self.names[i], self.start[i].elapsed_time(self.stop[i])) for i in range(self.count)]
 
 
 def rmm_status_read(ws: Optional[torch.Tensor] = None, device=None) -> int:

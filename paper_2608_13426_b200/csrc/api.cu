@@ -21,8 +21,30 @@ int fail(int code, const char *fmt, ...)
     return code;
 }
 
-int check_launch(const char *what)
+// Optional timing hook (rmm_profile_kernels): events recorded around launches whose name matches the filter.
+static struct {
+    cudaEvent_t *start = nullptr, *stop = nullptr;
+    int capacity = 0, used = 0;
+    bool pending = false;
+    char filter[64] = "";
+    const char *names[4096];
+} g_prof;
+
+void prof_begin(const char *name, cudaStream_t stream)
 {
+    if (g_prof.used >= g_prof.capacity || g_prof.used >= 4096) return;
+    if (g_prof.filter[0] != 0 && strstr(name, g_prof.filter) == nullptr) return;
+    cudaEventRecord(g_prof.start[g_prof.used], stream);
+    g_prof.names[g_prof.used] = name;
+    g_prof.pending = true;
+}
+
+int check_launch(const char *what, cudaStream_t stream)
+{
+    if (g_prof.pending) {
+        cudaEventRecord(g_prof.stop[g_prof.used++], stream);
+        g_prof.pending = false;
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "%s: launch failed: %s", what, cudaGetErrorString(e));
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -277,15 +299,22 @@ int rmm_status_read(void *ws, int *device_status)
     return RMM_OK;
 }
 
-int rmm_profile_gemm(void **start_events, void **stop_events, int n)
+int rmm_profile_kernels(void **start_events, void **stop_events, int n, const char *name_filter)
 {
-    if (n < 0 || ((start_events == nullptr || stop_events == nullptr) && n != 0))
-        return fail(RMM_ERR_INVALID_ARG, "profile_gemm: need two event arrays, or NULL, NULL, 0");
-    set_gemm_profile(start_events, stop_events, n);
+    if (n < 0 || n > 4096 || ((start_events == nullptr || stop_events == nullptr) && n != 0))
+        return fail(RMM_ERR_INVALID_ARG, "profile_kernels: need two event arrays and 0 <= n <= 4096, or NULL, NULL, 0");
+    g_prof.start = reinterpret_cast<cudaEvent_t *>(start_events);
+    g_prof.stop = reinterpret_cast<cudaEvent_t *>(stop_events);
+    g_prof.capacity = n;
+    g_prof.used = 0;
+    g_prof.pending = false;
+    snprintf(g_prof.filter, sizeof g_prof.filter, "%s", name_filter ? name_filter : "");
     return RMM_OK;
 }
 
-int rmm_profile_gemm_count(void) { return gemm_profile_used(); }
+int rmm_profile_count(void) { return g_prof.used; }
+
+const char *rmm_profile_name(int i) { return (i >= 0 && i < g_prof.used) ? g_prof.names[i] : ""; }
 
 const char *rmm_last_error(void) { return t_error; }
 

@@ -127,8 +127,9 @@ int launch_softmax_rows(const float *S, int64_t ld_s, int64_t heads, int64_t Lq,
                         __nv_bfloat16 *P, int64_t ld_p, cudaStream_t stream)
 {
     dim3 grid((unsigned)Lq, (unsigned)heads);
+    prof_begin("softmax_rows_kernel", stream);
     softmax_rows_kernel<<<grid, kSoftmaxThreads, 0, stream>>>(S, ld_s, Lq, Lk, causal, P, ld_p);
-    return check_launch("softmax_rows_kernel");
+    return check_launch("softmax_rows_kernel", stream);
 }
 
 }  // namespace rmm

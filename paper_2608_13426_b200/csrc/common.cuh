@@ -13,7 +13,8 @@ namespace rmm {
 // ---- error text (thread-local) and launch accounting -------------------------------------------
 int fail(int code, const char *fmt, ...);
 extern std::atomic<int64_t> g_launches;
-int check_launch(const char *what);  // cudaGetLastError -> RMM_OK / RMM_ERR_CUDA, counts the launch
+void prof_begin(const char *kernel_name, cudaStream_t stream);  // call right before a launch (timing hook)
+int check_launch(const char *what, cudaStream_t stream);  // right after: cudaGetLastError -> status, counts the launch
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -77,8 +78,6 @@ struct TcProblem {
     int *status;
 };
 int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream);
-void set_gemm_profile(void **start, void **stop, int n);
-int gemm_profile_used();
 
 // Gather columns: dst[b, r, j] = src[sb, r, idx[b, j]] for j < k with source batch sb = (b + b_off) / b_div
 // (dst row pitch ld_dst >= k; columns k..ld_dst are zeroed).  bf16 only.  idx_stride = elements between the

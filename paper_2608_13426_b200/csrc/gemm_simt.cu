@@ -140,11 +140,12 @@ int launch_gemm_simt(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx,
         return fail(RMM_ERR_UNSUPPORTED, "reduced_gemm (FMA path): batch or M/64 exceeds 65535");
     dim3 grid((unsigned)ceil_div(a.N, BN), (unsigned)ceil_div(a.M, BM), (unsigned)A->batch);
     const bool in_bf16 = A->dtype == RMM_BF16, out_bf16 = Y->dtype == RMM_BF16;
+    prof_begin("reduced_gemm_simt_kernel", stream);
     if (in_bf16 && out_bf16) reduced_gemm_simt_kernel<true, true><<<grid, THREADS, 0, stream>>>(a);
     else if (in_bf16) reduced_gemm_simt_kernel<true, false><<<grid, THREADS, 0, stream>>>(a);
     else if (out_bf16) reduced_gemm_simt_kernel<false, true><<<grid, THREADS, 0, stream>>>(a);
     else reduced_gemm_simt_kernel<false, false><<<grid, THREADS, 0, stream>>>(a);
-    return check_launch("reduced_gemm_simt_kernel");
+    return check_launch("reduced_gemm_simt_kernel", stream);
 }
 
 }  // namespace rmm

@@ -398,12 +398,6 @@ int sm_count()
     return n;
 }
 
-// Optional profiling hook (rmm_profile_gemm): events recorded around each launch of the GEMM kernel.
-struct GemmProfile {
-    cudaEvent_t *start = nullptr, *stop = nullptr;
-    int capacity = 0, used = 0;
-} g_profile;
-
 template <int BN, bool B_KMAJOR, bool OUT_BF16>
 int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const TcArgs &a, cudaStream_t stream)
 {
@@ -416,23 +410,12 @@ int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const TcArgs &a
     }
     int64_t tiles = a.batch * a.tiles_m * a.tiles_n;
     int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-    const bool prof = g_profile.used < g_profile.capacity;
-    if (prof) cudaEventRecord(g_profile.start[g_profile.used], stream);
+    prof_begin("reduced_gemm_tc_kernel", stream);
     kern<<<grid, kThreadsTc, SmemLayout<BN>::kTotal, stream>>>(ma, mb, a);
-    if (prof) cudaEventRecord(g_profile.stop[g_profile.used++], stream);
-    return check_launch("reduced_gemm_tc_kernel");
+    return check_launch("reduced_gemm_tc_kernel", stream);
 }
 
 }  // namespace
-
-void set_gemm_profile(void **start, void **stop, int n)
-{
-    g_profile.start = reinterpret_cast<cudaEvent_t *>(start);
-    g_profile.stop = reinterpret_cast<cudaEvent_t *>(stop);
-    g_profile.capacity = (start != nullptr && stop != nullptr) ? n : 0;
-    g_profile.used = 0;
-}
-int gemm_profile_used() { return g_profile.used; }
 
 bool tc_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y, TcPlan *plan)
 {

@@ -117,9 +117,10 @@ int launch_pack_cols(const __nv_bfloat16 *src, int64_t batch, int64_t rows, int6
     if (ld_dst % 2 != 0) return fail(RMM_ERR_UNSUPPORTED, "pack: destination pitch must be even");
     dim3 grid((unsigned)ceil_div(ld_dst, 256 * kWarps), (unsigned)ceil_div(rows, kRowsPerBlock), (unsigned)batch);
     if (grid.y > 65535u || grid.z > 65535u) return fail(RMM_ERR_UNSUPPORTED, "pack: rows/32 or batch exceeds 65535");
+    prof_begin("pack_cols_kernel", stream);
     pack_cols_kernel<<<grid, kWarps * 32, 0, stream>>>(src, rows, K, s_batch, s_row, b_off, b_div > 0 ? b_div : 1, idx, idx_stride, k, dst,
                                                                ld_dst, status);
-    return check_launch("pack_cols_kernel");
+    return check_launch("pack_cols_kernel", stream);
 }
 
 int launch_pack_rows(const __nv_bfloat16 *src, int64_t batch, int64_t K, int64_t n, int64_t s_batch, int64_t s_row,
@@ -133,10 +134,11 @@ int launch_pack_rows(const __nv_bfloat16 *src, int64_t batch, int64_t K, int64_t
     if (gx > 8) gx = 8;
     dim3 grid((unsigned)gx, (unsigned)ceil_div(k, 4), (unsigned)batch);
     if (grid.y > 65535u || grid.z > 65535u) return fail(RMM_ERR_UNSUPPORTED, "pack_rows: k/4 or batch exceeds 65535");
+    prof_begin("pack_rows_kernel", stream);
     pack_rows_kernel<<<grid, kRowVecThreads, 0, stream>>>(reinterpret_cast<const uint4 *>(src), K, nvec, s_batch / 8, s_row / 8, b_off,
                                                          b_div > 0 ? b_div : 1, idx, idx_stride, k,
                                                          reinterpret_cast<uint4 *>(dst), ld_dst / 8, status);
-    return check_launch("pack_rows_kernel");
+    return check_launch("pack_rows_kernel", stream);
 }
 
 }  // namespace rmm

@@ -504,11 +504,12 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
     const bool bf16 = A->dtype == RMM_BF16;
     size_t smem = (size_t)kThreads * p.vec * sizeof(double);
     if (fused && (size_t)p.n * 4 > smem) smem = (size_t)p.n * 4;
+    prof_begin("score_select_kernel", stream);
     if (bf16 && p.vec == 8) score_select_kernel<8, true><<<grid, kThreads, smem, stream>>>(a);
     else if (bf16) score_select_kernel<1, true><<<grid, kThreads, smem, stream>>>(a);
     else if (p.vec == 4) score_select_kernel<4, false><<<grid, kThreads, smem, stream>>>(a);
     else score_select_kernel<1, false><<<grid, kThreads, smem, stream>>>(a);
-    int rc = check_launch("score_select_kernel");
+    int rc = check_launch("score_select_kernel", stream);
     if (rc != RMM_OK || !do_select || fused) return rc;
     return launch_select(a.energy, A->batch, p.n, k, idx, retained, ws, stream);
 }
@@ -526,8 +527,9 @@ int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_
         if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "select: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         configured = true;
     }
+    prof_begin("select_kernel", stream);
     select_kernel<<<(unsigned)batch, threads, smem, stream>>>(keys, (int)K, (int)k, idx, retained, use_cache);
-    return check_launch("select_kernel");
+    return check_launch("select_kernel", stream);
 }
 
 }  // namespace rmm
