@@ -17,9 +17,9 @@ namespace rmm {
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kUnroll = 8;       // rows in flight per thread
-constexpr int kFlushEvery = 2;   // loop trips between fp32 -> fp64 flushes (kUnroll * kFlushEvery = 16 terms)
+constexpr int kThreads = 1024;     // one block per SM: its tail (the select) then has 32 warps to work with
+constexpr int kUnroll = 4;       // rows in flight per thread (1024 threads x 4 x 16 B = 64 KB in flight per SM)
+constexpr int kFlushEvery = 4;   // loop trips between fp32 -> fp64 flushes (kUnroll * kFlushEvery = 16 terms)
 constexpr int kFusedSelectMax = 8192;    // largest K whose select runs in the score kernel's tail (32 KB key cache)
 constexpr int kCachedSelectMax = 49152;  // largest K the stand-alone select kernel caches in shared memory (192 KB)
 
@@ -259,6 +259,180 @@ __device__ void block_select(const float *__restrict__ keys, int K, int k, int32
     __syncthreads();
 }
 
+// The same selection for K <= ITEMS * blockDim.x with every key held in a register of its thread (key j lives in
+// item j / blockDim.x of thread j % blockDim.x): all loops unroll, nothing is re-read, and the ordered emission needs
+// one scan over ITEMS * 32 per-warp counts.  Requires blockDim.x == 1024.
+template <int ITEMS>
+__device__ void block_select_reg(const float *__restrict__ keys, int K, int k, int32_t *__restrict__ idx, float *retained,
+                                 SelectSmem &sm)
+{
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+    unsigned u[ITEMS];
+    unsigned lo = 0xffffffffu, hi = 0u;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        const int j = tid + i * nthr;
+        u[i] = j < K ? key_image(__ldcg(keys + j)) : 0u;
+    }
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        if (tid + i * nthr < K) {
+            lo = min(lo, u[i]);
+            hi = max(hi, u[i]);
+        }
+    }
+    lo = __reduce_min_sync(0xffffffffu, lo);
+    hi = __reduce_max_sync(0xffffffffu, hi);
+    if (lane == 0) {
+        sm.warp_a[warp] = lo;
+        sm.warp_b[warp] = hi;
+    }
+    for (int i = tid; i < kBins; i += nthr) sm.hist[i] = 0;
+    if (tid == 0) sm.count = 0;
+    __syncthreads();
+    {
+        unsigned l = lane < nwarp ? sm.warp_a[lane] : 0xffffffffu, h = lane < nwarp ? sm.warp_b[lane] : 0u;
+        lo = __reduce_min_sync(0xffffffffu, l);
+        hi = __reduce_max_sync(0xffffffffu, h);
+    }
+    __syncthreads();
+
+    const int lcp = (lo ^ hi) ? __clz(lo ^ hi) : 32;
+    unsigned mask = lcp == 0 ? 0u : (lcp == 32 ? 0xffffffffu : ~(0xffffffffu >> lcp));
+    unsigned prefix = hi & mask;
+    unsigned remaining = (unsigned)k;
+    const unsigned lt = (1u << lane) - 1u;
+
+    if (lcp < 32) {
+        const int d1 = 32 - lcp < 11 ? 32 - lcp : 11;
+        int shift = 32 - lcp - d1;
+        const unsigned dmask = (1u << d1) - 1u;
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i)
+            if (tid + i * nthr < K) atomicAdd(&sm.hist[(u[i] >> shift) & dmask], 1u);
+        __syncthreads();
+        find_bin(sm, 1 << d1, remaining);
+        prefix |= sm.bin << shift;
+        mask |= dmask << shift;
+        remaining = sm.remaining;
+        const unsigned n_cand = sm.hist[sm.bin];
+        __syncthreads();
+        if (shift > 0) {
+            const bool listed = n_cand <= (unsigned)kCandMax;
+            if (listed) {
+#pragma unroll
+                for (int i = 0; i < ITEMS; ++i) {
+                    const bool live = tid + i * nthr < K && (u[i] & mask) == prefix;
+                    const unsigned act = __ballot_sync(0xffffffffu, live);
+                    if (act != 0u) {
+                        unsigned base = 0;
+                        if (lane == 0) base = atomicAdd(&sm.count, (unsigned)__popc(act));
+                        base = __shfl_sync(0xffffffffu, base, 0);
+                        if (live) sm.cand[base + __popc(act & lt)] = u[i];
+                    }
+                }
+                __syncthreads();
+            }
+            while (shift > 0) {
+                const int d = shift < 8 ? shift : 8;
+                shift -= d;
+                const unsigned m = (1u << d) - 1u;
+                if (tid < 256) sm.hist[tid] = 0;
+                __syncthreads();
+                if (listed) {
+                    for (int i = tid; i < (int)n_cand; i += nthr) {
+                        const unsigned c = sm.cand[i];
+                        if ((c & mask) == prefix) atomicAdd(&sm.hist[(c >> shift) & m], 1u);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < ITEMS; ++i)
+                        if (tid + i * nthr < K && (u[i] & mask) == prefix) atomicAdd(&sm.hist[(u[i] >> shift) & m], 1u);
+                }
+                __syncthreads();
+                find_bin(sm, 1 << d, remaining);
+                prefix |= sm.bin << shift;
+                mask |= m << shift;
+                remaining = sm.remaining;
+                __syncthreads();
+            }
+        }
+    }
+    const unsigned tau = prefix, need_eq = remaining;
+
+    // ---- ordered emission.  Index order = (item, warp, lane); per-(item, warp) counts, packed (greater << 16 | equal)
+    unsigned *cnt = sm.cand, *cnt_ex = sm.cand + ITEMS * 32;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        const bool in = tid + i * nthr < K;
+        const unsigned g = __ballot_sync(0xffffffffu, in && u[i] > tau), e = __ballot_sync(0xffffffffu, in && u[i] == tau);
+        if (lane == 0) cnt[i * nwarp + warp] = ((unsigned)__popc(g) << 16) | (unsigned)__popc(e);
+    }
+    __syncthreads();
+    if (tid < ITEMS * 32) {
+        const unsigned v = cnt[tid];
+        unsigned incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            unsigned o = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += o;
+        }
+        if (lane == 31) sm.warp_a[warp] = incl;
+        cnt_ex[tid] = incl - v;
+    }
+    __syncthreads();
+    double sum_kept = 0.0, sum_all = 0.0;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        const int j = tid + i * nthr;
+        const bool in = j < K;
+        unsigned base = cnt_ex[i * nwarp + warp];
+        for (int w = 0; w < i; ++w) base += sm.warp_a[w];  // entries of item i sit in scan warp i (nwarp == 32)
+        const bool gt = in && u[i] > tau, eq = in && u[i] == tau;
+        const unsigned g = __ballot_sync(0xffffffffu, gt), e = __ballot_sync(0xffffffffu, eq);
+        const unsigned gt_before = (base >> 16) + __popc(g & lt), eq_before = (base & 0xffffu) + __popc(e & lt);
+        if (in) {
+            const double f = (double)key_value(u[i]);
+            sum_all += f;
+            if (gt || (eq && eq_before < need_eq)) {
+                idx[gt_before + (eq_before < need_eq ? eq_before : need_eq)] = j;
+                sum_kept += f;
+            }
+        }
+    }
+    if (retained != nullptr) {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            sum_kept += __shfl_down_sync(0xffffffffu, sum_kept, d);
+            sum_all += __shfl_down_sync(0xffffffffu, sum_all, d);
+        }
+        __syncthreads();
+        if (lane == 0) {
+            sm.red[warp] = sum_kept;
+            sm.red[32 + warp] = sum_all;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            double a = 0.0, b = 0.0;
+            for (int w = 0; w < nwarp; ++w) {
+                a += sm.red[w];
+                b += sm.red[32 + w];
+            }
+            *retained = (b > 0.0) ? (float)(a / b) : 1.0f;
+        }
+    }
+    __syncthreads();
+}
+
+// Dispatch on the problem size: keys in registers when they fit (blocks of 1024 threads), else the cached form.
+__device__ __forceinline__ void block_select_any(const float *keys, int K, int k, int32_t *idx, float *retained,
+                                                 SelectSmem &sm, unsigned *kcache)
+{
+    if (blockDim.x == 1024 && K <= 1024) block_select_reg<1>(keys, K, k, idx, retained, sm);
+    else if (blockDim.x == 1024 && K <= 8192) block_select_reg<8>(keys, K, k, idx, retained, sm);
+    else block_select(keys, K, k, idx, retained, sm, kcache);
+}
+
 struct ScoreArgs {
     const void *A;
     int64_t s_batch, s_red, s_n;  // element strides: batch, reduced axis (rows), scored axis (columns)
@@ -301,7 +475,7 @@ __device__ __forceinline__ void load_vec(const void *A, int64_t off, int64_t s_n
 }
 
 template <int VEC, bool BF16>
-__global__ void __launch_bounds__(kThreads) score_select_kernel(ScoreArgs a)
+__global__ void __launch_bounds__(kThreads, 1) score_select_kernel(ScoreArgs a)
 {
     extern __shared__ __align__(16) unsigned char s_dyn[];  // row-lane partial sums, later the select's key cache
     double *s_part = reinterpret_cast<double *>(s_dyn);
@@ -405,8 +579,8 @@ __global__ void __launch_bounds__(kThreads) score_select_kernel(ScoreArgs a)
     __syncthreads();
     if (!s_flag) return;
     __threadfence();
-    block_select(a.energy + b * a.n, (int)a.n, a.k, a.idx + b * (int64_t)a.k,
-                 a.retained ? a.retained + b : nullptr, s_sel, reinterpret_cast<unsigned *>(s_dyn));
+    block_select_any(a.energy + b * a.n, (int)a.n, a.k, a.idx + b * (int64_t)a.k,
+                     a.retained ? a.retained + b : nullptr, s_sel, reinterpret_cast<unsigned *>(s_dyn));
 }
 
 __global__ void __launch_bounds__(1024) select_kernel(const float *keys, int K, int k, int32_t *idx, float *retained,
@@ -415,8 +589,8 @@ __global__ void __launch_bounds__(1024) select_kernel(const float *keys, int K, 
     extern __shared__ __align__(16) unsigned char s_dyn[];
     __shared__ SelectSmem s_sel;
     const int64_t b = blockIdx.x;
-    block_select(keys + b * K, K, k, idx + b * (int64_t)k, retained ? retained + b : nullptr, s_sel,
-                 use_cache ? reinterpret_cast<unsigned *>(s_dyn) : nullptr);
+    block_select_any(keys + b * K, K, k, idx + b * (int64_t)k, retained ? retained + b : nullptr, s_sel,
+                     use_cache ? reinterpret_cast<unsigned *>(s_dyn) : nullptr);
 }
 
 }  // namespace
@@ -449,9 +623,10 @@ int plan_score(const rmm_mat_t *A, int axis, ScorePlan *p)
     p->ty = kThreads / tx;
     p->col_blocks = (int)ceil_div(p->n, (int64_t)tx * p->vec);
 
-    // enough blocks to fill the machine several times over, but at least 4 loop trips of rows each
-    const int64_t want_blocks = 148 * 8;
-    int64_t splits = ceil_div(want_blocks, (int64_t)p->col_blocks * A->batch);
+    // one block of 1024 threads per SM: split the rows so that the grid is at most one wave, each block keeping
+    // at least two loop trips of rows
+    const int64_t want_blocks = 148;
+    int64_t splits = want_blocks / ((int64_t)p->col_blocks * A->batch);
     int64_t min_rows = (int64_t)p->ty * kUnroll * 2;
     int64_t max_splits = p->m / min_rows;
     if (max_splits < 1) max_splits = 1;
@@ -504,6 +679,16 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
     const bool bf16 = A->dtype == RMM_BF16;
     size_t smem = (size_t)kThreads * p.vec * sizeof(double);
     if (fused && (size_t)p.n * 4 > smem) smem = (size_t)p.n * 4;
+    static bool configured = false;
+    if (!configured) {
+        const int big = kThreads * 8 * (int)sizeof(double);
+        cudaError_t e = cudaFuncSetAttribute(score_select_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(score_select_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(score_select_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(score_select_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+        if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "score: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+        configured = true;
+    }
     prof_begin("score_select_kernel", stream);
     if (bf16 && p.vec == 8) score_select_kernel<8, true><<<grid, kThreads, smem, stream>>>(a);
     else if (bf16) score_select_kernel<1, true><<<grid, kThreads, smem, stream>>>(a);
@@ -518,7 +703,7 @@ int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_
                   cudaStream_t stream)
 {
     (void)ws;
-    int threads = K >= 4096 ? 1024 : (K >= 1024 ? 512 : 256);
+    const int threads = 1024;
     const int use_cache = K <= kCachedSelectMax;
     const size_t smem = use_cache ? (size_t)K * 4 : 0;
     static bool configured = false;
