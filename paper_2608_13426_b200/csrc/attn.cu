@@ -185,12 +185,12 @@ int rmm_reduced_attn(const rmm_attn_desc_t *d, const void *Q, const void *K, con
             if ((rc = launch_score_select(&qm, sq, true, p.kd, If, nullptr, nullptr, nullptr, w, st)) != RMM_OK) return rc;
 
             // Q[:, I_h] and K_{g(h)}[:, I_h]
-            rc = launch_pack_cols(static_cast<const __nv_bfloat16 *>(qm.ptr), hg, d->Lq, d->Dh, d->q_stride[1], d->q_stride[2], 0, 1,
-                                  If, p.kd, p.kd, Qp, p.ldd, status, st);
-            if (rc != RMM_OK) return rc;
-            rc = launch_pack_cols(kk + b * d->k_stride[0], hg, d->Lk, d->Dh, d->k_stride[1], d->k_stride[2], h0, group, If, p.kd,
-                                  p.kd, Kp, p.ldd, status, st);
-            if (rc != RMM_OK) return rc;
+            PackSpec qk[2];
+            qk[0] = pack_cols_spec(static_cast<const __nv_bfloat16 *>(qm.ptr), hg, d->Lq, d->Dh, d->q_stride[1], d->q_stride[2], 0, 1,
+                                   If, p.kd, p.kd, Qp, p.ldd);
+            qk[1] = pack_cols_spec(kk + b * d->k_stride[0], hg, d->Lk, d->Dh, d->k_stride[1], d->k_stride[2], h0, group, If, p.kd,
+                                   p.kd, Kp, p.ldd);
+            if ((rc = launch_pack(qk, 2, status, st)) != RMM_OK) return rc;
 
             // S~ = Q[:, I] K[:, I]^T / sqrt(Dh)  (the scale keeps the full head dimension)
             TcProblem g1 = {};
@@ -215,11 +215,11 @@ int rmm_reduced_attn(const rmm_attn_desc_t *d, const void *Q, const void *K, con
                 ScorePlan sp;
                 if ((rc = plan_score(&pm, 1, &sp)) != RMM_OK) return rc;
                 if ((rc = launch_score_select(&pm, sp, true, p.kt, It, nullptr, nullptr, nullptr, w, st)) != RMM_OK) return rc;
-                rc = launch_pack_cols(P, hg, d->Lq, d->Lk, d->Lq * p.ld_p, p.ld_p, 0, 1, It, p.kt, p.kt, Pp, p.ldt, status, st);
-                if (rc != RMM_OK) return rc;
-                rc = launch_pack_rows(v + b * d->v_stride[0], hg, d->Lk, d->Dh, d->v_stride[1], d->v_stride[2], h0, group, It, p.kt,
-                                      p.kt, Vp, d->Dh, status, st);
-                if (rc != RMM_OK) return rc;
+                PackSpec pv[2];
+                pv[0] = pack_cols_spec(P, hg, d->Lq, d->Lk, d->Lq * p.ld_p, p.ld_p, 0, 1, It, p.kt, p.kt, Pp, p.ldt);
+                pv[1] = pack_rows_spec(v + b * d->v_stride[0], hg, d->Lk, d->Dh, d->v_stride[1], d->v_stride[2], h0, group, It, p.kt,
+                                       p.kt, Vp, d->Dh);
+                if ((rc = launch_pack(pv, 2, status, st)) != RMM_OK) return rc;
                 g2.k = p.kt; g2.a = Pp; g2.a_ld = p.ldt; g2.a_sb = d->Lq * p.ldt;
                 g2.b = Vp; g2.b_ld = d->Dh; g2.b_sb = p.kt * d->Dh; g2.b_batches = hg; g2.b_batch_off = 0; g2.b_batch_div = 1;
             } else {

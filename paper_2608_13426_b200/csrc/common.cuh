@@ -79,18 +79,36 @@ struct TcProblem {
 };
 int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream);
 
-// Gather columns: dst[b, r, j] = src[sb, r, idx[b, j]] for j < k with source batch sb = (b + b_off) / b_div
-// (dst row pitch ld_dst >= k; columns k..ld_dst are zeroed).  bf16 only.  idx_stride = elements between the
-// index lists of two batch entries.
-int launch_pack_cols(const __nv_bfloat16 *src, int64_t batch, int64_t rows, int64_t K, int64_t s_batch, int64_t s_row,
-                     int64_t b_off, int64_t b_div, const int32_t *idx, int64_t idx_stride, int64_t k,
-                     __nv_bfloat16 *dst, int64_t ld_dst, int *status, cudaStream_t stream);
-
-// Gather rows: dst[b, j, 0:n] = src[sb, idx[b, j], 0:n] for j < k (NULL idx: rows 0 .. k-1), 16-byte vectors:
-// n, both pitches and both bases must be multiples of 8 elements.  Source batch sb = (b + b_off) / b_div.
-int launch_pack_rows(const __nv_bfloat16 *src, int64_t batch, int64_t K, int64_t n, int64_t s_batch, int64_t s_row,
-                     int64_t b_off, int64_t b_div, const int32_t *idx, int64_t idx_stride, int64_t k,
-                     __nv_bfloat16 *dst, int64_t ld_dst, int *status, cudaStream_t stream);
+// One gather of kept slices (see pack.cu).  Columns: dst[b, r, j] = src[sb, r, idx[b, j]], j < k, dst row pitch
+// ld_dst >= k (columns k .. ld_dst zeroed).  Rows: dst[b, j, 0:n] = src[sb, idx[b, j], 0:n].  NULL idx = 0 .. k-1.
+// Source batch sb = (b + b_off) / b_div; idx lists of two batch entries are idx_stride apart.  bf16 only.
+struct PackSpec {
+    int rows_gather;  // 0: column gather, 1: row gather
+    const __nv_bfloat16 *src;
+    __nv_bfloat16 *dst;
+    const int32_t *idx;
+    int64_t batch;
+    int64_t rows;     // column gather: rows of src and dst
+    int64_t K;        // index range: columns of src (column gather) or rows of src (row gather)
+    int64_t n;        // row gather: row length (multiple of 8)
+    int64_t s_batch, s_row, b_off, b_div, idx_stride, k, ld_dst;
+};
+static inline PackSpec pack_cols_spec(const __nv_bfloat16 *src, int64_t batch, int64_t rows, int64_t K, int64_t s_batch,
+                                      int64_t s_row, int64_t b_off, int64_t b_div, const int32_t *idx, int64_t idx_stride,
+                                      int64_t k, __nv_bfloat16 *dst, int64_t ld_dst)
+{
+    PackSpec s = {0, src, dst, idx, batch, rows, K, 0, s_batch, s_row, b_off, b_div, idx_stride, k, ld_dst};
+    return s;
+}
+static inline PackSpec pack_rows_spec(const __nv_bfloat16 *src, int64_t batch, int64_t K, int64_t n, int64_t s_batch,
+                                      int64_t s_row, int64_t b_off, int64_t b_div, const int32_t *idx, int64_t idx_stride,
+                                      int64_t k, __nv_bfloat16 *dst, int64_t ld_dst)
+{
+    PackSpec s = {1, src, dst, idx, batch, 0, K, n, s_batch, s_row, b_off, b_div, idx_stride, k, ld_dst};
+    return s;
+}
+// One launch for one or two gathers.
+int launch_pack(const PackSpec *specs, int n, int *status, cudaStream_t stream);
 
 // ---- attention helpers --------------------------------------------------------------------------------
 // Row softmax of fp32 logits S [heads, Lq, ld_s] with optional end-aligned causal mask; writes bf16

@@ -518,20 +518,21 @@ int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, i
         else { p.b_sb = B->stride_batch; }
         return launch_gemm_tc_problem(p, stream);
     }
-    rc = launch_pack_cols(a_src, batch, M, K, A->stride_batch, A->stride_row, 0, 1, idx, k, k, Ap, plan.ldp, status, stream);
-    if (rc != RMM_OK) return rc;
+    // A[:, I] and the kept slices of B are gathered by one launch
+    PackSpec specs[2];
+    specs[0] = pack_cols_spec(a_src, batch, M, K, A->stride_batch, A->stride_row, 0, 1, idx, k, k, Ap, plan.ldp);
     p.a = Ap; p.a_ld = plan.ldp; p.a_sb = M * plan.ldp;
     if (plan.b_kmajor) {
-        // B is K-contiguous ([N, K] in memory): pack B[idx, :]^T into Bp [batch, N, ldp]; a shared B
-        // (stride_batch 0) is packed once per index set
-        rc = launch_pack_cols(b_src, batch, N, K, B->stride_batch, B->stride_col, 0, 1, idx, k, k, Bp, plan.ldp, status, stream);
-        if (rc != RMM_OK) return rc;
+        // B is K-contiguous ([N, K] in memory): B[idx, :]^T goes to Bp [batch, N, ldp]; a shared B (stride_batch 0)
+        // is packed once per index set
+        specs[1] = pack_cols_spec(b_src, batch, N, K, B->stride_batch, B->stride_col, 0, 1, idx, k, k, Bp, plan.ldp);
         p.b = Bp; p.b_ld = plan.ldp; p.b_sb = N * plan.ldp;
     } else {
-        rc = launch_pack_rows(b_src, batch, K, N, B->stride_batch, B->stride_row, 0, 1, idx, k, k, Bp, N, status, stream);
-        if (rc != RMM_OK) return rc;
+        specs[1] = pack_rows_spec(b_src, batch, K, N, B->stride_batch, B->stride_row, 0, 1, idx, k, k, Bp, N);
         p.b = Bp; p.b_ld = N; p.b_sb = k * N;
     }
+    rc = launch_pack(specs, 2, status, stream);
+    if (rc != RMM_OK) return rc;
     return launch_gemm_tc_problem(p, stream);
 }
 

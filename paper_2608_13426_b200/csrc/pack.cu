@@ -1,60 +1,102 @@
-// Column gather dst[b, r, j] = src[b, r, idx[b, j]] (bf16): brings A[:, I] (paper Sec. 3.2) into a
-// contiguous K-major operand that a TMA tile load can fetch.  A's contraction axis is its contiguous
-// axis, so the gather is element-granular and no bulk-copy engine can do it.
+// Gathers that bring the kept slices of the contraction axis (paper Sec. 3.2: A[:, I] and B[I, :]) into
+// contiguous operands that TMA tile loads can fetch.  Up to two gathers run in ONE launch (e.g. A[:, I] and
+// B[I, :] of a product, or Q[:, I] and K[:, I] of an attention head group): block ranges are split between them.
 //
-// One warp owns 256 adjacent output columns of a few rows.  Lane l produces the output pairs
-// (2l, 2l+1) + 64 i, so that the 32 lanes of one load instruction read 64 neighbouring kept columns
-// (a few 32-byte sectors) and one store instruction writes 128 contiguous bytes.  The index pairs
-// are read once per warp and kept in registers for all of its rows.
+// Column gather  dst[b, r, j] = src[sb, r, idx[b, j]]   (the contraction axis is the contiguous one: element-granular,
+//                so no bulk-copy engine can do it).  A block stages R whole source rows in shared memory with
+//                coalesced 16-byte loads, then every thread builds pairs of output elements from shared memory and
+//                writes 4 bytes; the index pairs are read once per thread and reused for the R rows.  Rows too long
+//                for shared memory, or not 16-byte aligned, take the direct form (2-byte gathers from global memory).
+// Row gather     dst[b, j, :] = src[sb, idx[b, j], :]    16-byte vectors, 4 kept rows per block.
+// sb = (b + b_off) / b_div maps a batch entry to its source (grouped-query heads share K and V).
 #include "common.cuh"
 
 namespace rmm {
 namespace {
 
-constexpr int kWarps = 8;
-constexpr int kRowsPerBlock = 8;   // rows per warp, all in flight at once (the pass is latency-bound otherwise)
-constexpr int kRowVecThreads = 256;
+constexpr int kThreadsPack = 256;
+constexpr int kMaxStageBytes = 96 * 1024;  // longest source row that is staged in shared memory
+constexpr int kStageTarget = 32 * 1024;    // preferred staging size: several blocks per SM stay resident
+constexpr int kDirectRows = 8;
 
-__global__ void __launch_bounds__(kWarps * 32) pack_cols_kernel(const __nv_bfloat16 *__restrict__ src, int64_t rows,
-                                                                int64_t K, int64_t s_batch, int64_t s_row,
-                                                                int64_t b_off, int64_t b_div,
-                                                                const int32_t *__restrict__ idx, int64_t idx_stride,
-                                                                int64_t k, __nv_bfloat16 *__restrict__ dst,
-                                                                int64_t ld_dst, int *status)
+struct PackJob {
+    int type;  // 0 none, 1 columns staged, 2 columns direct, 3 rows
+    const __nv_bfloat16 *src;
+    __nv_bfloat16 *dst;
+    const int32_t *idx;
+    int64_t batch, rows, K, s_batch, s_row, b_off, b_div, idx_stride, k, ld_dst, n;
+    int R;                      // staged rows per block
+    int64_t bx, by, blocks;     // block grid of this job: bx * by * batch
+};
+
+struct PackArgs {
+    PackJob job[2];
+    int *status;
+};
+
+__device__ __forceinline__ int checked_index(const int32_t *ix, int64_t j, int64_t k, int64_t K, int *status)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t b = blockIdx.z;
-    const int64_t j0 = ((int64_t)blockIdx.x * kWarps + warp) * 256;  // first output column of this warp
-    if (j0 >= ld_dst) return;
-    const int32_t *ix = idx != nullptr ? idx + b * idx_stride : nullptr;  // NULL: columns 0 .. k-1 in order
+    if (j >= k) return -1;
+    int v = ix != nullptr ? __ldg(ix + j) : (int)j;
+    if (v < 0 || v >= K) {
+        atomicExch(status, (int)RMM_ERR_BOUNDS);
+        return -1;
+    }
+    return v;
+}
 
-    int c[8];  // source columns of this lane's 4 output pairs; -1 = write zero
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            int64_t j = j0 + 64 * i + 2 * lane + h;
-            int v = -1;
-            if (j < k) {
-                v = ix != nullptr ? __ldg(ix + j) : (int)j;
-                if (v < 0 || v >= K) {
-                    atomicExch(status, (int)RMM_ERR_BOUNDS);
-                    v = -1;
-                }
-            }
-            c[2 * i + h] = v;
+__device__ void pack_cols_staged(const PackJob &p, int64_t blk, int *status, unsigned char *smem)
+{
+    const int64_t b = blk / p.bx, r0 = (blk % p.bx) * p.R;
+    const int tid = threadIdx.x;
+    const int kv = (int)(p.K / 8);  // 16-byte vectors per source row
+    const unsigned short *s16 = reinterpret_cast<const unsigned short *>(p.src) + ((b + p.b_off) / p.b_div) * p.s_batch;
+    uint4 *stage = reinterpret_cast<uint4 *>(smem);
+    const int nrows = (int)min((int64_t)p.R, p.rows - r0);
+    for (int r = 0; r < nrows; ++r) {
+        const uint4 *srow = reinterpret_cast<const uint4 *>(s16 + (r0 + r) * p.s_row);
+        uint4 *drow = stage + (size_t)r * kv;
+#pragma unroll 4
+        for (int c = tid; c < kv; c += kThreadsPack) drow[c] = __ldg(srow + c);
+    }
+    __syncthreads();
+    const unsigned short *rows = reinterpret_cast<const unsigned short *>(smem);
+    const int32_t *ix = p.idx != nullptr ? p.idx + b * p.idx_stride : nullptr;
+    unsigned *d32 = reinterpret_cast<unsigned *>(p.dst + b * p.rows * p.ld_dst);
+    const int half = (int)(p.ld_dst / 2), K = (int)p.K;
+    unsigned *drow0 = d32 + ((r0 * p.ld_dst) >> 1);
+    for (int jp = tid; jp < half; jp += kThreadsPack) {
+        const int c0 = checked_index(ix, 2 * jp, p.k, p.K, status), c1 = checked_index(ix, 2 * jp + 1, p.k, p.K, status);
+        for (int r = 0; r < nrows; ++r) {
+            const unsigned short *row = rows + r * K;
+            const unsigned lo = c0 >= 0 ? row[c0] : 0u, hi = c1 >= 0 ? row[c1] : 0u;
+            drow0[(size_t)r * half + jp] = lo | (hi << 16);
         }
     }
+}
 
-    const unsigned short *s16 = reinterpret_cast<const unsigned short *>(src) + ((b + b_off) / b_div) * s_batch;
-    unsigned *d32 = reinterpret_cast<unsigned *>(dst + b * rows * ld_dst);
-    const int64_t r_begin = (int64_t)blockIdx.y * kRowsPerBlock;
-    const int64_t r_end = min(rows, r_begin + kRowsPerBlock);
-    unsigned out[kRowsPerBlock][4];
+// One warp owns 256 adjacent output columns of kDirectRows rows.  Lane l produces the output pairs (2l, 2l+1) + 64 i,
+// so the 32 lanes of one load read neighbouring kept columns and one store writes 128 contiguous bytes.
+__device__ void pack_cols_direct(const PackJob &p, int64_t blk, int *status)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t b = blk / (p.bx * p.by), rem = blk % (p.bx * p.by);
+    const int64_t j0 = ((rem % p.bx) * (kThreadsPack / 32) + warp) * 256;
+    const int64_t r_begin = (rem / p.bx) * kDirectRows, r_end = min(p.rows, r_begin + kDirectRows);
+    if (j0 >= p.ld_dst) return;
+    const int32_t *ix = p.idx != nullptr ? p.idx + b * p.idx_stride : nullptr;
+    int c[8];
 #pragma unroll
-    for (int rr = 0; rr < kRowsPerBlock; ++rr) {
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) c[2 * i + h] = checked_index(ix, j0 + 64 * i + 2 * lane + h, p.k, p.K, status);
+    const unsigned short *s16 = reinterpret_cast<const unsigned short *>(p.src) + ((b + p.b_off) / p.b_div) * p.s_batch;
+    unsigned *d32 = reinterpret_cast<unsigned *>(p.dst + b * p.rows * p.ld_dst);
+    unsigned out[kDirectRows][4];
+#pragma unroll
+    for (int rr = 0; rr < kDirectRows; ++rr) {
         const int64_t r = r_begin + rr;
-        const unsigned short *row = s16 + (r < r_end ? r : r_begin) * s_row;
+        const unsigned short *row = s16 + (r < r_end ? r : r_begin) * p.s_row;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             unsigned lo = c[2 * i] >= 0 ? (unsigned)__ldg(row + c[2 * i]) : 0u;
@@ -63,82 +105,117 @@ __global__ void __launch_bounds__(kWarps * 32) pack_cols_kernel(const __nv_bfloa
         }
     }
 #pragma unroll
-    for (int rr = 0; rr < kRowsPerBlock; ++rr) {
+    for (int rr = 0; rr < kDirectRows; ++rr) {
         const int64_t r = r_begin + rr;
         if (r >= r_end) break;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             int64_t j = j0 + 64 * i + 2 * lane;
-            if (j < ld_dst) d32[(r * ld_dst + j) >> 1] = out[rr][i];
+            if (j < p.ld_dst) d32[(r * p.ld_dst + j) >> 1] = out[rr][i];
         }
     }
 }
 
-// Row gather with 16-byte vectors: one block copies 4 kept rows.
-__global__ void __launch_bounds__(kRowVecThreads) pack_rows_kernel(const uint4 *__restrict__ src, int64_t K, int64_t nvec,
-                                                                   int64_t s_batch_v, int64_t s_row_v, int64_t b_off,
-                                                                   int64_t b_div, const int32_t *__restrict__ idx,
-                                                                   int64_t idx_stride, int64_t k, uint4 *__restrict__ dst,
-                                                                   int64_t ld_dst_v, int *status)
+__device__ void pack_rows(const PackJob &p, int64_t blk, int *status)
 {
-    const int64_t b = blockIdx.z;
-    const int64_t j0 = (int64_t)blockIdx.y * 4;
-    const uint4 *sbase = src + ((b + b_off) / b_div) * s_batch_v;
-    uint4 *dbase = dst + (b * k) * ld_dst_v;
+    const int64_t b = blk / (p.bx * p.by), rem = blk % (p.bx * p.by);
+    const int64_t j0 = (rem / p.bx) * 4, nvec = p.n / 8;
+    const uint4 *sbase = reinterpret_cast<const uint4 *>(p.src) + ((b + p.b_off) / p.b_div) * (p.s_batch / 8);
+    uint4 *dbase = reinterpret_cast<uint4 *>(p.dst) + (b * p.k) * (p.ld_dst / 8);
+    const int32_t *ix = p.idx != nullptr ? p.idx + b * p.idx_stride : nullptr;
     int rows[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        int v = -1;
-        if (j0 + i < k) {
-            v = idx != nullptr ? __ldg(idx + b * idx_stride + j0 + i) : (int)(j0 + i);
-            if (v < 0 || v >= K) {
-                if (threadIdx.x == 0) atomicExch(status, (int)RMM_ERR_BOUNDS);
-                v = -2;  // write zeros
-            }
-        }
-        rows[i] = v;
+        rows[i] = j0 + i < p.k ? checked_index(ix, j0 + i, p.k, p.K, status) : -2;  // -1: bad index, write zeros; -2: no row
     }
-    for (int64_t c = (int64_t)blockIdx.x * kRowVecThreads + threadIdx.x; c < nvec; c += (int64_t)gridDim.x * kRowVecThreads) {
+    for (int64_t c = (rem % p.bx) * kThreadsPack + threadIdx.x; c < nvec; c += p.bx * kThreadsPack) {
         uint4 v[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) v[i] = rows[i] >= 0 ? __ldg(sbase + rows[i] * s_row_v + c) : make_uint4(0, 0, 0, 0);
+        for (int i = 0; i < 4; ++i) v[i] = rows[i] >= 0 ? __ldg(sbase + rows[i] * (p.s_row / 8) + c) : make_uint4(0, 0, 0, 0);
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            if (rows[i] != -1) dbase[(j0 + i) * ld_dst_v + c] = v[i];
+            if (rows[i] != -2) dbase[(j0 + i) * (p.ld_dst / 8) + c] = v[i];
     }
+}
+
+__global__ void __launch_bounds__(kThreadsPack, 4) pack_kernel(const __grid_constant__ PackArgs a)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    int64_t blk = blockIdx.x;
+    const int which = blk < a.job[0].blocks ? 0 : 1;
+    if (which == 1) blk -= a.job[0].blocks;
+    const PackJob &p = a.job[which];
+    if (p.type == 1) pack_cols_staged(p, blk, a.status, smem);
+    else if (p.type == 2) pack_cols_direct(p, blk, a.status);
+    else if (p.type == 3) pack_rows(p, blk, a.status);
+}
+
+size_t plan_job(PackJob &p)
+{
+    size_t smem = 0;
+    if (p.type == 1) {
+        const bool staged = p.K % 8 == 0 && p.s_row % 8 == 0 && p.s_batch % 8 == 0 && reinterpret_cast<uintptr_t>(p.src) % 16 == 0 &&
+                            p.K * 2 <= kMaxStageBytes;
+        if (staged) {
+            int R = (int)(kStageTarget / (p.K * 2));
+            if (R < 1) R = 1;
+            if (R > 8) R = 8;
+            if (R > p.rows) R = (int)p.rows;
+            p.R = R;
+            p.bx = ceil_div(p.rows, R);
+            p.by = 1;
+            smem = (size_t)R * p.K * 2;
+        } else {
+            p.type = 2;
+            p.bx = ceil_div(p.ld_dst, 256 * (kThreadsPack / 32));
+            p.by = ceil_div(p.rows, kDirectRows);
+        }
+    } else if (p.type == 3) {
+        int64_t gx = ceil_div(p.n / 8, kThreadsPack);
+        p.bx = gx > 8 ? 8 : gx;
+        p.by = ceil_div(p.k, 4);
+    }
+    p.blocks = p.type == 0 ? 0 : p.bx * p.by * p.batch;
+    return smem;
 }
 
 }  // namespace
 
-int launch_pack_cols(const __nv_bfloat16 *src, int64_t batch, int64_t rows, int64_t K, int64_t s_batch, int64_t s_row,
-                     int64_t b_off, int64_t b_div, const int32_t *idx, int64_t idx_stride, int64_t k,
-                     __nv_bfloat16 *dst, int64_t ld_dst, int *status, cudaStream_t stream)
+int launch_pack(const PackSpec *specs, int n, int *status, cudaStream_t stream)
 {
-    if (ld_dst % 2 != 0) return fail(RMM_ERR_UNSUPPORTED, "pack: destination pitch must be even");
-    dim3 grid((unsigned)ceil_div(ld_dst, 256 * kWarps), (unsigned)ceil_div(rows, kRowsPerBlock), (unsigned)batch);
-    if (grid.y > 65535u || grid.z > 65535u) return fail(RMM_ERR_UNSUPPORTED, "pack: rows/32 or batch exceeds 65535");
-    prof_begin("pack_cols_kernel", stream);
-    pack_cols_kernel<<<grid, kWarps * 32, 0, stream>>>(src, rows, K, s_batch, s_row, b_off, b_div > 0 ? b_div : 1, idx, idx_stride, k, dst,
-                                                               ld_dst, status);
-    return check_launch("pack_cols_kernel", stream);
-}
-
-int launch_pack_rows(const __nv_bfloat16 *src, int64_t batch, int64_t K, int64_t n, int64_t s_batch, int64_t s_row,
-                     int64_t b_off, int64_t b_div, const int32_t *idx, int64_t idx_stride, int64_t k,
-                     __nv_bfloat16 *dst, int64_t ld_dst, int *status, cudaStream_t stream)
-{
-    if (n % 8 || s_batch % 8 || s_row % 8 || ld_dst % 8 || reinterpret_cast<uintptr_t>(src) % 16 || reinterpret_cast<uintptr_t>(dst) % 16)
-        return fail(RMM_ERR_UNSUPPORTED, "pack_rows: operands must be 16-byte aligned with pitches that are multiples of 8");
-    const int64_t nvec = n / 8;
-    int64_t gx = ceil_div(nvec, kRowVecThreads);
-    if (gx > 8) gx = 8;
-    dim3 grid((unsigned)gx, (unsigned)ceil_div(k, 4), (unsigned)batch);
-    if (grid.y > 65535u || grid.z > 65535u) return fail(RMM_ERR_UNSUPPORTED, "pack_rows: k/4 or batch exceeds 65535");
-    prof_begin("pack_rows_kernel", stream);
-    pack_rows_kernel<<<grid, kRowVecThreads, 0, stream>>>(reinterpret_cast<const uint4 *>(src), K, nvec, s_batch / 8, s_row / 8, b_off,
-                                                         b_div > 0 ? b_div : 1, idx, idx_stride, k,
-                                                         reinterpret_cast<uint4 *>(dst), ld_dst / 8, status);
-    return check_launch("pack_rows_kernel", stream);
+    if (n < 1 || n > 2) return fail(RMM_ERR_INVALID_ARG, "pack: one or two gathers per launch");
+    PackArgs a = {};
+    a.status = status;
+    size_t smem = 0;
+    int64_t blocks = 0;
+    for (int i = 0; i < n; ++i) {
+        const PackSpec &s = specs[i];
+        PackJob &p = a.job[i];
+        p.type = s.rows_gather ? 3 : 1;
+        p.src = s.src; p.dst = s.dst; p.idx = s.idx;
+        p.batch = s.batch; p.rows = s.rows; p.K = s.K; p.s_batch = s.s_batch; p.s_row = s.s_row;
+        p.b_off = s.b_off; p.b_div = s.b_div > 0 ? s.b_div : 1; p.idx_stride = s.idx_stride; p.k = s.k; p.ld_dst = s.ld_dst; p.n = s.n;
+        if (s.rows_gather) {
+            if (s.n % 8 || s.s_batch % 8 || s.s_row % 8 || s.ld_dst % 8 || reinterpret_cast<uintptr_t>(s.src) % 16 ||
+                reinterpret_cast<uintptr_t>(s.dst) % 16)
+                return fail(RMM_ERR_UNSUPPORTED, "pack: row gather needs 16-byte aligned operands and pitches that are multiples of 8");
+        } else if (s.ld_dst % 2 != 0) {
+            return fail(RMM_ERR_UNSUPPORTED, "pack: destination pitch must be even");
+        }
+        size_t sm = plan_job(p);
+        if (sm > smem) smem = sm;
+        blocks += p.blocks;
+    }
+    if (blocks > INT32_MAX) return fail(RMM_ERR_UNSUPPORTED, "pack: too many blocks");
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxStageBytes);
+        if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "pack: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+        configured = true;
+    }
+    prof_begin("pack_kernel", stream);
+    pack_kernel<<<(unsigned)blocks, kThreadsPack, smem, stream>>>(a);
+    return check_launch("pack_kernel", stream);
 }
 
 }  // namespace rmm
