@@ -90,6 +90,21 @@ size_t rmm_score_select_workspace_bytes(const rmm_mat_t *A, int axis);
 int rmm_score_select(const rmm_mat_t *A, int axis, double rho, int64_t k, int32_t *idx, float *scores, float *energy,
                      float *retained, void *ws, size_t ws_bytes, void *stream);
 
+/* rmm_score_select without a workspace argument (the paper has no counterpart).  For callers that cannot allocate
+ * device memory at all (code running where the allocator must not be touched: a frozen memory pool, a plugin that is
+ * handed inputs and outputs only, a latency-critical loop), the scratch lives in a device array built into the
+ * library: rmm_score_select_static_capacity() bytes (4 MiB), held by every GPU that loads the library until the
+ * process exits.  A problem whose scratch (about 8 * row_splits * n + 4 * n bytes per batch element, see
+ * rmm_score_select_workspace_bytes) exceeds the capacity is refused with RMM_ERR_WORKSPACE and a message; nothing is
+ * launched.  The call allocates nothing and frees nothing.  Its first call on each device looks the array's device
+ * address up (with that device current), so make that first call outside any stream capture.  All calls share the
+ * one array per device: it keeps the previous call's contents (the part that must start at zero is cleared on the
+ * stream by every call), and two calls that overlap on the GPU (different streams) race.  Results are those of
+ * rmm_score_select, bit for bit.  idx, scores, energy, retained as there. */
+size_t rmm_score_select_static_capacity(void);
+int rmm_score_select_static(const rmm_mat_t *A, int axis, double rho, int64_t k, int32_t *idx, float *scores,
+                            float *energy, float *retained, void *stream);
+
 /* Y = scale * A[:, I] B[I, :] (Sec. 3.2, RMM_rho(A,B); no rescaling: pass scale = 1).
  *   A    [b, M, K]; B [b or shared, K, N] (stride_batch 0 = shared); Y [b, M, N] (written in full)
  *   idx  int32 [b, k], each entry in [0, K) (NULL with k == K: the unreduced product, nothing is gathered); any set is accepted (so a cached or random set gives

@@ -15,6 +15,8 @@ from .binding import (  # noqa: F401
     rmm_reduced_gemm,
     rmm_score,
     rmm_score_select,
+    rmm_score_select_static,
+    rmm_score_select_static_capacity,
     rmm_select,
     rmm_status_read,
 )

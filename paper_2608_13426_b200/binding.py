@@ -46,7 +46,8 @@ class rmm_attn_desc_t(ctypes.Structure):
 
 
 EXPORTS = ["rmm_keep_count", "rmm_score_workspace_bytes", "rmm_score", "rmm_select_workspace_bytes", "rmm_select",
-           "rmm_score_select_workspace_bytes", "rmm_score_select", "rmm_reduced_gemm_workspace_bytes",
+           "rmm_score_select_workspace_bytes", "rmm_score_select", "rmm_score_select_static",
+           "rmm_score_select_static_capacity", "rmm_reduced_gemm_workspace_bytes",
            "rmm_reduced_gemm", "rmm_reduced_attn_workspace_bytes", "rmm_reduced_attn",
            "rmm_product_host_workspace_bytes", "rmm_product_host", "rmm_status_read", "rmm_last_error",
            "rmm_launch_count", "rmm_profile_kernels", "rmm_profile_count", "rmm_profile_name"]
@@ -75,6 +76,8 @@ def lib() -> ctypes.CDLL:
     L.rmm_score_select_workspace_bytes.argtypes = [mp, i32]
     L.rmm_score_select_workspace_bytes.restype = sz
     L.rmm_score_select.argtypes = [mp, i32, dbl, i64, vp, vp, vp, vp, vp, sz, vp]
+    L.rmm_score_select_static.argtypes = [mp, i32, dbl, i64, vp, vp, vp, vp, vp]
+    L.rmm_score_select_static_capacity.restype = sz
     L.rmm_reduced_gemm_workspace_bytes.argtypes = [mp, mp, i64, mp]
     L.rmm_reduced_gemm_workspace_bytes.restype = sz
     L.rmm_reduced_gemm.argtypes = [mp, mp, vp, i64, flt, mp, vp, sz, vp]
@@ -255,6 +258,21 @@ def rmm_score_select(A: torch.Tensor, rho: float = 0.0, k: int = 0, axis: int = 
                                   energy.data_ptr() if want_energy else None,
                                   ret.data_ptr() if want_retained else None, p, nb, _stream()))
     return idx, scores, energy, ret
+
+
+def rmm_score_select_static(A: torch.Tensor, idx: torch.Tensor, rho: float = 0.0, k: int = 0, axis: int = 1,
+                            energy: Optional[torch.Tensor] = None, retained: Optional[torch.Tensor] = None) -> None:
+    """Fused score + top-k for callers that cannot allocate: no workspace is passed, the scratch is a device array
+    built into the library.  Every buffer is the caller's: idx int32 [batch, k] (or [k]), optional energy fp32
+    [batch, n] and retained fp32 [batch] are written in place.  This wrapper itself allocates nothing on the device."""
+    m = as_mat(A)
+    _check(lib().rmm_score_select_static(ctypes.byref(m), axis, float(rho), int(k), idx.data_ptr(), None,
+                                         energy.data_ptr() if energy is not None else None,
+                                         retained.data_ptr() if retained is not None else None, _stream()))
+
+
+def rmm_score_select_static_capacity() -> int:
+    return int(lib().rmm_score_select_static_capacity())
 
 
 def rmm_reduced_gemm(A: torch.Tensor, B: torch.Tensor, idx: Optional[torch.Tensor], scale: float = 1.0,

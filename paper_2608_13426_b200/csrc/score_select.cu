@@ -718,3 +718,69 @@ int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_
 }
 
 }  // namespace rmm
+
+// ------------------------------------------------------------------------------------------------------------------
+// rmm_score_select_static: fused score + select for callers that cannot hand the library any scratch memory.
+//
+// Some callers run where device allocation is off the table: inside a region that must not touch the allocator (a
+// real-time loop, a plugin sandbox whose host gives it inputs and outputs only, code that runs after the memory pool
+// has been frozen), so they can neither cudaMalloc a workspace nor ask a framework for one.  For them the scratch of
+// the score pass (row-split partial sums, arrival counters, the energy keys) lives in the file-scope device array
+// below.  Every GPU that loads this library carries the array until the process exits.
+// ------------------------------------------------------------------------------------------------------------------
+#define RMM_STATIC_SCRATCH_BYTES (4u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[RMM_STATIC_SCRATCH_BYTES];
+
+namespace rmm {
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_ptr[kMaxDevices];  // device address of g_static_scratch, per device; NULL until set up
+
+// In host code `g_static_scratch` names a host-side shadow of the symbol, not device memory: the device address has
+// to be asked for, once per device, with that device current.
+int static_scratch(void **out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "score_select_static: cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= kMaxDevices) return fail(RMM_ERR_UNSUPPORTED, "score_select_static: device index %d is not covered", dev);
+    if (g_static_scratch_ptr[dev] == nullptr) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || p == nullptr)
+            return fail(RMM_ERR_CUDA, "score_select_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        g_static_scratch_ptr[dev] = p;
+    }
+    *out = g_static_scratch_ptr[dev];
+    return RMM_OK;
+}
+}  // namespace
+}  // namespace rmm
+
+extern "C" size_t rmm_score_select_static_capacity(void) { return RMM_STATIC_SCRATCH_BYTES; }
+
+extern "C" int rmm_score_select_static(const rmm_mat_t *A, int axis, double rho, int64_t k, int32_t *idx, float *scores,
+                                       float *energy, float *retained, void *stream)
+{
+    using namespace rmm;
+    ScorePlan p;
+    int rc = plan_score(A, axis, &p);
+    if (rc != RMM_OK) return rc;
+    if (idx == nullptr) return fail(RMM_ERR_INVALID_ARG, "score_select_static: idx is NULL");
+    int64_t kk = k;
+    if (k < 0 || k > p.n) return fail(RMM_ERR_INVALID_ARG, "score_select_static: k = %lld is outside [0, n]", (long long)k);
+    if (k == 0 && (rc = rmm_keep_count(rho, p.n, &kk)) != RMM_OK)
+        return fail(rc, "score_select_static: rho = %g is outside (0, 1]", rho);
+    if (p.total_bytes > RMM_STATIC_SCRATCH_BYTES)
+        return fail(RMM_ERR_WORKSPACE,
+                    "score_select_static: this problem needs %zu bytes of scratch but the built-in array holds %u; "
+                    "use rmm_score_select with a caller-provided workspace",
+                    p.total_bytes, (unsigned)RMM_STATIC_SCRATCH_BYTES);
+    void *ws = nullptr;
+    if ((rc = static_scratch(&ws)) != RMM_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the previous call left: the status word and the arrival counters must start at zero
+    cudaError_t e = cudaMemsetAsync(ws, 0, RMM_WS_HEADER_BYTES, st);
+    if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "score_select_static: cudaMemsetAsync: %s", cudaGetErrorString(e));
+    return launch_score_select(A, p, true, kk, idx, scores, energy, retained, ws, st);
+}
