@@ -121,16 +121,24 @@ def barrier(world):
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
-    torch.cuda.synchronize()
+    if torch.cuda.is_available():
+        torch.cuda.synchronize()
 
 
 def max_over_ranks(x: float, world: int) -> float:
+    """The slowest rank's time (replicas are independent: the job is as slow as its slowest replica)."""
     if world == 1:
         return x
     import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([x], dtype=torch.float64, device=dev)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def whole_job_value(ms_step: float, world: int, rho: float = RHO) -> float:
+    """TFLOP/s of the whole job: every replica retains the same FLOPs per step; ms_step is the max over ranks."""
+    return world * retained_flops(rho) / (ms_step * 1e-3) / 1e12
 
 
 def time_region(fn, steps: int, world: int) -> float:
@@ -259,7 +267,7 @@ def main():
     gemm_ms = [t for _, t in timer.times_ms()]
     gemm_ms_avg = sum(gemm_ms) / len(gemm_ms)
     assert rmm.rmm_status_read() == 0
-    value = world * retained_flops(RHO) / (ms_step * 1e-3) / 1e12
+    value = whole_job_value(ms_step, world)
 
     # ---- roofline of the dominant kernel (the tensor-core GEMM): retained FLOPs of one launch / its mean duration
     achieved = retained_flops(RHO) / (gemm_ms_avg * 1e-3) / 1e12

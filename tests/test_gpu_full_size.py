@@ -1,0 +1,126 @@
+"""Parity at the full sizes of the benchmark configurations (GPU only): index sets are checked in full against
+the oracle, products on sampled rows that the oracle computes one by one (tile edges included)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_13426_b200 as rmm
+from paper_2608_13426_b200 import synth
+from test_gpu_parity import TOL_BF16, check_index_set, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _device():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    torch.cuda.set_device(0)
+    yield
+    assert rmm.rmm_status_read() == 0
+
+
+def sample_rows(n, count, seed=0):
+    edges = [0, 1, 127, 128, 129, n // 2 - 1, n // 2, n - 2, n - 1]
+    extra = np.random.default_rng(seed).choice(n, count, replace=False).tolist()
+    return sorted({r for r in edges + extra if 0 <= r < n})
+
+
+@pytest.mark.parametrize("rho", [0.5, 0.75])
+def test_attention_prefill_qk_head_dim_reduction(oracle, rho):
+    """7B-class prefill: 32 heads, seq 4096, head_dim 128, 4 outlier dims per head x10; index set per head from Q,
+    S~ = Q[:, I] K[:, I]^T / sqrt(128) written as a batched product with K-contiguous B."""
+    H, L, Dh = 32, 4096, 128
+    Q, K, _ = synth.attention_qkv(1, H, H, L, L, Dh, seed=0)
+    Qd, Kd = Q[0].cuda(), K[0].cuda()
+    kd = oracle.keep_count(rho, Dh)
+    idx, _, _, _ = rmm.rmm_score_select(Qd, rho=rho)
+    S = rmm.rmm_reduced_gemm(Qd, Kd.transpose(1, 2), idx, scale=1.0 / math.sqrt(Dh))
+    assert S.shape == (H, L, L) and S.dtype == torch.bfloat16
+    idx_np = idx.cpu().numpy()
+    rows = sample_rows(L, 3)
+    for h in range(H):
+        e64, _ = oracle.score(Q[0, h])
+        check_index_set(idx_np[h], e64, kd)
+        for r in rows:
+            want = oracle.reduced_gemm(Q[0, h], K[0, h].T, idx_np[h], rows=(r, r + 1))[r] / math.sqrt(Dh)
+            assert rel_fro(S[h, r].float().cpu().numpy(), want) <= TOL_BF16
+
+
+@pytest.mark.parametrize("rho", [0.25, 0.5])
+def test_long_context_pv_sequence_reduction(oracle, rho):
+    """Long-context PV: seq 16384, head_dim 128, P = causal softmax given as a bf16 input, keys selected per head.
+    Two of the 32 heads (P alone is 0.5 GB per head)."""
+    H, L, Dh = 2, 16384, 128
+    P = synth.attention_probs(L, H, Dh, seed=3, causal=True, device="cuda")
+    V = synth.gaussian((H, L, Dh), 1.0, seed=5).cuda()
+    kt = oracle.keep_count(rho, L)
+    idx, _, _, ret = rmm.rmm_score_select(P, rho=rho, want_retained=True)
+    O = rmm.rmm_reduced_gemm(P, V, idx)
+    idx_np = idx.cpu().numpy()
+    Pc, Vc = P.cpu(), V.cpu()
+    rows = sample_rows(L, 4)
+    for h in range(H):
+        e64, _ = oracle.score(Pc[h])
+        check_index_set(idx_np[h], e64, kt)
+        _, kept = oracle.select(e64, kt)
+        assert float(ret[h]) == pytest.approx(kept / e64.sum(), rel=1e-5)
+        for r in rows:
+            want = oracle.reduced_gemm(Pc[h], Vc[h], idx_np[h], rows=(r, r + 1))[r]
+            got = O[h, r].float().cpu().numpy()
+            assert np.linalg.norm(got - want) <= TOL_BF16 * max(np.linalg.norm(want), 1e-3)
+
+
+def test_70b_class_projection_sampled(oracle):
+    """70B-class K/V projection: 32768 tokens x 8192 hidden -> 1024, activations with 1 % heavy-tailed channels;
+    the score pass and the select run at full size, the product is checked on sampled rows."""
+    M, K, N = 32768, 8192, 1024
+    A = synth.heavy_tailed_activations(M, K, seed=7, device="cuda")
+    B = synth.weight(K, N, seed=8, device="cuda")
+    Ac, Bc = A.cpu(), B.cpu()
+    e64, _ = oracle.score(Ac)
+    for rho in (0.25, 0.75):
+        k = oracle.keep_count(rho, K)
+        Y, idx = rmm.rmm(A, B, rho)
+        idx_np = idx.cpu().numpy()
+        check_index_set(idx_np, e64, k)
+        for r in sample_rows(M, 6, seed=1):
+            want = oracle.reduced_gemm(Ac, Bc, idx_np, rows=(r, r + 1))[r]
+            assert rel_fro(Y[r].float().cpu().numpy(), want) <= TOL_BF16
+
+
+def test_70b_class_down_projection_index_set(oracle):
+    """70B-class down projection: contraction over the 28672-wide intermediate axis (select in its own launch,
+    keys cached in shared memory); index set in full, product on sampled rows of a 4096-token slice."""
+    M, K, N = 4096, 28672, 8192
+    A = synth.heavy_tailed_activations(M, K, seed=9, device="cuda")
+    B = synth.weight(K, N, seed=10, device="cuda")
+    Ac, Bc = A.cpu(), B.cpu()
+    e64, _ = oracle.score(Ac)
+    k = oracle.keep_count(0.5, K)
+    Y, idx = rmm.rmm(A, B, 0.5)
+    idx_np = idx.cpu().numpy()
+    check_index_set(idx_np, e64, k)
+    for r in sample_rows(M, 3, seed=2):
+        want = oracle.reduced_gemm(Ac, Bc, idx_np, rows=(r, r + 1))[r]
+        assert rel_fro(Y[r].float().cpu().numpy(), want) <= TOL_BF16
+
+
+def test_reduced_attention_multi_tile(oracle):
+    """Reduced attention across several tiles and head groups: 8 query / 2 kv heads, 1536 x 1536, causal."""
+    B, Hq, Hkv, L, Dh = 1, 8, 2, 1536, 128
+    Q, K, V = synth.attention_qkv(B, Hq, Hkv, L, L, Dh, seed=11)
+    O, idx_feat, idx_tok = rmm.rmm_reduced_attn(Q.cuda(), K.cuda(), V.cuda(), True, 0.5, 0.5, want_idx=True)
+    Oo, If, It, P = oracle.attn(Q, K, V, True, 0.5, 0.5, round_p=True, want_p=True)
+    assert np.array_equal(idx_feat.cpu().numpy(), If)
+    got = idx_tok.cpu().numpy()
+    ok_heads = 0
+    for h in range(Hq):
+        a2 = (P[0, h] ** 2).sum(axis=0)
+        assert a2[got[0, h]].sum() >= (1 - 1e-6) * a2[It[0, h]].sum()
+        if np.array_equal(got[0, h], It[0, h]):
+            ok_heads += 1
+            assert rel_fro(O[0, h].float().cpu().numpy(), Oo[0, h]) <= TOL_BF16
+    assert ok_heads >= 1
