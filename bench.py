@@ -33,6 +33,9 @@ RHO = 0.5
 RHOS = (0.25, 0.5, 0.75, 1.0)
 METRIC = "reduced-GEMM retained TFLOP/s (whole RMM op: score + select + reduced product)"
 UNIT = "TFLOP/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the GEMM kernel on this workload at rho = 0.5, from the
+# ncu capture summarised in profiles/reduced_gemm_tc_kernel_mlp_2048x8192x2048_rho0.5.md
+GEMM_DRAM_TRAFFIC_BYTES = 33.67e6
 WORKLOAD = "1B-class MLP down-projection: A 2048x8192 bf16 N(0,1) with 1% Student-t(3) channels, B 8192x2048 bf16 N(0,0.02^2)"
 
 
@@ -221,6 +224,7 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU oracle timing (quick runs, profiling)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-rho sweep")
+    ap.add_argument("--sets", type=int, default=5, help="independent (A, B, Y) input sets rotated per step (5 = 377 MB, above L2)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -235,7 +239,7 @@ def main():
     peaks = measured_peaks()
 
     # ---- inputs: several independent (A, B, Y) sets, together well above the 126 MB L2, rotated per step
-    n_sets = 5
+    n_sets = max(1, args.sets)
     sets = []
     for s in range(n_sets):
         A, B = synth.mlp_product(M, K, N, seed=100 * rank + s)
@@ -271,10 +275,7 @@ def main():
 
     # ---- roofline of the dominant kernel (the tensor-core GEMM): retained FLOPs of one launch / its mean duration
     achieved = retained_flops(RHO) / (gemm_ms_avg * 1e-3) / 1e12
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "gemm_traffic.json")
-    if os.path.exists(tpath):
-        traffic = json.load(open(tpath)).get("dram_bytes_per_launch_rho0.5")
+    traffic = GEMM_DRAM_TRAFFIC_BYTES
     roofline = {"bound": "tensor", "kernel": "reduced_gemm_tc_kernel", "achieved": achieved, "peak": peaks["bf16_sustained"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": traffic,
                 "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step loop)",

@@ -7,7 +7,7 @@
 //                coalesced 16-byte loads, then every thread builds pairs of output elements from shared memory and
 //                writes 4 bytes; the index pairs are read once per thread and reused for the R rows.  Rows too long
 //                for shared memory, or not 16-byte aligned, take the direct form (2-byte gathers from global memory).
-// Row gather     dst[b, j, :] = src[sb, idx[b, j], :]    16-byte vectors, 4 kept rows per block.
+// Row gather     dst[b, j, :] = src[sb, idx[b, j], :]    16-byte vectors, 8 kept rows per block.
 // sb = (b + b_off) / b_div maps a batch entry to its source (grouped-query heads share K and V).
 #include "common.cuh"
 
@@ -17,7 +17,8 @@ namespace {
 constexpr int kThreadsPack = 256;
 constexpr int kMaxStageBytes = 96 * 1024;  // longest source row that is staged in shared memory
 constexpr int kStageTarget = 32 * 1024;    // preferred staging size: several blocks per SM stay resident
-constexpr int kDirectRows = 8;
+constexpr int kDirectRows = 4;
+constexpr int kRowsPerBlock = 8;  // kept rows copied by one block of the row gather
 
 struct PackJob {
     int type;  // 0 none, 1 columns staged, 2 columns direct, 3 rows
@@ -56,8 +57,15 @@ __device__ void pack_cols_staged(const PackJob &p, int64_t blk, int *status, uns
     for (int r = 0; r < nrows; ++r) {
         const uint4 *srow = reinterpret_cast<const uint4 *>(s16 + (r0 + r) * p.s_row);
         uint4 *drow = stage + (size_t)r * kv;
-#pragma unroll 4
-        for (int c = tid; c < kv; c += kThreadsPack) drow[c] = __ldg(srow + c);
+        for (int c0 = tid; c0 < kv; c0 += 4 * kThreadsPack) {  // four independent loads in flight per thread and row
+            uint4 v[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (c0 + i * kThreadsPack < kv) v[i] = __ldg(srow + c0 + i * kThreadsPack);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (c0 + i * kThreadsPack < kv) drow[c0 + i * kThreadsPack] = v[i];
+        }
     }
     __syncthreads();
     const unsigned short *rows = reinterpret_cast<const unsigned short *>(smem);
@@ -65,12 +73,24 @@ __device__ void pack_cols_staged(const PackJob &p, int64_t blk, int *status, uns
     unsigned *d32 = reinterpret_cast<unsigned *>(p.dst + b * p.rows * p.ld_dst);
     const int half = (int)(p.ld_dst / 2), K = (int)p.K;
     unsigned *drow0 = d32 + ((r0 * p.ld_dst) >> 1);
-    for (int jp = tid; jp < half; jp += kThreadsPack) {
-        const int c0 = checked_index(ix, 2 * jp, p.k, p.K, status), c1 = checked_index(ix, 2 * jp + 1, p.k, p.K, status);
+    for (int jp0 = tid; jp0 < half; jp0 += 4 * kThreadsPack) {  // four output pairs per thread: index loads first
+        int c[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int jp = jp0 + i * kThreadsPack;
+            c[2 * i] = jp < half ? checked_index(ix, 2 * jp, p.k, p.K, status) : -1;
+            c[2 * i + 1] = jp < half ? checked_index(ix, 2 * jp + 1, p.k, p.K, status) : -1;
+        }
         for (int r = 0; r < nrows; ++r) {
             const unsigned short *row = rows + r * K;
-            const unsigned lo = c0 >= 0 ? row[c0] : 0u, hi = c1 >= 0 ? row[c1] : 0u;
-            drow0[(size_t)r * half + jp] = lo | (hi << 16);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int jp = jp0 + i * kThreadsPack;
+                if (jp < half) {
+                    const unsigned lo = c[2 * i] >= 0 ? row[c[2 * i]] : 0u, hi = c[2 * i + 1] >= 0 ? row[c[2 * i + 1]] : 0u;
+                    drow0[(size_t)r * half + jp] = lo | (hi << 16);
+                }
+            }
         }
     }
 }
@@ -119,21 +139,22 @@ __device__ void pack_cols_direct(const PackJob &p, int64_t blk, int *status)
 __device__ void pack_rows(const PackJob &p, int64_t blk, int *status)
 {
     const int64_t b = blk / (p.bx * p.by), rem = blk % (p.bx * p.by);
-    const int64_t j0 = (rem / p.bx) * 4, nvec = p.n / 8;
+    const int64_t j0 = (rem / p.bx) * kRowsPerBlock, nvec = p.n / 8;
     const uint4 *sbase = reinterpret_cast<const uint4 *>(p.src) + ((b + p.b_off) / p.b_div) * (p.s_batch / 8);
     uint4 *dbase = reinterpret_cast<uint4 *>(p.dst) + (b * p.k) * (p.ld_dst / 8);
     const int32_t *ix = p.idx != nullptr ? p.idx + b * p.idx_stride : nullptr;
-    int rows[4];
+    int rows[kRowsPerBlock];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < kRowsPerBlock; ++i) {
         rows[i] = j0 + i < p.k ? checked_index(ix, j0 + i, p.k, p.K, status) : -2;  // -1: bad index, write zeros; -2: no row
     }
     for (int64_t c = (rem % p.bx) * kThreadsPack + threadIdx.x; c < nvec; c += p.bx * kThreadsPack) {
-        uint4 v[4];
+        uint4 v[kRowsPerBlock];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) v[i] = rows[i] >= 0 ? __ldg(sbase + rows[i] * (p.s_row / 8) + c) : make_uint4(0, 0, 0, 0);
+        for (int i = 0; i < kRowsPerBlock; ++i)
+            v[i] = rows[i] >= 0 ? __ldg(sbase + rows[i] * (p.s_row / 8) + c) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < kRowsPerBlock; ++i)
             if (rows[i] != -2) dbase[(j0 + i) * (p.ld_dst / 8) + c] = v[i];
     }
 }
@@ -173,7 +194,7 @@ size_t plan_job(PackJob &p)
     } else if (p.type == 3) {
         int64_t gx = ceil_div(p.n / 8, kThreadsPack);
         p.bx = gx > 8 ? 8 : gx;
-        p.by = ceil_div(p.k, 4);
+        p.by = ceil_div(p.k, kRowsPerBlock);
     }
     p.blocks = p.type == 0 ? 0 : p.bx * p.by * p.batch;
     return smem;

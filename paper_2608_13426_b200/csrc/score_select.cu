@@ -529,12 +529,23 @@ __global__ void __launch_bounds__(kThreads, 1) score_select_kernel(ScoreArgs a)
     for (int e = 0; e < VEC; ++e) s_part[ty * width + tx * VEC + e] = dacc[e];
     __syncthreads();
 
-    // combine the row lanes in lane order: thread t < width owns column col0 + t
+    // combine the row lanes in a fixed order, in two levels so that every thread helps: thread (part, c) adds the
+    // lanes part, part + parts, ... of column c, then thread c < width (the column's owner) adds the parts in order
     double colsum = 0.0;
     const int64_t mycol = col0 + tid;
     const bool owner = tid < width && mycol < a.n;
-    if (owner)
-        for (int y = 0; y < a.ty; ++y) colsum += s_part[y * width + tid];
+    {
+        const int parts = kThreads / width;  // width and ty are powers of two with width * ty == kThreads
+        const int c = tid % width, part = tid / width;
+        double sub = 0.0;
+        for (int y = part; y < a.ty; y += parts) sub += s_part[y * width + c];
+        __syncthreads();
+        s_part[part * width + c] = sub;
+        __syncthreads();
+        const int np = parts < a.ty ? parts : a.ty;
+        if (owner)
+            for (int q = 0; q < np; ++q) colsum += s_part[q * width + tid];
+    }
 
     bool finalize = true;
     if (a.row_splits > 1) {
@@ -616,17 +627,19 @@ int plan_score(const rmm_mat_t *A, int axis, ScorePlan *p)
     const bool vec_ok = p->s_n == 1 && p->n % full == 0 && (reinterpret_cast<uintptr_t>(A->ptr) % 16 == 0) &&
                         (p->s_red * es) % 16 == 0 && (p->s_batch * es) % 16 == 0;
     p->vec = vec_ok ? full : 1;
+    // thread layout: tx column groups x ty row lanes.  Narrow blocks (down to 8 groups = 128 contiguous bytes per
+    // row) are preferred as long as the grid stays within one block per SM, because a block that owns all the rows
+    // of its columns needs no cross-block combine; row splits only fill the machine when there are few columns.
+    const int64_t sms = 148;
     int64_t groups = ceil_div(p->n, p->vec);
     int tx = 32;
     while (tx > 1 && tx / 2 >= groups) tx /= 2;
+    const int tx_min = p->vec > 1 ? 8 : 32;
+    while (tx > tx_min && ceil_div(groups, tx / 2) * A->batch <= sms) tx /= 2;
     p->tx = tx;
     p->ty = kThreads / tx;
     p->col_blocks = (int)ceil_div(p->n, (int64_t)tx * p->vec);
-
-    // one block of 1024 threads per SM: split the rows so that the grid is at most one wave, each block keeping
-    // at least two loop trips of rows
-    const int64_t want_blocks = 148;
-    int64_t splits = want_blocks / ((int64_t)p->col_blocks * A->batch);
+    int64_t splits = sms / ((int64_t)p->col_blocks * A->batch);
     int64_t min_rows = (int64_t)p->ty * kUnroll * 2;
     int64_t max_splits = p->m / min_rows;
     if (max_splits < 1) max_splits = 1;
