@@ -17,6 +17,7 @@
 // Every mbarrier wait is bounded: on expiry the block records RMM_ERR_TIMEOUT in the workspace status
 // word, stops issuing work, lets copies in flight land, frees its TMEM and returns.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -98,34 +99,121 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
+// The same tile load issued by one CTA of a pair: the data lands in this CTA's shared memory, the byte count is
+// reported to an mbarrier that may live in the peer CTA (the pair's leader).  No multicast is involved.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar_cluster)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar_cluster)
+        : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address, in the cluster's shared window, of the variable at `local` in CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// TMEM allocation: with CTAS == 2 one warp of EACH CTA of the pair executes it, and the pair gets the same columns.
+template <int CTAS>
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols)
 {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (CTAS == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
 }
+template <int CTAS>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    if constexpr (CTAS == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    else
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// D[tmem] (+)= A[smem] B[smem].  CTAS == 2: issued by the pair's leader only; the tensor cores of both SMs work on a
+// 256-row tile, each reading A and its half of B from its own shared memory at the same offsets.
+template <int CTAS>
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
 {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if constexpr (CTAS == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
 }
-// Arrive on an mbarrier once every tcgen05 operation issued so far by this thread has completed.
+// The same with the 64-bit operand descriptors given as (low, high) words: within a tile only the low word (the
+// start address) changes, so the issuing thread needs one add per operand and instruction.
+template <int CTAS>
+__device__ __forceinline__ void umma_bf16_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                               uint32_t idesc, uint32_t accumulate)
+{
+    if constexpr (CTAS == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+            "setp.ne.b32 p, %6, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+            "setp.ne.b32 p, %6, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
+// Arrive on an mbarrier once every tcgen05 operation issued so far by this thread has completed.  CTAS == 2: the
+// arrival is delivered to the barrier at this offset in both CTAs of the pair.
+template <int CTAS>
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if constexpr (CTAS == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    } else {
+        const uint16_t both = 3;
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"(both) : "memory");
+    }
 }
-// 32 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+// 32 consecutive fp32 columns of this thread's TMEM lane; issue only (pair with tmem_ld_wait).
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32])
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -137,9 +225,8 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
         : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
-
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // Shared-memory operand descriptor (tcgen05 format): 128-byte swizzle, addresses and offsets in 16-byte units.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
 {
@@ -152,6 +239,15 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     return d;
 }
 
+#ifdef RMM_GEMM_STAMPS
+__device__ unsigned long long g_gstamps[16];
+#define GSTAMP_MIN(i) do { unsigned long long t_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_)); atomicMin(&g_gstamps[i], t_); } while (0)
+#define GSTAMP_MAX(i) do { unsigned long long t_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_)); atomicMax(&g_gstamps[i], t_); } while (0)
+#else
+#define GSTAMP_MIN(i)
+#define GSTAMP_MAX(i)
+#endif
+
 struct TcArgs {
     int64_t M, N, k, batch;
     int64_t b_batch_off, b_batch_div, b_batches;  // B batch entry of problem i = min((i + off) / div, b_batches - 1)
@@ -162,21 +258,38 @@ struct TcArgs {
     int *status;
 };
 
-template <int BN>
+// BN = tile columns (MMA N, accumulator columns); CTAS = CTAs per tile.  With CTAS == 2 a pair of CTAs on one TPC
+// shares a 256 x BN tile: each loads its own 128 rows of A and its own half of B's columns, so the operand bytes
+// per flop drop by a third against the single-CTA 128 x 256 tile.
+template <int BN, int CTAS>
 struct SmemLayout {
-    static constexpr int kStages = BN == 256 ? 4 : 6;
     static constexpr int kABytes = BM * BK * 2;
-    static constexpr int kBBytes = BN * BK * 2;
+    static constexpr int kBBytes = BN / CTAS * BK * 2;
+    static constexpr int kStages = (kABytes + kBBytes) > 32768 ? 4 : 6;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kBarOffset = kStages * kStageBytes;
     static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack to align the base to 1024 B
 };
 
-template <int BN, bool B_KMAJOR, bool OUT_BF16>
+// Tile order within one batch entry.
+__device__ __forceinline__ void tile_coords(int64_t t, int tiles_m, int tiles_n, int &tm, int &tn)
+{
+#ifdef RMM_GEMM_RASTER_M
+    tm = (int)(t % tiles_m);
+    tn = (int)(t / tiles_m);
+#else
+    tn = (int)(t % tiles_n);
+    tm = (int)(t / tiles_n);
+#endif
+}
+
+template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcArgs a)
 {
-    using L = SmemLayout<BN>;
+    using L = SmemLayout<BN, CTAS>;
+    constexpr int BNL = BN / CTAS;  // columns of B this CTA loads
+    const uint32_t rank = CTAS == 2 ? cluster_rank() : 0u;
     constexpr int kStages = L::kStages;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -190,9 +303,15 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + L::kBarOffset + 8 * (2 * kStages + 4) + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t num_tiles = a.batch * a.tiles_m * a.tiles_n;
+    if (threadIdx.x == 0) { GSTAMP_MIN(0); }
+    const int64_t num_tiles = a.batch * a.tiles_m * a.tiles_n;  // tiles of (128 * CTAS) x BN
+    const int64_t tile0 = blockIdx.x / CTAS, tile_step = gridDim.x / CTAS;
     const int num_kb = (int)((a.k + BK - 1) / BK);
 
+    if (threadIdx.x == 32) {  // descriptor fetch overlaps barrier set-up and the TMEM allocation
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(full_bar(s), 1);
@@ -200,141 +319,189 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(tfull_bar(i), 1);
-            mbar_init(tempty_bar(i), 4);
+            mbar_init(tempty_bar(i), 4 * CTAS);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), 2 * BN);
+    if (warp == 1) tmem_alloc<CTAS>(smem_u32(const_cast<uint32_t *>(tmem_slot)), 2 * BN);
     tc_fence_before();
-    __syncthreads();
+    if constexpr (CTAS == 2) cluster_sync_all();
+    else __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) { GSTAMP_MAX(1); }
 
     if (warp == 0) {
-        // ---------------------------------------------------------------- producer
-        uint32_t it = 0;
+        // ---------------------------------------------------------------- producer (one thread; the others idle)
+        uint32_t s = 0, ph = 0;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-            const int tn = (int)(tile % a.tiles_n);
-            const int tm = (int)((tile / a.tiles_n) % a.tiles_m);
+        for (int64_t tile = tile0; lane == 0 && tile < num_tiles && ok; tile += tile_step) {
+            int tm, tn;
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
+            tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, tm, tn);
             int64_t bb = (b + a.b_batch_off) / a.b_batch_div;
             if (bb >= a.b_batches) bb = a.b_batches - 1;
-            for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                const int s = it % kStages;
-                const uint32_t ph = (it / kStages) & 1u;
-                if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status)) { ok = false; break; }
-                if (lane == 0) {
+            for (int kb = 0; kb < num_kb; ++kb) {
+                if (!mbar_wait_lane(empty_bar(s), ph ^ 1u, abort_flag, a.status)) { ok = false; break; }
+                {
                     const uint32_t sa = base + s * L::kStageBytes;
                     const uint32_t sb = sa + L::kABytes;
-                    mbar_arrive_expect_tx(full_bar(s), L::kStageBytes);
-                    tma_load_3d(sa, &map_a, kb * BK, tm * BM, (int)b, full_bar(s));
-                    if constexpr (B_KMAJOR) {
-                        tma_load_3d(sb, &map_b, kb * BK, tn * BN, (int)bb, full_bar(s));
-                    } else {
-                        // 64 contraction rows x 64 columns per load; rows past k read as zeros
+                    const int row_a = tm * (BM * CTAS) + (int)rank * BM, col_b = tn * BN + (int)rank * BNL;
+#ifdef RMM_GEMM_SKIP_B
+                    if constexpr (CTAS == 1) {
+                        mbar_arrive_expect_tx(full_bar(s), L::kABytes);
+                        tma_load_3d(sa, &map_a, kb * BK, row_a, (int)b, full_bar(s));
+                    } else
+#endif
+                    if constexpr (CTAS == 1) {
+                        mbar_arrive_expect_tx(full_bar(s), L::kStageBytes);
+                        tma_load_3d(sa, &map_a, kb * BK, row_a, (int)b, full_bar(s));
+                        if constexpr (B_KMAJOR) {
+                            tma_load_3d(sb, &map_b, kb * BK, col_b, (int)bb, full_bar(s));
+                        } else {
+                            // 64 contraction rows x 64 columns per load; rows past k read as zeros
 #pragma unroll
-                        for (int c = 0; c < BN / 64; ++c)
-                            tma_load_3d(sb + c * (BK * 128), &map_b, tn * BN + c * 64, kb * BK, (int)bb, full_bar(s));
+                            for (int c = 0; c < BNL / 64; ++c)
+                                tma_load_3d(sb + c * (BK * 128), &map_b, col_b + c * 64, kb * BK, (int)bb, full_bar(s));
+                        }
+                    } else {
+                        // both CTAs report their bytes to the leader's barrier; the leader arms it for the pair
+                        const uint32_t lead_full = map_to_cta(full_bar(s), 0);
+                        if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * L::kStageBytes);
+                        tma_load_3d_pair(sa, &map_a, kb * BK, row_a, (int)b, lead_full);
+                        if constexpr (B_KMAJOR) {
+                            tma_load_3d_pair(sb, &map_b, kb * BK, col_b, (int)bb, lead_full);
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < BNL / 64; ++c)
+                                tma_load_3d_pair(sb + c * (BK * 128), &map_b, col_b + c * 64, kb * BK, (int)bb, lead_full);
+                        }
                     }
                 }
-                __syncwarp();
+                if (++s == kStages) { s = 0; ph ^= 1u; }
             }
         }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
+        __syncwarp();
+    } else if (warp == 1 && rank == 0) {
+        // ---------------------------------------------------------------- MMA issuer (the pair's leader only)
         // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B K- or MN-major, N = BN, M = 128
         constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((B_KMAJOR ? 0u : 1u) << 16) |
-                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-        uint32_t it = 0, tcount = 0;
+                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CTAS) >> 4) << 24);
+        // The issuing thread is the pacemaker of the whole kernel (one thread feeds the tensor cores of one or two
+        // SMs), so its loop is kept short: stage and phase are counters, descriptors advance by one add each.
+        // A, and a K-major B: 128-byte rows, 8-row groups 1024 B apart; 16 indices = 32 B along the row.
+        // MN-major B: 64-column chunks BK*128 B apart, 8-index groups 1024 B apart; 16 indices = 2048 B.
+        const uint64_t da0 = smem_desc(base, 16, 1024);
+        const uint64_t db0 = B_KMAJOR ? smem_desc(base + L::kABytes, 16, 1024) : smem_desc(base + L::kABytes, BK * 128, 1024);
+        const uint32_t a_hi = (uint32_t)(da0 >> 32), b_hi = (uint32_t)(db0 >> 32);
+        const uint32_t a_lo0 = (uint32_t)da0, b_lo0 = (uint32_t)db0;
+        constexpr uint32_t kStageUnits = L::kStageBytes >> 4, kAStep = 32 >> 4, kBStep = (B_KMAJOR ? 32 : 2048) >> 4;
+        const int last_steps = (int)((a.k - (int64_t)(num_kb - 1) * BK + UMMA_K - 1) / UMMA_K);  // MMAs of the last k-block
+        uint32_t stage = 0, phase = 0, tcount = 0;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+        for (int64_t tile = tile0; lane == 0 && tile < num_tiles && ok; tile += tile_step, ++tcount) {
             const uint32_t acc = tcount & 1u, acc_ph = (tcount >> 1) & 1u;
-            if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, a.status)) { ok = false; break; }
+            if (!mbar_wait_lane(tempty_bar(acc), acc_ph ^ 1u, abort_flag, a.status)) { ok = false; break; }
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * BN;
-            for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                const int s = it % kStages;
-                const uint32_t ph = (it / kStages) & 1u;
-                if (!mbar_wait(full_bar(s), ph, abort_flag, a.status)) { ok = false; break; }
+            uint32_t accumulate = 0;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                if (!mbar_wait_lane(full_bar(stage), phase, abort_flag, a.status)) { ok = false; break; }
                 tc_fence_after();
-                if (lane == 0) {
-                    const uint32_t sa = base + s * L::kStageBytes;
-                    const uint32_t sb = sa + L::kABytes;
-                    const int64_t left = a.k - (int64_t)kb * BK;
-                    const int steps = left >= BK ? BK / UMMA_K : (int)((left + UMMA_K - 1) / UMMA_K);
-                    for (int ks = 0; ks < steps; ++ks) {
-                        // A, and a K-major B: 128-byte rows, 8-row groups 1024 B apart; 16 indices = 32 B along the row
-                        const uint64_t da = smem_desc(sa + ks * 32, 16, 1024);
-                        // MN-major B: 64-column chunks BK*128 B apart, 8-index groups 1024 B apart; 16 indices = 2048 B
-                        const uint64_t db = B_KMAJOR ? smem_desc(sb + ks * 32, 16, 1024)
-                                                     : smem_desc(sb + ks * 2048, BK * 128, 1024);
-                        umma_bf16(d_tmem, da, db, idesc, (kb | ks) != 0 ? 1u : 0u);
+                if (kb == 0 && tcount == 0) { GSTAMP_MAX(2); }
+                const uint32_t a_lo = a_lo0 + stage * kStageUnits, b_lo = b_lo0 + stage * kStageUnits;
+                if (kb + 1 < num_kb || last_steps == BK / UMMA_K) {
+#pragma unroll
+                    for (int ks = 0; ks < BK / UMMA_K; ++ks) {
+                        umma_bf16_lohi<CTAS>(d_tmem, a_lo + ks * kAStep, a_hi, b_lo + ks * kBStep, b_hi, idesc, accumulate);
+                        accumulate = 1;
                     }
-                    umma_commit(empty_bar(s));
+                } else {
+                    for (int ks = 0; ks < last_steps; ++ks) {
+                        umma_bf16_lohi<CTAS>(d_tmem, a_lo + ks * kAStep, a_hi, b_lo + ks * kBStep, b_hi, idesc, accumulate);
+                        accumulate = 1;
+                    }
                 }
-                __syncwarp();
+                umma_commit<CTAS>(empty_bar(stage));
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
             }
-            if (ok && lane == 0) umma_commit(tfull_bar(acc));
-            __syncwarp();
+            if (ok) umma_commit<CTAS>(tfull_bar(acc));
+            GSTAMP_MAX(3);
         }
-    } else {
+        __syncwarp();
+    } else if (warp >= 2) {
         // ---------------------------------------------------------------- epilogue (warps 2..5)
         const int q = warp & 3;  // TMEM lane quarter this warp may read
         uint32_t tcount = 0;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
-            const int tn = (int)(tile % a.tiles_n);
-            const int tm = (int)((tile / a.tiles_n) % a.tiles_m);
+        for (int64_t tile = tile0; tile < num_tiles && ok; tile += tile_step, ++tcount) {
+            int tm, tn;
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
+            tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, tm, tn);
             const uint32_t acc = tcount & 1u, acc_ph = (tcount >> 1) & 1u;
             if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, a.status)) { ok = false; break; }
             tc_fence_after();
-            const int64_t m = (int64_t)tm * BM + q * 32 + lane;
+            if (lane == 0) { GSTAMP_MAX(4); }
+            const int64_t m = (int64_t)tm * (BM * CTAS) + rank * BM + q * 32 + lane;
             const int64_t n0 = (int64_t)tn * BN;
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + c * 32, r);
+            // scale, round and store 32 accumulator columns of this thread's row: 64 (bf16) or 128 (fp32) contiguous bytes
+            auto store_chunk = [&](const uint32_t (&r)[32], int c) {
                 const int64_t n = n0 + c * 32;
-                if (m < a.M && n < a.N) {
-                    if constexpr (OUT_BF16) {
-                        __nv_bfloat16 *y = reinterpret_cast<__nv_bfloat16 *>(a.Y) + b * a.y_sb + m * a.y_sr + n;
-                        if (n + 32 <= a.N) {
+                if (m >= a.M || n >= a.N) return;
+                if constexpr (OUT_BF16) {
+                    __nv_bfloat16 *y = reinterpret_cast<__nv_bfloat16 *>(a.Y) + b * a.y_sb + m * a.y_sr + n;
+                    if (n + 32 <= a.N) {
 #pragma unroll
-                            for (int v = 0; v < 4; ++v) {
-                                uint32_t w[4];
+                        for (int v = 0; v < 4; ++v) {
+                            uint32_t w[4];
 #pragma unroll
-                                for (int p = 0; p < 4; ++p) {
-                                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * v + 2 * p]) * a.scale,
-                                                                             __uint_as_float(r[8 * v + 2 * p + 1]) * a.scale);
-                                    w[p] = *reinterpret_cast<uint32_t *>(&h);
-                                }
-                                reinterpret_cast<uint4 *>(y)[v] = make_uint4(w[0], w[1], w[2], w[3]);
+                            for (int p = 0; p < 4; ++p) {
+                                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * v + 2 * p]) * a.scale,
+                                                                         __uint_as_float(r[8 * v + 2 * p + 1]) * a.scale);
+                                w[p] = *reinterpret_cast<uint32_t *>(&h);
                             }
-                        } else {
-                            for (int e = 0; e < 32 && n + e < a.N; ++e)
-                                y[e] = __float2bfloat16_rn(__uint_as_float(r[e]) * a.scale);
+                            reinterpret_cast<uint4 *>(y)[v] = make_uint4(w[0], w[1], w[2], w[3]);
                         }
                     } else {
-                        float *y = reinterpret_cast<float *>(a.Y) + b * a.y_sb + m * a.y_sr + n;
-                        if (n + 32 <= a.N) {
+                        for (int e = 0; e < 32 && n + e < a.N; ++e) y[e] = __float2bfloat16_rn(__uint_as_float(r[e]) * a.scale);
+                    }
+                } else {
+                    float *y = reinterpret_cast<float *>(a.Y) + b * a.y_sb + m * a.y_sr + n;
+                    if (n + 32 <= a.N) {
 #pragma unroll
-                            for (int v = 0; v < 8; ++v)
-                                reinterpret_cast<float4 *>(y)[v] =
-                                    make_float4(__uint_as_float(r[4 * v]) * a.scale, __uint_as_float(r[4 * v + 1]) * a.scale,
-                                                __uint_as_float(r[4 * v + 2]) * a.scale, __uint_as_float(r[4 * v + 3]) * a.scale);
-                        } else {
-                            for (int e = 0; e < 32 && n + e < a.N; ++e) y[e] = __uint_as_float(r[e]) * a.scale;
-                        }
+                        for (int v = 0; v < 8; ++v)
+                            reinterpret_cast<float4 *>(y)[v] =
+                                make_float4(__uint_as_float(r[4 * v]) * a.scale, __uint_as_float(r[4 * v + 1]) * a.scale,
+                                            __uint_as_float(r[4 * v + 2]) * a.scale, __uint_as_float(r[4 * v + 3]) * a.scale);
+                    } else {
+                        for (int e = 0; e < 32 && n + e < a.N; ++e) y[e] = __uint_as_float(r[e]) * a.scale;
                     }
                 }
+            };
+            // four TMEM loads in flight per wait: the load latency is paid BN / 128 times per tile instead of BN / 32
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; c += 4) {
+                uint32_t r0[32], r1[32], r2[32], r3[32];
+                tmem_ld32_issue(t_row + (c + 0) * 32, r0);
+                tmem_ld32_issue(t_row + (c + 1) * 32, r1);
+                tmem_ld32_issue(t_row + (c + 2) * 32, r2);
+                tmem_ld32_issue(t_row + (c + 3) * 32, r3);
+                tmem_ld_wait();
+                store_chunk(r0, c + 0);
+                store_chunk(r1, c + 1);
+                store_chunk(r2, c + 2);
+                store_chunk(r3, c + 3);
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            if (lane == 0) {
+                if constexpr (CTAS == 1) mbar_arrive(tempty_bar(acc));
+                else mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));  // the leader's MMA warp waits on it
+            }
+            if (lane == 0) { GSTAMP_MAX(5); }
         }
     }
 
@@ -346,8 +513,13 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         while (global_ns() - t0 < 200000ull) __nanosleep(1000);
         __syncthreads();
     }
+    if constexpr (CTAS == 2) {
+        tc_fence_before();
+        cluster_sync_all();  // the peer may still be reading operands or accumulators that involve this CTA
+    }
     tc_fence_after();
-    if (warp == 1) tmem_dealloc(tmem_base, 2 * BN);
+    if (warp == 1) tmem_dealloc<CTAS>(tmem_base, 2 * BN);
+    if (threadIdx.x == 0) { GSTAMP_MAX(6); }
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -398,20 +570,34 @@ int sm_count()
     return n;
 }
 
-template <int BN, bool B_KMAJOR, bool OUT_BF16>
+template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS>
 int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const TcArgs &a, cudaStream_t stream)
 {
-    auto kern = reduced_gemm_tc_kernel<BN, B_KMAJOR, OUT_BF16>;
+    auto kern = reduced_gemm_tc_kernel<BN, B_KMAJOR, OUT_BF16, CTAS>;
+    using L = SmemLayout<BN, CTAS>;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout<BN>::kTotal);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
         if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         configured = true;
     }
-    int64_t tiles = a.batch * a.tiles_m * a.tiles_n;
-    int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+    const int64_t tiles = a.batch * a.tiles_m * a.tiles_n;
+    const int64_t slots = sm_count() / CTAS;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((tiles < slots ? tiles : slots) * CTAS));
+    cfg.blockDim = dim3(kThreadsTc);
+    cfg.dynamicSmemBytes = L::kTotal;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CTAS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = CTAS == 2 ? 1 : 0;
     prof_begin("reduced_gemm_tc_kernel", stream);
-    kern<<<grid, kThreadsTc, SmemLayout<BN>::kTotal, stream>>>(ma, mb, a);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ma, mb, a);
+    if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "reduced_gemm_tc_kernel: launch: %s", cudaGetErrorString(e));
     return check_launch("reduced_gemm_tc_kernel", stream);
 }
 
@@ -462,19 +648,28 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
         if (rc != RMM_OK) return rc;
     }
     const int BN = p.N <= 128 ? 128 : 256;
+    // CTA pairs (256 x 256 tiles, a third fewer operand bytes per flop) pay off once there are enough pair tiles to
+    // keep every SM pair busy: measured 1.81-1.87 PFLOP/s against 1.51-1.59 for single CTAs on 8192 x 8192 outputs,
+    // while on a 2048 x 2048 output (64 pair tiles for 74 SM pairs) the pair's longer set-up and epilogue lose about
+    // 2 us.  RMM_GEMM_CTAS=1 or 2 forces a form (for measurements).
+    static const int forced = []() { const char *e = getenv("RMM_GEMM_CTAS"); return e ? atoi(e) : 0; }();
+    const int64_t pair_tiles = p.batch * ceil_div(p.M, 2 * BM) * ceil_div(p.N, 256);
+    int ctas = (BN == 256 && p.M > BM && pair_tiles >= sm_count() / 2) ? 2 : 1;
+    if (forced == 1) ctas = 1;
+    if (forced == 2 && BN == 256 && p.M > BM) ctas = 2;
     TcArgs a;
     a.M = p.M; a.N = p.N; a.k = p.k; a.batch = p.batch;
     a.b_batch_off = p.b_batch_off; a.b_batch_div = p.b_batch_div > 0 ? p.b_batch_div : 1; a.b_batches = p.b_batches;
     a.Y = p.y; a.y_sb = p.y_sb; a.y_sr = p.y_sr;
     a.scale = p.scale;
-    a.tiles_m = (int)ceil_div(p.M, BM);
+    a.tiles_m = (int)ceil_div(p.M, BM * ctas);
     a.tiles_n = (int)ceil_div(p.N, BN);
     a.status = p.status;
     const uint64_t b_sb = p.b_batches > 1 ? (uint64_t)p.b_sb * 2 : (uint64_t)p.b_ld * 2 * (uint64_t)(p.b_kmajor ? p.N : p.k);
     if (p.b_kmajor) {
         uint64_t dims[3] = {(uint64_t)p.k, (uint64_t)p.N, (uint64_t)p.b_batches};
         uint64_t st[2] = {(uint64_t)p.b_ld * 2, b_sb};
-        uint32_t box[3] = {BK, (uint32_t)BN, 1};
+        uint32_t box[3] = {BK, (uint32_t)(BN / ctas), 1};
         rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 3, dims, st, box);
     } else {
         uint64_t dims[3] = {(uint64_t)p.N, (uint64_t)p.k, (uint64_t)p.b_batches};
@@ -484,12 +679,16 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     }
     if (rc != RMM_OK) return rc;
     const bool out_bf16 = p.y_bf16 != 0;
-    if (BN == 256) {
-        if (p.b_kmajor) return out_bf16 ? launch_variant<256, true, true>(ma, mb, a, stream) : launch_variant<256, true, false>(ma, mb, a, stream);
-        return out_bf16 ? launch_variant<256, false, true>(ma, mb, a, stream) : launch_variant<256, false, false>(ma, mb, a, stream);
+    if (ctas == 2) {
+        if (p.b_kmajor) return out_bf16 ? launch_variant<256, true, true, 2>(ma, mb, a, stream) : launch_variant<256, true, false, 2>(ma, mb, a, stream);
+        return out_bf16 ? launch_variant<256, false, true, 2>(ma, mb, a, stream) : launch_variant<256, false, false, 2>(ma, mb, a, stream);
     }
-    if (p.b_kmajor) return out_bf16 ? launch_variant<128, true, true>(ma, mb, a, stream) : launch_variant<128, true, false>(ma, mb, a, stream);
-    return out_bf16 ? launch_variant<128, false, true>(ma, mb, a, stream) : launch_variant<128, false, false>(ma, mb, a, stream);
+    if (BN == 256) {
+        if (p.b_kmajor) return out_bf16 ? launch_variant<256, true, true, 1>(ma, mb, a, stream) : launch_variant<256, true, false, 1>(ma, mb, a, stream);
+        return out_bf16 ? launch_variant<256, false, true, 1>(ma, mb, a, stream) : launch_variant<256, false, false, 1>(ma, mb, a, stream);
+    }
+    if (p.b_kmajor) return out_bf16 ? launch_variant<128, true, true, 1>(ma, mb, a, stream) : launch_variant<128, true, false, 1>(ma, mb, a, stream);
+    return out_bf16 ? launch_variant<128, false, true, 1>(ma, mb, a, stream) : launch_variant<128, false, false, 1>(ma, mb, a, stream);
 }
 
 int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
