@@ -323,6 +323,21 @@ def main():
                             "score_select_frac_of_hbm": M * K * 2 / sel / 1e6 / peaks["hbm_gbs"],
                             "dense_cublas_ms": dense_ms, "speedup_vs_dense_cublas": dense_ms / whole})
 
+    # ---- the selection pass on a 70B-class activation (32768 tokens x 8192 hidden, 537 MB): the same kernel where it is
+    # bandwidth-bound rather than latency-bound (the benchmark product's 33.6 MB input is too small to show it)
+    selection_large = None
+    if not args.no_sweep and rank == 0:
+        Ml, Kl = 32768, 8192
+        big = [synth.heavy_tailed_activations(Ml, Kl, seed=50 + i, device=str(dev)) for i in range(2)]
+        idx_l = torch.empty(rmm.rmm_keep_count(RHO, Kl), dtype=torch.int32, device=dev)
+        for i in range(3):
+            rmm.rmm_score_select(big[i % 2], rho=RHO, idx=idx_l)
+        t = time_region(lambda i: rmm.rmm_score_select(big[i % 2], rho=RHO, idx=idx_l), 20, 1)
+        gbs = Ml * Kl * 2 / t / 1e6
+        selection_large = {"shape": [Ml, Kl], "ms": t, "gbs": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+                           "note": "fused score + top-k select, two alternating 537 MB inputs (above L2)"}
+        del big
+
     # ---- per-kernel breakdown of one step (a separate, untimed pass with every launch bracketed by events)
     breakdown = {}
     if rank == 0:
@@ -347,7 +362,7 @@ def main():
             "config": {"workload": WORKLOAD, "rho": RHO, "k": k, "M": M, "K": K, "N": N, "parallelism": f"replicas x{world}",
                        "l2_policy": f"inputs larger than L2: {n_sets} rotating (A, B, Y) sets, {resident_bytes / 1e6:.0f} MB resident"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
-            "kernel_breakdown": breakdown, "per_rho": per_rho, "peaks": peaks,
+            "kernel_breakdown": breakdown, "per_rho": per_rho, "selection_pass_large": selection_large, "peaks": peaks,
         }
         print(json.dumps(out))
     if world > 1:

@@ -8,6 +8,8 @@
 
 #include "rmm.h"
 
+struct CUtensorMap_st;  // the driver API's tensor-map type (cuda.h); opaque here
+
 namespace rmm {
 
 // ---- error text (thread-local) and launch accounting -------------------------------------------
@@ -19,6 +21,11 @@ int check_launch(const char *what, cudaStream_t stream);  // right after: cudaGe
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 static inline size_t dtype_size(int dt) { return dt == RMM_BF16 ? 2 : 4; }
+
+// ---- TMA tensor map for a bf16 tensor: dims / box innermost first, strides in bytes for dims 1..rank-1; 128-byte
+// swizzle or none.  `map` points to a CUtensorMap (opaque here so that only the users include <cuda.h>).
+int make_map(::CUtensorMap_st *map, void *ptr, int rank, const uint64_t *dims, const uint64_t *strides_bytes,
+             const uint32_t *box, bool swizzle128);
 
 // ---- workspace header: status word, then self-resetting arrival counters --------------------------
 struct WsHeader {
@@ -40,6 +47,7 @@ struct ScorePlan {
     int64_t s_batch, s_red, s_n;  // element strides: batch, reduced axis, scored axis
     size_t off_counters, off_partials, off_energy, total_bytes;
     bool counters_in_header;
+    bool use_tma;    // rows streamed through shared memory by TMA (bf16, 64-column blocks)
 };
 int plan_score(const rmm_mat_t *A, int axis, ScorePlan *plan);
 int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, int64_t k, int32_t *idx,

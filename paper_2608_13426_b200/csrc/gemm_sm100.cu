@@ -525,40 +525,6 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 // ----------------------------------------------------------------------------------------------
 // host side
 // ----------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (fn == nullptr) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-// bf16 tensor map with 128-byte swizzle; dims / strides innermost first, strides in bytes for dims 1..rank-1
-int make_map(CUtensorMap *map, void *ptr, int rank, const uint64_t *dims, const uint64_t *strides_bytes,
-             const uint32_t *box)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (fn == nullptr) return fail(RMM_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
-    cuuint64_t d[5], st[4];
-    cuuint32_t bx[5], es[5];
-    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
-    for (int i = 0; i + 1 < rank; ++i) st[i] = strides_bytes[i];
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, ptr, d, st, bx, es,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return fail(RMM_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
-    return RMM_OK;
-}
-
 int sm_count()
 {
     static int n = 0;
@@ -644,7 +610,7 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
         uint64_t dims[3] = {(uint64_t)p.k, (uint64_t)p.M, (uint64_t)p.batch};
         uint64_t st[2] = {(uint64_t)p.a_ld * 2, (uint64_t)p.a_sb * 2};
         uint32_t box[3] = {BK, BM, 1};
-        rc = make_map(&ma, const_cast<__nv_bfloat16 *>(p.a), 3, dims, st, box);
+        rc = make_map(&ma, const_cast<__nv_bfloat16 *>(p.a), 3, dims, st, box, true);
         if (rc != RMM_OK) return rc;
     }
     const int BN = p.N <= 128 ? 128 : 256;
@@ -670,12 +636,12 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
         uint64_t dims[3] = {(uint64_t)p.k, (uint64_t)p.N, (uint64_t)p.b_batches};
         uint64_t st[2] = {(uint64_t)p.b_ld * 2, b_sb};
         uint32_t box[3] = {BK, (uint32_t)(BN / ctas), 1};
-        rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 3, dims, st, box);
+        rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 3, dims, st, box, true);
     } else {
         uint64_t dims[3] = {(uint64_t)p.N, (uint64_t)p.k, (uint64_t)p.b_batches};
         uint64_t st[2] = {(uint64_t)p.b_ld * 2, b_sb};
         uint32_t box[3] = {64, BK, 1};
-        rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 3, dims, st, box);
+        rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 3, dims, st, box, true);
     }
     if (rc != RMM_OK) return rc;
     const bool out_bf16 = p.y_bf16 != 0;

@@ -11,6 +11,8 @@
 // Select: radix select on the order-preserving integer image of the fp32 keys (4 passes of 8 bits,
 // warp-aggregated shared-memory histograms), then one ordered compaction pass that emits the kept
 // indices ascending; among keys equal to the threshold the lowest indices are kept.
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace rmm {
@@ -474,57 +476,19 @@ __device__ __forceinline__ void load_vec(const void *A, int64_t off, int64_t s_n
     }
 }
 
-template <int VEC, bool BF16>
-__global__ void __launch_bounds__(kThreads, 1) score_select_kernel(ScoreArgs a)
+// Everything after a block's row loop: combine the row lanes, hand the column sums over (fp64 partials and an arrival
+// counter when the rows are split), write energies and scores, and let the last block of a batch element select.
+template <int VEC>
+__device__ __forceinline__ void score_finish(const ScoreArgs &a, const double (&dacc)[VEC], unsigned char *s_dyn,
+                                             SelectSmem &s_sel, int &s_flag)
 {
-    extern __shared__ __align__(16) unsigned char s_dyn[];  // row-lane partial sums, later the select's key cache
     double *s_part = reinterpret_cast<double *>(s_dyn);
-    __shared__ SelectSmem s_sel;
-    __shared__ int s_flag;
-
     const int tid = threadIdx.x;
     const int tx = tid % a.tx, ty = tid / a.tx;
     const int64_t b = blockIdx.z;
     const int split = blockIdx.y;
     const int width = a.tx * VEC;  // columns per block
     const int64_t col0 = (int64_t)blockIdx.x * width;
-    const int64_t col = col0 + (int64_t)tx * VEC;
-    const int64_t r_begin = (int64_t)split * a.rows_per_split;
-    const int64_t r_end = min(a.m, r_begin + a.rows_per_split);
-
-    double dacc[VEC];
-    float facc[VEC];
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) { dacc[e] = 0.0; facc[e] = 0.f; }
-
-    if (col < a.n) {
-        const int64_t base = b * a.s_batch + col * a.s_n;
-        int trips = 0;
-        for (int64_t r = r_begin + ty; r < r_end; r += (int64_t)a.ty * kUnroll) {
-            float v[kUnroll][VEC];
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                int64_t rr = r + (int64_t)u * a.ty;
-                if (rr < r_end) {
-                    load_vec<VEC, BF16>(a.A, base + rr * a.s_red, a.s_n, v[u]);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < VEC; ++e) v[u][e] = 0.f;
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u)
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) facc[e] = fmaf(v[u][e], v[u][e], facc[e]);
-            if (++trips == kFlushEvery) {
-                trips = 0;
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) { dacc[e] += (double)facc[e]; facc[e] = 0.f; }
-            }
-        }
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) dacc[e] += (double)facc[e];
-    }
 #pragma unroll
     for (int e = 0; e < VEC; ++e) s_part[ty * width + tx * VEC + e] = dacc[e];
     __syncthreads();
@@ -594,10 +558,173 @@ __global__ void __launch_bounds__(kThreads, 1) score_select_kernel(ScoreArgs a)
                      a.retained ? a.retained + b : nullptr, s_sel, reinterpret_cast<unsigned *>(s_dyn));
 }
 
+template <int VEC, bool BF16>
+__global__ void __launch_bounds__(kThreads, 1) score_select_kernel(ScoreArgs a)
+{
+    extern __shared__ __align__(128) unsigned char s_dyn[];  // row-lane partial sums, later the select's key cache
+    __shared__ SelectSmem s_sel;
+    __shared__ int s_flag;
+
+    const int tid = threadIdx.x;
+    const int tx = tid % a.tx, ty = tid / a.tx;
+    const int64_t b = blockIdx.z;
+    const int split = blockIdx.y;
+    const int width = a.tx * VEC;  // columns per block
+    const int64_t col0 = (int64_t)blockIdx.x * width;
+    const int64_t col = col0 + (int64_t)tx * VEC;
+    const int64_t r_begin = (int64_t)split * a.rows_per_split;
+    const int64_t r_end = min(a.m, r_begin + a.rows_per_split);
+
+    double dacc[VEC];
+    float facc[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) { dacc[e] = 0.0; facc[e] = 0.f; }
+
+    if (col < a.n) {
+        const int64_t base = b * a.s_batch + col * a.s_n;
+        int trips = 0;
+        for (int64_t r = r_begin + ty; r < r_end; r += (int64_t)a.ty * kUnroll) {
+            float v[kUnroll][VEC];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                int64_t rr = r + (int64_t)u * a.ty;
+                if (rr < r_end) {
+                    load_vec<VEC, BF16>(a.A, base + rr * a.s_red, a.s_n, v[u]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) v[u][e] = 0.f;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) facc[e] = fmaf(v[u][e], v[u][e], facc[e]);
+            if (++trips == kFlushEvery) {
+                trips = 0;
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) { dacc[e] += (double)facc[e]; facc[e] = 0.f; }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) dacc[e] += (double)facc[e];
+    }
+    score_finish<VEC>(a, dacc, s_dyn, s_sel, s_flag);
+}
+
+// ---- the same pass with the rows streamed through shared memory by TMA ------------------------------------------------
+// For bf16 matrices that satisfy the TMA rules.  A block owns 64 columns (128 contiguous bytes per row) and streams
+// its rows as 256-row tiles (32 KB) through a ring of kTmaStages buffers: the copies in flight cost no registers, so
+// about 128 KB per SM are outstanding, against the 64 KB that 1024 threads x 4 register loads allow.  Rows or columns
+// outside the matrix arrive as zeros (tensor-map bounds), so the loop has no edge cases.  Thread (tx, ty) reads the
+// 16-byte group tx of rows ty and ty + 128 of every tile.
+constexpr int kTmaStages = 6, kTmaRows = 256, kTmaCols = 64;
+constexpr int kTmaStageBytes = kTmaRows * kTmaCols * 2;
+constexpr unsigned long long kScoreWaitNs = 2000000000ull;
+
+__device__ __forceinline__ bool score_wait(uint32_t bar, uint32_t parity, int *status)
+{
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((it & 255u) == 255u) {  // bounded: give up after 2 s, report, and let the block finish with what it has
+            unsigned long long now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kScoreWaitNs) {
+                atomicExch(status, (int)RMM_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1) score_tma_kernel(const __grid_constant__ CUtensorMap map_a, ScoreArgs a, int *status)
+{
+    extern __shared__ __align__(128) unsigned char s_dyn[];  // the tile ring; afterwards partial sums and the key cache
+    __shared__ SelectSmem s_sel;
+    __shared__ int s_flag;
+    __shared__ __align__(8) unsigned long long s_bar[2 * kTmaStages];
+
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int tx = tid & 7, ty = tid >> 3;  // 8 column groups x 128 row lanes
+    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(s_dyn);
+    const uint32_t bars = (uint32_t)__cvta_generic_to_shared(s_bar);
+    auto full_bar = [&](int st) { return bars + 8u * st; };
+    auto empty_bar = [&](int st) { return bars + 8u * (kTmaStages + st); };
+    const int64_t r_begin = (int64_t)blockIdx.y * a.rows_per_split;
+    const int64_t r_end = min(a.m, r_begin + a.rows_per_split);
+    const int n_tiles = (int)((r_end - r_begin + kTmaRows - 1) / kTmaRows);
+    const int col0 = (int)blockIdx.x * kTmaCols;
+
+    if (tid == 0) {
+        for (int st = 0; st < kTmaStages; ++st) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full_bar(st)), "r"(1) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_bar(st)), "r"(kThreads / 32) : "memory");
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    }
+    __syncthreads();
+
+    auto issue = [&](int t) {  // thread 0 only: fetch tile t into its ring slot
+        const int st = t % kTmaStages;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full_bar(st)), "r"(kTmaStageBytes) : "memory");
+        asm volatile(
+            "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+            ::"r"(ring + st * kTmaStageBytes), "l"(&map_a), "r"(col0), "r"((int)(r_begin + (int64_t)t * kTmaRows)),
+              "r"((int)blockIdx.z), "r"(full_bar(st))
+            : "memory");
+    };
+    constexpr int kAhead = kTmaStages - 2;  // tiles in flight ahead of the consumers
+    if (tid == 0)
+        for (int t = 0; t < kAhead && t < n_tiles; ++t) issue(t);
+
+    double dacc[8];
+    float facc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { dacc[e] = 0.0; facc[e] = 0.f; }
+    bool ok = true;
+    for (int t = 0; t < n_tiles && ok; ++t) {
+        const int st = t % kTmaStages;
+        const uint32_t ph = (uint32_t)(t / kTmaStages) & 1u;
+        if (tid == 0 && t + kAhead < n_tiles) {
+            // the slot of tile t + kAhead was last used by tile t - 2: wait until every warp has released it
+            const int nt = t + kAhead, ns = nt % kTmaStages;
+            if (nt >= kTmaStages && !score_wait(empty_bar(ns), (uint32_t)(nt / kTmaStages - 1) & 1u, status)) ok = false;
+            if (ok) issue(nt);
+        }
+        if (!score_wait(full_bar(st), ph, status)) { ok = false; }
+        const uint4 *tile = reinterpret_cast<const uint4 *>(s_dyn + st * kTmaStageBytes);
+        const uint4 q0 = tile[ty * 8 + tx], q1 = tile[(ty + 128) * 8 + tx];
+        const unsigned w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float lo0 = __uint_as_float(w[i] << 16), hi0 = __uint_as_float(w[i] & 0xffff0000u);
+            const float lo1 = __uint_as_float(w[4 + i] << 16), hi1 = __uint_as_float(w[4 + i] & 0xffff0000u);
+            facc[2 * i] = fmaf(lo1, lo1, fmaf(lo0, lo0, facc[2 * i]));
+            facc[2 * i + 1] = fmaf(hi1, hi1, fmaf(hi0, hi0, facc[2 * i + 1]));
+        }
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(st)) : "memory");
+        if ((t & 7) == 7) {  // 16 terms per fp32 chain, then fp64
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { dacc[e] += (double)facc[e]; facc[e] = 0.f; }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) dacc[e] += (double)facc[e];
+    __syncthreads();  // every tile has landed and been read: the ring can be reused for the partial sums
+    score_finish<8>(a, dacc, s_dyn, s_sel, s_flag);
+}
+
 __global__ void __launch_bounds__(1024) select_kernel(const float *keys, int K, int k, int32_t *idx, float *retained,
                                                       int use_cache)
 {
-    extern __shared__ __align__(16) unsigned char s_dyn[];
+    extern __shared__ __align__(128) unsigned char s_dyn[];
     __shared__ SelectSmem s_sel;
     const int64_t b = blockIdx.x;
     block_select_any(keys + b * K, K, k, idx + b * (int64_t)k, retained ? retained + b : nullptr, s_sel,
@@ -636,17 +763,21 @@ int plan_score(const rmm_mat_t *A, int axis, ScorePlan *p)
     while (tx > 1 && tx / 2 >= groups) tx /= 2;
     const int tx_min = p->vec > 1 ? 8 : 32;
     while (tx > tx_min && ceil_div(groups, tx / 2) * A->batch <= sms) tx /= 2;
+    // bf16 matrices that meet the TMA rules stream through shared memory in 64-column blocks (score_tma_kernel)
+    p->use_tma = p->vec == 8 && A->dtype == RMM_BF16 && p->n >= kTmaCols && p->m <= INT32_MAX;
+    if (p->use_tma) tx = 8;
     p->tx = tx;
     p->ty = kThreads / tx;
     p->col_blocks = (int)ceil_div(p->n, (int64_t)tx * p->vec);
     int64_t splits = sms / ((int64_t)p->col_blocks * A->batch);
-    int64_t min_rows = (int64_t)p->ty * kUnroll * 2;
+    int64_t min_rows = p->use_tma ? 2 * kTmaRows : (int64_t)p->ty * kUnroll * 2;
     int64_t max_splits = p->m / min_rows;
     if (max_splits < 1) max_splits = 1;
     if (splits > max_splits) splits = max_splits;
     if (splits > 64) splits = 64;
     if (splits < 1) splits = 1;
     p->rows_per_split = ceil_div(p->m, splits);
+    if (p->use_tma && splits > 1) p->rows_per_split = ceil_div(p->rows_per_split, kTmaRows) * kTmaRows;  // whole tiles
     p->row_splits = (int)ceil_div(p->m, p->rows_per_split);
 
     int64_t n_counters = A->batch * (p->col_blocks + 1);
@@ -692,6 +823,25 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
     const bool bf16 = A->dtype == RMM_BF16;
     size_t smem = (size_t)kThreads * p.vec * sizeof(double);
     if (fused && (size_t)p.n * 4 > smem) smem = (size_t)p.n * 4;
+    if (p.use_tma) {
+        CUtensorMap map;
+        const uint64_t dims[3] = {(uint64_t)p.n, (uint64_t)p.m, (uint64_t)A->batch};
+        const uint64_t st[2] = {(uint64_t)p.s_red * 2, A->batch > 1 ? (uint64_t)p.s_batch * 2 : (uint64_t)p.s_red * 2 * (uint64_t)p.m};
+        const uint32_t box[3] = {kTmaCols, kTmaRows, 1};
+        int rc = make_map(&map, const_cast<void *>(a.A), 3, dims, st, box, false);
+        if (rc != RMM_OK) return rc;
+        static bool tma_configured = false;
+        if (!tma_configured) {
+            cudaError_t e = cudaFuncSetAttribute(score_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTmaStages * kTmaStageBytes);
+            if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "score: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+            tma_configured = true;
+        }
+        prof_begin("score_select_kernel", stream);
+        score_tma_kernel<<<grid, kThreads, kTmaStages * kTmaStageBytes, stream>>>(map, a, &hdr->status);
+        int rc2 = check_launch("score_select_kernel", stream);
+        if (rc2 != RMM_OK || !do_select || fused) return rc2;
+        return launch_select(a.energy, A->batch, p.n, k, idx, retained, ws, stream);
+    }
     static bool configured = false;
     if (!configured) {
         const int big = kThreads * 8 * (int)sizeof(double);
