@@ -151,13 +151,14 @@ int rmm_product_host(const void *A_host, const void *B_host, int64_t M, int64_t 
  * Synchronous: call it after the stream the workspace was used on has been synchronised. */
 int rmm_status_read(void *ws, int *device_status);
 
-/* Timing hook for benchmarks (the paper has no counterpart).  After rmm_profile_kernels(start, stop, n, filter),
- * the next launches of library kernels whose name contains `name_filter` (NULL or "" = every kernel), up to n of
- * them, are bracketed by cudaEventRecord(start[i]) and cudaEventRecord(stop[i]) on their stream.  The host arrays
+/* Timing hook for benchmarks (the paper has no counterpart).  After rmm_profile_kernels(start, stop, n, filter, every),
+ * launches of library kernels whose name contains `name_filter` (NULL or "" = every kernel) are bracketed by
+ * cudaEventRecord(start[i]) and cudaEventRecord(stop[i]) on their stream: one matching launch in `every` (<= 1: all of
+ * them), up to n pairs.  (Event records between kernels cost a few microseconds of launch overlap, hence `every`.)  The host arrays
  * hold cudaEvent_t handles created by the caller with timing enabled and must stay alive until the hook is cleared
- * with (NULL, NULL, 0, NULL).  n <= 4096.  Not thread-safe.  rmm_profile_count() tells how many pairs have been
+ * with (NULL, NULL, 0, NULL, 0).  n <= 4096.  Not thread-safe.  rmm_profile_count() tells how many pairs have been
  * recorded, rmm_profile_name(i) the kernel the i-th pair brackets (a static string). */
-int rmm_profile_kernels(void **start_events, void **stop_events, int n, const char *name_filter);
+int rmm_profile_kernels(void **start_events, void **stop_events, int n, const char *name_filter, int every);
 int rmm_profile_count(void);
 const char *rmm_profile_name(int i);
 

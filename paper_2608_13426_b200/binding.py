@@ -90,7 +90,7 @@ def lib() -> ctypes.CDLL:
     L.rmm_status_read.argtypes = [vp, ctypes.POINTER(i32)]
     L.rmm_last_error.restype = ctypes.c_char_p
     L.rmm_launch_count.restype = i64
-    L.rmm_profile_kernels.argtypes = [vp, vp, i32, ctypes.c_char_p]
+    L.rmm_profile_kernels.argtypes = [vp, vp, i32, ctypes.c_char_p, i32]
     L.rmm_profile_name.argtypes = [i32]
     L.rmm_profile_name.restype = ctypes.c_char_p
     _lib = L
@@ -159,11 +159,12 @@ def rmm_launch_count() -> int:
 
 
 class KernelTimer:
-    """Brackets the next n launches of library kernels whose name contains `name_filter` with CUDA events
-    (rmm_profile_kernels).  Use as a context manager; times_ms() then gives (kernel name, duration) pairs."""
+    """Brackets launches of library kernels whose name contains `name_filter` with CUDA events (one matching launch
+    in `every`, at most n of them; rmm_profile_kernels).  Use as a context manager; times_ms() then gives (kernel name, duration) pairs."""
 
-    def __init__(self, n: int, name_filter: str = ""):
+    def __init__(self, n: int, name_filter: str = "", every: int = 1):
         self.n = n
+        self.every = every
         self.filter = name_filter.encode()
         self.start = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
         self.stop = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
@@ -176,13 +177,13 @@ class KernelTimer:
         self.names = []
 
     def __enter__(self):
-        _check(lib().rmm_profile_kernels(self._s, self._e, self.n, self.filter))
+        _check(lib().rmm_profile_kernels(self._s, self._e, self.n, self.filter, self.every))
         return self
 
     def __exit__(self, *exc):
         self.count = int(lib().rmm_profile_count())
         self.names = [lib().rmm_profile_name(i).decode() for i in range(self.count)]
-        _check(lib().rmm_profile_kernels(None, None, 0, None))
+        _check(lib().rmm_profile_kernels(None, None, 0, None, 0))
         return False
 
     def times_ms(self):

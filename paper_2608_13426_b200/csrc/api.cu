@@ -24,7 +24,7 @@ int fail(int code, const char *fmt, ...)
 // Optional timing hook (rmm_profile_kernels): events recorded around launches whose name matches the filter.
 static struct {
     cudaEvent_t *start = nullptr, *stop = nullptr;
-    int capacity = 0, used = 0;
+    int capacity = 0, used = 0, every = 1, seen = 0;
     bool pending = false;
     char filter[64] = "";
     const char *names[4096];
@@ -34,6 +34,7 @@ void prof_begin(const char *name, cudaStream_t stream)
 {
     if (g_prof.used >= g_prof.capacity || g_prof.used >= 4096) return;
     if (g_prof.filter[0] != 0 && strstr(name, g_prof.filter) == nullptr) return;
+    if (g_prof.seen++ % g_prof.every != 0) return;  // bracket one matching launch in `every`
     cudaEventRecord(g_prof.start[g_prof.used], stream);
     g_prof.names[g_prof.used] = name;
     g_prof.pending = true;
@@ -299,10 +300,12 @@ int rmm_status_read(void *ws, int *device_status)
     return RMM_OK;
 }
 
-int rmm_profile_kernels(void **start_events, void **stop_events, int n, const char *name_filter)
+int rmm_profile_kernels(void **start_events, void **stop_events, int n, const char *name_filter, int every)
 {
     if (n < 0 || n > 4096 || ((start_events == nullptr || stop_events == nullptr) && n != 0))
         return fail(RMM_ERR_INVALID_ARG, "profile_kernels: need two event arrays and 0 <= n <= 4096, or NULL, NULL, 0");
+    g_prof.every = every > 1 ? every : 1;
+    g_prof.seen = 0;
     g_prof.start = reinterpret_cast<cudaEvent_t *>(start_events);
     g_prof.stop = reinterpret_cast<cudaEvent_t *>(stop_events);
     g_prof.capacity = n;
