@@ -47,6 +47,7 @@ __global__ void __launch_bounds__(kSoftmaxThreads) softmax_rows_kernel(const flo
                                                                        __nv_bfloat16 *__restrict__ P, int64_t ld_p)
 {
     __shared__ float sh[32];
+    pdl_wait();
     const int64_t i = blockIdx.x, h = blockIdx.y;
     const float *s = S + (h * Lq + i) * ld_s;
     __nv_bfloat16 *p = P + (h * Lq + i) * ld_p;
@@ -128,7 +129,7 @@ int launch_softmax_rows(const float *S, int64_t ld_s, int64_t heads, int64_t Lq,
 {
     dim3 grid((unsigned)Lq, (unsigned)heads);
     prof_begin("softmax_rows_kernel", stream);
-    softmax_rows_kernel<<<grid, kSoftmaxThreads, 0, stream>>>(S, ld_s, Lq, Lk, causal, P, ld_p);
+    launch_kernel(softmax_rows_kernel, grid, dim3(kSoftmaxThreads), 0, stream, 1, S, ld_s, Lq, Lk, causal, P, ld_p);
     return check_launch("softmax_rows_kernel", stream);
 }
 

@@ -18,6 +18,44 @@ extern std::atomic<int64_t> g_launches;
 void prof_begin(const char *kernel_name, cudaStream_t stream);  // call right before a launch (timing hook)
 int check_launch(const char *what, cudaStream_t stream);  // right after: cudaGetLastError -> status, counts the launch
 
+// Every kernel is launched with programmatic stream serialization allowed: its blocks may be scheduled, and run
+// their set-up (barrier initialisation, descriptor prefetch, TMEM allocation), while the previous kernel on the stream
+// drains.  A kernel touches global memory only after pdl_wait(), which returns once the previous grid has completed
+// and its writes are visible, so results do not depend on the overlap.  cluster_x > 1 adds a cluster dimension.
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                        int cluster_x, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster_x > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)cluster_x;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#ifdef __CUDACC__
+// Let the next kernel on the stream start its set-up, then wait for the previous kernel's results.
+__device__ __forceinline__ void pdl_wait()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 static inline size_t dtype_size(int dt) { return dt == RMM_BF16 ? 2 : 4; }

@@ -37,6 +37,7 @@ __global__ void __launch_bounds__(THREADS) reduced_gemm_simt_kernel(SimtArgs a)
     __shared__ float sA[BK][BM + 1];
     __shared__ float sB[BK][BN + 1];
     __shared__ int sIdx[BK];
+    pdl_wait();
 
     const int tid = threadIdx.x;
     const int64_t b = blockIdx.z;
@@ -141,10 +142,10 @@ int launch_gemm_simt(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx,
     dim3 grid((unsigned)ceil_div(a.N, BN), (unsigned)ceil_div(a.M, BM), (unsigned)A->batch);
     const bool in_bf16 = A->dtype == RMM_BF16, out_bf16 = Y->dtype == RMM_BF16;
     prof_begin("reduced_gemm_simt_kernel", stream);
-    if (in_bf16 && out_bf16) reduced_gemm_simt_kernel<true, true><<<grid, THREADS, 0, stream>>>(a);
-    else if (in_bf16) reduced_gemm_simt_kernel<true, false><<<grid, THREADS, 0, stream>>>(a);
-    else if (out_bf16) reduced_gemm_simt_kernel<false, true><<<grid, THREADS, 0, stream>>>(a);
-    else reduced_gemm_simt_kernel<false, false><<<grid, THREADS, 0, stream>>>(a);
+    if (in_bf16 && out_bf16) launch_kernel(reduced_gemm_simt_kernel<true, true>, grid, dim3(THREADS), 0, stream, 1, a);
+    else if (in_bf16) launch_kernel(reduced_gemm_simt_kernel<true, false>, grid, dim3(THREADS), 0, stream, 1, a);
+    else if (out_bf16) launch_kernel(reduced_gemm_simt_kernel<false, true>, grid, dim3(THREADS), 0, stream, 1, a);
+    else launch_kernel(reduced_gemm_simt_kernel<false, false>, grid, dim3(THREADS), 0, stream, 1, a);
     return check_launch("reduced_gemm_simt_kernel", stream);
 }
 

@@ -332,6 +332,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     if (threadIdx.x == 0) { GSTAMP_MAX(1); }
+    pdl_wait();  // set-up above overlapped the previous kernel's tail; operands are read from here on
 
     if (warp == 0) {
         // ---------------------------------------------------------------- producer (one thread; the others idle)
@@ -549,20 +550,9 @@ int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const TcArgs &a
     }
     const int64_t tiles = a.batch * a.tiles_m * a.tiles_n;
     const int64_t slots = sm_count() / CTAS;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((tiles < slots ? tiles : slots) * CTAS));
-    cfg.blockDim = dim3(kThreadsTc);
-    cfg.dynamicSmemBytes = L::kTotal;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = CTAS;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = CTAS == 2 ? 1 : 0;
     prof_begin("reduced_gemm_tc_kernel", stream);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, ma, mb, a);
+    cudaError_t e = launch_kernel(kern, dim3((unsigned)((tiles < slots ? tiles : slots) * CTAS)), dim3(kThreadsTc), L::kTotal, stream,
+                                  CTAS, ma, mb, a);
     if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "reduced_gemm_tc_kernel: launch: %s", cudaGetErrorString(e));
     return check_launch("reduced_gemm_tc_kernel", stream);
 }

@@ -162,6 +162,7 @@ __device__ void pack_rows(const PackJob &p, int64_t blk, int *status)
 __global__ void __launch_bounds__(kThreadsPack, 4) pack_kernel(const __grid_constant__ PackArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem[];
+    pdl_wait();
     int64_t blk = blockIdx.x;
     const int which = blk < a.job[0].blocks ? 0 : 1;
     if (which == 1) blk -= a.job[0].blocks;
@@ -235,7 +236,7 @@ int launch_pack(const PackSpec *specs, int n, int *status, cudaStream_t stream)
         configured = true;
     }
     prof_begin("pack_kernel", stream);
-    pack_kernel<<<(unsigned)blocks, kThreadsPack, smem, stream>>>(a);
+    launch_kernel(pack_kernel, dim3((unsigned)blocks), dim3(kThreadsPack), smem, stream, 1, a);
     return check_launch("pack_kernel", stream);
 }
 

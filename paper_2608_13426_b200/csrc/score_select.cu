@@ -564,6 +564,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_select_kernel(ScoreArgs a)
     extern __shared__ __align__(128) unsigned char s_dyn[];  // row-lane partial sums, later the select's key cache
     __shared__ SelectSmem s_sel;
     __shared__ int s_flag;
+    pdl_wait();
 
     const int tid = threadIdx.x;
     const int tx = tid % a.tx, ty = tid / a.tx;
@@ -669,6 +670,7 @@ __global__ void __launch_bounds__(kThreads, 1) score_tma_kernel(const __grid_con
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     }
     __syncthreads();
+    pdl_wait();
 
     auto issue = [&](int t) {  // thread 0 only: fetch tile t into its ring slot
         const int st = t % kTmaStages;
@@ -726,6 +728,7 @@ __global__ void __launch_bounds__(1024) select_kernel(const float *keys, int K, 
 {
     extern __shared__ __align__(128) unsigned char s_dyn[];
     __shared__ SelectSmem s_sel;
+    pdl_wait();
     const int64_t b = blockIdx.x;
     block_select_any(keys + b * K, K, k, idx + b * (int64_t)k, retained ? retained + b : nullptr, s_sel,
                      use_cache ? reinterpret_cast<unsigned *>(s_dyn) : nullptr);
@@ -837,7 +840,7 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
             tma_configured = true;
         }
         prof_begin("score_select_kernel", stream);
-        score_tma_kernel<<<grid, kThreads, kTmaStages * kTmaStageBytes, stream>>>(map, a, &hdr->status);
+        launch_kernel(score_tma_kernel, grid, dim3(kThreads), kTmaStages * kTmaStageBytes, stream, 1, map, a, &hdr->status);
         int rc2 = check_launch("score_select_kernel", stream);
         if (rc2 != RMM_OK || !do_select || fused) return rc2;
         return launch_select(a.energy, A->batch, p.n, k, idx, retained, ws, stream);
@@ -853,10 +856,10 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
         configured = true;
     }
     prof_begin("score_select_kernel", stream);
-    if (bf16 && p.vec == 8) score_select_kernel<8, true><<<grid, kThreads, smem, stream>>>(a);
-    else if (bf16) score_select_kernel<1, true><<<grid, kThreads, smem, stream>>>(a);
-    else if (p.vec == 4) score_select_kernel<4, false><<<grid, kThreads, smem, stream>>>(a);
-    else score_select_kernel<1, false><<<grid, kThreads, smem, stream>>>(a);
+    if (bf16 && p.vec == 8) launch_kernel(score_select_kernel<8, true>, grid, dim3(kThreads), smem, stream, 1, a);
+    else if (bf16) launch_kernel(score_select_kernel<1, true>, grid, dim3(kThreads), smem, stream, 1, a);
+    else if (p.vec == 4) launch_kernel(score_select_kernel<4, false>, grid, dim3(kThreads), smem, stream, 1, a);
+    else launch_kernel(score_select_kernel<1, false>, grid, dim3(kThreads), smem, stream, 1, a);
     int rc = check_launch("score_select_kernel", stream);
     if (rc != RMM_OK || !do_select || fused) return rc;
     return launch_select(a.energy, A->batch, p.n, k, idx, retained, ws, stream);
@@ -876,7 +879,7 @@ int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_
         configured = true;
     }
     prof_begin("select_kernel", stream);
-    select_kernel<<<(unsigned)batch, threads, smem, stream>>>(keys, (int)K, (int)k, idx, retained, use_cache);
+    launch_kernel(select_kernel, dim3((unsigned)batch), dim3(threads), smem, stream, 1, keys, (int)K, (int)k, idx, retained, use_cache);
     return check_launch("select_kernel", stream);
 }
 
