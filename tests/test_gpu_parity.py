@@ -137,6 +137,42 @@ def test_select_ties_and_extremes(oracle):
         assert np.array_equal(idx[b], want)
 
 
+@pytest.mark.parametrize("K", [3000, 8192, 20000])
+def test_select_many_equal_keys(oracle, K):
+    """Thousands of keys equal to the threshold (more than the kernel's short candidate list holds), mixed with
+    distinct ones: the lowest indices among the equal keys are kept, bit for bit."""
+    g = torch.Generator().manual_seed(K)
+    keys = torch.rand(K, generator=g) + 1.0
+    dup = torch.randperm(K, generator=g)[: (2 * K) // 3]
+    keys[dup] = 1.5                                   # two thirds of the keys tie at one value inside the range
+    for k in (K // 10, K // 2, (9 * K) // 10):
+        want, _ = oracle.select(keys.double().numpy(), k)
+        got = rmm.rmm_select(dev(keys), k=k).cpu().numpy()
+        assert np.array_equal(got, want)
+    # two clusters that straddle a power of two (no common leading bits beyond the sign)
+    keys = torch.cat([torch.full((K // 2,), 2047.5), torch.full((K - K // 2,), 2048.5)])[torch.randperm(K, generator=g)]
+    want, _ = oracle.select(keys.double().numpy(), K // 3)
+    assert np.array_equal(rmm.rmm_select(dev(keys), k=K // 3).cpu().numpy(), want)
+
+
+def test_static_and_random_index_controls(oracle):
+    """The paper's ablation controls need no extra entry point: a set chosen once (static) or drawn at random with the
+    same budget is simply passed to the reduced product; the retained-energy diagnostic orders them as Theorem 1 says."""
+    A0, B = synth.mlp_product(512, 1024, 256, seed=21)
+    A1 = synth.heavy_tailed_activations(512, 1024, seed=22)          # a later input with other heavy channels
+    k = 256
+    idx_static, _, e0, ret0 = rmm.rmm_score_select(dev(A0), k=k, want_energy=True, want_retained=True)
+    idx_dyn, _, e1, ret1 = rmm.rmm_score_select(dev(A1), k=k, want_energy=True, want_retained=True)
+    idx_rand = torch.sort(torch.randperm(1024, generator=torch.Generator().manual_seed(5))[:k]).values.int()
+    e1c = e1.double().cpu().numpy()
+    kept = lambda ix: float(e1c[ix.cpu().numpy()].sum() / e1c.sum())
+    assert kept(idx_dyn) == pytest.approx(float(ret1[0]), rel=1e-5)
+    assert kept(idx_dyn) >= kept(idx_static) >= 0.0 and kept(idx_dyn) >= kept(idx_rand)
+    for ix in (idx_static, idx_rand.cuda()):
+        Y = rmm.rmm_reduced_gemm(dev(A1), dev(B), ix, out_dtype=torch.float32)
+        assert rel_fro(Y.cpu().numpy(), oracle.reduced_gemm(A1, B, ix.cpu().numpy())) <= 1e-5
+
+
 # ------------------------------------------------------------------------------------------------
 # fused score + select
 # ------------------------------------------------------------------------------------------------
