@@ -341,6 +341,27 @@ def main():
                            "note": "fused score + top-k select, two alternating 537 MB inputs (above L2)"}
         del big
 
+    # ---- decode step (one activation row) on a 70B-class gate/up projection: the gathered GEMV reads only the kept rows
+    decode = None
+    if not args.no_sweep and rank == 0:
+        Kd, Nd = 8192, 28672
+        Ws = [synth.weight(Kd, Nd, seed=70 + i, device=str(dev)) for i in range(3)]     # 3 x 470 MB, rotated
+        x = synth.heavy_tailed_activations(1, Kd, seed=73, device=str(dev))
+        yd = torch.empty(1, Nd, dtype=torch.bfloat16, device=dev)
+        decode = []
+        for i in range(3):
+            torch.matmul(x, Ws[i], out=yd)
+        dense = time_region(lambda i: torch.matmul(x, Ws[i % 3], out=yd), 30, 1)
+        for rho in (0.25, 0.5, 1.0):
+            idx_d, _, _, _ = rmm.rmm_score_select(x, rho=rho)
+            for i in range(3):
+                rmm.rmm_reduced_gemm(x, Ws[i % 3], idx_d, out=yd)
+            t = time_region(lambda i: rmm.rmm_reduced_gemm(x, Ws[i % 3], idx_d, out=yd), 30, 1)
+            gbs = idx_d.numel() * Nd * 2 / t / 1e6
+            decode.append({"rho": rho, "shape": [1, Kd, Nd], "reduced_gemv_ms": t, "kept_rows_gbs": gbs,
+                           "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "dense_cublas_ms": dense, "speedup_vs_dense": dense / t})
+        del Ws
+
     # ---- per-kernel breakdown of one step (a separate, untimed pass with every launch bracketed by events)
     breakdown = {}
     if rank == 0:
@@ -365,7 +386,7 @@ def main():
             "config": {"workload": WORKLOAD, "rho": RHO, "k": k, "M": M, "K": K, "N": N, "parallelism": f"replicas x{world}",
                        "l2_policy": f"inputs larger than L2: {n_sets} rotating (A, B, Y) sets, {resident_bytes / 1e6:.0f} MB resident"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
-            "kernel_breakdown": breakdown, "per_rho": per_rho, "selection_pass_large": selection_large, "peaks": peaks,
+            "kernel_breakdown": breakdown, "per_rho": per_rho, "selection_pass_large": selection_large, "decode_step": decode, "peaks": peaks,
         }
         print(json.dumps(out))
     if world > 1:

@@ -112,7 +112,9 @@ int rmm_score_select_static(const rmm_mat_t *A, int axis, double rho, int64_t k,
  *   bf16 operands run on the tensor cores (fp32 accumulation) when A has stride_col 1, B has
  *   stride_col 1 (slices of the contraction axis contiguous) or stride_row 1, Y has stride_col 1, and
  *   pointers / leading strides are 16-byte aligned; Y may be bf16 or fp32.  Every other layout, and
- *   fp32 operands, run on a plain FMA kernel (fp32 accumulation).  A and B must share a dtype. */
+ *   fp32 operands, run on a plain FMA kernel (fp32 accumulation).  A and B must share a dtype.
+ *   Decode-step shapes (batch 1, M <= 4, bf16, B with contiguous rows; App. "Complexity Analysis", decoding step)
+ *   take a gathered GEMV that reads only the kept rows of B (k N 2 bytes) and packs nothing. */
 size_t rmm_reduced_gemm_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y);
 int rmm_reduced_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
                      const rmm_mat_t *Y, void *ws, size_t ws_bytes, void *stream);

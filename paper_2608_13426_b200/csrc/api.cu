@@ -192,6 +192,8 @@ size_t rmm_reduced_gemm_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, 
 {
     if (A == nullptr || B == nullptr || Y == nullptr) return 0;
     rmm_mat_t b = shared_b(A, B);
+    GemvPlan gplan;
+    if (gemv_eligible(A, &b, k, Y, &gplan)) return gplan.total_bytes;
     TcPlan plan;
     if (tc_eligible(A, &b, k, Y, &plan)) return plan.total_bytes;
     return RMM_WS_HEADER_BYTES;
@@ -203,6 +205,12 @@ int rmm_reduced_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx,
     int rc = check_gemm(A, B, idx, k, Y);
     if (rc != RMM_OK) return rc;
     rmm_mat_t b = shared_b(A, B);
+    GemvPlan gplan;
+    if (gemv_eligible(A, &b, k, Y, &gplan)) {  // decode-step shapes: only the kept rows of B are read
+        rc = check_ws(ws, ws_bytes, gplan.total_bytes, "reduced_gemm");
+        if (rc != RMM_OK) return rc;
+        return launch_gemv(A, &b, idx, k, scale, Y, gplan, ws, static_cast<cudaStream_t>(stream));
+    }
     TcPlan plan;
     if (tc_eligible(A, &b, k, Y, &plan)) {
         rc = check_ws(ws, ws_bytes, plan.total_bytes, "reduced_gemm");

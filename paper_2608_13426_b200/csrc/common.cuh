@@ -98,6 +98,15 @@ int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_
 int launch_gemm_simt(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
                      const rmm_mat_t *Y, void *ws, cudaStream_t stream);
 
+// Decode-step path (M <= 4 rows of bf16 activations, B rows contiguous): HBM-bound gathered GEMV, no packing.
+struct GemvPlan {
+    int splits, rows_per_split;
+    size_t off_partials, total_bytes;
+};
+bool gemv_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y, GemvPlan *plan);
+int launch_gemv(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale, const rmm_mat_t *Y,
+                const GemvPlan &plan, void *ws, cudaStream_t stream);
+
 // Tensor-core path (tcgen05, TMEM accumulators).  Operands must satisfy tc_eligible().
 struct TcPlan {
     int b_kmajor;       // 0: B rows (contraction slices) contiguous, kept rows copied; 1: B is K-contiguous, packed like A

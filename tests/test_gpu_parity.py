@@ -290,6 +290,29 @@ def test_reduced_gemm_fma_path(oracle, M, K, N, rho, dtype):
     assert rel_fro(Yb.float().cpu().numpy(), want) <= TOL_BF16
 
 
+@pytest.mark.parametrize("M,K,N,rho", [(1, 8192, 4096, 0.5), (1, 4096, 1000, 0.25), (2, 1024, 256, 0.75), (3, 8192, 2048, 0.1),
+                                       (8, 2048, 28672, 0.5), (5, 512, 8, 1.0)])
+def test_decode_step_gathered_gemv(oracle, M, K, N, rho):
+    """Decode-step shapes (a handful of activation rows): s_j = |x_j| for one row, the kept rows of W are the only
+    ones read; fp32 accumulation of exact bf16 products."""
+    A = synth.heavy_tailed_activations(M, K, seed=60 + M, frac=0.05)
+    B = synth.weight(K, N, seed=61 + M)
+    e64, _ = oracle.score(A)
+    k = oracle.keep_count(rho, K)
+    idx, _, _, _ = rmm.rmm_score_select(dev(A), rho=rho)
+    check_index_set(idx.cpu().numpy(), e64, k)
+    if M == 1:                                           # one row: the norm of a column is the magnitude of its entry
+        order = np.argsort(-np.abs(A[0].double().numpy()), kind="stable")[:k]
+        assert set(order.tolist()) == set(oracle.select(e64, k)[0].tolist())
+    want = oracle.reduced_gemm(A, B, idx.cpu().numpy())
+    Y = rmm.rmm_reduced_gemm(dev(A), dev(B), idx, out_dtype=torch.float32)
+    assert rel_fro(Y.cpu().numpy(), want) <= 1e-5
+    Yb = rmm.rmm_reduced_gemm(dev(A), dev(B), idx, scale=0.5)
+    assert rel_fro(Yb.float().cpu().numpy(), 0.5 * want) <= TOL_BF16
+    Y2 = rmm.rmm_reduced_gemm(dev(A), dev(B), idx, out_dtype=torch.float32)
+    assert torch.equal(Y, Y2)                            # deterministic
+
+
 def test_reduced_gemm_any_index_set_and_bad_index(oracle):
     """A cached or random set is accepted (static / random controls); an out-of-range index is skipped and reported."""
     A, B = synth.mlp_product(256, 512, 256, seed=11)
