@@ -56,6 +56,18 @@ __device__ __forceinline__ void pdl_wait()
 }
 #endif
 
+// Function attributes (the opt-in to more than 48 KB of dynamic shared memory) belong to a device: a flag per device
+// and call site says whether the current device has been set up.  Returns true exactly once per device.
+struct PerDeviceOnce {
+    std::atomic<bool> done[64];
+    bool first()
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;  // unknown: set up every time
+        return !done[dev].exchange(true);
+    }
+};
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 static inline size_t dtype_size(int dt) { return dt == RMM_BF16 ? 2 : 4; }

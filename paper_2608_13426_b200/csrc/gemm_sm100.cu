@@ -528,12 +528,9 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 // ----------------------------------------------------------------------------------------------
 int sm_count()
 {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    }
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
     return n;
 }
 
@@ -542,11 +539,10 @@ int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const TcArgs &a
 {
     auto kern = reduced_gemm_tc_kernel<BN, B_KMAJOR, OUT_BF16, CTAS>;
     using L = SmemLayout<BN, CTAS>;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    if (configured.first()) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
         if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        configured = true;
     }
     const int64_t tiles = a.batch * a.tiles_m * a.tiles_n;
     const int64_t slots = sm_count() / CTAS;

@@ -16,7 +16,7 @@ namespace {
 
 constexpr int kThreadsPack = 256;
 constexpr int kMaxStageBytes = 96 * 1024;  // longest source row that is staged in shared memory
-constexpr int kStageTarget = 32 * 1024;    // preferred staging size: several blocks per SM stay resident
+constexpr int kStageTarget = 36 * 1024;    // preferred staging size (two 8192-column rows with their zero pads): several blocks per SM stay resident
 constexpr int kDirectRows = 4;
 constexpr int kRowsPerBlock = 8;  // kept rows copied by one block of the row gather
 
@@ -46,17 +46,27 @@ __device__ __forceinline__ int checked_index(const int32_t *ix, int64_t j, int64
     return v;
 }
 
+__device__ __forceinline__ unsigned lds_u16(uint32_t addr)
+{
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+    return v;
+}
+
+// Staged rows have a pitch of K + 8 elements; the 8 spare elements are zero, so a missing or bad index simply
+// points at column K and the inner loop has no predicates.  All inner-loop addressing is 32-bit.
 __device__ void pack_cols_staged(const PackJob &p, int64_t blk, int *status, unsigned char *smem)
 {
     const int64_t b = blk / p.bx, r0 = (blk % p.bx) * p.R;
     const int tid = threadIdx.x;
-    const int kv = (int)(p.K / 8);  // 16-byte vectors per source row
+    const int K = (int)p.K, kv = K / 8, pitch_v = kv + 1;  // 16-byte vectors per source row / per staged row
     const unsigned short *s16 = reinterpret_cast<const unsigned short *>(p.src) + ((b + p.b_off) / p.b_div) * p.s_batch;
     uint4 *stage = reinterpret_cast<uint4 *>(smem);
     const int nrows = (int)min((int64_t)p.R, p.rows - r0);
     for (int r = 0; r < nrows; ++r) {
         const uint4 *srow = reinterpret_cast<const uint4 *>(s16 + (r0 + r) * p.s_row);
-        uint4 *drow = stage + (size_t)r * kv;
+        uint4 *drow = stage + r * pitch_v;
+        if (tid == 0) drow[kv] = make_uint4(0, 0, 0, 0);
         for (int c0 = tid; c0 < kv; c0 += 4 * kThreadsPack) {  // four independent loads in flight per thread and row
             uint4 v[4];
 #pragma unroll
@@ -68,28 +78,37 @@ __device__ void pack_cols_staged(const PackJob &p, int64_t blk, int *status, uns
         }
     }
     __syncthreads();
-    const unsigned short *rows = reinterpret_cast<const unsigned short *>(smem);
+    const uint32_t rows_s = (uint32_t)__cvta_generic_to_shared(smem);
+    const uint32_t pitch_b = (uint32_t)pitch_v * 16u;
     const int32_t *ix = p.idx != nullptr ? p.idx + b * p.idx_stride : nullptr;
-    unsigned *d32 = reinterpret_cast<unsigned *>(p.dst + b * p.rows * p.ld_dst);
-    const int half = (int)(p.ld_dst / 2), K = (int)p.K;
-    unsigned *drow0 = d32 + ((r0 * p.ld_dst) >> 1);
+    const int half = (int)(p.ld_dst / 2), k = (int)p.k;
+    unsigned *drow0 = reinterpret_cast<unsigned *>(p.dst + b * p.rows * p.ld_dst) + ((r0 * p.ld_dst) >> 1);
     for (int jp0 = tid; jp0 < half; jp0 += 4 * kThreadsPack) {  // four output pairs per thread: index loads first
-        int c[8];
+        uint32_t cb[8];  // byte offsets of the source columns inside a staged row
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int jp = jp0 + i * kThreadsPack;
-            c[2 * i] = jp < half ? checked_index(ix, 2 * jp, p.k, p.K, status) : -1;
-            c[2 * i + 1] = jp < half ? checked_index(ix, 2 * jp + 1, p.k, p.K, status) : -1;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int j = 2 * jp + h;
+                int c = K;  // the zero column
+                if (jp < half && j < k) {
+                    c = ix != nullptr ? __ldg(ix + j) : j;
+                    if (c < 0 || c >= K) {
+                        atomicExch(status, (int)RMM_ERR_BOUNDS);
+                        c = K;
+                    }
+                }
+                cb[2 * i + h] = (uint32_t)c * 2u;
+            }
         }
-        for (int r = 0; r < nrows; ++r) {
-            const unsigned short *row = rows + r * K;
+        uint32_t row_s = rows_s;
+        unsigned *d = drow0 + jp0;
+        for (int r = 0; r < nrows; ++r, row_s += pitch_b, d += half) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int jp = jp0 + i * kThreadsPack;
-                if (jp < half) {
-                    const unsigned lo = c[2 * i] >= 0 ? row[c[2 * i]] : 0u, hi = c[2 * i + 1] >= 0 ? row[c[2 * i + 1]] : 0u;
-                    drow0[(size_t)r * half + jp] = lo | (hi << 16);
-                }
+                const unsigned v = lds_u16(row_s + cb[2 * i]) | (lds_u16(row_s + cb[2 * i + 1]) << 16);
+                if (jp0 + i * kThreadsPack < half) d[i * kThreadsPack] = v;
             }
         }
     }
@@ -177,16 +196,16 @@ size_t plan_job(PackJob &p)
     size_t smem = 0;
     if (p.type == 1) {
         const bool staged = p.K % 8 == 0 && p.s_row % 8 == 0 && p.s_batch % 8 == 0 && reinterpret_cast<uintptr_t>(p.src) % 16 == 0 &&
-                            p.K * 2 <= kMaxStageBytes;
+                            (p.K + 8) * 2 <= kMaxStageBytes && p.K <= INT32_MAX / 4 && p.ld_dst <= INT32_MAX / 4;
         if (staged) {
-            int R = (int)(kStageTarget / (p.K * 2));
+            int R = (int)(kStageTarget / ((p.K + 8) * 2));
             if (R < 1) R = 1;
             if (R > 8) R = 8;
             if (R > p.rows) R = (int)p.rows;
             p.R = R;
             p.bx = ceil_div(p.rows, R);
             p.by = 1;
-            smem = (size_t)R * p.K * 2;
+            smem = (size_t)R * (p.K + 8) * 2;
         } else {
             p.type = 2;
             p.bx = ceil_div(p.ld_dst, 256 * (kThreadsPack / 32));
@@ -229,11 +248,10 @@ int launch_pack(const PackSpec *specs, int n, int *status, cudaStream_t stream)
         blocks += p.blocks;
     }
     if (blocks > INT32_MAX) return fail(RMM_ERR_UNSUPPORTED, "pack: too many blocks");
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    if (configured.first()) {
         cudaError_t e = cudaFuncSetAttribute(pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxStageBytes);
         if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "pack: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        configured = true;
     }
     prof_begin("pack_kernel", stream);
     launch_kernel(pack_kernel, dim3((unsigned)blocks), dim3(kThreadsPack), smem, stream, 1, a);

@@ -833,11 +833,10 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
         const uint32_t box[3] = {kTmaCols, kTmaRows, 1};
         int rc = make_map(&map, const_cast<void *>(a.A), 3, dims, st, box, false);
         if (rc != RMM_OK) return rc;
-        static bool tma_configured = false;
-        if (!tma_configured) {
+        static PerDeviceOnce tma_configured;
+        if (tma_configured.first()) {
             cudaError_t e = cudaFuncSetAttribute(score_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTmaStages * kTmaStageBytes);
             if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "score: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-            tma_configured = true;
         }
         prof_begin("score_select_kernel", stream);
         launch_kernel(score_tma_kernel, grid, dim3(kThreads), kTmaStages * kTmaStageBytes, stream, 1, map, a, &hdr->status);
@@ -845,15 +844,14 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
         if (rc2 != RMM_OK || !do_select || fused) return rc2;
         return launch_select(a.energy, A->batch, p.n, k, idx, retained, ws, stream);
     }
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    if (configured.first()) {
         const int big = kThreads * 8 * (int)sizeof(double);
         cudaError_t e = cudaFuncSetAttribute(score_select_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(score_select_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(score_select_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(score_select_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
         if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "score: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        configured = true;
     }
     prof_begin("score_select_kernel", stream);
     if (bf16 && p.vec == 8) launch_kernel(score_select_kernel<8, true>, grid, dim3(kThreads), smem, stream, 1, a);
@@ -872,11 +870,10 @@ int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_
     const int threads = 1024;
     const int use_cache = K <= kCachedSelectMax;
     const size_t smem = use_cache ? (size_t)K * 4 : 0;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    if (configured.first()) {
         cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kCachedSelectMax * 4);
         if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "select: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-        configured = true;
     }
     prof_begin("select_kernel", stream);
     launch_kernel(select_kernel, dim3((unsigned)batch), dim3(threads), smem, stream, 1, keys, (int)K, (int)k, idx, retained, use_cache);
