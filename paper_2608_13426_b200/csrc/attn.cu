@@ -8,6 +8,7 @@
 //   rho_t = 1: O = P V_g (same kernel, P and V loaded in place)
 // S~ and P live in the workspace (materialised), so this form is bound by HBM traffic, not by the tensor cores.
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -70,8 +71,19 @@ __global__ void __launch_bounds__(kSoftmaxThreads) softmax_rows_kernel(const flo
 
 struct AttnPlan {
     int64_t kd, kt, ldd, ldt, ld_s, ld_p, hg;
+    bool fused;
     size_t inner_bytes, off_idxf, off_idxt, off_qp, off_kp, off_s, off_p, off_pp, off_vp, total;
 };
+
+// rho_t = 1 with head_dim and kept features up to 128 runs fused (RMM_ATTN_FUSED=0 keeps the composed form, for comparison).
+bool use_fused(const rmm_attn_desc_t *d, int64_t kd)
+{
+    static const bool enabled = [] {
+        const char *e = getenv("RMM_ATTN_FUSED");
+        return e == nullptr || e[0] != '0';
+    }();
+    return enabled && fused_attn_eligible(d, kd);
+}
 
 int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
 {
@@ -97,7 +109,8 @@ int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
     const double per_head = (double)d->Lq * ((double)p->ld_s * 4 + (double)p->ld_p * 2 + (double)p->ldt * 2);
     int64_t hg = (int64_t)(6.0 * 1073741824.0 / per_head);
     if (hg < 1) hg = 1;
-    if (hg > d->Hq) hg = d->Hq;
+    p->fused = use_fused(d, p->kd);
+    if (hg > d->Hq || p->fused) hg = d->Hq;  // the fused form materialises neither S~ nor P: all heads at once
     p->hg = hg;
 
     // workspace of the inner score/select calls (the larger of the Q pass and the P pass)
@@ -114,10 +127,11 @@ int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
     p->off_idxt = off; off += align_up((size_t)hg * p->kt * 4, 256);
     p->off_qp = off; off += align_up((size_t)hg * d->Lq * p->ldd * 2, 256);
     p->off_kp = off; off += align_up((size_t)hg * d->Lk * p->ldd * 2, 256);
-    p->off_s = off; off += align_up((size_t)hg * d->Lq * p->ld_s * 4, 256);
-    p->off_p = off; off += align_up((size_t)hg * d->Lq * p->ld_p * 2, 256);
-    p->off_pp = off; off += align_up((size_t)hg * d->Lq * p->ldt * 2, 256);
-    p->off_vp = off; off += align_up((size_t)hg * p->kt * d->Dh * 2, 256);
+    const size_t mat = p->fused ? 0 : 1;
+    p->off_s = off; off += mat * align_up((size_t)hg * d->Lq * p->ld_s * 4, 256);
+    p->off_p = off; off += mat * align_up((size_t)hg * d->Lq * p->ld_p * 2, 256);
+    p->off_pp = off; off += mat * align_up((size_t)hg * d->Lq * p->ldt * 2, 256);
+    p->off_vp = off; off += mat * align_up((size_t)hg * p->kt * d->Dh * 2, 256);
     p->total = off;
     return RMM_OK;
 }
@@ -192,6 +206,14 @@ int rmm_reduced_attn(const rmm_attn_desc_t *d, const void *Q, const void *K, con
             qk[1] = pack_cols_spec(kk + b * d->k_stride[0], hg, d->Lk, d->Dh, d->k_stride[1], d->k_stride[2], h0, group, If, p.kd,
                                    p.kd, Kp, p.ldd);
             if ((rc = launch_pack(qk, 2, status, st)) != RMM_OK) return rc;
+
+            if (p.fused) {
+                rc = launch_fused_attn(Qp, Kp, p.ldd, p.kd, v, d->v_stride[2], d->v_stride[1], d->B * d->Hkv, b * d->Hq + h0, group,
+                                       o + b * d->o_stride[0] + h0 * d->o_stride[1], d->o_stride[1], d->o_stride[2], hg, d->Lq, d->Lk,
+                                       d->Dh, d->causal, status, st);
+                if (rc != RMM_OK) return rc;
+                continue;
+            }
 
             // S~ = Q[:, I] K[:, I]^T / sqrt(Dh)  (the scale keeps the full head dimension)
             TcProblem g1 = {};

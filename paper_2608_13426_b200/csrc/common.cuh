@@ -182,5 +182,13 @@ int launch_pack(const PackSpec *specs, int n, int *status, cudaStream_t stream);
 // P [heads, Lq, ld_p] (columns Lk .. ld_p zeroed).
 int launch_softmax_rows(const float *S, int64_t ld_s, int64_t heads, int64_t Lq, int64_t Lk, int causal,
                         __nv_bfloat16 *P, int64_t ld_p, cudaStream_t stream);
+// Fused form for rho_t = 1 (S~ and P stay on the SM): O = softmax(Qp Kp^T / sqrt(Dh) + mask) V for packed
+// Qp [heads, Lq, ldd], Kp [heads, Lk, ldd] (kd valid columns) and V [v_batches, Lk, Dh] read in place
+// (row pitch v_ld, batch pitch v_sb; head h uses batch entry (h + v_off) / v_div).
+bool fused_attn_eligible(const rmm_attn_desc_t *d, int64_t kd);
+int launch_fused_attn(const __nv_bfloat16 *Qp, const __nv_bfloat16 *Kp, int64_t ldd, int64_t kd, const __nv_bfloat16 *V,
+                      int64_t v_ld, int64_t v_sb, int64_t v_batches, int64_t v_off, int64_t v_div, __nv_bfloat16 *O,
+                      int64_t o_sh, int64_t o_sr, int64_t heads, int64_t Lq, int64_t Lk, int64_t Dh, int causal,
+                      int *status, cudaStream_t stream);
 
 }  // namespace rmm

@@ -200,7 +200,7 @@ size_t plan_job(PackJob &p)
         if (staged) {
             int R = (int)(kStageTarget / ((p.K + 8) * 2));
             if (R < 1) R = 1;
-            if (R > 8) R = 8;
+            if (R > 64) R = 64;  // short rows (attention heads): many rows per block
             if (R > p.rows) R = (int)p.rows;
             p.R = R;
             p.bx = ceil_div(p.rows, R);

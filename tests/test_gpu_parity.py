@@ -413,3 +413,29 @@ def test_reduced_attention_gqa_and_ragged(oracle):
     assert check_attention(oracle, 2, 8, 2, 100, 173, 128, True, 0.5, 0.5, seed=31)
     assert check_attention(oracle, 1, 4, 1, 257, 257, 128, False, 0.75, 0.3, seed=32)
     assert check_attention(oracle, 1, 2, 2, 1, 300, 64, True, 0.5, 1.0, seed=33)      # a single query row (decode shape)
+
+
+@pytest.mark.parametrize("shape", [
+    # B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d
+    (1, 2, 2, 128, 128, 128, True, 0.5),       # one tile
+    (1, 4, 2, 300, 300, 128, True, 0.5),       # ragged tail, two heads per kv head
+    (2, 4, 4, 257, 515, 64, True, 0.75),       # Lk > Lq: every query sees the prefix
+    (1, 2, 1, 384, 200, 128, True, 1.0),       # Lq > Lk: the first rows see no key and give zeros
+    (1, 3, 3, 200, 391, 128, False, 0.25),     # no mask
+    (1, 2, 2, 640, 640, 72, False, 0.5),       # head_dim that is no multiple of 64
+    (1, 8, 2, 1024, 1024, 128, True, 0.5),     # several blocks per head and a key ring that wraps
+])
+def test_fused_attention_feature_reduction_only(oracle, shape):
+    """rho_t = 1 runs the fused kernel (S~ and P stay on the SM); parity with the oracle's unfused definition."""
+    B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d = shape
+    assert check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, 1.0, seed=40 + Lq % 7)
+    assert rmm.rmm_status_read() == 0
+
+
+def test_fused_attention_rows_without_keys_are_zero():
+    B, Hq, Hkv, Lq, Lk, Dh = 1, 2, 2, 300, 100, 64
+    Q, K, V = synth.attention_qkv(B, Hq, Hkv, Lq, Lk, Dh, seed=47)
+    O = rmm.rmm_reduced_attn(dev(Q), dev(K), dev(V), True, 0.5, 1.0)
+    O = O[0] if isinstance(O, tuple) else O
+    assert torch.count_nonzero(O[:, :, : Lq - Lk]) == 0          # end-aligned mask: query i sees keys <= i - (Lq - Lk)
+    assert torch.isfinite(O.float()).all()
