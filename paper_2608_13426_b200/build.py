@@ -33,7 +33,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, *NVCC_FLAGS, "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB, *sources(),
+    extra = os.environ.get("RMM_NVCC_EXTRA", "").split()  # e.g. -DRMM_GEMM_STAMPS for the debug time stamps
+    cmd = [nvcc, *NVCC_FLAGS, *extra, "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB, *sources(),
            "-lcudart"]
     if verbose:
         cmd.insert(1, "-Xptxas")

@@ -63,18 +63,41 @@ __device__ void pack_cols_staged(const PackJob &p, int64_t blk, int *status, uns
     const unsigned short *s16 = reinterpret_cast<const unsigned short *>(p.src) + ((b + p.b_off) / p.b_div) * p.s_batch;
     uint4 *stage = reinterpret_cast<uint4 *>(smem);
     const int nrows = (int)min((int64_t)p.R, p.rows - r0);
-    for (int r = 0; r < nrows; ++r) {
-        const uint4 *srow = reinterpret_cast<const uint4 *>(s16 + (r0 + r) * p.s_row);
-        uint4 *drow = stage + r * pitch_v;
-        if (tid == 0) drow[kv] = make_uint4(0, 0, 0, 0);
-        for (int c0 = tid; c0 < kv; c0 += 4 * kThreadsPack) {  // four independent loads in flight per thread and row
+    if (kv >= kThreadsPack) {
+        for (int r = 0; r < nrows; ++r) {
+            const uint4 *srow = reinterpret_cast<const uint4 *>(s16 + (r0 + r) * p.s_row);
+            uint4 *drow = stage + r * pitch_v;
+            if (tid == 0) drow[kv] = make_uint4(0, 0, 0, 0);
+            for (int c0 = tid; c0 < kv; c0 += 4 * kThreadsPack) {  // four independent loads in flight per thread and row
+                uint4 v[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (c0 + i * kThreadsPack < kv) v[i] = __ldg(srow + c0 + i * kThreadsPack);
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (c0 + i * kThreadsPack < kv) drow[c0 + i * kThreadsPack] = v[i];
+            }
+        }
+    } else {
+        // short rows (attention heads): the block's rows are staged as one flat list of 16-byte vectors
+        const int total = nrows * kv;
+        const unsigned short *s0 = s16 + r0 * p.s_row;
+        for (int r = tid; r < nrows; r += kThreadsPack) stage[r * pitch_v + kv] = make_uint4(0, 0, 0, 0);
+        for (int f0 = tid; f0 < total; f0 += 4 * kThreadsPack) {
             uint4 v[4];
+            int at[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int f = f0 + i * kThreadsPack;
+                if (f < total) {
+                    const int r = f / kv, c = f - r * kv;
+                    v[i] = __ldg(reinterpret_cast<const uint4 *>(s0 + (int64_t)r * p.s_row) + c);
+                    at[i] = r * pitch_v + c;
+                }
+            }
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                if (c0 + i * kThreadsPack < kv) v[i] = __ldg(srow + c0 + i * kThreadsPack);
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (c0 + i * kThreadsPack < kv) drow[c0 + i * kThreadsPack] = v[i];
+                if (f0 + i * kThreadsPack < total) stage[at[i]] = v[i];
         }
     }
     __syncthreads();
@@ -83,6 +106,31 @@ __device__ void pack_cols_staged(const PackJob &p, int64_t blk, int *status, uns
     const int32_t *ix = p.idx != nullptr ? p.idx + b * p.idx_stride : nullptr;
     const int half = (int)(p.ld_dst / 2), k = (int)p.k;
     unsigned *drow0 = reinterpret_cast<unsigned *>(p.dst + b * p.rows * p.ld_dst) + ((r0 * p.ld_dst) >> 1);
+    if (2 * half <= kThreadsPack) {
+        // short rows: thread = (output pair, row phase); every thread keeps its two source columns for all its rows
+        const int rows_par = kThreadsPack / half, jp = tid % half, rsub = tid / half;
+        if (rsub < rows_par) {
+            uint32_t cb[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int j = 2 * jp + h;
+                int c = K;
+                if (j < k) {
+                    c = ix != nullptr ? __ldg(ix + j) : j;
+                    if (c < 0 || c >= K) {
+                        atomicExch(status, (int)RMM_ERR_BOUNDS);
+                        c = K;
+                    }
+                }
+                cb[h] = (uint32_t)c * 2u;
+            }
+            for (int r = rsub; r < nrows; r += rows_par) {
+                const uint32_t row_s = rows_s + (uint32_t)r * pitch_b;
+                drow0[r * half + jp] = lds_u16(row_s + cb[0]) | (lds_u16(row_s + cb[1]) << 16);
+            }
+        }
+        return;
+    }
     for (int jp0 = tid; jp0 < half; jp0 += 4 * kThreadsPack) {  // four output pairs per thread: index loads first
         uint32_t cb[8];  // byte offsets of the source columns inside a staged row
 #pragma unroll
@@ -200,7 +248,7 @@ size_t plan_job(PackJob &p)
         if (staged) {
             int R = (int)(kStageTarget / ((p.K + 8) * 2));
             if (R < 1) R = 1;
-            if (R > 64) R = 64;  // short rows (attention heads): many rows per block
+            if (R > 128) R = 128;  // short rows (attention heads): many rows per block
             if (R > p.rows) R = (int)p.rows;
             p.R = R;
             p.bx = ceil_div(p.rows, R);
