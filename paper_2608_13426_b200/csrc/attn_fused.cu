@@ -41,7 +41,6 @@ constexpr int kOffQ = 0, kOffKv = kGroups * kQTile, kOffP = kOffKv + kKvStages *
 constexpr int kFusedSmem = kOffBar + 512;
 constexpr int kTmemCols = 512;        // per group: S~ double buffer (2 x 64 columns); then O (128 columns per group)
 constexpr uint32_t kTmemO = kGroups * 2 * FN;
-constexpr unsigned kStaggerNs = 400;
 constexpr float kGrowLimit = 40.f;    // log2 of the largest p taken against a stale maximum
 
 // Debug aid (-DRMM_ATTN_STAMPS): clocks spent per phase by the MMA issuer of group 0 and by one softmax warp of
@@ -279,9 +278,6 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             }
             const int64_t last_key = a.causal ? min(a.Lk - 1, i + diag) : a.Lk - 1;  // < 0: this row sees nothing
             float m = -INFINITY, l = 0.f;  // m: the maximum that p is taken against (scaled, log2 domain)
-            // Start the second group half a step late: the exp phase of one group (bound by the special-function
-            // unit) then overlaps the other phases of its neighbour on the same scheduler, and the two stay apart.
-            if (g == 1) __nanosleep(kStaggerNs);
             for (int j = 0; j < nt; ++j, ++s_it, ++p_it) {
                 const uint32_t sb = s_it & 1u;
                 ASTAMP(7);

@@ -95,6 +95,13 @@ __device__ __forceinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity, 
     }
 }
 
+// Whole-warp form of the sleeping wait.
+__device__ __forceinline__ bool mbar_wait_sleepy_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+{
+    bool ok = mbar_wait_sleepy(bar, parity, abort_flag, status);
+    return __all_sync(0xffffffffu, ok);
+}
+
 // Whole-warp form: every lane waits, and the warp takes one common decision.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
