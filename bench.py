@@ -362,6 +362,35 @@ def main():
                            "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "dense_cublas_ms": dense, "speedup_vs_dense": dense / t})
         del Ws
 
+    # ---- reduced attention on a 7B-class prefill (32 heads, 4096 tokens, head_dim 128, causal): feature reduction
+    # only (fused kernel: S~ and P stay on the SM) and feature + token reduction (composed from the library's kernels,
+    # S~ and P materialised); torch's dense scaled_dot_product_attention at the same shape is context, not a target
+    attention = None
+    if not args.no_sweep and rank == 0:
+        Ha, La, Da = 32, 4096, 128
+        Qa, Ka, Va = synth.attention_qkv(1, Ha, Ha, La, La, Da, seed=0, device=str(dev))
+        for _ in range(3):
+            torch.nn.functional.scaled_dot_product_attention(Qa, Ka, Va, is_causal=True)
+        dense = time_region(lambda i: torch.nn.functional.scaled_dot_product_attention(Qa, Ka, Va, is_causal=True), 10, 1)
+        attention = []
+        for rho_d, rho_t, reps in ((0.5, 1.0, 10), (0.75, 1.0, 10), (0.5, 0.5, 3)):
+            for _ in range(2):
+                rmm.rmm_reduced_attn(Qa, Ka, Va, True, rho_d, rho_t)
+            t = time_region(lambda i: rmm.rmm_reduced_attn(Qa, Ka, Va, True, rho_d, rho_t), reps, 1)
+            kt = binding.KernelTimer(64)
+            with kt:
+                rmm.rmm_reduced_attn(Qa, Ka, Va, True, rho_d, rho_t)
+            parts = {}
+            for name, x in kt.times_ms():
+                parts[name] = parts.get(name, 0.0) + 1e3 * x
+            kd = rmm.rmm_keep_count(rho_d, Da)
+            # causal flops actually needed: (kd + Dh * rho_t) multiply-adds per visible (query, key) pair
+            fl = 2.0 * Ha * (La * (La + 1) / 2) * (kd + Da * rho_t)
+            attention.append({"rho_d": rho_d, "rho_t": rho_t, "shape": [Ha, La, Da], "causal": True, "ms": t,
+                              "retained_tflops": fl / t / 1e9, "kernels_us": parts, "dense_sdpa_ms": dense,
+                              "path": "fused" if rho_t >= 1.0 else "composed"})
+        del Qa, Ka, Va
+
     # ---- per-kernel breakdown of one step (a separate, untimed pass with every launch bracketed by events)
     breakdown = {}
     if rank == 0:
@@ -386,7 +415,8 @@ def main():
             "config": {"workload": WORKLOAD, "rho": RHO, "k": k, "M": M, "K": K, "N": N, "parallelism": f"replicas x{world}",
                        "l2_policy": f"inputs larger than L2: {n_sets} rotating (A, B, Y) sets, {resident_bytes / 1e6:.0f} MB resident"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
-            "kernel_breakdown": breakdown, "per_rho": per_rho, "selection_pass_large": selection_large, "decode_step": decode, "peaks": peaks,
+            "kernel_breakdown": breakdown, "per_rho": per_rho, "selection_pass_large": selection_large, "decode_step": decode,
+            "attention_prefill": attention, "peaks": peaks,
         }
         print(json.dumps(out))
     if world > 1:
