@@ -7,6 +7,12 @@
 //   rho_t < 1: score + select on P -> T; pack P[:, T] and V_g[T, :]; O = P[:, T] V_g[T, :]
 //   rho_t = 1: O = P V_g (same kernel, P and V loaded in place)
 // S~ and P live in the workspace (materialised), so this form is bound by HBM traffic, not by the tensor cores.
+//
+// With head_dim and kept features up to 128 the steps after the packing run fused instead (attn_fused.cu), S~ and P
+// staying on the SM:
+//   rho_t = 1: one pass, O = softmax(S~ + mask) V;
+//   rho_t < 1: row normalisers (sweep 1), token scores of the bf16-rounded P (sweep 2), select T, pack K[T] and V[T],
+//              O = P[:, T] V[T, :] (sweep 3).
 #include <math.h>
 #include <stdlib.h>
 
@@ -70,12 +76,12 @@ __global__ void __launch_bounds__(kSoftmaxThreads) softmax_rows_kernel(const flo
 }
 
 struct AttnPlan {
-    int64_t kd, kt, ldd, ldt, ld_s, ld_p, hg;
+    int64_t kd, kt, ldd, ldt, ld_s, ld_p, hg, lse_ld;
     bool fused;
-    size_t inner_bytes, off_idxf, off_idxt, off_qp, off_kp, off_s, off_p, off_pp, off_vp, total;
+    size_t inner_bytes, off_idxf, off_idxt, off_qp, off_kp, off_s, off_p, off_pp, off_vp, off_lse, off_energy, off_kpt, total;
 };
 
-// rho_t = 1 with head_dim and kept features up to 128 runs fused (RMM_ATTN_FUSED=0 keeps the composed form, for comparison).
+// head_dim and kept features up to 128 run fused (RMM_ATTN_FUSED=0 keeps the composed form, for comparison).
 bool use_fused(const rmm_attn_desc_t *d, int64_t kd)
 {
     static const bool enabled = [] {
@@ -131,7 +137,13 @@ int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
     p->off_s = off; off += mat * align_up((size_t)hg * d->Lq * p->ld_s * 4, 256);
     p->off_p = off; off += mat * align_up((size_t)hg * d->Lq * p->ld_p * 2, 256);
     p->off_pp = off; off += mat * align_up((size_t)hg * d->Lq * p->ldt * 2, 256);
-    p->off_vp = off; off += mat * align_up((size_t)hg * p->kt * d->Dh * 2, 256);
+    p->off_vp = off; off += align_up((size_t)hg * p->kt * d->Dh * 2, 256);
+    // fused token reduction: row normalisers, token scores, K[T]
+    const size_t tokf = p->fused && d->rho_t < 1.0 ? 1 : 0;
+    p->lse_ld = (d->Lq + 63) / 64 * 64;
+    p->off_lse = off; off += tokf * align_up((size_t)hg * p->lse_ld * 4, 256);
+    p->off_energy = off; off += tokf * align_up((size_t)hg * d->Lk * 4, 256);
+    p->off_kpt = off; off += tokf * align_up((size_t)hg * p->kt * p->ldd * 2, 256);
     p->total = off;
     return RMM_OK;
 }
@@ -208,9 +220,29 @@ int rmm_reduced_attn(const rmm_attn_desc_t *d, const void *Q, const void *K, con
             if ((rc = launch_pack(qk, 2, status, st)) != RMM_OK) return rc;
 
             if (p.fused) {
-                rc = launch_fused_attn(Qp, Kp, p.ldd, p.kd, v, d->v_stride[2], d->v_stride[1], d->B * d->Hkv, b * d->Hq + h0, group,
-                                       o + b * d->o_stride[0] + h0 * d->o_stride[1], d->o_stride[1], d->o_stride[2], hg, d->Lq, d->Lk,
-                                       d->Dh, d->causal, status, st);
+                __nv_bfloat16 *og = o + b * d->o_stride[0] + h0 * d->o_stride[1];
+                if (!tok) {
+                    rc = launch_fused_attn(Qp, Kp, p.ldd, p.kd, v, d->v_stride[2], d->v_stride[1], d->B * d->Hkv, b * d->Hq + h0, group,
+                                           og, d->o_stride[1], d->o_stride[2], hg, d->Lq, d->Lk, d->Dh, d->causal, d->Lk - d->Lq,
+                                           nullptr, 0, nullptr, status, st);
+                    if (rc != RMM_OK) return rc;
+                    continue;
+                }
+                float *lse = reinterpret_cast<float *>(w + p.off_lse), *energy = reinterpret_cast<float *>(w + p.off_energy);
+                __nv_bfloat16 *KpT = reinterpret_cast<__nv_bfloat16 *>(w + p.off_kpt);
+                // sweeps 1 and 2: row normalisers, then token scores of the bf16-rounded P; one token set per query head
+                rc = launch_fused_attn_scores(Qp, Kp, p.ldd, p.kd, hg, d->Lq, d->Lk, d->Dh, d->causal, lse, p.lse_ld, energy, status, st);
+                if (rc != RMM_OK) return rc;
+                if ((rc = launch_select(energy, hg, d->Lk, p.kt, It, nullptr, w, st)) != RMM_OK) return rc;
+                // K[T] (already reduced to the kept features) and V[T]
+                PackSpec kv[2];
+                kv[0] = pack_rows_spec(Kp, hg, d->Lk, p.ldd, d->Lk * p.ldd, p.ldd, 0, 1, It, p.kt, p.kt, KpT, p.ldd);
+                kv[1] = pack_rows_spec(v + b * d->v_stride[0], hg, d->Lk, d->Dh, d->v_stride[1], d->v_stride[2], h0, group, It, p.kt,
+                                       p.kt, Vp, d->Dh);
+                if ((rc = launch_pack(kv, 2, status, st)) != RMM_OK) return rc;
+                // sweep 3: O = P[:, T] V[T, :] against the full-row normalisers
+                rc = launch_fused_attn(Qp, KpT, p.ldd, p.kd, Vp, d->Dh, p.kt * d->Dh, hg, 0, 1, og, d->o_stride[1], d->o_stride[2], hg,
+                                       d->Lq, p.kt, d->Dh, d->causal, d->Lk - d->Lq, lse, p.lse_ld, It, status, st);
                 if (rc != RMM_OK) return rc;
                 continue;
             }

@@ -182,13 +182,21 @@ int launch_pack(const PackSpec *specs, int n, int *status, cudaStream_t stream);
 // P [heads, Lq, ld_p] (columns Lk .. ld_p zeroed).
 int launch_softmax_rows(const float *S, int64_t ld_s, int64_t heads, int64_t Lq, int64_t Lk, int causal,
                         __nv_bfloat16 *P, int64_t ld_p, cudaStream_t stream);
-// Fused form for rho_t = 1 (S~ and P stay on the SM): O = softmax(Qp Kp^T / sqrt(Dh) + mask) V for packed
-// Qp [heads, Lq, ldd], Kp [heads, Lk, ldd] (kd valid columns) and V [v_batches, Lk, Dh] read in place
-// (row pitch v_ld, batch pitch v_sb; head h uses batch entry (h + v_off) / v_div).
+// Fused forms (S~ and P stay on the SM; head_dim and kept features up to 128) on packed Qp [heads, Lq, ldd],
+// Kp [heads, Lk, ldd] (kd valid columns) and V [v_batches, Lk, Dh] (row pitch v_ld, batch pitch v_sb; head h uses
+// batch entry (h + v_off) / v_div).
 bool fused_attn_eligible(const rmm_attn_desc_t *d, int64_t kd);
+// lse == tok == NULL: O = softmax(Qp Kp^T / sqrt(Dh) + mask) V.  With lse [heads, lse_ld] and tok [heads, Lk] given,
+// Kp and V hold the kept keys only (Lk of them, at positions tok): O = P V with P = bf16(2^(x - lse)), not
+// renormalised.  diag = Lk - Lq of the unpacked problem (causal: query i sees key t iff t <= i + diag).
 int launch_fused_attn(const __nv_bfloat16 *Qp, const __nv_bfloat16 *Kp, int64_t ldd, int64_t kd, const __nv_bfloat16 *V,
                       int64_t v_ld, int64_t v_sb, int64_t v_batches, int64_t v_off, int64_t v_div, __nv_bfloat16 *O,
-                      int64_t o_sh, int64_t o_sr, int64_t heads, int64_t Lq, int64_t Lk, int64_t Dh, int causal,
-                      int *status, cudaStream_t stream);
+                      int64_t o_sh, int64_t o_sr, int64_t heads, int64_t Lq, int64_t Lk, int64_t Dh, int causal, int64_t diag,
+                      const float *lse, int64_t lse_ld, const int32_t *tok, int *status, cudaStream_t stream);
+// Two sweeps: lse [heads, lse_ld] (lse_ld a multiple of 64, >= Lq) = log2-domain row normalisers of softmax(S~ + mask);
+// energy [heads, Lk] = squared token scores sum_i bf16(P_it)^2.
+int launch_fused_attn_scores(const __nv_bfloat16 *Qp, const __nv_bfloat16 *Kp, int64_t ldd, int64_t kd, int64_t heads,
+                             int64_t Lq, int64_t Lk, int64_t Dh, int causal, float *lse, int64_t lse_ld, float *energy,
+                             int *status, cudaStream_t stream);
 
 }  // namespace rmm

@@ -226,6 +226,31 @@ __device__ void pack_rows(const PackJob &p, int64_t blk, int *status)
     }
 }
 
+// Row gather of short rows (fewer 16-byte vectors per row than threads per block): a thread owns one vector position
+// and kRowsPerBlock rows, so a block covers (threads / vectors) * kRowsPerBlock rows with every thread busy.
+__device__ void pack_rows_short(const PackJob &p, int64_t blk, int *status)
+{
+    const int nvec = (int)(p.n / 8), rows_par = kThreadsPack / nvec, rows_blk = rows_par * kRowsPerBlock;
+    const int64_t b = blk / p.by, j0 = (blk % p.by) * rows_blk;
+    const int c = threadIdx.x % nvec, rsub = threadIdx.x / nvec;
+    if (rsub >= rows_par) return;
+    const uint4 *sbase = reinterpret_cast<const uint4 *>(p.src) + ((b + p.b_off) / p.b_div) * (p.s_batch / 8);
+    uint4 *dbase = reinterpret_cast<uint4 *>(p.dst) + (b * p.k) * (p.ld_dst / 8);
+    const int32_t *ix = p.idx != nullptr ? p.idx + b * p.idx_stride : nullptr;
+    int rows[kRowsPerBlock];
+#pragma unroll
+    for (int i = 0; i < kRowsPerBlock; ++i) {
+        const int64_t j = j0 + rsub + (int64_t)rows_par * i;
+        rows[i] = j < p.k ? checked_index(ix, j, p.k, p.K, status) : -2;  // -1: bad index, write zeros; -2: no row
+    }
+    uint4 v[kRowsPerBlock];
+#pragma unroll
+    for (int i = 0; i < kRowsPerBlock; ++i) v[i] = rows[i] >= 0 ? __ldg(sbase + rows[i] * (p.s_row / 8) + c) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int i = 0; i < kRowsPerBlock; ++i)
+        if (rows[i] != -2) dbase[(j0 + rsub + (int64_t)rows_par * i) * (p.ld_dst / 8) + c] = v[i];
+}
+
 __global__ void __launch_bounds__(kThreadsPack, 4) pack_kernel(const __grid_constant__ PackArgs a)
 {
     extern __shared__ __align__(16) unsigned char smem[];
@@ -237,6 +262,7 @@ __global__ void __launch_bounds__(kThreadsPack, 4) pack_kernel(const __grid_cons
     if (p.type == 1) pack_cols_staged(p, blk, a.status, smem);
     else if (p.type == 2) pack_cols_direct(p, blk, a.status);
     else if (p.type == 3) pack_rows(p, blk, a.status);
+    else if (p.type == 4) pack_rows_short(p, blk, a.status);
 }
 
 size_t plan_job(PackJob &p)
@@ -259,6 +285,10 @@ size_t plan_job(PackJob &p)
             p.bx = ceil_div(p.ld_dst, 256 * (kThreadsPack / 32));
             p.by = ceil_div(p.rows, kDirectRows);
         }
+    } else if (p.type == 3 && p.n / 8 <= kThreadsPack / 2) {
+        p.type = 4;  // short rows
+        p.bx = 1;
+        p.by = ceil_div(p.k, (int64_t)(kThreadsPack / (p.n / 8)) * kRowsPerBlock);
     } else if (p.type == 3) {
         int64_t gx = ceil_div(p.n / 8, kThreadsPack);
         p.bx = gx > 8 ? 8 : gx;

@@ -439,3 +439,45 @@ def test_fused_attention_rows_without_keys_are_zero():
     O = O[0] if isinstance(O, tuple) else O
     assert torch.count_nonzero(O[:, :, : Lq - Lk]) == 0          # end-aligned mask: query i sees keys <= i - (Lq - Lk)
     assert torch.isfinite(O.float()).all()
+
+
+@pytest.mark.parametrize("shape", [
+    # B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t
+    (1, 2, 2, 128, 128, 128, True, 0.5, 0.5),       # one tile
+    (1, 4, 2, 300, 300, 128, True, 0.5, 0.25),      # ragged tail, two heads per kv head
+    (2, 4, 4, 257, 515, 64, True, 0.75, 0.5),       # Lk > Lq
+    (1, 2, 1, 384, 200, 128, True, 1.0, 0.5),       # Lq > Lk: the first rows see no key
+    (1, 3, 3, 200, 391, 128, False, 0.25, 0.3),     # no mask
+    (1, 2, 2, 640, 640, 72, False, 0.5, 0.75),      # head_dim that is no multiple of 64
+    (1, 4, 2, 1024, 1024, 128, True, 0.5, 0.5),     # several blocks per head and a key ring that wraps
+])
+def test_fused_attention_token_reduction(oracle, shape):
+    """rho_t < 1 through the fused sweeps (row normalisers, token scores of the rounded P, gathered P V): the token
+    sets meet Theorem 1's criterion against the oracle's P, and O matches wherever the sets agree."""
+    B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t = shape
+    assert check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t, seed=60 + Lq % 7)
+    assert rmm.rmm_status_read() == 0
+
+
+def test_fused_and_composed_attention_agree(oracle, monkeypatch):
+    """The fused sweeps and the composed form (S~ and P materialised) are two routes to the same result."""
+    import subprocess, sys, os
+    code = (
+        "import torch, paper_2608_13426_b200 as rmm\n"
+        "from paper_2608_13426_b200 import synth\n"
+        "Q, K, V = synth.attention_qkv(1, 4, 2, 300, 420, 128, seed=71, device='cuda')\n"
+        "O, f, t = rmm.rmm_reduced_attn(Q, K, V, True, 0.5, 0.5, want_idx=True)\n"
+        "torch.save((O.cpu(), f.cpu(), t.cpu()), __import__('sys').argv[1])\n")
+    outs = []
+    for flag in ("1", "0"):
+        path = os.path.join(os.environ.get("TMPDIR", "/tmp"), f"rmm_attn_{flag}_{os.getpid()}.pt")
+        env = dict(os.environ, RMM_ATTN_FUSED=flag)
+        subprocess.run([sys.executable, "-c", code, path], check=True, env=env, cwd=os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+        outs.append(torch.load(path))
+        os.remove(path)
+    (O1, f1, t1), (O0, f0, t0) = outs
+    assert torch.equal(f1, f0)
+    same = [h for h in range(4) if torch.equal(t1[0, h], t0[0, h])]
+    assert len(same) >= 2
+    for h in same:
+        assert rel_fro(O1[0, h].float().numpy(), O0[0, h].float().numpy().astype(np.float64)) <= TOL_BF16
