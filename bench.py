@@ -216,6 +216,44 @@ def run_reference(args):
     }))
 
 
+def attention_case(rmm, binding, synth, dev, heads, seq, head_dim=128, reps=10):
+    """Reduced attention on a prefill shape (heads x seq x head_dim, causal): feature reduction only (one fused pass) and
+    feature + token reduction (three fused sweeps: row normalisers, token scores, gathered P V); S~ and P stay on the SM
+    in both.  torch's dense scaled_dot_product_attention at the same shape is context, not a target."""
+    Qa, Ka, Va = synth.attention_qkv(1, heads, heads, seq, seq, head_dim, seed=0, device=str(dev))
+    for _ in range(3):
+        torch.nn.functional.scaled_dot_product_attention(Qa, Ka, Va, is_causal=True)
+    dense = time_region(lambda i: torch.nn.functional.scaled_dot_product_attention(Qa, Ka, Va, is_causal=True), reps, 1)
+    out = []
+    for rho_d, rho_t in ((0.5, 1.0), (0.75, 1.0), (0.5, 0.5), (0.5, 0.25)):
+        for _ in range(2):
+            rmm.rmm_reduced_attn(Qa, Ka, Va, True, rho_d, rho_t)
+        t = time_region(lambda i: rmm.rmm_reduced_attn(Qa, Ka, Va, True, rho_d, rho_t), reps, 1)
+        kt = binding.KernelTimer(64)
+        with kt:
+            rmm.rmm_reduced_attn(Qa, Ka, Va, True, rho_d, rho_t)
+        parts = {}
+        for name, x in kt.times_ms():
+            parts[name] = parts.get(name, 0.0) + 1e3 * x
+        kd = rmm.rmm_keep_count(rho_d, head_dim)
+        # causal flops actually needed: (kd + Dh * rho_t) multiply-adds per visible (query, key) pair
+        fl = 2.0 * heads * (seq * (seq + 1) / 2) * (kd + head_dim * rho_t)
+        out.append({"rho_d": rho_d, "rho_t": rho_t, "shape": [heads, seq, head_dim], "causal": True, "ms": t,
+                    "retained_tflops": fl / t / 1e9, "kernels_us": parts, "dense_sdpa_ms": dense,
+                    "path": "fused, one pass" if rho_t >= 1.0 else "fused, three sweeps"})
+    return out
+
+
+def run_attention_only(args):
+    import paper_2608_13426_b200 as rmm
+    from paper_2608_13426_b200 import binding, synth
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    res = attention_case(rmm, binding, synth, dev, args.attn_heads, args.attn_seq, reps=3)
+    assert rmm.rmm_status_read() == 0
+    print(json.dumps({"attention_prefill": res}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -225,9 +263,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU oracle timing (quick runs, profiling)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-rho sweep")
     ap.add_argument("--sets", type=int, default=5, help="independent (A, B, Y) input sets rotated per step (5 = 377 MB, above L2)")
+    ap.add_argument("--attention-only", action="store_true",
+                    help="run only the reduced-attention case (a few launches: for profiler captures) and print its own JSON line")
+    ap.add_argument("--attn-heads", type=int, default=32)
+    ap.add_argument("--attn-seq", type=int, default=4096)
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.attention_only:
+        return run_attention_only(args)
     if args.warmup < 3:
         args.warmup = 3
 
@@ -362,35 +406,10 @@ def main():
                            "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "dense_cublas_ms": dense, "speedup_vs_dense": dense / t})
         del Ws
 
-    # ---- reduced attention on a 7B-class prefill (32 heads, 4096 tokens, head_dim 128, causal): feature reduction
-    # only (one fused pass) and feature + token reduction (three fused sweeps: row normalisers, token scores, gathered
-    # P V); S~ and P stay on the SM in both.  torch's dense scaled_dot_product_attention at the same shape is context,
-    # not a target
+    # ---- reduced attention on a 7B-class prefill (32 heads, 4096 tokens, head_dim 128, causal)
     attention = None
     if not args.no_sweep and rank == 0:
-        Ha, La, Da = 32, 4096, 128
-        Qa, Ka, Va = synth.attention_qkv(1, Ha, Ha, La, La, Da, seed=0, device=str(dev))
-        for _ in range(3):
-            torch.nn.functional.scaled_dot_product_attention(Qa, Ka, Va, is_causal=True)
-        dense = time_region(lambda i: torch.nn.functional.scaled_dot_product_attention(Qa, Ka, Va, is_causal=True), 10, 1)
-        attention = []
-        for rho_d, rho_t, reps in ((0.5, 1.0, 10), (0.75, 1.0, 10), (0.5, 0.5, 10), (0.5, 0.25, 10)):
-            for _ in range(2):
-                rmm.rmm_reduced_attn(Qa, Ka, Va, True, rho_d, rho_t)
-            t = time_region(lambda i: rmm.rmm_reduced_attn(Qa, Ka, Va, True, rho_d, rho_t), reps, 1)
-            kt = binding.KernelTimer(64)
-            with kt:
-                rmm.rmm_reduced_attn(Qa, Ka, Va, True, rho_d, rho_t)
-            parts = {}
-            for name, x in kt.times_ms():
-                parts[name] = parts.get(name, 0.0) + 1e3 * x
-            kd = rmm.rmm_keep_count(rho_d, Da)
-            # causal flops actually needed: (kd + Dh * rho_t) multiply-adds per visible (query, key) pair
-            fl = 2.0 * Ha * (La * (La + 1) / 2) * (kd + Da * rho_t)
-            attention.append({"rho_d": rho_d, "rho_t": rho_t, "shape": [Ha, La, Da], "causal": True, "ms": t,
-                              "retained_tflops": fl / t / 1e9, "kernels_us": parts, "dense_sdpa_ms": dense,
-                              "path": "fused, one pass" if rho_t >= 1.0 else "fused, three sweeps"})
-        del Qa, Ka, Va
+        attention = attention_case(rmm, binding, synth, dev, 32, 4096)
 
     # ---- per-kernel breakdown of one step (a separate, untimed pass with every launch bracketed by events)
     breakdown = {}

@@ -124,3 +124,23 @@ def test_reduced_attention_multi_tile(oracle):
             ok_heads += 1
             assert rel_fro(O[0, h].float().cpu().numpy(), Oo[0, h]) <= TOL_BF16
     assert ok_heads >= 1
+
+
+@pytest.mark.parametrize("rho_t", [1.0, 0.5])
+def test_long_context_fused_attention(oracle, rho_t):
+    """Fused reduced attention at 8192 tokens (a key ring that wraps many times, several items per block, all four
+    kernel modes): 2 query heads on 1 kv head, head_dim 128, causal, rho_d = 0.5."""
+    B, Hq, Hkv, L, Dh = 1, 2, 1, 8192, 128
+    Q, K, V = synth.attention_qkv(B, Hq, Hkv, L, L, Dh, seed=21)
+    O, idx_feat, idx_tok = rmm.rmm_reduced_attn(Q.cuda(), K.cuda(), V.cuda(), True, 0.5, rho_t, want_idx=True)
+    Oo, If, It, P = oracle.attn(Q, K, V, True, 0.5, rho_t, round_p=True, want_p=True)
+    assert np.array_equal(idx_feat.cpu().numpy(), If)
+    for h in range(Hq):
+        if rho_t < 1.0:
+            got = idx_tok.cpu().numpy()[0, h]
+            a2 = (P[0, h] ** 2).sum(axis=0)
+            assert np.all(np.diff(got) > 0)
+            assert a2[got].sum() >= (1 - 1e-6) * a2[It[0, h]].sum()
+            if not np.array_equal(got, It[0, h]):
+                continue
+        assert rel_fro(O[0, h].float().cpu().numpy(), Oo[0, h]) <= TOL_BF16
