@@ -244,6 +244,46 @@ def attention_case(rmm, binding, synth, dev, heads, seq, head_dim=128, reps=10):
     return out
 
 
+def layer_sweep_70b(rmm, synth, dev, peaks, tokens=32768, hidden=8192, inter=28672, reps=3):
+    """Whole reduced product (score + select + gathers + GEMM) per projection shape and rho, dense cuBLAS beside it."""
+    shapes = [("q_o_proj", tokens, hidden, hidden), ("k_v_proj", tokens, hidden, 1024),
+              ("gate_up_proj", tokens, hidden, inter), ("down_proj", tokens, inter, hidden)]
+    out = []
+    for name, m, kk, n in shapes:
+        A = synth.heavy_tailed_activations(m, kk, seed=7, device=str(dev))
+        B = synth.weight(kk, n, seed=8, device=str(dev))
+        Y = torch.empty(m, n, dtype=torch.bfloat16, device=dev)
+        for _ in range(2):
+            torch.matmul(A, B, out=Y)
+        dense = time_region(lambda i: torch.matmul(A, B, out=Y), reps, 1)
+        for rho in RHOS:
+            k = rmm.rmm_keep_count(rho, kk)
+            idx = torch.empty(k, dtype=torch.int32, device=dev)
+
+            def op(i):
+                rmm.rmm_score_select(A, rho=rho, idx=idx)
+                rmm.rmm_reduced_gemm(A, B, idx, out=Y)
+
+            op(0)
+            t = time_region(op, reps, 1)
+            fl = 2.0 * m * k * n
+            out.append({"layer": name, "shape": [m, kk, n], "rho": rho, "whole_op_ms": t, "whole_op_tflops": fl / t / 1e9,
+                        "frac_of_sustained_peak": fl / t / 1e9 / peaks["bf16_sustained"], "dense_cublas_ms": dense,
+                        "dense_cublas_tflops": 2.0 * m * kk * n / dense / 1e9, "speedup_vs_dense_cublas": dense / t})
+        del A, B, Y
+    # attention of one layer: 64 query heads on 8 kv heads, causal
+    Q, Kx, V = synth.attention_qkv(1, 64, 8, tokens, tokens, 128, seed=0, device=str(dev))
+    for _ in range(2):
+        torch.nn.functional.scaled_dot_product_attention(Q, Kx, V, is_causal=True, enable_gqa=True)
+    dense = time_region(lambda i: torch.nn.functional.scaled_dot_product_attention(Q, Kx, V, is_causal=True, enable_gqa=True), reps, 1)
+    for rho_d, rho_t in ((0.5, 1.0), (0.5, 0.5), (0.5, 0.25)):
+        rmm.rmm_reduced_attn(Q, Kx, V, True, rho_d, rho_t)
+        t = time_region(lambda i: rmm.rmm_reduced_attn(Q, Kx, V, True, rho_d, rho_t), reps, 1)
+        out.append({"layer": "attention", "shape": [64, 8, tokens, 128], "rho_d": rho_d, "rho_t": rho_t, "ms": t,
+                    "dense_sdpa_ms": dense, "speedup_vs_dense_sdpa": dense / t})
+    return out
+
+
 def run_attention_only(args):
     import paper_2608_13426_b200 as rmm
     from paper_2608_13426_b200 import binding, synth
@@ -411,6 +451,12 @@ def main():
     if not args.no_sweep and rank == 0:
         attention = attention_case(rmm, binding, synth, dev, 32, 4096)
 
+    # ---- 70B-class layer (hidden 8192, intermediate 28672, 64 query / 8 kv heads, 32768 prefill tokens): every
+    # projection at every rho beside dense cuBLAS, and the attention of one layer
+    layer70 = None
+    if not args.no_sweep and rank == 0:
+        layer70 = layer_sweep_70b(rmm, synth, dev, peaks)
+
     # ---- per-kernel breakdown of one step (a separate, untimed pass with every launch bracketed by events)
     breakdown = {}
     if rank == 0:
@@ -436,7 +482,7 @@ def main():
                        "l2_policy": f"inputs larger than L2: {n_sets} rotating (A, B, Y) sets, {resident_bytes / 1e6:.0f} MB resident"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "kernel_breakdown": breakdown, "per_rho": per_rho, "selection_pass_large": selection_large, "decode_step": decode,
-            "attention_prefill": attention, "peaks": peaks,
+            "attention_prefill": attention, "layer_sweep_70b": layer70, "peaks": peaks,
         }
         print(json.dumps(out))
     if world > 1:

@@ -481,3 +481,9 @@ def test_fused_and_composed_attention_agree(oracle, monkeypatch):
     assert len(same) >= 2
     for h in same:
         assert rel_fro(O1[0, h].float().numpy(), O0[0, h].float().numpy().astype(np.float64)) <= TOL_BF16
+
+
+def test_composed_attention_for_wide_heads(oracle):
+    """head_dim above 128 runs the composed form (S~ and P in the workspace); both reductions."""
+    assert check_attention(oracle, 1, 2, 1, 130, 200, 256, True, 0.5, 0.5, seed=81)
+    assert check_attention(oracle, 1, 2, 2, 96, 96, 256, False, 0.75, 1.0, seed=82)
