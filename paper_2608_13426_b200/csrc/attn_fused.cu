@@ -244,66 +244,71 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         ASTAMP_DECL(blockIdx.x == 0 && lane == 0 && g == 0);
         auto step_s = [&](int j) -> bool {  // S~ of tile j (if this group needs it); consumes one ring entry
             ASTAMP(7);
-            if (!mbar_wait_lane(kv_full(ks), kph, abort_flag, a.status)) return false;
+            if (!mbar_wait(kv_full(ks), kph, abort_flag, a.status)) return false;
             ASTAMP(0);
             if (j >= gb && j < ge) {
                 const uint32_t sb = s_it & 1u;
-                if (!mbar_wait_lane(s_empty(g, sb), ((s_it >> 1) & 1u) ^ 1u, abort_flag, a.status)) return false;
+                if (!mbar_wait(s_empty(g, sb), ((s_it >> 1) & 1u) ^ 1u, abort_flag, a.status)) return false;
                 ASTAMP(1);
                 tc_fence_after();
                 uint32_t ql = q_lo, kl = k_lo + ks * (kKvTile >> 4), acc = 0;
-                for (int left = steps_s; left > 0; left -= 4, ql += kQChunk >> 4, kl += kKvChunk >> 4) {  // 64-feature chunks
-                    const int ns = left < 4 ? left : 4;
-                    for (int st = 0; st < ns; ++st, acc = 1u)  // 16 features = 32 bytes per step
-                        umma_bf16_lohi<1>(t_s + sb * FN, ql + 2 * st, q_hi, kl + 2 * st, k_hi, idesc_s, acc);
+                if (elect_one()) {
+                    for (int left = steps_s; left > 0; left -= 4, ql += kQChunk >> 4, kl += kKvChunk >> 4) {  // 64-feature chunks
+                        const int ns = left < 4 ? left : 4;
+                        for (int st = 0; st < ns; ++st, acc = 1u)  // 16 features = 32 bytes per step
+                            umma_bf16_lohi<1>(t_s + sb * FN, ql + 2 * st, q_hi, kl + 2 * st, k_hi, idesc_s, acc);
+                    }
+                    umma_commit<1>(s_full(g, sb));
                 }
-                umma_commit<1>(s_full(g, sb));
                 ++s_it;
             }
-            umma_commit<1>(kv_empty(ks));
+            if (elect_one()) umma_commit<1>(kv_empty(ks));
+            __syncwarp();
             if (++ks == kKvStages) { ks = 0; kph ^= 1u; }
             ASTAMP(2);
             return true;
         };
-        for (int64_t n = 0; lane == 0 && n < rounds && ok; ++n) {
+        for (int64_t n = 0; n < rounds && ok; ++n) {
             int64_t head, r0;
             if (!item_of(n, &head, &r0)) continue;
             int jb, je;
             block_range(head, r0, &jb, &je);
             if (je <= jb) continue;
             tile_range(head, r0 + g * FM, &gb, &ge);
-            if (!mbar_wait_lane(q_full, n_item & 1u, abort_flag, a.status)) { ok = false; break; }
+            if (!mbar_wait(q_full, n_item & 1u, abort_flag, a.status)) { ok = false; break; }
             ok = step_s(jb);
             for (int j = jb; j < je && ok; ++j) {
                 if (j + 1 < je) ok = step_s(j + 1);                        // S~ of the next tile runs ahead of this P V
                 if (!ok) break;
                 if constexpr (kHasV) {
                     ASTAMP(7);
-                    if (!mbar_wait_lane(kv_full(ks), kph, abort_flag, a.status)) { ok = false; break; }
+                    if (!mbar_wait(kv_full(ks), kph, abort_flag, a.status)) { ok = false; break; }
                     ASTAMP(3);
                     if (j >= gb && j < ge) {
-                        if (j == gb && !mbar_wait_lane(o_empty(g), (o_it & 1u) ^ 1u, abort_flag, a.status)) { ok = false; break; }
+                        if (j == gb && !mbar_wait(o_empty(g), (o_it & 1u) ^ 1u, abort_flag, a.status)) { ok = false; break; }
                         ASTAMP(4);
-                        if (!mbar_wait_lane(p_full(g), p_it & 1u, abort_flag, a.status)) { ok = false; break; }
+                        if (!mbar_wait(p_full(g), p_it & 1u, abort_flag, a.status)) { ok = false; break; }
                         ASTAMP(5);
                         tc_fence_after();
                         const uint32_t vl = v_lo + ks * (kKvTile >> 4);
+                        if (elect_one()) {
 #pragma unroll
-                        for (int st = 0; st < FN / 16; ++st)  // P: K-major, 32 bytes per step; V: MN-major (rows = keys), 16 keys = 2048 bytes
-                            umma_bf16_lohi<1>(t_o, p_lo + st * 2, p_hi, vl + st * (2048 >> 4), v_hi, idesc_o, (j != gb || st != 0) ? 1u : 0u);
-                        umma_commit<1>(p_empty(g));   // "P V of this tile is complete": P may be rewritten, O may be rescaled
-                        ++p_it;
-                        if (j == ge - 1) {
-                            umma_commit<1>(o_full(g));
-                            ++o_it;
+                            for (int st = 0; st < FN / 16; ++st)  // P: K-major, 32 bytes per step; V: MN-major (rows = keys), 16 keys = 2048 bytes
+                                umma_bf16_lohi<1>(t_o, p_lo + st * 2, p_hi, vl + st * (2048 >> 4), v_hi, idesc_o, (j != gb || st != 0) ? 1u : 0u);
+                            umma_commit<1>(p_empty(g));   // "P V of this tile is complete": P may be rewritten, O may be rescaled
+                            if (j == ge - 1) umma_commit<1>(o_full(g));
                         }
+                        ++p_it;
+                        if (j == ge - 1) ++o_it;
                     }
-                    umma_commit<1>(kv_empty(ks));
+                    if (elect_one()) umma_commit<1>(kv_empty(ks));
+                    __syncwarp();
                     if (++ks == kKvStages) { ks = 0; kph ^= 1u; }
                     ASTAMP(6);
                 }
             }
-            if (ok) umma_commit<1>(q_empty);
+            if (ok && elect_one()) umma_commit<1>(q_empty);
+            __syncwarp();
             ++n_item;
         }
         ASTAMP_FLUSH(0);

@@ -95,6 +95,19 @@ __device__ __forceinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity, 
     }
 }
 
+// One lane of the (converged) warp: the code around it stays warp-uniform, so descriptors and counters can live in
+// uniform registers, which is where the tensor-core instructions take their operands from.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 // Whole-warp form of the sleeping wait.
 __device__ __forceinline__ bool mbar_wait_sleepy_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
 {
