@@ -146,12 +146,6 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     const uint32_t sa = base + s * L::kStageBytes;
                     const uint32_t sb = sa + L::kABytes;
                     const int row_a = tm * (BM * CTAS) + (int)rank * BM, col_b = tn * BN + (int)rank * BNL;
-#ifdef RMM_GEMM_SKIP_B
-                    if constexpr (CTAS == 1) {
-                        mbar_arrive_expect_tx(full_bar(s), L::kABytes);
-                        tma_load_3d(sa, &map_a, kb * BK, row_a, (int)b, full_bar(s));
-                    } else
-#endif
                     if constexpr (CTAS == 1) {
                         mbar_arrive_expect_tx(full_bar(s), L::kStageBytes);
                         tma_load_3d(sa, &map_a, kb * BK, row_a, (int)b, full_bar(s));
