@@ -91,6 +91,27 @@ bool use_fused(const rmm_attn_desc_t *d, int64_t kd)
     return enabled && fused_attn_eligible(d, kd);
 }
 
+// A batch of sequences whose (batch, head) pairs are evenly spaced in memory is one sequence with B * Hq heads on
+// B * Hkv kv heads (head h of sequence b reads kv head b * Hkv + h / group either way): one pass of launches
+// instead of B.
+rmm_attn_desc_t fold_batch(const rmm_attn_desc_t &d)
+{
+    rmm_attn_desc_t f = d;
+    const bool even = d.B > 1 && d.Hkv >= 1 && d.Hq % d.Hkv == 0 && d.B * d.Hq <= 65535 &&
+                      d.q_stride[0] == d.Hq * d.q_stride[1] && d.k_stride[0] == d.Hkv * d.k_stride[1] &&
+                      d.v_stride[0] == d.Hkv * d.v_stride[1] && d.o_stride[0] == d.Hq * d.o_stride[1];
+    if (even) {
+        f.B = 1;
+        f.Hq = d.B * d.Hq;
+        f.Hkv = d.B * d.Hkv;
+        f.q_stride[0] = f.Hq * d.q_stride[1];
+        f.k_stride[0] = f.Hkv * d.k_stride[1];
+        f.v_stride[0] = f.Hkv * d.v_stride[1];
+        f.o_stride[0] = f.Hq * d.o_stride[1];
+    }
+    return f;
+}
+
 int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
 {
     if (d == nullptr) return fail(RMM_ERR_INVALID_ARG, "reduced_attn: NULL description");
@@ -168,14 +189,19 @@ extern "C" {
 size_t rmm_reduced_attn_workspace_bytes(const rmm_attn_desc_t *desc)
 {
     AttnPlan p;
-    if (plan_attn(desc, &p) != RMM_OK) return 0;
+    if (desc == nullptr) return 0;
+    const rmm_attn_desc_t folded = fold_batch(*desc);
+    if (plan_attn(&folded, &p) != RMM_OK) return 0;
     return p.total;
 }
 
-int rmm_reduced_attn(const rmm_attn_desc_t *d, const void *Q, const void *K, const void *V, void *O, int32_t *idx_feat,
+int rmm_reduced_attn(const rmm_attn_desc_t *desc, const void *Q, const void *K, const void *V, void *O, int32_t *idx_feat,
                      int32_t *idx_tok, void *ws, size_t ws_bytes, void *stream)
 {
     AttnPlan p;
+    if (desc == nullptr) return fail(RMM_ERR_INVALID_ARG, "reduced_attn: NULL description");
+    const rmm_attn_desc_t folded = fold_batch(*desc);
+    const rmm_attn_desc_t *d = &folded;
     int rc = plan_attn(d, &p);
     if (rc != RMM_OK) return rc;
     if (Q == nullptr || K == nullptr || V == nullptr || O == nullptr) return fail(RMM_ERR_INVALID_ARG, "reduced_attn: NULL tensor");

@@ -487,3 +487,21 @@ def test_composed_attention_for_wide_heads(oracle):
     """head_dim above 128 runs the composed form (S~ and P in the workspace); both reductions."""
     assert check_attention(oracle, 1, 2, 1, 130, 200, 256, True, 0.5, 0.5, seed=81)
     assert check_attention(oracle, 1, 2, 2, 96, 96, 256, False, 0.75, 1.0, seed=82)
+
+
+def test_attention_batch_folding_and_uneven_batch_stride(oracle):
+    """A contiguous batch is folded into the head axis (one pass of launches); a Q whose batch stride is not
+    Hq * head stride takes the per-sequence loop.  Both must give the same result."""
+    B, Hq, Hkv, Lq, Lk, Dh = 3, 4, 2, 150, 150, 64
+    Q, K, V = synth.attention_qkv(B, Hq, Hkv, Lq, Lk, Dh, seed=91)
+    Qd, Kd, Vd = dev(Q), dev(K), dev(V)
+    O1, f1, _ = rmm.rmm_reduced_attn(Qd, Kd, Vd, True, 0.5, 1.0, want_idx=True)
+    big = torch.zeros(B, Hq + 1, Lq, Dh, dtype=torch.bfloat16, device="cuda")
+    big[:, :Hq] = Qd
+    Qv = big[:, :Hq]
+    assert Qv.stride(0) != Hq * Qv.stride(1)
+    O2, f2, _ = rmm.rmm_reduced_attn(Qv, Kd, Vd, True, 0.5, 1.0, want_idx=True)
+    assert torch.equal(f1, f2) and torch.equal(O1, O2)
+    Oo, If, _ = oracle.attn(Q, K, V, True, 0.5, 1.0, round_p=True)[:3]
+    assert np.array_equal(f1.cpu().numpy(), If)
+    assert rel_fro(O1.float().cpu().numpy(), Oo) <= TOL_BF16
