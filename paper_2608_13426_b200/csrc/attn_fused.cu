@@ -11,10 +11,11 @@
 //   GATHERED  rho_t < 1, sweep 3:  O = P[:, T] V[T, :] on the kept keys (K[T], V[T] packed), P_it = bf16(2^(x_it -
 //             lse_i)) against the full-row normaliser of sweep 1: no renormalisation (Sec. 3.3).
 //
-// One block owns 256 rows of one head as two groups of 128 and walks the other axis in tiles of 64; both groups
+// One block owns 256 rows of one head as two groups of 128 and walks the other axis in tiles of 128; both groups
 // consume the same tiles, so each crosses from L2 to the SM once per 256 rows.  Per tile and group: S~ on the tensor
-// cores (kd of the Dh features); one thread per row takes p = 2^(x - m), rounds it once to bf16 and writes it to
-// shared memory as the A operand of O += P V.  In FULL mode m is the row maximum seen so far, refreshed only when
+// cores (kd of the Dh features; 128 columns of tensor memory, released as soon as the softmax warps hold the tile in
+// registers); one thread per row takes p = 2^(x - m) in two chunks of 64 columns, rounds it once to bf16 and writes it
+// to shared memory as the A operand of O += P V.  In FULL mode m is the row maximum seen so far, refreshed only when
 // the new maximum exceeds it by more than 40 (p up to 2^40 and row sums up to 2^71 are far from the bf16 and fp32
 // range limits, and floating point keeps the same relative precision at any scale): then l and the O row in tensor
 // memory are multiplied by 2^(m_old - m_new); the epilogue divides by l.  The paper rounds the normalised weight P
@@ -36,20 +37,21 @@ using namespace ptx;
 
 enum { MODE_FULL = 0, MODE_STATS = 1, MODE_ENERGY = 2, MODE_GATHERED = 3 };
 
-constexpr int FM = 128, FN = 64;      // rows per group, columns per step
+constexpr int FM = 128, FN = 128;     // rows per group, columns per step
 constexpr int kGroups = 2;
 constexpr int kFusedThreads = 64 + kGroups * 128 + 32;  // producer, MMA issuer 0, 8 softmax warps, MMA issuer 1
 constexpr int kMmaWarp1 = 10;
-constexpr int kKvStages = 8;
+constexpr int kKvStages = 3;
 constexpr int kQChunk = 16384;        // row-side chunk: 128 rows x 64 features (128 bytes per row, 128-byte swizzle)
 constexpr int kQTile = 2 * kQChunk;   // up to 128 kept features
-constexpr int kKvChunk = 8192;        // column-side chunk: 64 keys x 64 features (or 64 keys x 64 columns of V)
+constexpr int kKvChunk = 16384;       // column-side chunk: 128 keys x 64 features (or 128 keys x 64 columns of V)
 constexpr int kKvTile = 2 * kKvChunk; // ring entry: a K tile (up to 128 kept features) or a V tile (up to 128 columns)
-constexpr int kPTile = 16384;         // P tile: 128 rows x 64 keys
+constexpr int kPChunk = 16384;        // P chunk: 128 rows x 64 keys (128 bytes per row, 128-byte swizzle)
+constexpr int kPTile = 2 * kPChunk;   // P tile: 128 rows x 128 keys
 constexpr int kOffQ = 0, kOffKv = kGroups * kQTile, kOffP = kOffKv + kKvStages * kKvTile, kOffBar = kOffP + kGroups * kPTile;
 constexpr int kFusedSmem = kOffBar + 512;
-constexpr int kTmemCols = 512;        // per group: S~ double buffer (2 x 64 columns); then O (128 columns per group)
-constexpr uint32_t kTmemO = kGroups * 2 * FN;
+constexpr int kTmemCols = 512;        // per group: S~ (128 columns); then O (128 columns per group)
+constexpr uint32_t kTmemO = kGroups * FN;
 constexpr float kGrowLimit = 40.f;    // log2 of the largest p taken against a stale maximum
 
 // Debug aid (-DRMM_ATTN_STAMPS): clocks spent per phase by the MMA issuer of group 0 and by one softmax warp of
@@ -237,7 +239,7 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const uint32_t q_hi = (uint32_t)(dq0 >> 32), k_hi = (uint32_t)(dk0 >> 32), p_hi = (uint32_t)(dp0 >> 32), v_hi = (uint32_t)(dv0 >> 32);
         const uint32_t q_lo = (uint32_t)dq0, k_lo = (uint32_t)dk0, p_lo = (uint32_t)dp0, v_lo = (uint32_t)dv0;
         const int steps_s = (a.kd + 15) / 16;
-        const uint32_t t_s = tmem_base + g * 2 * FN, t_o = tmem_base + kTmemO + g * 128;
+        const uint32_t t_s = tmem_base + g * FN, t_o = tmem_base + kTmemO + g * 128;
         uint32_t ks = 0, kph = 0, n_item = 0, s_it = 0, p_it = 0, o_it = 0;
         bool ok = true;
         int gb = 0, ge = 0;  // this group's tile range in the current item
@@ -247,8 +249,8 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (!mbar_wait(kv_full(ks), kph, abort_flag, a.status)) return false;
             ASTAMP(0);
             if (j >= gb && j < ge) {
-                const uint32_t sb = s_it & 1u;
-                if (!mbar_wait(s_empty(g, sb), ((s_it >> 1) & 1u) ^ 1u, abort_flag, a.status)) return false;
+                // S~ is single-buffered: the softmax warps release it as soon as they hold the tile in registers
+                if (!mbar_wait(s_empty(g, 0), (s_it & 1u) ^ 1u, abort_flag, a.status)) return false;
                 ASTAMP(1);
                 tc_fence_after();
                 uint32_t ql = q_lo, kl = k_lo + ks * (kKvTile >> 4), acc = 0;
@@ -256,9 +258,9 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     for (int left = steps_s; left > 0; left -= 4, ql += kQChunk >> 4, kl += kKvChunk >> 4) {  // 64-feature chunks
                         const int ns = left < 4 ? left : 4;
                         for (int st = 0; st < ns; ++st, acc = 1u)  // 16 features = 32 bytes per step
-                            umma_bf16_lohi<1>(t_s + sb * FN, ql + 2 * st, q_hi, kl + 2 * st, k_hi, idesc_s, acc);
+                            umma_bf16_lohi<1>(t_s, ql + 2 * st, q_hi, kl + 2 * st, k_hi, idesc_s, acc);
                     }
-                    umma_commit<1>(s_full(g, sb));
+                    umma_commit<1>(s_full(g, 0));
                 }
                 ++s_it;
             }
@@ -293,8 +295,9 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         const uint32_t vl = v_lo + ks * (kKvTile >> 4);
                         if (elect_one()) {
 #pragma unroll
-                            for (int st = 0; st < FN / 16; ++st)  // P: K-major, 32 bytes per step; V: MN-major (rows = keys), 16 keys = 2048 bytes
-                                umma_bf16_lohi<1>(t_o, p_lo + st * 2, p_hi, vl + st * (2048 >> 4), v_hi, idesc_o, (j != gb || st != 0) ? 1u : 0u);
+                            for (int st = 0; st < FN / 16; ++st)  // P: K-major, 64-key chunks, 32 bytes per step; V: MN-major (rows = keys), 16 keys = 2048 bytes
+                                umma_bf16_lohi<1>(t_o, p_lo + (st >> 2) * (kPChunk >> 4) + (st & 3) * 2, p_hi, vl + st * (2048 >> 4), v_hi, idesc_o,
+                                                  (j != gb || st != 0) ? 1u : 0u);
                             umma_commit<1>(p_empty(g));   // "P V of this tile is complete": P may be rewritten, O may be rescaled
                             if (j == ge - 1) umma_commit<1>(o_full(g));
                         }
@@ -315,12 +318,13 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ softmax and epilogue (one row per thread)
+        // A step is 128 columns, taken as two chunks of 64 so that a thread never holds more than 64 logits.
         const int g = (warp - 2) >> 2, q = warp & 3, r = q * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
-        const uint32_t t_s = t_lane + g * 2 * FN, t_o = t_lane + kTmemO + g * 128;
+        const uint32_t t_s = t_lane + g * FN, t_o = t_lane + kTmemO + g * 128;
         const float c2 = a.scale_log2;
         const uint64_t c22 = pack2(c2, c2);
-        uint8_t *prow = base_ptr + kOffP + g * kPTile + r * 128;  // row r: 64 keys = 128 bytes, 16-byte units swizzled
+        uint8_t *prow = base_ptr + kOffP + g * kPTile + r * 128;  // row r of each 64-key chunk: 128 bytes, 16-byte units swizzled
         uint32_t s_it = 0, p_it = 0, o_it = 0;
         bool ok = true;
         ASTAMP_DECL(blockIdx.x == 0 && warp == 2 && lane == 0);
@@ -354,107 +358,46 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             float m = -INFINITY, l = 0.f;  // FULL / STATS: the maximum that p is taken against (log2 domain), the row sum
             float row_lse = 0.f;           // GATHERED: this row's normaliser
             if constexpr (MODE == MODE_GATHERED) row_lse = i < a.lse_ld ? a.lse[head * a.lse_ld + i] : INFINITY;
-            for (int j = jb; j < je; ++j, ++s_it) {
-                const uint32_t sb = s_it & 1u;
-                // ENERGY: the normalisers of this tile's 64 queries (the same for every thread), fetched ahead of the wait
-                float4 cl[MODE == MODE_ENERGY ? 16 : 1];
-                if constexpr (MODE == MODE_ENERGY) {
-                    const float4 *lp = reinterpret_cast<const float4 *>(a.lse + head * a.lse_ld + (int64_t)j * FN);
-#pragma unroll
-                    for (int u = 0; u < 16; ++u) cl[u] = __ldg(lp + u);
-                }
-                ASTAMP(7);
-                if (!mbar_wait(s_full(g, sb), (s_it >> 1) & 1u, abort_flag, a.status)) { ok = false; break; }
-                ASTAMP(0);
-                tc_fence_after();
-                uint32_t v0[32], v1[32];
-                tmem_ld32_issue(t_s + sb * FN + 0, v0);
-                tmem_ld32_issue(t_s + sb * FN + 32, v1);
-                tmem_ld_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(s_empty(g, sb));
-                ASTAMP(1);
 
-                // boundary tiles only (the diagonal and the ragged end): hidden columns become -inf
-                const int64_t c0 = (int64_t)j * FN;
+            // 64 logits of the current tile (columns c_off .. c_off + 63) into registers; hidden columns become -inf on
+            // boundary tiles (the diagonal and the ragged end)
+            auto load_chunk = [&](int j, int c_off, uint32_t (&v0)[32], uint32_t (&v1)[32]) {
+                tmem_ld32_issue(t_s + c_off, v0);
+                tmem_ld32_issue(t_s + c_off + 32, v1);
+                tmem_ld_wait();
+                const int64_t c0 = (int64_t)j * FN + c_off;
                 const int64_t rel_hi = last_col - c0, rel_lo = first_col - c0;
-                const int hi = rel_hi > FN - 1 ? FN - 1 : (rel_hi < -1 ? -1 : (int)rel_hi);
-                const int lo = rel_lo < 0 ? 0 : (rel_lo > FN ? FN : (int)rel_lo);
-                if (!__all_sync(0xffffffffu, hi >= FN - 1 && lo <= 0)) {
+                const int hi = rel_hi > 63 ? 63 : (rel_hi < -1 ? -1 : (int)rel_hi);
+                const int lo = rel_lo < 0 ? 0 : (rel_lo > 64 ? 64 : (int)rel_lo);
+                if (!__all_sync(0xffffffffu, hi >= 63 && lo <= 0)) {
 #pragma unroll
                     for (int e = 0; e < 32; ++e) {
                         if (e > hi || e < lo) v0[e] = 0xff800000u;
                         if (e + 32 > hi || e + 32 < lo) v1[e] = 0xff800000u;
                     }
                 }
-
-                if constexpr (MODE == MODE_ENERGY) {
-                    // p = bf16(2^(x - lse_i)); this key's score accumulates p^2 over the queries
-                    float acc0 = 0.f, acc1 = 0.f;
-                    auto fold = [&](const uint32_t (&v)[32], int c) {
+            };
+            auto release_s = [&]() {  // this warp holds what it needs of the S~ tile
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(s_empty(g, 0));
+            };
+            auto max_chunk = [&](const uint32_t (&v0)[32], const uint32_t (&v1)[32]) -> float {
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                        for (int e = 0; e < 32; e += 4) {
-                            const float4 ls = cl[(c + e) >> 2];
-                            const float p0 = ex2(fmaf(__uint_as_float(v[e]), c2, -ls.x)), p1 = ex2(fmaf(__uint_as_float(v[e + 1]), c2, -ls.y));
-                            const float p2 = ex2(fmaf(__uint_as_float(v[e + 2]), c2, -ls.z)), p3 = ex2(fmaf(__uint_as_float(v[e + 3]), c2, -ls.w));
-                            const float2 ra = __bfloat1622float2(__floats2bfloat162_rn(p0, p1));
-                            const float2 rb = __bfloat1622float2(__floats2bfloat162_rn(p2, p3));
-                            acc0 = fmaf(ra.x, ra.x, acc0);
-                            acc1 = fmaf(ra.y, ra.y, acc1);
-                            acc0 = fmaf(rb.x, rb.x, acc0);
-                            acc1 = fmaf(rb.y, rb.y, acc1);
-                        }
-                    };
-                    fold(v0, 0);
-                    fold(v1, 32);
-                    l += acc0 + acc1;
-                    continue;
+                for (int e = 0; e < 32; e += 4) {
+                    mx0 = fmax3(mx0, __uint_as_float(v0[e]), __uint_as_float(v0[e + 1]));
+                    mx1 = fmax3(mx1, __uint_as_float(v0[e + 2]), __uint_as_float(v0[e + 3]));
+                    mx2 = fmax3(mx2, __uint_as_float(v1[e]), __uint_as_float(v1[e + 1]));
+                    mx3 = fmax3(mx3, __uint_as_float(v1[e + 2]), __uint_as_float(v1[e + 3]));
                 }
-
-                if constexpr (MODE == MODE_FULL || MODE == MODE_STATS) {
-                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        mx0 = fmax3(mx0, __uint_as_float(v0[e]), __uint_as_float(v0[e + 1]));
-                        mx1 = fmax3(mx1, __uint_as_float(v0[e + 2]), __uint_as_float(v0[e + 3]));
-                        mx2 = fmax3(mx2, __uint_as_float(v1[e]), __uint_as_float(v1[e + 1]));
-                        mx3 = fmax3(mx3, __uint_as_float(v1[e + 2]), __uint_as_float(v1[e + 3]));
-                    }
-                    const float mc = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * c2;
-                    const bool grow = mc > m + kGrowLimit;
-                    if (__any_sync(0xffffffffu, grow)) {
-                        const float alpha = (grow && m > -INFINITY) ? ex2(m - mc) : 1.f;
-                        l *= alpha;
-                        if (grow) m = mc;
-                        if constexpr (MODE == MODE_FULL) {
-                            if (j > jb) {  // rows of O already hold sums taken against the old maximum
-                                if (!mbar_wait(p_empty(g), (p_it & 1u) ^ 1u, abort_flag, a.status)) { ok = false; break; }
-                                tc_fence_after();
-                                for (int c = 0; c < nv * 64; c += 32) {
-                                    uint32_t o[32];
-                                    tmem_ld32_issue(t_o + c, o);
-                                    tmem_ld_wait();
-#pragma unroll
-                                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                                    tmem_st32_issue(t_o + c, o);
-                                }
-                                tmem_st_wait();
-                            }
-                        }
-                    }
-                }
-                float neg_m;
-                if constexpr (MODE == MODE_GATHERED) neg_m = -row_lse;   // +inf normaliser (row sees nothing): p = 0
-                else neg_m = m > -INFINITY ? -m : 0.f;
+                return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+            };
+            // p = 2^(x - m) for 64 logits: row sum (unless GATHERED) and, with V, the bf16 values packed into w
+            auto emit_chunk = [&](const uint32_t (&v0)[32], const uint32_t (&v1)[32], float neg_m, uint32_t (&w)[kHasV ? 32 : 1]) {
                 const uint64_t nm2 = pack2(neg_m, neg_m);
-                ASTAMP(2);
-
-                // p for the 64 keys, rounded and packed in registers; the shared-memory tile is written once the
-                // tensor cores are done with the previous one
-                uint64_t sum_a = 0, sum_b = 0;  // two packed pairs of partial row sums
-                uint32_t w[kHasV ? 32 : 1];
-                auto emit = [&](const uint32_t (&v)[32], int c) {
+                uint64_t sum_a = 0, sum_b = 0;
+                auto half = [&](const uint32_t (&v)[32], int c) {
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
                         float x0, x1;
@@ -467,28 +410,142 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         }
                     }
                 };
-                emit(v0, 0);
-                emit(v1, 32);
+                half(v0, 0);
+                half(v1, 32);
                 if constexpr (MODE != MODE_GATHERED) {
                     float s0, s1;
                     unpack2(fadd2(sum_a, sum_b), s0, s1);
                     l += s0 + s1;
                 }
+            };
+            auto store_chunk = [&](int chunk, const uint32_t (&w)[kHasV ? 32 : 1]) {
                 if constexpr (kHasV) {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)  // 16-byte units of 8 keys
+                        *reinterpret_cast<uint4 *>(prow + chunk * kPChunk + ((u ^ (r & 7)) << 4)) =
+                            make_uint4(w[4 * u], w[4 * u + 1], w[4 * u + 2], w[4 * u + 3]);
+                }
+            };
+            // m and l follow a new chunk maximum (log2 domain); returns the factor the sums taken so far have to be scaled by
+            auto follow_max = [&](float mc, bool *any_grow) -> float {
+                const bool grow = mc > m + kGrowLimit;
+                *any_grow = __any_sync(0xffffffffu, grow);
+                const float alpha = (grow && m > -INFINITY) ? ex2(m - mc) : 1.f;
+                l *= alpha;
+                if (grow) m = mc;
+                return alpha;
+            };
+
+            for (int j = jb; j < je; ++j, ++s_it) {
+                if constexpr (MODE == MODE_ENERGY) {
+                    // the 128 normalisers of the next tile (512 bytes, the same for every thread) are pulled into L1
+                    // one step ahead; the first tile's are fetched cold
+                    const int64_t nxt = (int64_t)(j + 1) * FN + lane * 32;
+                    if (lane < 4 && j + 1 < je && nxt < a.lse_ld)
+                        asm volatile("prefetch.global.L1 [%0];" ::"l"(a.lse + head * a.lse_ld + nxt));
+                }
+                ASTAMP(7);
+                if (!mbar_wait(s_full(g, 0), s_it & 1u, abort_flag, a.status)) { ok = false; break; }
+                ASTAMP(0);
+                tc_fence_after();
+                uint32_t v0[32], v1[32];
+
+                if constexpr (MODE == MODE_ENERGY) {
+                    // p = bf16(2^(x - lse_i)); this key's score accumulates p^2 over the tile's 128 queries
+                    float acc0 = 0.f, acc1 = 0.f;
+                    for (int c_off = 0; c_off < FN; c_off += 64) {
+                        float4 cl[16];  // the normalisers of these 64 queries (the same for every thread)
+                        const float4 *lp = reinterpret_cast<const float4 *>(a.lse + head * a.lse_ld + (int64_t)j * FN + c_off);
+#pragma unroll
+                        for (int u = 0; u < 16; ++u) cl[u] = (int64_t)j * FN + c_off + 4 * u < a.lse_ld ? __ldg(lp + u) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        load_chunk(j, c_off, v0, v1);
+                        if (c_off == 64) release_s();
+                        auto fold = [&](const uint32_t (&v)[32], int c) {
+#pragma unroll
+                            for (int e = 0; e < 32; e += 4) {
+                                const float4 ls = cl[(c + e) >> 2];
+                                const float p0 = ex2(fmaf(__uint_as_float(v[e]), c2, -ls.x)), p1 = ex2(fmaf(__uint_as_float(v[e + 1]), c2, -ls.y));
+                                const float p2 = ex2(fmaf(__uint_as_float(v[e + 2]), c2, -ls.z)), p3 = ex2(fmaf(__uint_as_float(v[e + 3]), c2, -ls.w));
+                                const float2 ra = __bfloat1622float2(__floats2bfloat162_rn(p0, p1));
+                                const float2 rb = __bfloat1622float2(__floats2bfloat162_rn(p2, p3));
+                                acc0 = fmaf(ra.x, ra.x, acc0);
+                                acc1 = fmaf(ra.y, ra.y, acc1);
+                                acc0 = fmaf(rb.x, rb.x, acc0);
+                                acc1 = fmaf(rb.y, rb.y, acc1);
+                            }
+                        };
+                        fold(v0, 0);
+                        fold(v1, 32);
+                    }
+                    l += acc0 + acc1;
+                    continue;
+                }
+
+                if constexpr (MODE == MODE_STATS) {
+                    // no P and no O: the two chunks are folded one after the other, each against its own maximum
+                    for (int c_off = 0; c_off < FN; c_off += 64) {
+                        load_chunk(j, c_off, v0, v1);
+                        if (c_off == 64) release_s();
+                        bool any_grow;
+                        follow_max(max_chunk(v0, v1) * c2, &any_grow);
+                        uint32_t w[1];
+                        emit_chunk(v0, v1, m > -INFINITY ? -m : 0.f, w);
+                    }
+                    continue;
+                }
+
+                uint32_t w[kHasV ? 32 : 1];
+                if constexpr (MODE == MODE_GATHERED) {
+                    const float neg_m = -row_lse;   // +inf normaliser (row sees nothing): p = 0
+                    load_chunk(j, 0, v0, v1);
+                    emit_chunk(v0, v1, neg_m, w);
+                    if (!mbar_wait(p_empty(g), (p_it & 1u) ^ 1u, abort_flag, a.status)) { ok = false; break; }
+                    store_chunk(0, w);
+                    load_chunk(j, 64, v0, v1);
+                    release_s();
+                    emit_chunk(v0, v1, neg_m, w);
+                    store_chunk(1, w);
+                } else {
+                    // FULL: the maximum of all 128 logits decides about a rescale before any p is taken; the second
+                    // chunk is still in registers then, the first is read from tensor memory once more
+                    load_chunk(j, 0, v0, v1);
+                    const float mx_a = max_chunk(v0, v1);
+                    load_chunk(j, 64, v0, v1);
+                    const float mc = fmaxf(mx_a, max_chunk(v0, v1)) * c2;
+                    bool any_grow;
+                    const float alpha = follow_max(mc, &any_grow);
+                    if (any_grow && j > jb) {  // rows of O already hold sums taken against the old maximum
+                        if (!mbar_wait(p_empty(g), (p_it & 1u) ^ 1u, abort_flag, a.status)) { ok = false; break; }
+                        tc_fence_after();
+                        for (int c = 0; c < nv * 64; c += 16) {
+                            uint32_t o[16];
+                            tmem_ld16_issue(t_o + c, o);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tmem_st16_issue(t_o + c, o);
+                        }
+                        tmem_st_wait();
+                    }
+                    const float neg_m = m > -INFINITY ? -m : 0.f;
+                    ASTAMP(2);
+                    emit_chunk(v0, v1, neg_m, w);
                     ASTAMP(3);
                     // (a repeated wait on a completed phase returns at once: the rescale above may have waited already)
                     if (!mbar_wait(p_empty(g), (p_it & 1u) ^ 1u, abort_flag, a.status)) { ok = false; break; }
                     ASTAMP(4);
-#pragma unroll
-                    for (int u = 0; u < 8; ++u)  // 16-byte units of 8 keys
-                        *reinterpret_cast<uint4 *>(prow + ((u ^ (r & 7)) << 4)) = make_uint4(w[4 * u], w[4 * u + 1], w[4 * u + 2], w[4 * u + 3]);
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the tensor cores
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(p_full(g));
-                    ++p_it;
-                    ASTAMP(5);
+                    store_chunk(1, w);
+                    load_chunk(j, 0, v0, v1);
+                    release_s();
+                    emit_chunk(v0, v1, neg_m, w);
+                    store_chunk(0, w);
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the tensor cores
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p_full(g));
+                ++p_it;
+                ASTAMP(5);
             }
             if (!ok) break;
             if constexpr (MODE == MODE_STATS) {
