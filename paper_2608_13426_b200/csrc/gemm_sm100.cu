@@ -12,8 +12,10 @@
 //   MMA       one elected thread issues tcgen05.mma (bf16 x bf16 -> fp32, M=128, N=BN, K=16 per instruction);
 //             accumulators live in TMEM, double buffered (2 x BN columns) so that the epilogue of one tile
 //             overlaps the main loop of the next.
-//   epilogue  4 warps read TMEM with tcgen05.ld (one accumulator row per thread), scale, round to bf16
-//             (or keep fp32) and store 64 contiguous bytes per thread.
+//   epilogue  4 warps read TMEM with tcgen05.ld (one accumulator row per thread) and scale.  bf16 output: each warp
+//             rounds its 32 x 64 slab into swizzled shared memory and hands it to a TMA tile store (full 128-byte
+//             lines per row, edges clipped by the tensor map; direct 64-byte row pieces reached 1.9 TB/s on an
+//             output-bound product, the tile stores follow the copy rate).  fp32 output: 128 contiguous bytes per thread.
 // Every mbarrier wait is bounded: on expiry the block records RMM_ERR_TIMEOUT in the workspace status
 // word, stops issuing work, lets copies in flight land, frees its TMEM and returns.
 #include <cuda.h>
@@ -60,7 +62,9 @@ struct SmemLayout {
     static constexpr int kBBytes = BN / CTAS * BK * 2;
     static constexpr int kStages = (kABytes + kBBytes) > 32768 ? 4 : 6;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kBarOffset = kStages * kStageBytes;
+    static constexpr int kEpiOffset = kStages * kStageBytes;  // epilogue staging: 4 warps x 2 slabs of 32 rows x 128 bytes
+    static constexpr int kEpiBytes = 4 * 2 * 4096;
+    static constexpr int kBarOffset = kEpiOffset + kEpiBytes;
     static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack to align the base to 1024 B
 };
 
@@ -81,7 +85,8 @@ __device__ __forceinline__ void tile_coords(int64_t t, int tiles_m, int tiles_n,
 
 template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS>
 __global__ void __launch_bounds__(kThreadsTc, 1)
-reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcArgs a)
+reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                       const __grid_constant__ CUtensorMap map_y, TcArgs a)
 {
     using L = SmemLayout<BN, CTAS>;
     constexpr int BNL = BN / CTAS;  // columns of B this CTA loads
@@ -107,6 +112,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     if (threadIdx.x == 32) {  // descriptor fetch overlaps barrier set-up and the TMEM allocation
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+        if constexpr (OUT_BF16) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_y) : "memory");
     }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -225,8 +231,10 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     } else if (warp >= 2) {
         // ---------------------------------------------------------------- epilogue (warps 2..5)
         const int q = warp & 3;  // TMEM lane quarter this warp may read
-        uint32_t tcount = 0;
+        uint32_t tcount = 0, ebuf = 0;
         bool ok = true;
+        uint8_t *slab = base_ptr + L::kEpiOffset + q * 8192 + lane * 128;   // this thread's row of the warp's staging slabs
+        const uint32_t slab_s = base + L::kEpiOffset + q * 8192;
         for (int64_t tile = tile0; tile < num_tiles && ok; tile += tile_step, ++tcount) {
             int tm, tn;
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
@@ -235,15 +243,23 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, a.status)) { ok = false; break; }
             tc_fence_after();
             if (lane == 0) { GSTAMP_MAX(4); }
-            const int64_t m = (int64_t)tm * (BM * CTAS) + rank * BM + q * 32 + lane;
+            const int64_t m_warp = (int64_t)tm * (BM * CTAS) + rank * BM + q * 32, m = m_warp + lane;
             const int64_t n0 = (int64_t)tn * BN;
-            // scale, round and store 32 accumulator columns of this thread's row: 64 (bf16) or 128 (fp32) contiguous bytes
-            auto store_chunk = [&](const uint32_t (&r)[32], int c) {
-                const int64_t n = n0 + c * 32;
-                if (m >= a.M || n >= a.N) return;
-                if constexpr (OUT_BF16) {
-                    __nv_bfloat16 *y = reinterpret_cast<__nv_bfloat16 *>(a.Y) + b * a.y_sb + m * a.y_sr + n;
-                    if (n + 32 <= a.N) {
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
+            if constexpr (OUT_BF16) {
+                // 64 columns at a time: two TMEM loads, scale and round, one 32 x 64 slab per warp through a TMA store
+#pragma unroll 1
+                for (int c = 0; c < BN / 64; ++c) {
+                    const int64_t n = n0 + c * 64;
+                    if (n >= a.N || m_warp >= a.M) break;  // warp-uniform: nothing of this slab lies inside Y
+                    uint32_t r0[32], r1[32];
+                    tmem_ld32_issue(t_row + c * 64, r0);
+                    tmem_ld32_issue(t_row + c * 64 + 32, r1);
+                    tmem_ld_wait();
+                    if (lane == 0) bulk_wait_read<1>();  // the slab written two chunks ago has been read by its store
+                    __syncwarp();
+                    uint8_t *row = slab + ebuf * 4096;
+                    auto put = [&](const uint32_t (&r)[32], int u0) {
 #pragma unroll
                         for (int v = 0; v < 4; ++v) {
                             uint32_t w[4];
@@ -253,12 +269,24 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                                                                          __uint_as_float(r[8 * v + 2 * p + 1]) * a.scale);
                                 w[p] = *reinterpret_cast<uint32_t *>(&h);
                             }
-                            reinterpret_cast<uint4 *>(y)[v] = make_uint4(w[0], w[1], w[2], w[3]);
+                            *reinterpret_cast<uint4 *>(row + (((u0 + v) ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                         }
-                    } else {
-                        for (int e = 0; e < 32 && n + e < a.N; ++e) y[e] = __float2bfloat16_rn(__uint_as_float(r[e]) * a.scale);
+                    };
+                    put(r0, 0);
+                    put(r1, 4);
+                    fence_proxy_async();  // generic writes -> visible to the copy engine
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_3d(&map_y, slab_s + ebuf * 4096, (int)n, (int)m_warp, (int)b);
+                        bulk_commit();
                     }
-                } else {
+                    ebuf ^= 1u;
+                }
+            } else {
+                // 128 contiguous bytes per thread and 32-column chunk
+                auto store_chunk = [&](const uint32_t (&r)[32], int c) {
+                    const int64_t n = n0 + c * 32;
+                    if (m >= a.M || n >= a.N) return;
                     float *y = reinterpret_cast<float *>(a.Y) + b * a.y_sb + m * a.y_sr + n;
                     if (n + 32 <= a.N) {
 #pragma unroll
@@ -269,22 +297,21 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     } else {
                         for (int e = 0; e < 32 && n + e < a.N; ++e) y[e] = __uint_as_float(r[e]) * a.scale;
                     }
-                }
-            };
-            // four TMEM loads in flight per wait: the load latency is paid BN / 128 times per tile instead of BN / 32
-            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
+                };
+                // four TMEM loads in flight per wait: the load latency is paid BN / 128 times per tile instead of BN / 32
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; c += 4) {
-                uint32_t r0[32], r1[32], r2[32], r3[32];
-                tmem_ld32_issue(t_row + (c + 0) * 32, r0);
-                tmem_ld32_issue(t_row + (c + 1) * 32, r1);
-                tmem_ld32_issue(t_row + (c + 2) * 32, r2);
-                tmem_ld32_issue(t_row + (c + 3) * 32, r3);
-                tmem_ld_wait();
-                store_chunk(r0, c + 0);
-                store_chunk(r1, c + 1);
-                store_chunk(r2, c + 2);
-                store_chunk(r3, c + 3);
+                for (int c = 0; c < BN / 32; c += 4) {
+                    uint32_t r0[32], r1[32], r2[32], r3[32];
+                    tmem_ld32_issue(t_row + (c + 0) * 32, r0);
+                    tmem_ld32_issue(t_row + (c + 1) * 32, r1);
+                    tmem_ld32_issue(t_row + (c + 2) * 32, r2);
+                    tmem_ld32_issue(t_row + (c + 3) * 32, r3);
+                    tmem_ld_wait();
+                    store_chunk(r0, c + 0);
+                    store_chunk(r1, c + 1);
+                    store_chunk(r2, c + 2);
+                    store_chunk(r3, c + 3);
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -293,6 +320,10 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 else mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));  // the leader's MMA warp waits on it
             }
             if (lane == 0) { GSTAMP_MAX(5); }
+        }
+        if constexpr (OUT_BF16) {
+            if (lane == 0) bulk_wait_read<0>();  // shared memory stays valid until every store has read its slab
+            __syncwarp();
         }
     }
 
@@ -325,7 +356,7 @@ int sm_count()
 }
 
 template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS>
-int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const TcArgs &a, cudaStream_t stream)
+int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &my, const TcArgs &a, cudaStream_t stream)
 {
     auto kern = reduced_gemm_tc_kernel<BN, B_KMAJOR, OUT_BF16, CTAS>;
     using L = SmemLayout<BN, CTAS>;
@@ -338,7 +369,7 @@ int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const TcArgs &a
     const int64_t slots = sm_count() / CTAS;
     prof_begin("reduced_gemm_tc_kernel", stream);
     cudaError_t e = launch_kernel(kern, dim3((unsigned)((tiles < slots ? tiles : slots) * CTAS)), dim3(kThreadsTc), L::kTotal, stream,
-                                  CTAS, ma, mb, a);
+                                  CTAS, ma, mb, my, a);
     if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "reduced_gemm_tc_kernel: launch: %s", cudaGetErrorString(e));
     return check_launch("reduced_gemm_tc_kernel", stream);
 }
@@ -421,16 +452,25 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     }
     if (rc != RMM_OK) return rc;
     const bool out_bf16 = p.y_bf16 != 0;
+    CUtensorMap my = ma;  // fp32 output is stored without a tensor map
+    if (out_bf16) {
+        // per-warp store slabs: 64 columns x 32 rows; rows and columns past M and N are clipped by the map
+        uint64_t dims[3] = {(uint64_t)p.N, (uint64_t)p.M, (uint64_t)p.batch};
+        uint64_t st[2] = {(uint64_t)p.y_sr * 2, p.batch > 1 ? (uint64_t)p.y_sb * 2 : (uint64_t)p.y_sr * 2 * (uint64_t)p.M};
+        uint32_t box[3] = {64, 32, 1};
+        rc = make_map(&my, p.y, 3, dims, st, box, true);
+        if (rc != RMM_OK) return rc;
+    }
     if (ctas == 2) {
-        if (p.b_kmajor) return out_bf16 ? launch_variant<256, true, true, 2>(ma, mb, a, stream) : launch_variant<256, true, false, 2>(ma, mb, a, stream);
-        return out_bf16 ? launch_variant<256, false, true, 2>(ma, mb, a, stream) : launch_variant<256, false, false, 2>(ma, mb, a, stream);
+        if (p.b_kmajor) return out_bf16 ? launch_variant<256, true, true, 2>(ma, mb, my, a, stream) : launch_variant<256, true, false, 2>(ma, mb, my, a, stream);
+        return out_bf16 ? launch_variant<256, false, true, 2>(ma, mb, my, a, stream) : launch_variant<256, false, false, 2>(ma, mb, my, a, stream);
     }
     if (BN == 256) {
-        if (p.b_kmajor) return out_bf16 ? launch_variant<256, true, true, 1>(ma, mb, a, stream) : launch_variant<256, true, false, 1>(ma, mb, a, stream);
-        return out_bf16 ? launch_variant<256, false, true, 1>(ma, mb, a, stream) : launch_variant<256, false, false, 1>(ma, mb, a, stream);
+        if (p.b_kmajor) return out_bf16 ? launch_variant<256, true, true, 1>(ma, mb, my, a, stream) : launch_variant<256, true, false, 1>(ma, mb, my, a, stream);
+        return out_bf16 ? launch_variant<256, false, true, 1>(ma, mb, my, a, stream) : launch_variant<256, false, false, 1>(ma, mb, my, a, stream);
     }
-    if (p.b_kmajor) return out_bf16 ? launch_variant<128, true, true, 1>(ma, mb, a, stream) : launch_variant<128, true, false, 1>(ma, mb, a, stream);
-    return out_bf16 ? launch_variant<128, false, true, 1>(ma, mb, a, stream) : launch_variant<128, false, false, 1>(ma, mb, a, stream);
+    if (p.b_kmajor) return out_bf16 ? launch_variant<128, true, true, 1>(ma, mb, my, a, stream) : launch_variant<128, true, false, 1>(ma, mb, my, a, stream);
+    return out_bf16 ? launch_variant<128, false, true, 1>(ma, mb, my, a, stream) : launch_variant<128, false, false, 1>(ma, mb, my, a, stream);
 }
 
 int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
