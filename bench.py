@@ -244,7 +244,7 @@ def attention_case(rmm, binding, synth, dev, heads, seq, head_dim=128, reps=10):
     return out
 
 
-def layer_sweep_70b(rmm, synth, dev, peaks, tokens=32768, hidden=8192, inter=28672, reps=3):
+def layer_sweep_70b(rmm, synth, dev, peaks, tokens=32768, hidden=8192, inter=28672, reps=5):
     """Whole reduced product (score + select + gathers + GEMM) per projection shape and rho, dense cuBLAS beside it."""
     shapes = [("q_o_proj", tokens, hidden, hidden), ("k_v_proj", tokens, hidden, 1024),
               ("gate_up_proj", tokens, hidden, inter), ("down_proj", tokens, inter, hidden)]
@@ -265,6 +265,7 @@ def layer_sweep_70b(rmm, synth, dev, peaks, tokens=32768, hidden=8192, inter=286
                 rmm.rmm_reduced_gemm(A, B, idx, out=Y)
 
             op(0)
+            op(1)
             t = time_region(op, reps, 1)
             fl = 2.0 * m * k * n
             out.append({"layer": name, "shape": [m, kk, n], "rho": rho, "whole_op_ms": t, "whole_op_tflops": fl / t / 1e9,
