@@ -505,3 +505,16 @@ def test_attention_batch_folding_and_uneven_batch_stride(oracle):
     Oo, If, _ = oracle.attn(Q, K, V, True, 0.5, 1.0, round_p=True)[:3]
     assert np.array_equal(f1.cpu().numpy(), If)
     assert rel_fro(O1.float().cpu().numpy(), Oo) <= TOL_BF16
+
+
+def test_long_rows_with_an_unsorted_index_list(oracle):
+    """Rows above 36 KB take the streaming column gather; any index list is accepted (here: shuffled, with repeats)."""
+    M, K, N = 300, 20000, 256
+    A = synth.heavy_tailed_activations(M, K, seed=95)
+    B = synth.weight(K, N, seed=96)
+    rng = np.random.default_rng(97)
+    idx = rng.integers(0, K, size=5001).astype(np.int32)
+    Y = rmm.rmm_reduced_gemm(dev(A), dev(B), torch.from_numpy(idx).cuda())
+    want = oracle.reduced_gemm(A, B, idx)
+    assert rel_fro(Y.float().cpu().numpy(), want) <= TOL_BF16
+    assert rmm.rmm_status_read() == 0
