@@ -157,7 +157,7 @@ def test_select_many_equal_keys(oracle, K):
 
 def test_static_and_random_index_controls(oracle):
     """The paper's ablation controls need no extra entry point: a set chosen once (static) or drawn at random with the
-    same budget is simply passed to the reduced product; the retained-energy diagnostic orders them as Theorem 1 says."""
+    same keep count is simply passed to the reduced product; the retained-energy diagnostic orders them as Theorem 1 says."""
     A0, B = synth.mlp_product(512, 1024, 256, seed=21)
     A1 = synth.heavy_tailed_activations(512, 1024, seed=22)          # a later input with other heavy channels
     k = 256
