@@ -519,6 +519,20 @@ def main():
             gbs = idx_d.numel() * Nd * 2 / t / 1e6
             decode.append({"rho": rho, "shape": [1, Kd, Nd], "reduced_gemv_ms": t, "kept_rows_gbs": gbs,
                            "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "dense_cublas_ms": dense, "speedup_vs_dense": dense / t})
+        # small decode batches (2 .. 128 rows): up to 4 rows the gathered GEMV, above it the tensor-core kernel that
+        # fetches the kept rows of W itself (no packed copy of W); rho = 0.5
+        for Mb in (4, 16, 64, 128):
+            xb = synth.heavy_tailed_activations(Mb, Kd, seed=74, device=str(dev))
+            yb = torch.empty(Mb, Nd, dtype=torch.bfloat16, device=dev)
+            idx_b, _, _, _ = rmm.rmm_score_select(xb, rho=0.5)
+            for i in range(3):
+                rmm.rmm_reduced_gemm(xb, Ws[i % 3], idx_b, out=yb)
+                torch.matmul(xb, Ws[i % 3], out=yb)
+            t = time_region(lambda i: rmm.rmm_reduced_gemm(xb, Ws[i % 3], idx_b, out=yb), 30, 1)
+            dn = time_region(lambda i: torch.matmul(xb, Ws[i % 3], out=yb), 30, 1)
+            gbs = idx_b.numel() * Nd * 2 / t / 1e6
+            decode.append({"rho": 0.5, "shape": [Mb, Kd, Nd], "reduced_product_ms": t, "kept_rows_gbs": gbs,
+                           "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "dense_cublas_ms": dn, "speedup_vs_dense": dn / t})
         del Ws
 
     # ---- reduced attention on a 7B-class prefill (32 heads, 4096 tokens, head_dim 128, causal)

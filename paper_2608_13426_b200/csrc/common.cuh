@@ -138,6 +138,10 @@ struct TcProblem {
     const __nv_bfloat16 *b;  // K-major: [b_batches, N, b_ld] (kept columns first); MN-major: [b_batches, k, b_ld], rows = kept slices
     int64_t b_ld, b_sb, b_batches;
     int64_t b_batch_off, b_batch_div;  // B batch entry used by problem i = min((i + off) / div, b_batches - 1)
+    // MN-major B only: when b_idx is set, b is the UNPACKED matrix [b_batches, b_rows, b_ld] and the kernel fetches the
+    // kept rows b_idx[i * b_idx_stride + 0 .. k-1] itself (no packed copy of B; outputs of up to 128 rows)
+    const int32_t *b_idx;
+    int64_t b_idx_stride, b_rows;
     void *y;
     int y_bf16;
     int64_t y_sb, y_sr;

@@ -9,6 +9,12 @@
 //             K-contiguous (K^T in attention) it is packed like A and loaded as K-major tiles.  (Fetching the
 //             kept rows inside the producer with TMA gather4 was measured first: at 512 bytes per instruction
 //             the copy engine sustained about one instruction per 70 clocks, 2.5x slower than this form.)
+//             Outputs of up to 256 rows (small decode batches) skip the packed copy of B: eight gather warps fetch
+//             the kept rows straight from B with 16-byte cp.async into the same swizzled layout (one row of the tile
+//             = one 512-byte warp request).  There every tile of B is used once, the product is bound by reading the
+//             kept rows from HBM, and the copy would triple that traffic.  (For taller outputs the same gather was
+//             measured at 1480 clocks per k-block against 590 for TMA tiles of the packed copy: the load/store path
+//             does not sustain the L2-to-SM rate that re-used tiles need.)
 //   MMA       one elected thread issues tcgen05.mma (bf16 x bf16 -> fp32, M=128, N=BN, K=16 per instruction);
 //             accumulators live in TMEM, double buffered (2 x BN columns) so that the epilogue of one tile
 //             overlaps the main loop of the next.
@@ -33,6 +39,7 @@ constexpr int BM = 128;
 constexpr int BK = 64;           // contraction indices per pipeline stage (128 bytes of bf16)
 constexpr int UMMA_K = 16;
 constexpr int kThreadsTc = 192;  // warp 0 producer, warp 1 MMA + TMEM owner, warps 2-5 epilogue
+constexpr int kGatherWarps = 8;  // B_GATHER: warps 6-13 fetch the kept rows of B
 
 #ifdef RMM_GEMM_STAMPS
 __device__ unsigned long long g_gstamps[16];
@@ -51,6 +58,10 @@ struct TcArgs {
     float scale;
     int tiles_m, tiles_n;
     int *status;
+    // B_GATHER: the unpacked B and the kept row numbers
+    const __nv_bfloat16 *b_src;
+    const int32_t *b_idx;
+    int64_t b_ld, b_sb, b_idx_stride, b_rows;
 };
 
 // BN = tile columns (MMA N, accumulator columns); CTAS = CTAs per tile.  With CTAS == 2 a pair of CTAs on one TPC
@@ -83,8 +94,8 @@ __device__ __forceinline__ void tile_coords(int64_t t, int tiles_m, int tiles_n,
     tm = (int)(r / width);
 }
 
-template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS>
-__global__ void __launch_bounds__(kThreadsTc, 1)
+template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS, bool B_GATHER>
+__global__ void __launch_bounds__(kThreadsTc + (B_GATHER ? 32 * kGatherWarps : 0), 1)
 reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                        const __grid_constant__ CUtensorMap map_y, TcArgs a)
 {
@@ -116,7 +127,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_bar(s), 1);
+            mbar_init(full_bar(s), B_GATHER ? 1 + 32 * kGatherWarps : 1);
             mbar_init(empty_bar(s), 1);
         }
         for (int i = 0; i < 2; ++i) {
@@ -152,7 +163,10 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     const uint32_t sa = base + s * L::kStageBytes;
                     const uint32_t sb = sa + L::kABytes;
                     const int row_a = tm * (BM * CTAS) + (int)rank * BM, col_b = tn * BN + (int)rank * BNL;
-                    if constexpr (CTAS == 1) {
+                    if constexpr (B_GATHER) {
+                        mbar_arrive_expect_tx(full_bar(s), L::kABytes);
+                        tma_load_3d(sa, &map_a, kb * BK, row_a, (int)b, full_bar(s));
+                    } else if constexpr (CTAS == 1) {
                         mbar_arrive_expect_tx(full_bar(s), L::kStageBytes);
                         tma_load_3d(sa, &map_a, kb * BK, row_a, (int)b, full_bar(s));
                         if constexpr (B_KMAJOR) {
@@ -206,6 +220,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             uint32_t accumulate = 0;
             for (int kb = 0; kb < num_kb; ++kb) {
                 if (!mbar_wait_lane(full_bar(stage), phase, abort_flag, a.status)) { ok = false; break; }
+                if constexpr (B_GATHER) fence_proxy_async();  // B arrived through the generic proxy (cp.async)
                 tc_fence_after();
                 if (kb == 0 && tcount == 0) { GSTAMP_MAX(2); }
                 const uint32_t a_lo = a_lo0 + stage * kStageUnits, b_lo = b_lo0 + stage * kStageUnits;
@@ -228,7 +243,62 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             GSTAMP_MAX(3);
         }
         __syncwarp();
-    } else if (warp >= 2) {
+    } else if (B_GATHER && warp >= 6) {
+        // ---------------------------------------------------------------- gather warps: kept rows of B -> MN-major tile
+        // Row r of the k-block is one warp request: lane l copies 16 bytes (8 columns) to chunk l / 8, row r, 16-byte
+        // unit (l % 8) ^ (r % 8) -- the layout a 128-byte-swizzled TMA tile load would have produced.  The thread does
+        // not wait for its copies: the stage's barrier receives this thread's arrival when they have landed, so every
+        // free stage has copies in flight.  The MMA thread orders the landed data before the tensor cores'
+        // (asynchronous-proxy) reads with a proxy fence.  Row numbers are fetched one k-block ahead.
+        static_assert(!B_GATHER || (!B_KMAJOR && CTAS == 1 && BN == 256), "gather form: single-CTA 128 x 256 tiles, row-contiguous B");
+        constexpr int kRowsPerWarp = BK / kGatherWarps;
+        const int gw = warp - 6;
+        uint32_t s = 0, ph = 0;
+        bool ok = true;
+        for (int64_t tile = tile0; tile < num_tiles && ok; tile += tile_step) {
+            int tm, tn;
+            const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
+            tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, tm, tn);
+            int64_t bb = (b + a.b_batch_off) / a.b_batch_div;
+            if (bb >= a.b_batches) bb = a.b_batches - 1;
+            const int32_t *ix = a.b_idx + b * a.b_idx_stride;
+            const int64_t col = (int64_t)tn * BN + lane * 8;
+            const __nv_bfloat16 *bcol = a.b_src + bb * a.b_sb + (col < a.N ? col : 0);
+            const uint32_t col_bytes = col < a.N ? 16u : 0u;
+            const uint32_t lane_off = (uint32_t)(lane >> 3) * (BK * 128);
+            int rows[kRowsPerWarp], rows_next[kRowsPerWarp];
+            auto fetch_rows = [&](int kb, int (&out)[kRowsPerWarp]) {
+#pragma unroll
+                for (int i = 0; i < kRowsPerWarp; ++i) {
+                    const int64_t kk = (int64_t)kb * BK + gw + kGatherWarps * i;
+                    out[i] = kk < a.k ? __ldg(ix + kk) : -1;
+                }
+            };
+            fetch_rows(0, rows_next);
+            for (int kb = 0; kb < num_kb; ++kb) {
+#pragma unroll
+                for (int i = 0; i < kRowsPerWarp; ++i) rows[i] = rows_next[i];
+                if (kb + 1 < num_kb) fetch_rows(kb + 1, rows_next);
+                if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status)) { ok = false; break; }
+                const uint32_t sb = base + s * L::kStageBytes + L::kABytes + lane_off;
+#pragma unroll
+                for (int i = 0; i < kRowsPerWarp; ++i) {
+                    const int r = gw + kGatherWarps * i;
+                    int row = rows[i];
+                    if (row >= a.b_rows || (row < 0 && (int64_t)kb * BK + r < a.k)) {
+                        atomicExch(a.status, (int)RMM_ERR_BOUNDS);
+                        row = -1;
+                    }
+                    const uint32_t dst = sb + r * 128 + (((uint32_t)(lane & 7) ^ (uint32_t)(r & 7)) << 4);
+                    cp_async_16(dst, row >= 0 ? bcol + (int64_t)row * a.b_ld : bcol, row >= 0 ? col_bytes : 0u);
+                }
+                cp_async_arrive_noinc(full_bar(s));
+                if (++s == kStages) { s = 0; ph ^= 1u; }
+            }
+        }
+        cp_async_commit();
+        cp_async_wait<0>();  // nothing of this thread is in flight when the block tears down
+    } else if (warp >= 2 && warp < 6) {
         // ---------------------------------------------------------------- epilogue (warps 2..5)
         const int q = warp & 3;  // TMEM lane quarter this warp may read
         uint32_t tcount = 0, ebuf = 0;
@@ -355,10 +425,10 @@ int sm_count()
     return n;
 }
 
-template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS>
+template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS, bool B_GATHER = false>
 int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &my, const TcArgs &a, cudaStream_t stream)
 {
-    auto kern = reduced_gemm_tc_kernel<BN, B_KMAJOR, OUT_BF16, CTAS>;
+    auto kern = reduced_gemm_tc_kernel<BN, B_KMAJOR, OUT_BF16, CTAS, B_GATHER>;
     using L = SmemLayout<BN, CTAS>;
     static PerDeviceOnce configured;
     if (configured.first()) {
@@ -368,7 +438,8 @@ int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorM
     const int64_t tiles = a.batch * a.tiles_m * a.tiles_n;
     const int64_t slots = sm_count() / CTAS;
     prof_begin("reduced_gemm_tc_kernel", stream);
-    cudaError_t e = launch_kernel(kern, dim3((unsigned)((tiles < slots ? tiles : slots) * CTAS)), dim3(kThreadsTc), L::kTotal, stream,
+    cudaError_t e = launch_kernel(kern, dim3((unsigned)((tiles < slots ? tiles : slots) * CTAS)),
+                                  dim3(kThreadsTc + (B_GATHER ? 32 * kGatherWarps : 0)), L::kTotal, stream,
                                   CTAS, ma, mb, my, a);
     if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "reduced_gemm_tc_kernel: launch: %s", cudaGetErrorString(e));
     return check_launch("reduced_gemm_tc_kernel", stream);
@@ -430,6 +501,7 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     int ctas = (BN == 256 && p.M > BM && pair_tiles >= sm_count() / 2) ? 2 : 1;
     if (forced == 1) ctas = 1;
     if (forced == 2 && BN == 256 && p.M > BM) ctas = 2;
+    if (p.b_idx != nullptr) ctas = 1;  // the in-kernel row gather exists for single-CTA tiles
     TcArgs a;
     a.M = p.M; a.N = p.N; a.k = p.k; a.batch = p.batch;
     a.b_batch_off = p.b_batch_off; a.b_batch_div = p.b_batch_div > 0 ? p.b_batch_div : 1; a.b_batches = p.b_batches;
@@ -438,6 +510,22 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     a.tiles_m = (int)ceil_div(p.M, BM * ctas);
     a.tiles_n = (int)ceil_div(p.N, BN);
     a.status = p.status;
+    a.b_src = p.b; a.b_idx = p.b_idx; a.b_ld = p.b_ld; a.b_sb = p.b_batches > 1 ? p.b_sb : 0; a.b_idx_stride = p.b_idx_stride;
+    a.b_rows = p.b_rows;
+    if (p.b_idx != nullptr) {
+        if (p.b_kmajor || ctas != 1 || BN != 256)
+            return fail(RMM_ERR_UNSUPPORTED, "reduced_gemm_tc: in-kernel row gather needs single-CTA 128 x 256 tiles and row-contiguous B");
+        CUtensorMap my_g = ma;  // (the tensor map of B is unused in this form; A's stands in)
+        if (p.y_bf16) {
+            uint64_t dims[3] = {(uint64_t)p.N, (uint64_t)p.M, (uint64_t)p.batch};
+            uint64_t st[2] = {(uint64_t)p.y_sr * 2, p.batch > 1 ? (uint64_t)p.y_sb * 2 : (uint64_t)p.y_sr * 2 * (uint64_t)p.M};
+            uint32_t box[3] = {64, 32, 1};
+            rc = make_map(&my_g, p.y, 3, dims, st, box, true);
+            if (rc != RMM_OK) return rc;
+            return launch_variant<256, false, true, 1, true>(ma, ma, my_g, a, stream);
+        }
+        return launch_variant<256, false, false, 1, true>(ma, ma, my_g, a, stream);
+    }
     const uint64_t b_sb = p.b_batches > 1 ? (uint64_t)p.b_sb * 2 : (uint64_t)p.b_ld * 2 * (uint64_t)(p.b_kmajor ? p.N : p.k);
     if (p.b_kmajor) {
         uint64_t dims[3] = {(uint64_t)p.k, (uint64_t)p.N, (uint64_t)p.b_batches};
@@ -503,6 +591,17 @@ int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, i
     PackSpec specs[2];
     specs[0] = pack_cols_spec(a_src, batch, M, K, A->stride_batch, A->stride_row, 0, 1, idx, k, k, Ap, plan.ldp);
     p.a = Ap; p.a_ld = plan.ldp; p.a_sb = M * plan.ldp;
+    if (!plan.b_kmajor && M <= 2 * BM && N > 128) {
+        // one or two tile rows: a tile of B is used once or twice (the second time from L2), so the kernel fetches the
+        // kept rows itself and only A[:, I] is packed
+        p.b = b_src; p.b_ld = B->stride_row; p.b_rows = K;
+        if (B->stride_batch == 0) { p.b_batches = 1; p.b_sb = 0; }
+        else { p.b_sb = B->stride_batch; }
+        p.b_idx = idx; p.b_idx_stride = k;
+        rc = launch_pack(specs, 1, status, stream);
+        if (rc != RMM_OK) return rc;
+        return launch_gemm_tc_problem(p, stream);
+    }
     if (plan.b_kmajor) {
         // B is K-contiguous ([N, K] in memory): B[idx, :]^T goes to Bp [batch, N, ldp]; a shared B (stride_batch 0)
         // is packed once per index set

@@ -175,6 +175,21 @@ __device__ __forceinline__ void cluster_sync_all()
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// 16-byte asynchronous copy global -> shared (generic proxy); `bytes` < 16 zero-fills the rest (0: all zeros, nothing read).
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// The mbarrier receives one arrival (already counted at initialisation: .noinc) once every cp.async issued so far by
+// this thread has landed; the thread itself does not wait.
+__device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
 // TMEM allocation: with CTAS == 2 one warp of EACH CTA of the pair executes it, and the pair gets the same columns.
 template <int CTAS>
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols)

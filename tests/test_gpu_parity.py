@@ -518,3 +518,24 @@ def test_long_rows_with_an_unsorted_index_list(oracle):
     want = oracle.reduced_gemm(A, B, idx)
     assert rel_fro(Y.float().cpu().numpy(), want) <= TOL_BF16
     assert rmm.rmm_status_read() == 0
+
+
+@pytest.mark.parametrize("M,K,N,rho", [(5, 4096, 2048, 0.5), (17, 1000, 520, 0.3), (100, 2048, 1024, 0.25), (128, 512, 264, 0.75),
+                                       (129, 1024, 512, 0.5), (256, 1536, 2048, 0.5)])
+def test_small_batch_product_fetches_rows_of_b_in_the_kernel(oracle, M, K, N, rho):
+    """Up to 256 output rows (and N > 128) the tensor-core kernel gathers the kept rows of B itself; ragged k-blocks,
+    ragged column tiles and a second tile row are covered."""
+    A = synth.heavy_tailed_activations(M, K, seed=M)
+    B = synth.weight(K, N, seed=M + 1)
+    Y, idx = rmm.rmm(dev(A), dev(B), rho)
+    idx_np = idx.cpu().numpy()
+    e64, _ = oracle.score(A)
+    check_index_set(idx_np, e64, oracle.keep_count(rho, K))
+    assert rel_fro(Y.float().cpu().numpy(), oracle.reduced_gemm(A, B, idx_np)) <= TOL_BF16
+    # a bad index is reported through the status word, not dereferenced
+    bad = idx.clone()
+    bad[0] = K + 5
+    rmm.rmm_reduced_gemm(dev(A), dev(B), bad)
+    torch.cuda.synchronize()
+    assert rmm.rmm_status_read() == 6          # RMM_ERR_BOUNDS, cleared by the read
+    assert rmm.rmm_status_read() == 0
