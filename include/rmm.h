@@ -114,7 +114,9 @@ int rmm_score_select_static(const rmm_mat_t *A, int axis, double rho, int64_t k,
  *   pointers / leading strides are 16-byte aligned; Y may be bf16 or fp32.  Every other layout, and
  *   fp32 operands, run on a plain FMA kernel (fp32 accumulation).  A and B must share a dtype.
  *   Decode-step shapes (batch 1, M <= 4, bf16, B with contiguous rows; App. "Complexity Analysis", decoding step)
- *   take a gathered GEMV that reads only the kept rows of B (k N 2 bytes) and packs nothing. */
+ *   take a gathered GEMV that reads only the kept rows of B (k N 2 bytes) and packs nothing; outputs of up to 256
+ *   rows (small decode batches, B with contiguous rows, N > 128) run on the tensor cores with the kept rows of B
+ *   fetched by the kernel itself, so W is read once and never copied. */
 size_t rmm_reduced_gemm_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y);
 int rmm_reduced_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
                      const rmm_mat_t *Y, void *ws, size_t ws_bytes, void *stream);
@@ -128,7 +130,11 @@ int rmm_reduced_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx,
  *   rho_t == 1: O = P V
  * Q [B,Hq,Lq,Dh], K,V [B,Hkv,Lk,Dh], O [B,Hq,Lq,Dh] are bf16 with explicit element strides
  * (batch, head, row, 1).  idx_feat int32 [B,Hq,kd] and idx_tok int32 [B,Hq,kt] receive the index sets
- * (either may be NULL).  S~ and P are materialised in the workspace one group of heads at a time. */
+ * (either may be NULL).  With head_dim and kept features up to 128, S~ and P stay on the SM (fused kernel: one pass
+ * for rho_t == 1; row normalisers, token scores and a gathered P V pass for rho_t < 1, where the normalised P is
+ * what is rounded, scored and multiplied; for rho_t == 1 the bf16 rounding is applied to P times a per-row factor,
+ * which changes O by rounding noise only).  Wider heads materialise S~ and P in the workspace one group of heads at a
+ * time.  An evenly strided batch is processed as B * Hq heads in one pass of launches. */
 typedef struct {
     int64_t B, Hq, Hkv, Lq, Lk, Dh;
     int32_t causal;
