@@ -39,6 +39,7 @@ constexpr int BM = 128;
 constexpr int BK = 64;           // contraction indices per pipeline stage (128 bytes of bf16)
 constexpr int UMMA_K = 16;
 constexpr int kThreadsTc = 192;  // warp 0 producer, warp 1 MMA + TMEM owner, warps 2-5 epilogue
+constexpr int kThreadsTc2 = 320; // ... and warps 6-9 a second epilogue set, for products with a handful of k-blocks
 constexpr int kGatherWarps = 8;  // B_GATHER: warps 6-13 fetch the kept rows of B
 
 #ifdef RMM_GEMM_STAMPS
@@ -57,6 +58,7 @@ struct TcArgs {
     int64_t y_sb, y_sr;     // element strides of Y (column stride 1)
     float scale;
     int tiles_m, tiles_n;
+    int epi_sets;           // 1, or 2: a second set of four epilogue warps takes every other 64-column chunk
     int *status;
     // B_GATHER: the unpacked B and the kept row numbers
     const __nv_bfloat16 *b_src;
@@ -95,7 +97,7 @@ __device__ __forceinline__ void tile_coords(int64_t t, int tiles_m, int tiles_n,
 }
 
 template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS, bool B_GATHER>
-__global__ void __launch_bounds__(kThreadsTc + (B_GATHER ? 32 * kGatherWarps : 0), 1)
+__global__ void __launch_bounds__(B_GATHER ? kThreadsTc + 32 * kGatherWarps : kThreadsTc2, 1)
 reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                        const __grid_constant__ CUtensorMap map_y, TcArgs a)
 {
@@ -132,7 +134,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(tfull_bar(i), 1);
-            mbar_init(tempty_bar(i), 4 * CTAS);
+            mbar_init(tempty_bar(i), 4 * CTAS * a.epi_sets);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -298,13 +300,18 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         }
         cp_async_commit();
         cp_async_wait<0>();  // nothing of this thread is in flight when the block tears down
-    } else if (warp >= 2 && warp < 6) {
-        // ---------------------------------------------------------------- epilogue (warps 2..5)
+    } else if (warp >= 2 && warp < 2 + 4 * a.epi_sets) {
+        // ---------------------------------------------------------------- epilogue (warps 2..5, and 6..9 as a second set)
+        // With two sets, set s takes the 64-column chunks c with c % 2 == s and every warp has one staging slab
+        // instead of two: products with very few k-blocks are bound by this code, and one epilogue warp per scheduler
+        // issues too few instructions per clock to keep up with the stores.
         const int q = warp & 3;  // TMEM lane quarter this warp may read
+        const int eset = (warp - 2) >> 2, slabs = a.epi_sets == 2 ? 1 : 2;
         uint32_t tcount = 0, ebuf = 0;
         bool ok = true;
-        uint8_t *slab = base_ptr + L::kEpiOffset + q * 8192 + lane * 128;   // this thread's row of the warp's staging slabs
-        const uint32_t slab_s = base + L::kEpiOffset + q * 8192;
+        const int slab_id = a.epi_sets == 2 ? eset * 4 + q : q * 2;        // 4 KB slabs; a single set has two per warp
+        uint8_t *slab = base_ptr + L::kEpiOffset + slab_id * 4096 + lane * 128;   // this thread's row of the warp's staging slabs
+        const uint32_t slab_s = base + L::kEpiOffset + slab_id * 4096;
         for (int64_t tile = tile0; tile < num_tiles && ok; tile += tile_step, ++tcount) {
             int tm, tn;
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
@@ -319,14 +326,17 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             if constexpr (OUT_BF16) {
                 // 64 columns at a time: two TMEM loads, scale and round, one 32 x 64 slab per warp through a TMA store
 #pragma unroll 1
-                for (int c = 0; c < BN / 64; ++c) {
+                for (int c = eset; c < BN / 64; c += a.epi_sets) {
                     const int64_t n = n0 + c * 64;
                     if (n >= a.N || m_warp >= a.M) break;  // warp-uniform: nothing of this slab lies inside Y
                     uint32_t r0[32], r1[32];
                     tmem_ld32_issue(t_row + c * 64, r0);
                     tmem_ld32_issue(t_row + c * 64 + 32, r1);
                     tmem_ld_wait();
-                    if (lane == 0) bulk_wait_read<1>();  // the slab written two chunks ago has been read by its store
+                    if (lane == 0) {  // the slab about to be rewritten has been read by its store
+                        if (slabs == 2) bulk_wait_read<1>();
+                        else bulk_wait_read<0>();
+                    }
                     __syncwarp();
                     uint8_t *row = slab + ebuf * 4096;
                     auto put = [&](const uint32_t (&r)[32], int u0) {
@@ -350,9 +360,9 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                         tma_store_3d(&map_y, slab_s + ebuf * 4096, (int)n, (int)m_warp, (int)b);
                         bulk_commit();
                     }
-                    ebuf ^= 1u;
+                    if (slabs == 2) ebuf ^= 1u;
                 }
-            } else {
+            } else if (eset == 0) {
                 // 128 contiguous bytes per thread and 32-column chunk
                 auto store_chunk = [&](const uint32_t (&r)[32], int c) {
                     const int64_t n = n0 + c * 32;
@@ -439,7 +449,7 @@ int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorM
     const int64_t slots = sm_count() / CTAS;
     prof_begin("reduced_gemm_tc_kernel", stream);
     cudaError_t e = launch_kernel(kern, dim3((unsigned)((tiles < slots ? tiles : slots) * CTAS)),
-                                  dim3(kThreadsTc + (B_GATHER ? 32 * kGatherWarps : 0)), L::kTotal, stream,
+                                  dim3(B_GATHER ? kThreadsTc + 32 * kGatherWarps : (a.epi_sets == 2 ? kThreadsTc2 : kThreadsTc)), L::kTotal, stream,
                                   CTAS, ma, mb, my, a);
     if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "reduced_gemm_tc_kernel: launch: %s", cudaGetErrorString(e));
     return check_launch("reduced_gemm_tc_kernel", stream);
@@ -510,6 +520,8 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     a.tiles_m = (int)ceil_div(p.M, BM * ctas);
     a.tiles_n = (int)ceil_div(p.N, BN);
     a.status = p.status;
+    // products with at most four k-blocks per tile are bound by the epilogue: two sets of epilogue warps
+    a.epi_sets = (p.y_bf16 && p.b_idx == nullptr && ceil_div(p.k, BK) <= 4) ? 2 : 1;
     a.b_src = p.b; a.b_idx = p.b_idx; a.b_ld = p.b_ld; a.b_sb = p.b_batches > 1 ? p.b_sb : 0; a.b_idx_stride = p.b_idx_stride;
     a.b_rows = p.b_rows;
     if (p.b_idx != nullptr) {
