@@ -246,7 +246,9 @@ def attention_case(rmm, binding, synth, dev, heads, seq, head_dim=128, reps=10):
 
 def layer_sweep_70b(rmm, synth, dev, peaks, tokens=32768, hidden=8192, inter=28672, reps=5):
     """Whole reduced product (score + select + gathers + GEMM) per projection shape and rho, dense cuBLAS beside it."""
-    shapes = [("q_o_proj", tokens, hidden, hidden), ("k_v_proj", tokens, hidden, 1024),
+    # (Q, K and V read the same activations, hence the same index set: fused into one product they share the selection
+    # and the gather of A, which the narrow K/V projection alone cannot repay)
+    shapes = [("q_o_proj", tokens, hidden, hidden), ("k_v_proj", tokens, hidden, 1024), ("qkv_fused_proj", tokens, hidden, hidden + 2048),
               ("gate_up_proj", tokens, hidden, inter), ("down_proj", tokens, inter, hidden)]
     out = []
     for name, m, kk, n in shapes:
