@@ -8,9 +8,11 @@
 // shared memory, row splits through an fp64 partial array combined in split order by the last
 // block to arrive (self-resetting atomicInc counter).  Results are therefore run-to-run identical.
 //
-// Select: radix select on the order-preserving integer image of the fp32 keys (4 passes of 8 bits,
-// warp-aggregated shared-memory histograms), then one ordered compaction pass that emits the kept
-// indices ascending; among keys equal to the threshold the lowest indices are kept.
+// Select: radix select on the order-preserving integer image of the fp32 keys (the bits common to all
+// keys are skipped, one digit of up to 11 bits over all keys, then 8-bit digits over the keys that share
+// the threshold's digit), then one ordered compaction pass that emits the kept indices ascending; among
+// keys equal to the threshold the lowest indices are kept.  bf16 matrices that meet the TMA rules are
+// streamed by score_tma_kernel (64-column blocks, 256-row tiles through a ring of shared-memory buffers).
 #include <cuda.h>
 
 #include "common.cuh"
