@@ -1,7 +1,7 @@
 // Reduced attention (paper Sec. 3.3) composed from the library's own kernels, one group of query heads
 // at a time:
-//   score + select on Q          -> I per query head              (score_select_kernel)
-//   pack Q[:, I], K_g[:, I]      -> K-major operands              (pack_cols_kernel)
+//   score + select on Q          -> I per query head              (score_tma_kernel / score_select_kernel)
+//   pack Q[:, I], K_g[:, I]      -> K-major operands              (pack_kernel)
 //   S~ = Q[:, I] K[:, I]^T / sqrt(Dh), fp32                        (reduced_gemm_tc_kernel, K-major B)
 //   P  = bf16(softmax(S~ + causal mask))                            (softmax_rows_kernel)
 //   rho_t < 1: score + select on P -> T; pack P[:, T] and V_g[T, :]; O = P[:, T] V_g[T, :]
