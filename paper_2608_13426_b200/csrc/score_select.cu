@@ -840,9 +840,9 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
             cudaError_t e = cudaFuncSetAttribute(score_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTmaStages * kTmaStageBytes);
             if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "score: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         }
-        prof_begin("score_select_kernel", stream);
+        prof_begin("score_tma_kernel", stream);
         launch_kernel(score_tma_kernel, grid, dim3(kThreads), kTmaStages * kTmaStageBytes, stream, 1, map, a, &hdr->status);
-        int rc2 = check_launch("score_select_kernel", stream);
+        int rc2 = check_launch("score_tma_kernel", stream);
         if (rc2 != RMM_OK || !do_select || fused) return rc2;
         return launch_select(a.energy, A->batch, p.n, k, idx, retained, ws, stream);
     }
