@@ -230,11 +230,12 @@ __device__ void block_select(const float *__restrict__ keys, int K, int k, int32
         const unsigned g = __ballot_sync(0xffffffffu, gt), e = __ballot_sync(0xffffffffu, eq);
         const unsigned gt_before = gt_base + __popc(g & lt), eq_before = eq_base + __popc(e & lt);
         if (in) {
-            const double f = (double)key_value(u);
-            sum_all += f;
-            if (gt || (eq && eq_before < need_eq)) {
-                idx[gt_before + (eq_before < need_eq ? eq_before : need_eq)] = j;
-                sum_kept += f;
+            const bool keep = gt || (eq && eq_before < need_eq);
+            if (keep) idx[gt_before + (eq_before < need_eq ? eq_before : need_eq)] = j;
+            if (retained != nullptr) {  // the energy sums (fp64 conversions and adds) only when they are asked for
+                const double f = (double)key_value(u);
+                sum_all += f;
+                if (keep) sum_kept += f;
             }
         }
         gt_base += __popc(g);
@@ -396,11 +397,12 @@ __device__ void block_select_reg(const float *__restrict__ keys, int K, int k, i
         const unsigned g = __ballot_sync(0xffffffffu, gt), e = __ballot_sync(0xffffffffu, eq);
         const unsigned gt_before = (base >> 16) + __popc(g & lt), eq_before = (base & 0xffffu) + __popc(e & lt);
         if (in) {
-            const double f = (double)key_value(u[i]);
-            sum_all += f;
-            if (gt || (eq && eq_before < need_eq)) {
-                idx[gt_before + (eq_before < need_eq ? eq_before : need_eq)] = j;
-                sum_kept += f;
+            const bool keep = gt || (eq && eq_before < need_eq);
+            if (keep) idx[gt_before + (eq_before < need_eq ? eq_before : need_eq)] = j;
+            if (retained != nullptr) {  // the energy sums (fp64 conversions and adds) only when they are asked for
+                const double f = (double)key_value(u[i]);
+                sum_all += f;
+                if (keep) sum_kept += f;
             }
         }
     }
