@@ -59,6 +59,9 @@ def _load():
     L.orc_attn.restype = None
     L.orc_attn.argtypes = [vp, vp, vp, i32, i64, i64, i64, i64, i64, i64, vp, vp, vp,
                            i32, dbl, dbl, i32, vp, vp, vp, vp]
+    L.orc_attn_sets.restype = i32
+    L.orc_attn_sets.argtypes = [vp, vp, vp, i32, i64, i64, i64, i64, i64, i64, vp, vp, vp,
+                                i32, dbl, dbl, i32, vp, vp, vp, i64, vp, vp, vp, vp]
     _lib = L
     return L
 
@@ -170,10 +173,16 @@ def rmm(A, B, rho: float):
     return reduced_gemm(A, B, idx), idx, e
 
 
-def attn(Q, K, V, causal: bool, rho_d: float, rho_t: float, round_p: bool = True, want_p: bool = False):
+def attn(Q, K, V, causal: bool, rho_d: float, rho_t: float, round_p: bool = True, want_p: bool = False,
+         idx_feat=None, idx_tok=None, rows=None):
     """Reduced attention of Sec. 3.3.  Q [B,Hq,Lq,Dh]; K, V [B,Hkv,Lk,Dh] (same dtype).
 
-    Returns (O [B,Hq,Lq,Dh] fp64, idx_feat [B,Hq,kd], idx_tok [B,Hq,kt] or None, P or None).
+    idx_feat [B,Hq,kd] / idx_tok [B,Hq,kt] (int32), if given, replace the TopK choice of the feature / token set
+    (the formulas for S~ and O~ hold for any set); rows (a list of query rows), if given, restricts the evaluation
+    to those rows (with rho_t < 1 the token set must then be given, because token scores need every row).
+
+    Returns (O [B,Hq,Lq or len(rows),Dh] fp64, idx_feat [B,Hq,kd], idx_tok [B,Hq,kt] or None, P or None):
+    the sets are the ones that were used.
     """
     Q, K, V = as_np(Q), as_np(K), as_np(V)
     assert Q.ndim == 4 and K.ndim == 4 and V.ndim == 4 and Q.dtype == K.dtype == V.dtype
@@ -182,14 +191,29 @@ def attn(Q, K, V, causal: bool, rho_d: float, rho_t: float, round_p: bool = True
     assert Hq % Hkv == 0
     kd = keep_count(rho_d, Dh)
     kt = keep_count(rho_t, Lk)
-    O = np.zeros((B, Hq, Lq, Dh), np.float64)
-    idx_feat = np.zeros((B, Hq, kd), np.int32)
-    idx_tok = np.zeros((B, Hq, kt), np.int32) if rho_t < 1.0 else None
-    P = np.zeros((B, Hq, Lq, Lk), np.float64) if want_p else None
+    assert kd >= 1 and kt >= 1
+    feat_in = tok_in = rows_in = None
+    if idx_feat is not None:
+        feat_in = np.ascontiguousarray(as_np(idx_feat), dtype=np.int32)
+        assert feat_in.shape == (B, Hq, kd) and feat_in.min() >= 0 and feat_in.max() < Dh
+    if idx_tok is not None and rho_t < 1.0:
+        tok_in = np.ascontiguousarray(as_np(idx_tok), dtype=np.int32)
+        assert tok_in.shape == (B, Hq, kt) and tok_in.min() >= 0 and tok_in.max() < Lk
+    nq = Lq
+    if rows is not None:
+        rows_in = np.ascontiguousarray(np.asarray(rows), dtype=np.int64)
+        assert rows_in.ndim == 1 and rows_in.size >= 1 and rows_in.min() >= 0 and rows_in.max() < Lq
+        assert rho_t >= 1.0 or tok_in is not None, "token scores need every query row"
+        nq = rows_in.size
+    O = np.zeros((B, Hq, nq, Dh), np.float64)
+    out_feat = np.zeros((B, Hq, kd), np.int32)
+    out_tok = np.zeros((B, Hq, kt), np.int32) if rho_t < 1.0 else None
+    P = np.zeros((B, Hq, nq, Lk), np.float64) if want_p else None
     s3 = [(ctypes.c_int64 * 4)(*_estr(x)) for x in (Q, K, V)]
-    _load().orc_attn(Q.ctypes.data, K.ctypes.data, V.ctypes.data, _dt(Q), B, Hq, Hkv, Lq, Lk, Dh,
-                     s3[0], s3[1], s3[2], int(bool(causal)), float(rho_d), float(rho_t),
-                     int(bool(round_p)), O.ctypes.data, idx_feat.ctypes.data,
-                     idx_tok.ctypes.data if idx_tok is not None else None,
-                     P.ctypes.data if P is not None else None)
-    return O, idx_feat, idx_tok, P
+    ptr = lambda a: a.ctypes.data if a is not None else None
+    rc = _load().orc_attn_sets(Q.ctypes.data, K.ctypes.data, V.ctypes.data, _dt(Q), B, Hq, Hkv, Lq, Lk, Dh,
+                               s3[0], s3[1], s3[2], int(bool(causal)), float(rho_d), float(rho_t),
+                               int(bool(round_p)), ptr(feat_in), ptr(tok_in), ptr(rows_in), nq,
+                               O.ctypes.data, out_feat.ctypes.data, ptr(out_tok), ptr(P))
+    assert rc == 0
+    return O, out_feat, out_tok, P

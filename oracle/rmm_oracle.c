@@ -16,6 +16,8 @@
  *   orc_attn           Sec. 3.3 "Attention": feature scores on Q, S~ = Q[:,I] K[:,I]^T / sqrt(d_h),
  *                      P = softmax(S~ + M), token scores a_t = ||P[:, t]||_2,
  *                      O~ = P[:, T] V[T, :]; grouped-query rule of the same paragraph
+ *   orc_attn_sets      the same formulas of Sec. 3.3 evaluated on a feature set I and / or token set T that
+ *                      the caller hands in (and, optionally, on a subset of the query rows)
  *
  * Readings taken where the paper is silent (all listed in the design document):
  *   - ties in TopK go to the lower index; the index set is reported ascending;
@@ -255,20 +257,39 @@ double orc_round_bf16(double x)
  *   4. if round_p: P <- bf16(P)
  *   5. if rho_t < 1: a_t = ||P[:, t]||_2, T = TopK(a, ceil(rho_t Lk))     -> idx_tok[b,h,:]
  *      O~ = P[:, T] V_g[T, :]  (no renormalisation); else O~ = P V_g
- * O [B, Hq, Lq, Dh] contiguous doubles.  idx_feat / idx_tok may be NULL.
- * P_out, if non-NULL, receives P for every (b,h) as [B,Hq,Lq,Lk] doubles (small cases only).
+ *
+ * Sec. 3.3 defines S~ and O~ for ANY feature set I and token set T; the TopK rule only says which sets RMM
+ * picks.  So that a result can be judged on somebody else's sets (the same way orc_reduced_gemm takes idx),
+ * either set may be handed in:
+ *   idx_feat_in [B,Hq,kd] non-NULL: step 1 is skipped and I = idx_feat_in[b,h,:], used in the order given;
+ *   idx_tok_in  [B,Hq,kt] non-NULL (rho_t < 1 only): the scoring of step 5 is skipped and T = idx_tok_in[b,h,:].
+ * Every other step is unchanged.  The sets actually used are reported in idx_feat / idx_tok (either may be NULL).
+ *
+ * rows [n_rows] non-NULL: only these query rows are evaluated (steps 2-4 and the product of step 5 are row by
+ * row, so nothing else changes); O is then [B, Hq, n_rows, Dh] and P_out [B, Hq, n_rows, Lk].  Token scores need
+ * every row, so with rows given and rho_t < 1 the token set must be handed in; otherwise -1 is returned and
+ * nothing is written.  Returns 0 on success.
+ * O [B, Hq, Lq (or n_rows), Dh] contiguous doubles.
+ * P_out, if non-NULL, receives P for every (b,h) as [B,Hq,Lq (or n_rows),Lk] doubles (small cases only).
  */
-void orc_attn(const void *Q, const void *Kt, const void *V, int dtype,
-              int64_t B, int64_t Hq, int64_t Hkv, int64_t Lq, int64_t Lk, int64_t Dh,
-              const int64_t *sq, const int64_t *sk, const int64_t *sv,
-              int causal, double rho_d, double rho_t, int round_p,
-              double *O, int32_t *idx_feat, int32_t *idx_tok, double *P_out)
+int orc_attn_sets(const void *Q, const void *Kt, const void *V, int dtype,
+                  int64_t B, int64_t Hq, int64_t Hkv, int64_t Lq, int64_t Lk, int64_t Dh,
+                  const int64_t *sq, const int64_t *sk, const int64_t *sv,
+                  int causal, double rho_d, double rho_t, int round_p,
+                  const int32_t *idx_feat_in, const int32_t *idx_tok_in,
+                  const int64_t *rows, int64_t n_rows,
+                  double *O, int32_t *idx_feat, int32_t *idx_tok, double *P_out)
 {
     int64_t kd = orc_keep_count(rho_d, Dh);
     int64_t kt = orc_keep_count(rho_t, Lk);
+    if (kd < 1 || kt < 1)
+        return -1;
+    if (rows != NULL && rho_t < 1.0 && idx_tok_in == NULL)
+        return -1;
+    int64_t nq = rows != NULL ? n_rows : Lq; /* query rows evaluated */
     int64_t group = Hq / Hkv;
     double scale = 1.0 / sqrt((double)Dh);
-    double *P = (double *)malloc((size_t)Lq * (size_t)Lk * sizeof(double));
+    double *P = (double *)malloc((size_t)nq * (size_t)Lk * sizeof(double));
     double *e_feat = (double *)malloc((size_t)Dh * sizeof(double));
     double *e_tok = (double *)malloc((size_t)Lk * sizeof(double));
     int32_t *I = (int32_t *)malloc((size_t)kd * sizeof(int32_t));
@@ -281,16 +302,21 @@ void orc_attn(const void *Q, const void *Kt, const void *V, int dtype,
             int64_t k0 = b * sk[0] + g * sk[1];
             int64_t v0 = b * sv[0] + g * sv[1];
 
-            /* 1. feature scores on Q only, and the feature set */
-            orc_column_energy(Q, dtype, q0, Lq, Dh, sq[2], sq[3], e_feat);
-            orc_select(e_feat, Dh, kd, I);
+            /* 1. feature scores on Q only (all of its rows), and the feature set */
+            if (idx_feat_in != NULL) {
+                memcpy(I, idx_feat_in + (b * Hq + h) * kd, (size_t)kd * sizeof(int32_t));
+            } else {
+                orc_column_energy(Q, dtype, q0, Lq, Dh, sq[2], sq[3], e_feat);
+                orc_select(e_feat, Dh, kd, I);
+            }
             if (idx_feat)
                 memcpy(idx_feat + (b * Hq + h) * kd, I, (size_t)kd * sizeof(int32_t));
 
             /* 2-4. reduced scores, mask, softmax, rounding */
 #pragma omp parallel for schedule(static)
-            for (int64_t i = 0; i < Lq; ++i) {
-                double *row = P + i * Lk;
+            for (int64_t ii = 0; ii < nq; ++ii) {
+                int64_t i = rows != NULL ? rows[ii] : ii;
+                double *row = P + ii * Lk;
                 int64_t last = causal ? i + (Lk - Lq) : Lk - 1; /* last visible key */
                 double mx = -INFINITY;
                 for (int64_t t = 0; t < Lk; ++t) {
@@ -319,21 +345,25 @@ void orc_attn(const void *Q, const void *Kt, const void *V, int dtype,
                 }
             }
             if (P_out)
-                memcpy(P_out + (b * Hq + h) * Lq * Lk, P, (size_t)Lq * (size_t)Lk * sizeof(double));
+                memcpy(P_out + (b * Hq + h) * nq * Lk, P, (size_t)nq * (size_t)Lk * sizeof(double));
 
             /* 5. token scores on the very P that is multiplied, and the token set */
             int64_t kt_used = Lk;
             if (rho_t < 1.0) {
-                orc_column_energy(P, ORC_F64, 0, Lq, Lk, Lk, 1, e_tok);
-                orc_select(e_tok, Lk, kt, T);
+                if (idx_tok_in != NULL) {
+                    memcpy(T, idx_tok_in + (b * Hq + h) * kt, (size_t)kt * sizeof(int32_t));
+                } else {
+                    orc_column_energy(P, ORC_F64, 0, Lq, Lk, Lk, 1, e_tok);
+                    orc_select(e_tok, Lk, kt, T);
+                }
                 kt_used = kt;
                 if (idx_tok)
                     memcpy(idx_tok + (b * Hq + h) * kt, T, (size_t)kt * sizeof(int32_t));
             }
 
-            double *Oh = O + (b * Hq + h) * Lq * Dh;
+            double *Oh = O + (b * Hq + h) * nq * Dh;
 #pragma omp parallel for schedule(static)
-            for (int64_t i = 0; i < Lq; ++i) {
+            for (int64_t i = 0; i < nq; ++i) {
                 for (int64_t c = 0; c < Dh; ++c) {
                     double acc = 0.0;
                     for (int64_t r = 0; r < kt_used; ++r) {
@@ -350,4 +380,16 @@ void orc_attn(const void *Q, const void *Kt, const void *V, int dtype,
     free(e_tok);
     free(I);
     free(T);
+    return 0;
+}
+
+/* The method as the paper states it: both sets chosen by the TopK rule, every query row evaluated. */
+void orc_attn(const void *Q, const void *Kt, const void *V, int dtype,
+              int64_t B, int64_t Hq, int64_t Hkv, int64_t Lq, int64_t Lk, int64_t Dh,
+              const int64_t *sq, const int64_t *sk, const int64_t *sv,
+              int causal, double rho_d, double rho_t, int round_p,
+              double *O, int32_t *idx_feat, int32_t *idx_tok, double *P_out)
+{
+    (void)orc_attn_sets(Q, Kt, V, dtype, B, Hq, Hkv, Lq, Lk, Dh, sq, sk, sv, causal, rho_d, rho_t, round_p,
+                        NULL, NULL, NULL, 0, O, idx_feat, idx_tok, P_out);
 }

@@ -376,3 +376,60 @@ def test_attention_rounded_p_is_scored_and_multiplied(oracle):
         assert np.allclose(O[0, h], want, rtol=1e-12, atol=1e-14)
     # causal, Lq < Lk: query i sees keys t <= i + (Lk - Lq)
     assert P[0, 0][0, 4:].sum() == 0.0 and P[0, 0][0, 3] > 0.0
+
+
+def test_attention_on_given_sets(oracle):
+    """Sec. 3.3 defines S~ = Q[:, I] K[:, I]^T / sqrt(d_h) and O~ = P[:, T] V[T, :] for any I and T.  Handing the
+    oracle's own choice back reproduces its result bit for bit; a foreign feature set equals the library on Q with
+    the other dims zeroed; a foreign token set equals P[:, T] V[T, :] from the returned P; sets are reported back."""
+    B, Hq, Hkv, Lq, Lk, Dh = 2, 4, 2, 9, 13, 16
+    Q, K, V = synth.attention_qkv(B, Hq, Hkv, Lq, Lk, Dh, seed=24, n_outlier=2)
+    O, If, It, P = oracle.attn(Q, K, V, True, 0.5, 0.5, round_p=True, want_p=True)
+    O2, If2, It2, P2 = oracle.attn(Q, K, V, True, 0.5, 0.5, round_p=True, want_p=True, idx_feat=If, idx_tok=It)
+    assert np.array_equal(O, O2) and np.array_equal(P, P2) and np.array_equal(If, If2) and np.array_equal(It, It2)
+    # only one of the two handed in: the other is still chosen by TopK
+    O3, _, It3, _ = oracle.attn(Q, K, V, True, 0.5, 0.5, round_p=True, idx_feat=If)
+    assert np.array_equal(O3, O) and np.array_equal(It3, It)
+
+    # a foreign feature set (not the TopK one), unrounded P: library attention on Q with the other dims zeroed
+    rng = np.random.default_rng(0)
+    kd = 8
+    feat = np.stack([np.sort(rng.choice(Dh, kd, replace=False)) for _ in range(B * Hq)]).reshape(B, Hq, kd).astype(np.int32)
+    assert not np.array_equal(feat, If)
+    Of, Iff, _, _ = oracle.attn(Q, K, V, True, 0.5, 1.0, round_p=False, idx_feat=feat)
+    assert np.array_equal(Iff, feat)
+    Qz = torch.zeros_like(Q)
+    for b in range(B):
+        for h in range(Hq):
+            Qz[b, h][:, feat[b, h].tolist()] = Q[b, h][:, feat[b, h].tolist()]
+    assert np.allclose(Of, sdpa_reference(Qz, K, V, True).numpy(), rtol=1e-11, atol=1e-12)
+
+    # a foreign token set: O = P[:, T] V[T, :] with the P of the same call, no renormalisation
+    kt = oracle.keep_count(0.5, Lk)
+    tok = np.stack([np.sort(rng.choice(Lk, kt, replace=False)) for _ in range(B * Hq)]).reshape(B, Hq, kt).astype(np.int32)
+    Ot, _, Itt, Pt = oracle.attn(Q, K, V, True, 0.5, 0.5, round_p=True, want_p=True, idx_feat=If, idx_tok=tok)
+    assert np.array_equal(Itt, tok) and np.array_equal(Pt, P)       # P does not depend on T
+    for b in range(B):
+        for h in range(Hq):
+            want = P[b, h][:, tok[b, h]] @ V[b, h // (Hq // Hkv)].double().numpy()[tok[b, h], :]
+            assert np.allclose(Ot[b, h], want, rtol=1e-12, atol=1e-14)
+    assert not np.allclose(Ot, O)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_on_sampled_query_rows(oracle, causal):
+    """Steps 2-4 of Sec. 3.3 and the final product are row by row: evaluating a subset of the query rows gives
+    exactly those rows of the full result (the feature set still comes from every row of Q)."""
+    B, Hq, Hkv, Lq, Lk, Dh = 1, 4, 2, 21, 30, 16
+    Q, K, V = synth.attention_qkv(B, Hq, Hkv, Lq, Lk, Dh, seed=25, n_outlier=2)
+    rows = [0, 3, 20, 7]
+    O, If, _, P = oracle.attn(Q, K, V, causal, 0.5, 1.0, round_p=True, want_p=True)
+    Or, Ifr, _, Pr = oracle.attn(Q, K, V, causal, 0.5, 1.0, round_p=True, want_p=True, rows=rows)
+    assert Or.shape == (B, Hq, 4, Dh) and Pr.shape == (B, Hq, 4, Lk)
+    assert np.array_equal(Ifr, If) and np.array_equal(Or, O[:, :, rows]) and np.array_equal(Pr, P[:, :, rows])
+    # with token reduction the set must be handed in (scores need every row); then rows are again independent
+    O5, _, It, _ = oracle.attn(Q, K, V, causal, 0.5, 0.4, round_p=True)
+    O5r, _, Itr, _ = oracle.attn(Q, K, V, causal, 0.5, 0.4, round_p=True, idx_tok=It, rows=rows)
+    assert np.array_equal(Itr, It) and np.array_equal(O5r, O5[:, :, rows])
+    with pytest.raises(AssertionError):
+        oracle.attn(Q, K, V, causal, 0.5, 0.4, rows=rows)
