@@ -128,6 +128,23 @@ def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 
 
+_poison = os.environ.get("RMM_POISON_OUTPUTS", "0") not in ("", "0")
+
+
+def poison_outputs(on: bool) -> None:
+    """Testing aid: when on, every output tensor this module allocates is filled with NaN (floating point) or
+    INT32_MIN (indices) before the library is called, so that an element no kernel wrote cannot pass for a result."""
+    global _poison
+    _poison = bool(on)
+
+
+def _out(shape, dtype: torch.dtype, device) -> torch.Tensor:
+    t = torch.empty(shape, dtype=dtype, device=device)
+    if _poison:
+        t.fill_(float("nan") if dtype.is_floating_point else torch.iinfo(dtype).min)
+    return t
+
+
 _ws_cache = {}
 
 
@@ -214,8 +231,8 @@ def rmm_score(A: torch.Tensor, axis: int = 1, want_scores: bool = True, want_ene
     ws = workspace(need, A.device) if ws is None else ws
     p, nb = _ws_ptr(ws)
     shape = (m.batch, n) if A.dim() == 3 else (n,)
-    scores = torch.empty(shape, dtype=torch.float32, device=A.device) if want_scores else None
-    energy = torch.empty(shape, dtype=torch.float32, device=A.device) if want_energy else None
+    scores = _out(shape, torch.float32, A.device) if want_scores else None
+    energy = _out(shape, torch.float32, A.device) if want_energy else None
     _check(lib().rmm_score(ctypes.byref(m), axis, scores.data_ptr() if want_scores else None,
                            energy.data_ptr() if want_energy else None, p, nb, _stream()))
     return scores, energy
@@ -230,8 +247,8 @@ def rmm_select(keys: torch.Tensor, rho: float = 0.0, k: int = 0, want_retained: 
     kk = int(k) if k > 0 else rmm_keep_count(rho, K)
     ws = workspace(lib().rmm_select_workspace_bytes(batch, K), keys.device) if ws is None else ws
     p, nb = _ws_ptr(ws)
-    idx = torch.empty((batch, kk) if keys.dim() == 2 else (kk,), dtype=torch.int32, device=keys.device)
-    ret = torch.empty((batch,), dtype=torch.float32, device=keys.device) if want_retained else None
+    idx = _out((batch, kk) if keys.dim() == 2 else (kk,), torch.int32, keys.device)
+    ret = _out((batch,), torch.float32, keys.device) if want_retained else None
     _check(lib().rmm_select(keys.data_ptr(), batch, K, float(rho), int(k), idx.data_ptr(),
                             ret.data_ptr() if want_retained else None, p, nb, _stream()))
     return (idx, ret) if want_retained else idx
@@ -249,11 +266,11 @@ def rmm_score_select(A: torch.Tensor, rho: float = 0.0, k: int = 0, axis: int = 
     p, nb = _ws_ptr(ws)
     three = A.dim() == 3
     if idx is None:
-        idx = torch.empty((m.batch, kk) if three else (kk,), dtype=torch.int32, device=A.device)
+        idx = _out((m.batch, kk) if three else (kk,), torch.int32, A.device)
     shape = (m.batch, n) if three else (n,)
-    scores = torch.empty(shape, dtype=torch.float32, device=A.device) if want_scores else None
-    energy = torch.empty(shape, dtype=torch.float32, device=A.device) if want_energy else None
-    ret = torch.empty((m.batch,), dtype=torch.float32, device=A.device) if want_retained else None
+    scores = _out(shape, torch.float32, A.device) if want_scores else None
+    energy = _out(shape, torch.float32, A.device) if want_energy else None
+    ret = _out((m.batch,), torch.float32, A.device) if want_retained else None
     _check(lib().rmm_score_select(ctypes.byref(m), axis, float(rho), int(k), idx.data_ptr(),
                                   scores.data_ptr() if want_scores else None,
                                   energy.data_ptr() if want_energy else None,
@@ -293,7 +310,7 @@ def rmm_reduced_gemm(A: torch.Tensor, B: torch.Tensor, idx: Optional[torch.Tenso
     if out is None:
         dt = out_dtype if out_dtype is not None else A.dtype
         shape = (ma.batch, ma.rows, mb.cols) if A.dim() == 3 else (ma.rows, mb.cols)
-        out = torch.empty(shape, dtype=dt, device=A.device)
+        out = _out(shape, dt, A.device)
     my = as_mat(out)
     need = lib().rmm_reduced_gemm_workspace_bytes(ctypes.byref(ma), ctypes.byref(mb), k, ctypes.byref(my))
     ws = workspace(need, A.device) if ws is None else ws
@@ -312,7 +329,7 @@ def rmm_reduced_attn(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, causal: 
             raise RmmError(RMM_ERR_UNSUPPORTED, "Q, K, V must be 4-D bf16 CUDA tensors with a contiguous last dim")
     B, Hq, Lq, Dh = Q.shape
     _, Hkv, Lk, _ = K.shape
-    O = torch.empty((B, Hq, Lq, Dh), dtype=torch.bfloat16, device=Q.device)
+    O = _out((B, Hq, Lq, Dh), torch.bfloat16, Q.device)
     d = rmm_attn_desc_t(B, Hq, Hkv, Lq, Lk, Dh, int(bool(causal)), float(rho_d), float(rho_t),
                         (ctypes.c_int64 * 3)(*Q.stride()[:3]), (ctypes.c_int64 * 3)(*K.stride()[:3]),
                         (ctypes.c_int64 * 3)(*V.stride()[:3]), (ctypes.c_int64 * 3)(*O.stride()[:3]))
@@ -323,9 +340,9 @@ def rmm_reduced_attn(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, causal: 
     p, nb = _ws_ptr(ws)
     idx_feat = idx_tok = None
     if want_idx:
-        idx_feat = torch.empty((B, Hq, rmm_keep_count(rho_d, Dh)), dtype=torch.int32, device=Q.device)
+        idx_feat = _out((B, Hq, rmm_keep_count(rho_d, Dh)), torch.int32, Q.device)
         if rho_t < 1.0:
-            idx_tok = torch.empty((B, Hq, rmm_keep_count(rho_t, Lk)), dtype=torch.int32, device=Q.device)
+            idx_tok = _out((B, Hq, rmm_keep_count(rho_t, Lk)), torch.int32, Q.device)
     _check(lib().rmm_reduced_attn(ctypes.byref(d), Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(),
                                   idx_feat.data_ptr() if idx_feat is not None else None,
                                   idx_tok.data_ptr() if idx_tok is not None else None, p, nb, _stream()))

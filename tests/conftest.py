@@ -18,3 +18,14 @@ def oracle():
 
     orc.build()
     return orc
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _poisoned_outputs():
+    """Every output tensor the binding allocates during the tests starts as NaN / INT32_MIN, so an element that no
+    kernel wrote fails the comparison instead of passing on whatever a recycled allocation held."""
+    from paper_2608_13426_b200 import binding
+
+    binding.poison_outputs(True)
+    yield
+    binding.poison_outputs(False)

@@ -371,35 +371,44 @@ def test_host_buffer_entry_point(oracle):
 # ------------------------------------------------------------------------------------------------
 # attention
 # ------------------------------------------------------------------------------------------------
-def check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t, seed, n_outlier=4):
+def check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t, seed, n_outlier=4, tok_band=1e-4):
+    """Feature sets: strict 1e-6 band against the oracle's TopK on Q.  Everything after that is judged on the GPU's
+    OWN sets: the oracle is evaluated on the GPU's feature sets (its P and its TopK token sets are then the
+    reference for the token sets) and on the GPU's token sets (its O is the reference for O).  No comparison is
+    conditional on the sets coinciding.  Returns whether the feature sets coincided with the oracle's."""
     Q, K, V = synth.attention_qkv(B, Hq, Hkv, Lq, Lk, Dh, seed=seed, n_outlier=n_outlier)
     O, idx_feat, idx_tok = rmm.rmm_reduced_attn(dev(Q), dev(K), dev(V), causal, rho_d, rho_t, want_idx=True)
-    Oo, If, It, P = oracle.attn(Q, K, V, causal, rho_d, rho_t, round_p=True, want_p=True)
     kd = oracle.keep_count(rho_d, Dh)
+    feat = idx_feat.cpu().numpy()
+    same_feat = True
     for b in range(B):
         for h in range(Hq):
             e64, _ = oracle.score(Q[b, h])
-            check_index_set(idx_feat[b, h].cpu().numpy(), e64, kd)
-    same_feat = np.array_equal(idx_feat.cpu().numpy(), If)
+            same_feat &= check_index_set(feat[b, h], e64, kd) == 0
+    tok = None
     if rho_t < 1.0:
         kt = oracle.keep_count(rho_t, Lk)
-        got = idx_tok.cpu().numpy()
-        assert got.shape == (B, Hq, kt)
-        if same_feat:
-            for b in range(B):
-                for h in range(Hq):
-                    # token scores come from an fp32 softmax on the GPU: judge the criterion (Theorem 1) --
-                    # the oracle-evaluated retained energy of the GPU's set is within 1e-6 of the optimum --
-                    # and set equality outside a 1e-4 * max band
-                    a2 = (P[b, h] ** 2).sum(axis=0)
-                    assert np.all(np.diff(got[b, h]) > 0)
-                    assert a2[got[b, h]].sum() >= (1 - 1e-6) * a2[It[b, h]].sum()
-                    s = np.sqrt(a2)
-                    tau = np.sort(s)[::-1][kt - 1]
-                    diff = np.setxor1d(got[b, h], It[b, h])
-                    assert np.all(np.abs(s[diff] - tau) <= 1e-4 * s.max())
-    if same_feat and (rho_t == 1.0 or np.array_equal(idx_tok.cpu().numpy(), It)):
-        assert rel_fro(O.float().cpu().numpy(), Oo) <= TOL_BF16
+        tok = idx_tok.cpu().numpy()
+        assert tok.shape == (B, Hq, kt)
+        _, _, It, P = oracle.attn(Q, K, V, causal, rho_d, rho_t, round_p=True, want_p=True, idx_feat=feat)
+        for b in range(B):
+            for h in range(Hq):
+                # token scores come from an fp32 softmax on the GPU: judge the criterion (Theorem 1) --
+                # the oracle-evaluated retained energy of the GPU's set is within 1e-6 of the optimum --
+                # and set equality outside a 1e-4 * max band
+                a2 = (P[b, h] ** 2).sum(axis=0)
+                assert np.all(np.diff(tok[b, h]) > 0) and tok[b, h].min() >= 0 and tok[b, h].max() < Lk
+                assert a2[tok[b, h]].sum() >= (1 - 1e-6) * a2[It[b, h]].sum()
+                s = np.sqrt(a2)
+                tau = np.sort(s)[::-1][kt - 1]
+                diff = np.setxor1d(tok[b, h], It[b, h])
+                assert np.all(np.abs(s[diff] - tau) <= tok_band * s.max())
+    Oo, _, _, _ = oracle.attn(Q, K, V, causal, rho_d, rho_t, round_p=True, idx_feat=feat, idx_tok=tok)
+    Og = O.float().cpu().numpy()
+    assert np.isfinite(Og).all()
+    for b in range(B):
+        for h in range(Hq):
+            assert rel_fro(Og[b, h], Oo[b, h]) <= TOL_BF16, (b, h)
     return same_feat
 
 
@@ -453,18 +462,20 @@ def test_fused_attention_rows_without_keys_are_zero():
 ])
 def test_fused_attention_token_reduction(oracle, shape):
     """rho_t < 1 through the fused sweeps (row normalisers, token scores of the rounded P, gathered P V): the token
-    sets meet Theorem 1's criterion against the oracle's P, and O matches wherever the sets agree."""
+    sets meet Theorem 1's criterion against the oracle's P, and O matches the oracle evaluated on the GPU's sets."""
     B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t = shape
     assert check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t, seed=60 + Lq % 7)
     assert rmm.rmm_status_read() == 0
 
 
 def test_fused_and_composed_attention_agree(oracle, monkeypatch):
-    """The fused sweeps and the composed form (S~ and P materialised) are two routes to the same result."""
+    """The fused sweeps and the composed form (S~ and P materialised) are two routes to the same result: same
+    feature sets, and each form's O matches the oracle evaluated on that form's own token sets."""
     import subprocess, sys, os
     code = (
         "import torch, paper_2608_13426_b200 as rmm\n"
-        "from paper_2608_13426_b200 import synth\n"
+        "from paper_2608_13426_b200 import synth, binding\n"
+        "binding.poison_outputs(True)\n"
         "Q, K, V = synth.attention_qkv(1, 4, 2, 300, 420, 128, seed=71, device='cuda')\n"
         "O, f, t = rmm.rmm_reduced_attn(Q, K, V, True, 0.5, 0.5, want_idx=True)\n"
         "torch.save((O.cpu(), f.cpu(), t.cpu()), __import__('sys').argv[1])\n")
@@ -477,10 +488,11 @@ def test_fused_and_composed_attention_agree(oracle, monkeypatch):
         os.remove(path)
     (O1, f1, t1), (O0, f0, t0) = outs
     assert torch.equal(f1, f0)
-    same = [h for h in range(4) if torch.equal(t1[0, h], t0[0, h])]
-    assert len(same) >= 2
-    for h in same:
-        assert rel_fro(O1[0, h].float().numpy(), O0[0, h].float().numpy().astype(np.float64)) <= TOL_BF16
+    Q, K, V = synth.attention_qkv(1, 4, 2, 300, 420, 128, seed=71)
+    for O, f, t in outs:
+        Oo, _, _, _ = oracle.attn(Q, K, V, True, 0.5, 0.5, round_p=True, idx_feat=f.numpy(), idx_tok=t.numpy())
+        for h in range(4):
+            assert rel_fro(O[0, h].float().numpy(), Oo[0, h]) <= TOL_BF16
 
 
 def test_composed_attention_for_wide_heads(oracle):
@@ -502,8 +514,7 @@ def test_attention_batch_folding_and_uneven_batch_stride(oracle):
     assert Qv.stride(0) != Hq * Qv.stride(1)
     O2, f2, _ = rmm.rmm_reduced_attn(Qv, Kd, Vd, True, 0.5, 1.0, want_idx=True)
     assert torch.equal(f1, f2) and torch.equal(O1, O2)
-    Oo, If, _ = oracle.attn(Q, K, V, True, 0.5, 1.0, round_p=True)[:3]
-    assert np.array_equal(f1.cpu().numpy(), If)
+    Oo = oracle.attn(Q, K, V, True, 0.5, 1.0, round_p=True, idx_feat=f1.cpu().numpy())[0]
     assert rel_fro(O1.float().cpu().numpy(), Oo) <= TOL_BF16
 
 
