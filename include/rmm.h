@@ -59,8 +59,8 @@ typedef struct {
 #define RMM_WS_HEADER_BYTES 4096
 
 /* |I| = ceil(rho K) (Sec. 3.2), host only.  rho is taken as a double; the product rho*K is snapped
- * to the nearest integer when it lies within 1e-9*K of it (so 0.07*100 gives 7, not 8), then
- * rounded up and clamped to [1, K].  RMM_ERR_INVALID_ARG if rho is not in (0, 1], K < 1 or k is NULL. */
+ * to the nearest integer when it lies within 4 ulps (4 * 2^-52 * rho*K) of it (so 0.07*100 gives 7, not 8,
+ * while a ratio that is genuinely a little above j/K gives j + 1 at any K), then rounded up and clamped to [1, K].  RMM_ERR_INVALID_ARG if rho is not in (0, 1], K < 1 or k is NULL. */
 int rmm_keep_count(double rho, int64_t K, int64_t *k);
 
 /* Importance scores s_j = ||A[:, j]||_2 (Sec. 3.2 "Activation-aware dimension selection"; in
@@ -74,7 +74,8 @@ size_t rmm_score_workspace_bytes(const rmm_mat_t *A, int axis);
 int rmm_score(const rmm_mat_t *A, int axis, float *scores, float *energy, void *ws, size_t ws_bytes, void *stream);
 
 /* I = TopK(keys, k) (Sec. 3.2; Theorem 1 shows it minimises the discarded energy).  One index set per
- * batch element.  k > 0 is used as given, otherwise k = rmm_keep_count(rho, K).
+ * batch element.  k in [1, K] is used as given; k == 0 means k = rmm_keep_count(rho, K); k < 0 or k > K is
+ * RMM_ERR_INVALID_ARG.
  *   keys     fp32 [batch, K], non-negative
  *   idx      int32 [batch, k], ASCENDING; among equal keys the lower index is kept
  *   retained fp32 [batch] or NULL: sum of the kept keys / sum of all keys (1 - eps_A(rho) of Eq. 5
@@ -100,10 +101,16 @@ int rmm_score_select(const rmm_mat_t *A, int axis, double rho, int64_t k, int32_
  * address up (with that device current), so make that first call outside any stream capture.  All calls share the
  * one array per device: it keeps the previous call's contents (the part that must start at zero is cleared on the
  * stream by every call), and two calls that overlap on the GPU (different streams) race.  Results are those of
- * rmm_score_select, bit for bit.  idx, scores, energy, retained as there. */
+ * rmm_score_select, bit for bit.  idx, scores, energy, retained as there.
+ * The device status word of these calls lives in the built-in array, where rmm_status_read cannot reach it:
+ * rmm_score_select_static_status copies it to *device_status (an rmm_status_t) and clears it, for the current device.
+ * It is a blocking copy: synchronise the stream first.  The word is sticky (a later call does not erase an error an
+ * earlier one reported).  The cached address of the array belongs to the device's primary context and does not
+ * survive cudaDeviceReset(). */
 size_t rmm_score_select_static_capacity(void);
 int rmm_score_select_static(const rmm_mat_t *A, int axis, double rho, int64_t k, int32_t *idx, float *scores,
                             float *energy, float *retained, void *stream);
+int rmm_score_select_static_status(int *device_status);
 
 /* Y = scale * A[:, I] B[I, :] (Sec. 3.2, RMM_rho(A,B); no rescaling: pass scale = 1).
  *   A    [b, M, K]; B [b or shared, K, N] (stride_batch 0 = shared); Y [b, M, N] (written in full)

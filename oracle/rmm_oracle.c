@@ -21,8 +21,9 @@
  *
  * Readings taken where the paper is silent (all listed in the design document):
  *   - ties in TopK go to the lower index; the index set is reported ascending;
- *   - ceil(rho*K) is taken on the double product with a 1e-9*K guard against products that
- *     are integral in exact arithmetic but land a hair above the integer in binary;
+ *   - ceil(rho*K) is taken on the double product; a product within 4 ulps (4 * 2^-52 * rho*K) of an
+ *     integer is that integer, which guards ratios such as 0.07 * 100 that are integral in exact
+ *     arithmetic but land a hair above the integer in binary, and nothing else;
  *   - selection compares squared norms (monotone in the norm, no sqrt collapse);
  *   - the softmax scale keeps the full 1/sqrt(d_h); no renormalisation after dropping tokens;
  *   - P is rounded once to bf16 (round-to-nearest-even) before it is scored and multiplied
@@ -86,7 +87,9 @@ int64_t orc_keep_count(double rho, int64_t K)
     double x = rho * (double)K;
     double r = nearbyint(x);
     int64_t k;
-    if (fabs(x - r) <= 1e-9 * (double)K)
+    /* rho and the product each carry at most half an ulp of rounding error, so a product that is integral in exact
+     * arithmetic lands within a few ulps of that integer; anything further away is genuinely fractional */
+    if (fabs(x - r) <= 4.0 * 2.220446049250313e-16 * x)
         k = (int64_t)r;
     else
         k = (int64_t)ceil(x);

@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     rmm_score_select,
     rmm_score_select_static,
     rmm_score_select_static_capacity,
+    rmm_score_select_static_status,
     rmm_select,
     rmm_status_read,
 )

@@ -47,7 +47,7 @@ class rmm_attn_desc_t(ctypes.Structure):
 
 EXPORTS = ["rmm_keep_count", "rmm_score_workspace_bytes", "rmm_score", "rmm_select_workspace_bytes", "rmm_select",
            "rmm_score_select_workspace_bytes", "rmm_score_select", "rmm_score_select_static",
-           "rmm_score_select_static_capacity", "rmm_reduced_gemm_workspace_bytes",
+           "rmm_score_select_static_capacity", "rmm_score_select_static_status", "rmm_reduced_gemm_workspace_bytes",
            "rmm_reduced_gemm", "rmm_reduced_attn_workspace_bytes", "rmm_reduced_attn",
            "rmm_product_host_workspace_bytes", "rmm_product_host", "rmm_status_read", "rmm_last_error",
            "rmm_launch_count", "rmm_profile_kernels", "rmm_profile_count", "rmm_profile_name"]
@@ -78,6 +78,7 @@ def lib() -> ctypes.CDLL:
     L.rmm_score_select.argtypes = [mp, i32, dbl, i64, vp, vp, vp, vp, vp, sz, vp]
     L.rmm_score_select_static.argtypes = [mp, i32, dbl, i64, vp, vp, vp, vp, vp]
     L.rmm_score_select_static_capacity.restype = sz
+    L.rmm_score_select_static_status.argtypes = [ctypes.POINTER(i32)]
     L.rmm_reduced_gemm_workspace_bytes.argtypes = [mp, mp, i64, mp]
     L.rmm_reduced_gemm_workspace_bytes.restype = sz
     L.rmm_reduced_gemm.argtypes = [mp, mp, vp, i64, flt, mp, vp, sz, vp]
@@ -284,6 +285,18 @@ def rmm_score_select_static(A: torch.Tensor, idx: torch.Tensor, rho: float = 0.0
     built into the library.  Every buffer is the caller's: idx int32 [batch, k] (or [k]), optional energy fp32
     [batch, n] and retained fp32 [batch] are written in place.  This wrapper itself allocates nothing on the device."""
     m = as_mat(A)
+    n = m.cols if axis == 1 else m.rows
+    kk = int(k) if k > 0 else rmm_keep_count(rho, n)
+
+    def buf(t, dtype, numel, name):
+        if t.dtype != dtype or not t.is_cuda or not t.is_contiguous() or t.numel() != numel:
+            raise RmmError(RMM_ERR_INVALID_ARG, f"score_select_static: {name} must be a contiguous {dtype} CUDA tensor of {numel} elements")
+
+    buf(idx, torch.int32, m.batch * kk, "idx")
+    if energy is not None:
+        buf(energy, torch.float32, m.batch * n, "energy")
+    if retained is not None:
+        buf(retained, torch.float32, m.batch, "retained")
     _check(lib().rmm_score_select_static(ctypes.byref(m), axis, float(rho), int(k), idx.data_ptr(), None,
                                          energy.data_ptr() if energy is not None else None,
                                          retained.data_ptr() if retained is not None else None, _stream()))
@@ -291,6 +304,14 @@ def rmm_score_select_static(A: torch.Tensor, idx: torch.Tensor, rho: float = 0.0
 
 def rmm_score_select_static_capacity() -> int:
     return int(lib().rmm_score_select_static_capacity())
+
+
+def rmm_score_select_static_status() -> int:
+    """Synchronise the current stream, then read and clear the status word of the built-in scratch array."""
+    torch.cuda.current_stream().synchronize()
+    st = ctypes.c_int(0)
+    _check(lib().rmm_score_select_static_status(ctypes.byref(st)))
+    return int(st.value)
 
 
 def rmm_reduced_gemm(A: torch.Tensor, B: torch.Tensor, idx: Optional[torch.Tensor], scale: float = 1.0,

@@ -96,7 +96,8 @@ int rmm_keep_count(double rho, int64_t K, int64_t *k)
         return fail(RMM_ERR_INVALID_ARG, "keep_count: need rho in (0, 1], K >= 1 and a non-NULL result");
     const double x = rho * (double)K;
     const double r = nearbyint(x);
-    int64_t v = fabs(x - r) <= 1e-9 * (double)K ? (int64_t)r : (int64_t)ceil(x);
+    // the product of two doubles is off by at most a few ulps: only that close to an integer does it count as integral
+    int64_t v = fabs(x - r) <= 4.0 * 2.220446049250313e-16 * x ? (int64_t)r : (int64_t)ceil(x);
     if (v < 1) v = 1;
     if (v > K) v = K;
     *k = v;

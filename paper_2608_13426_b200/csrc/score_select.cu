@@ -14,6 +14,7 @@
 // keys equal to the threshold the lowest indices are kept.  bf16 matrices that meet the TMA rules are
 // streamed by score_tma_kernel (64-column blocks, 256-row tiles through a ring of shared-memory buffers).
 #include <cuda.h>
+#include <stddef.h>
 
 #include "common.cuh"
 
@@ -901,7 +902,11 @@ static __device__ __align__(256) unsigned char g_static_scratch[RMM_STATIC_SCRAT
 namespace rmm {
 namespace {
 constexpr int kMaxDevices = 64;
-void *g_static_scratch_ptr[kMaxDevices];  // device address of g_static_scratch, per device; NULL until set up
+// Device address of g_static_scratch, per device ordinal; NULL until set up.  Two host threads that make their first
+// call at the same time both look the address up and store the same value.  The address belongs to the device's
+// primary context: it does not survive cudaDeviceReset() (a process that resets a device must not call these entry
+// points on it afterwards).
+std::atomic<void *> g_static_scratch_ptr[kMaxDevices];
 
 // In host code `g_static_scratch` names a host-side shadow of the symbol, not device memory: the device address has
 // to be asked for, once per device, with that device current.
@@ -911,14 +916,14 @@ int static_scratch(void **out)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "score_select_static: cudaGetDevice: %s", cudaGetErrorString(e));
     if (dev < 0 || dev >= kMaxDevices) return fail(RMM_ERR_UNSUPPORTED, "score_select_static: device index %d is not covered", dev);
-    if (g_static_scratch_ptr[dev] == nullptr) {
-        void *p = nullptr;
+    void *p = g_static_scratch_ptr[dev].load(std::memory_order_acquire);
+    if (p == nullptr) {
         e = cudaGetSymbolAddress(&p, g_static_scratch);
         if (e != cudaSuccess || p == nullptr)
             return fail(RMM_ERR_CUDA, "score_select_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
-        g_static_scratch_ptr[dev] = p;
+        g_static_scratch_ptr[dev].store(p, std::memory_order_release);
     }
-    *out = g_static_scratch_ptr[dev];
+    *out = p;
     return RMM_OK;
 }
 }  // namespace
@@ -946,8 +951,20 @@ extern "C" int rmm_score_select_static(const rmm_mat_t *A, int axis, double rho,
     void *ws = nullptr;
     if ((rc = static_scratch(&ws)) != RMM_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // the array keeps whatever the previous call left: the status word and the arrival counters must start at zero
-    cudaError_t e = cudaMemsetAsync(ws, 0, RMM_WS_HEADER_BYTES, st);
+    // the array keeps whatever the previous call left: the arrival counters must start at zero.  The status word in front
+    // of them is left alone, so that an error a kernel reported stays there until rmm_score_select_static_status reads it.
+    cudaError_t e = cudaMemsetAsync(static_cast<char *>(ws) + offsetof(WsHeader, counters), 0,
+                                    RMM_WS_HEADER_BYTES - offsetof(WsHeader, counters), st);
     if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "score_select_static: cudaMemsetAsync: %s", cudaGetErrorString(e));
     return launch_score_select(A, p, true, kk, idx, scores, energy, retained, ws, st);
+}
+
+extern "C" int rmm_score_select_static_status(int *device_status)
+{
+    using namespace rmm;
+    if (device_status == nullptr) return fail(RMM_ERR_INVALID_ARG, "score_select_static_status: NULL argument");
+    void *ws = nullptr;
+    int rc = static_scratch(&ws);
+    if (rc != RMM_OK) return rc;
+    return rmm_status_read(ws, device_status);  // blocking 4-byte copy; clears the word if it was set
 }

@@ -476,8 +476,8 @@ def test_fused_and_composed_attention_agree(oracle, monkeypatch):
         "import torch, paper_2608_13426_b200 as rmm\n"
         "from paper_2608_13426_b200 import synth, binding\n"
         "binding.poison_outputs(True)\n"
-        "Q, K, V = synth.attention_qkv(1, 4, 2, 300, 420, 128, seed=71, device='cuda')\n"
-        "O, f, t = rmm.rmm_reduced_attn(Q, K, V, True, 0.5, 0.5, want_idx=True)\n"
+        "Q, K, V = synth.attention_qkv(1, 4, 2, 300, 420, 128, seed=71)\n"
+        "O, f, t = rmm.rmm_reduced_attn(Q.cuda(), K.cuda(), V.cuda(), True, 0.5, 0.5, want_idx=True)\n"
         "torch.save((O.cpu(), f.cpu(), t.cpu()), __import__('sys').argv[1])\n")
     outs = []
     for flag in ("1", "0"):

@@ -38,6 +38,27 @@ def test_keep_count_exact_rationals(oracle):
                 assert oracle.keep_count(p / q, K) == want, (p, q, K)
 
 
+def test_keep_count_large_axes_and_near_integers(oracle):
+    """The snap to an integer is a matter of a few ulps at any size: on axes of 2^15 .. 2^30 a ratio that is
+    integral in exact arithmetic gives that integer, and a ratio a little above j / K (from 1e-7 down to a few
+    hundred ulps) gives j + 1, as exact rational arithmetic on the double that was passed says."""
+    for K in (32768, 28672, 1 << 20, (1 << 24) + 3, 1 << 30):
+        for q in (3, 5, 7, 10, 100, 1000):
+            for p in (1, q // 2, q - 1):
+                rho = p / q
+                exact = Fraction(p, q) * K
+                if exact.denominator == 1:                      # integral in exact arithmetic: no rounding up
+                    assert oracle.keep_count(rho, K) == int(exact), (p, q, K)
+                else:
+                    assert oracle.keep_count(rho, K) == math.ceil(Fraction(rho) * K), (p, q, K)
+        for j in (1, K // 3, K - 2):
+            for above in (1e-3, 1e-5, 1e-7 * K / 32768):
+                rho = (j + above) / K                           # genuinely fractional: ceil gives j + 1
+                assert math.ceil(Fraction(rho) * K) == j + 1
+                assert oracle.keep_count(rho, K) == j + 1, (j, above, K)
+            assert oracle.keep_count(j / K, K) == j             # j / K itself rounds to j even if the product is a hair off
+
+
 def test_keep_count_paper_values(oracle):
     for line in open(os.path.join(GOLDEN, "keep_count_paper.txt")):
         if line.startswith("#") or not line.strip():

@@ -34,6 +34,7 @@ def test_static_scratch_matches_workspace_entry_point_twice():
         assert torch.equal(idx, want_idx)
         assert torch.equal(energy, want_energy)
         assert torch.equal(retained, want_ret)
+        assert rmm.rmm_score_select_static_status() == 0        # no kernel of this call reported an error
     # a batched problem that still fits
     Q = synth.gaussian((6, 300, 128), 1.0, seed=43).cuda()
     idx = torch.empty((6, 64), dtype=torch.int32, device="cuda")
@@ -56,3 +57,8 @@ def test_static_scratch_rejects_oversize():
     assert e.value.code == binding.RMM_ERR_WORKSPACE and "built-in array" in str(e.value)
     torch.cuda.synchronize()
     assert int(idx.min()) == -7 and int(idx.max()) == -7                        # nothing was launched
+    # the wrapper checks the caller's buffers before the call: a short idx would be written past its end
+    small = torch.zeros((8, 64, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.RmmError) as e:
+        rmm.rmm_score_select_static(small, torch.empty(100, dtype=torch.int32, device="cuda"), rho=0.5)
+    assert e.value.code == binding.RMM_ERR_INVALID_ARG
