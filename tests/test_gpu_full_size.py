@@ -52,8 +52,8 @@ def test_attention_prefill_qk_head_dim_reduction(oracle, rho):
 @pytest.mark.parametrize("rho", [0.25, 0.5])
 def test_long_context_pv_sequence_reduction(oracle, rho):
     """Long-context PV: seq 16384, head_dim 128, P = causal softmax given as a bf16 input, keys selected per head.
-    Two of the 32 heads (P alone is 0.5 GB per head)."""
-    H, L, Dh = 2, 16384, 128
+    Eight of the 32 heads (P alone is 0.5 GB per head; heads are independent problems of identical shape)."""
+    H, L, Dh = 8, 16384, 128
     P = synth.attention_probs(L, H, Dh, seed=3, causal=True, device="cuda")
     V = synth.gaussian((H, L, Dh), 1.0, seed=5).cuda()
     kt = oracle.keep_count(rho, L)
@@ -158,3 +158,51 @@ def test_long_context_fused_attention(oracle, rho_t):
     Oo = oracle.attn(Q, K, V, True, 0.5, rho_t, round_p=True, idx_feat=feat, idx_tok=tok)[0]
     for h in range(Hq):
         assert rel_fro(O[0, h].float().cpu().numpy(), Oo[0, h]) <= TOL_BF16
+
+
+# ------------------------------------------------------------------------------------------------
+# 70B-class layer at the sizes the benchmark times (32768 prefill tokens): index sets in full, products on tile-edge
+# and seeded rows that the oracle computes one by one
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,K,N", [("gate_up", 8192, 28672), ("q_o", 8192, 8192), ("down", 28672, 8192)])
+def test_70b_class_layer_products_full_size(oracle, name, K, N):
+    M = 32768
+    A = synth.heavy_tailed_activations(M, K, seed=13, device="cuda")
+    B = synth.weight(K, N, seed=14, device="cuda")
+    Ac, Bc = A.cpu(), B.cpu()
+    e64, _ = oracle.score(Ac)
+    rows = sample_rows(M, 4, seed=3) + [255, 256, 257]          # 256: the edge of a CTA pair's tile
+    for rho in (0.25, 0.5):
+        k = oracle.keep_count(rho, K)
+        Y, idx = rmm.rmm(A, B, rho)
+        idx_np = idx.cpu().numpy()
+        check_index_set(idx_np, e64, k)
+        Yr = Y[rows].float().cpu().numpy()
+        assert np.isfinite(Y.float().sum().item())               # no element of the 32768 x N output was left unwritten
+        del Y
+        for i, r in enumerate(rows):
+            want = oracle.reduced_gemm(Ac, Bc, idx_np, rows=(r, r + 1))[r]
+            assert rel_fro(Yr[i], want) <= TOL_BF16, (name, rho, r)
+    assert rmm.rmm_status_read() == 0
+
+
+def test_70b_class_attention_full_size(oracle):
+    """64 query heads on 8 kv heads, 32768 tokens, head_dim 128, causal, rho_d = 0.5 (feature reduction, one fused
+    pass).  Feature sets of every head in full; O of two query heads (from different kv groups) on sampled query rows,
+    against the oracle evaluated on the GPU's feature sets for those rows only."""
+    Hq, Hkv, L, Dh = 64, 8, 32768, 128
+    Q, K, V = synth.attention_qkv(1, Hq, Hkv, L, L, Dh, seed=17, device="cuda")
+    O, idx_feat, _ = rmm.rmm_reduced_attn(Q, K, V, True, 0.5, 1.0, want_idx=True)
+    assert bool(torch.isfinite(O.float().sum()))
+    feat = idx_feat.cpu().numpy()
+    for h in range(Hq):
+        check_index_set(feat[0, h], oracle.score(Q[0, h].cpu())[0], 64)
+    rows = sample_rows(L, 6, seed=4)
+    for h in (5, 62):
+        g = h // (Hq // Hkv)
+        Qh, Kg, Vg = Q[:, h:h + 1].cpu(), K[:, g:g + 1].cpu(), V[:, g:g + 1].cpu()
+        Oo = oracle.attn(Qh, Kg, Vg, True, 0.5, 1.0, round_p=True, idx_feat=feat[:, h:h + 1], rows=rows)[0]
+        got = O[0, h][rows].float().cpu().numpy()
+        for i, r in enumerate(rows):
+            assert rel_fro(got[i], Oo[0, 0, i]) <= TOL_BF16, (h, r)
+    assert rmm.rmm_status_read() == 0
