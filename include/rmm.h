@@ -153,9 +153,21 @@ size_t rmm_reduced_attn_workspace_bytes(const rmm_attn_desc_t *desc);
 int rmm_reduced_attn(const rmm_attn_desc_t *desc, const void *Q, const void *K, const void *V, void *O,
                      int32_t *idx_feat, int32_t *idx_tok, void *ws, size_t ws_bytes, void *stream);
 
+/* The whole operation of Sec. 3.2 on device operands: I = TopK of the column norms of A with |I| = k (k == 0:
+ * ceil(rho K)), Y = scale * A[:, I] B[I, :].  The result is that of rmm_score_select followed by rmm_reduced_gemm, bit
+ * for bit; idx [batch, k] and retained [batch] (or NULL) as there.  For one bf16 product (batch 1) whose A has 2048 to
+ * 8192 columns and more than 256 rows, and whose operands meet the tensor-core layout rules, the scores, the selection
+ * and both gathers run in ONE launch (every block owns 64 columns of A, a grid-wide barrier makes all column energies
+ * visible, every block then selects and gathers its own kept columns and the matching rows of B), followed by the
+ * tensor-core product; this form expects the GPU to itself (all of its blocks must be resident at once; if they are
+ * not, the barrier's bounded wait expires and RMM_ERR_TIMEOUT is reported).  Everything else runs as the two calls. */
+size_t rmm_product_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, const rmm_mat_t *Y);
+int rmm_product(const rmm_mat_t *A, const rmm_mat_t *B, double rho, int64_t k, float scale, const rmm_mat_t *Y, int32_t *idx,
+                float *retained, void *ws, size_t ws_bytes, void *stream);
+
 /* The whole operation of Sec. 3.2 on one bf16 product held in HOST memory (pinned for speed):
  * copies A [M,K] and B [K,N] (row-major, contiguous) to the device staging area inside ws, runs
- * rmm_score_select and rmm_reduced_gemm, and copies Y [M,N] bf16 and idx [k] back, all asynchronously on
+ * rmm_product, and copies Y [M,N] bf16 and idx [k] back, all asynchronously on
  * `stream`; the caller synchronises the stream before reading Y_host / idx_host.  copy_B = 0 reuses the
  * B already staged by an earlier call on the same workspace (a resident weight). */
 size_t rmm_product_host_workspace_bytes(int64_t M, int64_t K, int64_t N);

@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     rmm,
     rmm_keep_count,
     rmm_launch_count,
+    rmm_product,
     rmm_product_host,
     rmm_reduced_attn,
     rmm_reduced_gemm,

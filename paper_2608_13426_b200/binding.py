@@ -49,7 +49,7 @@ EXPORTS = ["rmm_keep_count", "rmm_score_workspace_bytes", "rmm_score", "rmm_sele
            "rmm_score_select_workspace_bytes", "rmm_score_select", "rmm_score_select_static",
            "rmm_score_select_static_capacity", "rmm_score_select_static_status", "rmm_reduced_gemm_workspace_bytes",
            "rmm_reduced_gemm", "rmm_reduced_attn_workspace_bytes", "rmm_reduced_attn",
-           "rmm_product_host_workspace_bytes", "rmm_product_host", "rmm_status_read", "rmm_last_error",
+           "rmm_product_workspace_bytes", "rmm_product", "rmm_product_host_workspace_bytes", "rmm_product_host", "rmm_status_read", "rmm_last_error",
            "rmm_launch_count", "rmm_profile_kernels", "rmm_profile_count", "rmm_profile_name"]
 
 _lib = None
@@ -85,6 +85,9 @@ def lib() -> ctypes.CDLL:
     L.rmm_reduced_attn_workspace_bytes.argtypes = [ctypes.POINTER(rmm_attn_desc_t)]
     L.rmm_reduced_attn_workspace_bytes.restype = sz
     L.rmm_reduced_attn.argtypes = [ctypes.POINTER(rmm_attn_desc_t), vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.rmm_product_workspace_bytes.argtypes = [mp, mp, mp]
+    L.rmm_product_workspace_bytes.restype = sz
+    L.rmm_product.argtypes = [mp, mp, dbl, i64, flt, mp, vp, vp, vp, sz, vp]
     L.rmm_product_host_workspace_bytes.argtypes = [i64, i64, i64]
     L.rmm_product_host_workspace_bytes.restype = sz
     L.rmm_product_host.argtypes = [vp, vp, i64, i64, i64, dbl, i32, vp, vp, vp, sz, vp]
@@ -385,8 +388,31 @@ def rmm_product_host(A_host: torch.Tensor, B_host: torch.Tensor, rho: float, Y_h
                                   p, nb, _stream()))
 
 
+def rmm_product(A: torch.Tensor, B: torch.Tensor, rho: float = 0.0, k: int = 0, scale: float = 1.0,
+                out: Optional[torch.Tensor] = None, idx: Optional[torch.Tensor] = None, want_retained: bool = False,
+                ws: Optional[torch.Tensor] = None):
+    """RMM_rho(A, B) of Sec. 3.2 on device tensors in one call: (Y, idx) or (Y, idx, retained)."""
+    ma, mb = as_mat(A), as_mat(B)
+    kk = int(k) if k > 0 else rmm_keep_count(rho, ma.cols)
+    three = A.dim() == 3
+    if out is None:
+        out = _out((ma.batch, ma.rows, mb.cols) if three else (ma.rows, mb.cols), A.dtype, A.device)
+    if idx is None:
+        idx = _out((ma.batch, kk) if three else (kk,), torch.int32, A.device)
+    elif idx.dtype != torch.int32 or not idx.is_cuda or not idx.is_contiguous() or idx.numel() != ma.batch * kk:
+        raise RmmError(RMM_ERR_INVALID_ARG, "idx must be a contiguous int32 CUDA tensor of batch * k elements")
+    ret = _out((ma.batch,), torch.float32, A.device) if want_retained else None
+    my = as_mat(out)
+    need = lib().rmm_product_workspace_bytes(ctypes.byref(ma), ctypes.byref(mb), ctypes.byref(my))
+    if need == 0:
+        raise RmmError(RMM_ERR_UNSUPPORTED, "rmm_product: operands not covered")
+    ws = workspace(need, A.device) if ws is None else ws
+    p, nb = _ws_ptr(ws)
+    _check(lib().rmm_product(ctypes.byref(ma), ctypes.byref(mb), float(rho), int(k), float(scale), ctypes.byref(my),
+                             idx.data_ptr(), ret.data_ptr() if want_retained else None, p, nb, _stream()))
+    return (out, idx, ret) if want_retained else (out, idx)
+
+
 def rmm(A: torch.Tensor, B: torch.Tensor, rho: float, out: Optional[torch.Tensor] = None):
-    """RMM_rho(A, B) of Sec. 3.2 on device tensors: fused score + select, then the reduced product.
-    Returns (Y, idx)."""
-    idx, _, _, _ = rmm_score_select(A, rho=rho)
-    return rmm_reduced_gemm(A, B, idx, out=out), idx
+    """RMM_rho(A, B) of Sec. 3.2 on device tensors (rmm_product).  Returns (Y, idx)."""
+    return rmm_product(A, B, rho=rho, out=out)

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -50,6 +51,27 @@ int check_launch(const char *what, cudaStream_t stream)
     if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "%s: launch failed: %s", what, cudaGetErrorString(e));
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return RMM_OK;
+}
+
+int sm_count()
+{
+    static std::atomic<int> cached[64];
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = -1;
+    if (dev >= 0 && (n = cached[dev].load(std::memory_order_relaxed)) > 0) return n;
+    if (dev < 0 || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    cached[dev].store(n, std::memory_order_relaxed);
+    return n;
+}
+
+unsigned long long wait_limit_ns()
+{
+    static const unsigned long long limit = []() -> unsigned long long {
+        const char *e = getenv("RMM_SPIN_LIMIT_MS");
+        const double ms = e != nullptr ? atof(e) : 0.0;
+        return ms > 0.0 ? (unsigned long long)(ms * 1e6) : 2000000000ull;
+    }();
+    return limit;
 }
 
 static int check_ws(void *ws, size_t ws_bytes, size_t need, const char *who)
@@ -223,6 +245,79 @@ int rmm_reduced_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx,
     return launch_gemm_simt(A, &b, idx, k, scale, Y, ws, static_cast<cudaStream_t>(stream));
 }
 
+// ---- whole operation on device operands ------------------------------------------------------------
+struct ProductPlan {
+    bool fused;
+    FrontPlan front;
+    size_t total;
+};
+
+static int plan_product(const rmm_mat_t *A, const rmm_mat_t *B, const rmm_mat_t *Y, int64_t k, ProductPlan *pp)
+{
+    rmm_mat_t b = shared_b(A, B);
+    pp->fused = front_eligible(A, &b, Y, k, &pp->front);
+    if (pp->fused) {
+        pp->total = pp->front.total_bytes;
+        return RMM_OK;
+    }
+    const size_t s1 = rmm_score_select_workspace_bytes(A, 1);
+    const size_t s2 = rmm_reduced_gemm_workspace_bytes(A, B, k, Y);
+    if (s1 == 0 || s2 == 0) return RMM_ERR_UNSUPPORTED;
+    pp->total = s1 > s2 ? s1 : s2;
+    return RMM_OK;
+}
+
+size_t rmm_product_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, const rmm_mat_t *Y)
+{
+    if (A == nullptr || B == nullptr || Y == nullptr || A->cols < 1) return 0;
+    ProductPlan pp;
+    if (plan_product(A, B, Y, A->cols, &pp) != RMM_OK) return 0;  // k = K bounds every k
+    size_t need = pp.total;
+    if (pp.fused) {  // a k for which the fused form does not apply falls back to the two-call form
+        const size_t s1 = rmm_score_select_workspace_bytes(A, 1), s2 = rmm_reduced_gemm_workspace_bytes(A, B, A->cols, Y);
+        if (s1 > need) need = s1;
+        if (s2 > need) need = s2;
+    }
+    return need;
+}
+
+int rmm_product(const rmm_mat_t *A, const rmm_mat_t *B, double rho, int64_t k, float scale, const rmm_mat_t *Y, int32_t *idx,
+                float *retained, void *ws, size_t ws_bytes, void *stream)
+{
+    if (A == nullptr || A->ptr == nullptr || A->cols < 1) return fail(RMM_ERR_INVALID_ARG, "product: A is NULL or empty");
+    if (idx == nullptr) return fail(RMM_ERR_INVALID_ARG, "product: idx is NULL");
+    int64_t kk;
+    int rc = resolve_k(rho, k, A->cols, &kk, "product");
+    if (rc != RMM_OK) return rc;
+    rc = check_gemm(A, B, idx, kk, Y);
+    if (rc != RMM_OK) return rc;
+    ProductPlan pp;
+    rc = plan_product(A, B, Y, kk, &pp);
+    if (rc != RMM_OK) return fail(rc, "product: operands not covered");
+    rc = check_ws(ws, ws_bytes, pp.total, "product");
+    if (rc != RMM_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!pp.fused) {
+        rc = rmm_score_select(A, 1, rho, kk, idx, nullptr, nullptr, retained, ws, ws_bytes, stream);
+        if (rc != RMM_OK) return rc;
+        return rmm_reduced_gemm(A, B, idx, kk, scale, Y, ws, ws_bytes, stream);
+    }
+    rmm_mat_t b = shared_b(A, B);
+    rc = launch_front(A, &b, kk, idx, nullptr, retained, pp.front, ws, st);
+    if (rc != RMM_OK) return rc;
+    char *w = static_cast<char *>(ws);
+    TcProblem p = {};
+    p.batch = 1; p.M = A->rows; p.N = B->cols; p.k = kk;
+    p.a = reinterpret_cast<const __nv_bfloat16 *>(w + pp.front.off_ap); p.a_ld = pp.front.ldp; p.a_sb = A->rows * pp.front.ldp;
+    p.b_kmajor = 0;
+    p.b = reinterpret_cast<const __nv_bfloat16 *>(w + pp.front.off_bp); p.b_ld = B->cols; p.b_sb = kk * B->cols; p.b_batches = 1;
+    p.b_batch_off = 0; p.b_batch_div = 1;
+    p.y = Y->ptr; p.y_bf16 = Y->dtype == RMM_BF16; p.y_sb = Y->stride_batch; p.y_sr = Y->stride_row;
+    p.scale = scale;
+    p.status = &reinterpret_cast<WsHeader *>(w)->status;
+    return launch_gemm_tc_problem(p, st);
+}
+
 // ---- whole operation on host buffers -------------------------------------------------------------
 struct HostPlan {
     size_t off_a, off_b, off_y, off_idx, off_inner, inner_bytes, total;
@@ -240,10 +335,9 @@ static int plan_host(int64_t M, int64_t K, int64_t N, void *ws, HostPlan *h)
     rmm_mat_t Y = {nullptr, RMM_BF16, 1, M, N, M * N, N, 1};
     // sizes that do not depend on the pointers: use aligned dummies for the planners
     A.ptr = B.ptr = Y.ptr = reinterpret_cast<void *>(uintptr_t(256));
-    size_t s1 = rmm_score_select_workspace_bytes(&A, 1);
-    size_t s2 = rmm_reduced_gemm_workspace_bytes(&A, &B, K, &Y);  // k = K bounds every k
-    if (s1 == 0 || s2 == 0) return RMM_ERR_UNSUPPORTED;
-    h->inner_bytes = align_up(s1 > s2 ? s1 : s2, 256);
+    size_t s1 = rmm_product_workspace_bytes(&A, &B, &Y);
+    if (s1 == 0) return RMM_ERR_UNSUPPORTED;
+    h->inner_bytes = align_up(s1, 256);
     off += h->inner_bytes;
     h->off_a = off; off += align_up((size_t)M * K * 2, 256);
     h->off_b = off; off += align_up((size_t)K * N * 2, 256);
@@ -283,9 +377,7 @@ int rmm_product_host(const void *A_host, const void *B_host, int64_t M, int64_t 
     cudaError_t e = cudaMemcpyAsync(h.A.ptr, A_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess && copy_B) e = cudaMemcpyAsync(h.B.ptr, B_host, (size_t)K * N * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "product_host: host-to-device copy: %s", cudaGetErrorString(e));
-    rc = rmm_score_select(&h.A, 1, rho, k, idx, nullptr, nullptr, nullptr, w + h.off_inner, h.inner_bytes, stream);
-    if (rc != RMM_OK) return rc;
-    rc = rmm_reduced_gemm(&h.A, &h.B, idx, k, 1.0f, &h.Y, w + h.off_inner, h.inner_bytes, stream);
+    rc = rmm_product(&h.A, &h.B, rho, k, 1.0f, &h.Y, idx, nullptr, w + h.off_inner, h.inner_bytes, stream);
     if (rc != RMM_OK) return rc;
     e = cudaMemcpyAsync(Y_host, h.Y.ptr, (size_t)M * N * 2, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess && idx_host != nullptr)

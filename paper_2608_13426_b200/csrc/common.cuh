@@ -68,6 +68,9 @@ struct PerDeviceOnce {
     }
 };
 
+int sm_count();                      // multiprocessors of the current device
+unsigned long long wait_limit_ns();  // bound of every device-side wait: 2 s, or RMM_SPIN_LIMIT_MS from the environment
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 static inline size_t dtype_size(int dt) { return dt == RMM_BF16 ? 2 : 4; }
@@ -104,6 +107,16 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
                         float *scores, float *energy, float *retained, void *ws, cudaStream_t stream);
 int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_t *idx, float *retained, void *ws,
                   cudaStream_t stream);
+
+// Front end of a whole product in one launch (scores, selection, packed A[:, I] and B[I, :]); see score_select.cu.
+struct FrontPlan {
+    int col_blocks;
+    int64_t ldp;  // row pitch of the packed A (multiple of 8)
+    size_t off_energy, off_ap, off_bp, total_bytes;
+};
+bool front_eligible(const rmm_mat_t *A, const rmm_mat_t *B, const rmm_mat_t *Y, int64_t k, FrontPlan *plan);
+int launch_front(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, int32_t *idx, float *energy, float *retained,
+                 const FrontPlan &plan, void *ws, cudaStream_t stream);
 
 // ---- reduced GEMM ------------------------------------------------------------------------------------
 // Plain FMA kernel: any strides, bf16 or fp32 operands, fp32 accumulation, bf16 or fp32 output.

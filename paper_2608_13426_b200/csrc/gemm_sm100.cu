@@ -427,14 +427,6 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 // ----------------------------------------------------------------------------------------------
 // host side
 // ----------------------------------------------------------------------------------------------
-int sm_count()
-{
-    int dev = 0, n = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    return n;
-}
-
 template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS, bool B_GATHER = false>
 int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &my, const TcArgs &a, cudaStream_t stream)
 {

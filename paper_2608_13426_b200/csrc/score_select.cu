@@ -15,6 +15,7 @@
 // streamed by score_tma_kernel (64-column blocks, 256-row tiles through a ring of shared-memory buffers).
 #include <cuda.h>
 #include <stddef.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 #include "select.cuh"
@@ -218,7 +219,7 @@ constexpr int kTmaStages = 6, kTmaRows = 256, kTmaCols = 64;
 constexpr int kTmaStageBytes = kTmaRows * kTmaCols * 2;
 constexpr unsigned long long kScoreWaitNs = 2000000000ull;
 
-__device__ __forceinline__ bool score_wait(uint32_t bar, uint32_t parity, int *status)
+__device__ __forceinline__ bool score_wait(uint32_t bar, uint32_t parity, int *status, unsigned long long limit_ns = kScoreWaitNs)
 {
     unsigned long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
@@ -230,7 +231,7 @@ __device__ __forceinline__ bool score_wait(uint32_t bar, uint32_t parity, int *s
             unsigned long long now;
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
             if (t0 == 0) t0 = now;
-            if (now - t0 > kScoreWaitNs) {
+            if (now - t0 > limit_ns) {
                 atomicExch(status, (int)RMM_ERR_TIMEOUT);
                 return false;
             }
@@ -319,6 +320,385 @@ __global__ void __launch_bounds__(kThreads, 1) score_tma_kernel(const __grid_con
     score_finish<8>(a, dacc, s_dyn, s_sel, s_flag);
 }
 
+// ---- the front end of a whole product in ONE launch: scores, selection, and both gathers ---------------------------
+// For one bf16 product Y = A[:, I] B[I, :] whose score pass needs no row split (every block owns 64 columns and all
+// the rows) and whose keys fit in registers (n <= 8192).  Phases of a block:
+//   1. stream its 64 columns of A through the ring and sum the squares (as score_tma_kernel), publish 64 energies;
+//   2. grid-wide barrier (an arrival counter and a generation word in the workspace header; the grid is at most one
+//      block per SM, all resident; the wait is bounded like every other);
+//   3. EVERY block runs the selection on all n energies (redundantly: a block-wide select costs the same whether one
+//      block or all of them run it, and nobody then waits for a second barrier), so each knows the threshold, the kept
+//      columns among its own 64 and their positions in the index list; block 0 writes the list itself;
+//   4. (warps 0-15) its kept columns of A go to Ap[:, pos0 .. pos0 + cnt): the last six tiles of the stream are still in
+//      the ring and are gathered from there, the earlier ones are copied again (from L2 when A is small); a warp copies
+//      2-byte elements from shared memory to 4-byte stores;
+//   5. (warps 16-31, at the same time) the rows of B that belong to its kept columns, requested into L2 right after the
+//      selection, go to Bp[pos0 .. pos0 + cnt, :] as 16-byte vectors.
+// The reduced product then reads Ap and Bp with TMA tile loads.  Against separate score, select and gather launches
+// this saves two launches, the hand-off to a single selecting block, and the gather kernel's own staging of A.
+#ifdef RMM_FRONT_STAMPS
+// Debug build: %globaltimer stamps of the front kernel's phases (first start / last end over all blocks), read back by
+// rmm_debug_front_stamps.  Slot 0 is a minimum, the others maxima.
+__device__ unsigned long long g_fstamps[16];
+#define FSTAMP_MIN(i) do { if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); atomicMin(&g_fstamps[i], t_); } } while (0)
+#define FSTAMP_MAX(i) do { if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); atomicMax(&g_fstamps[i], t_); } } while (0)
+#else
+#define FSTAMP_MIN(i)
+#define FSTAMP_MAX(i)
+#endif
+
+struct FrontArgs {
+    ScoreArgs sc;             // A, n, m, energy, scores, k, idx, retained (row_splits == 1; counters unused)
+    unsigned *grid_bar;       // [2] in the workspace header: arrivals, generation
+    __nv_bfloat16 *Ap;        // [m, ldp]
+    int64_t ldp;
+    const __nv_bfloat16 *B;   // [n, N], row pitch b_sr
+    int64_t b_sr, N;
+    __nv_bfloat16 *Bp;        // [k, N]
+    unsigned long long wait_ns;
+};
+
+constexpr int kFrontCombBytes = (kThreads / 32) * kTmaCols * 8;              // per-warp column sums (fp64)
+constexpr int kFrontSmemBytes = kTmaStages * kTmaStageBytes + kFrontCombBytes;
+
+__global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_constant__ CUtensorMap map_a, FrontArgs fa, int *status)
+{
+    extern __shared__ __align__(128) unsigned char s_dyn[];  // the tile ring, then the per-warp column sums
+    __shared__ SelectSmem s_sel;
+    __shared__ __align__(8) unsigned long long s_bar[2 * kTmaStages];
+    __shared__ int s_ok, s_first, s_end;
+    __shared__ int s_pos[kTmaCols];           // position in the index list of each own column, or -1
+    __shared__ unsigned short s_own[kTmaCols];  // own kept columns (0 .. 63) in list order
+
+    const ScoreArgs &a = fa.sc;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tx = tid & 7, ty = tid >> 3;  // 8 column groups x 128 row lanes
+    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(s_dyn);
+    const uint32_t bars = (uint32_t)__cvta_generic_to_shared(s_bar);
+    auto full_bar = [&](int st) { return bars + 8u * st; };
+    auto empty_bar = [&](int st) { return bars + 8u * (kTmaStages + st); };
+    const int n_tiles = (int)((a.m + kTmaRows - 1) / kTmaRows);
+    const int col0 = (int)blockIdx.x * kTmaCols;
+
+    if (tid == 0) {
+        for (int st = 0; st < kTmaStages; ++st) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(full_bar(st)), "r"(1) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_bar(st)), "r"(kThreads / 32) : "memory");
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+        s_ok = 1;
+    }
+    __syncthreads();
+    pdl_wait();
+    FSTAMP_MIN(0);
+    unsigned gen0 = 0;
+    if (tid == 0) gen0 = *reinterpret_cast<volatile unsigned *>(fa.grid_bar + 1);  // before this block can have arrived
+
+    // Ring protocol.  A slot's `full` barrier completes once per fill, its `empty` barrier once every time all 32 warps
+    // have released it.  full_par (every thread) and empty_par (thread 0) hold, per slot, the parity of the next
+    // completion to wait for; every completion is waited for exactly once, in order.
+    uint32_t full_par = 0, empty_par = 0;
+    auto fill = [&](int slot, int tile) {  // thread 0 only: rows of `tile` -> slot
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full_bar(slot)), "r"(kTmaStageBytes) : "memory");
+        asm volatile(
+            "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+            ::"r"(ring + slot * kTmaStageBytes), "l"(&map_a), "r"(col0), "r"(tile * kTmaRows), "r"(0), "r"(full_bar(slot))
+            : "memory");
+    };
+    auto wait_empty = [&](int slot) -> bool {  // thread 0 only
+        const bool done = score_wait(empty_bar(slot), (empty_par >> slot) & 1u, status, fa.wait_ns);
+        empty_par ^= 1u << slot;
+        return done;
+    };
+    auto wait_full = [&](int slot) -> bool {
+        const bool done = score_wait(full_bar(slot), (full_par >> slot) & 1u, status, fa.wait_ns);
+        full_par ^= 1u << slot;
+        return done;
+    };
+    constexpr int kAhead = kTmaStages - 2;
+    if (tid == 0)
+        for (int t = 0; t < kAhead && t < n_tiles; ++t) fill(t, t);
+
+    // ---- 1. scores
+    double dacc[8];
+    float facc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { dacc[e] = 0.0; facc[e] = 0.f; }
+    bool ok = true;
+    for (int t = 0; t < n_tiles && ok; ++t) {
+        const int st = t % kTmaStages;
+        if (tid == 0 && t + kAhead < n_tiles) {
+            const int nt = t + kAhead, ns = nt % kTmaStages;
+            if (nt >= kTmaStages && !wait_empty(ns)) ok = false;
+            if (ok) fill(ns, nt);
+        }
+        if (!wait_full(st)) { ok = false; break; }
+        const uint4 *tile = reinterpret_cast<const uint4 *>(s_dyn + st * kTmaStageBytes);
+        const uint4 q0 = tile[ty * 8 + tx], q1 = tile[(ty + 128) * 8 + tx];
+        const unsigned w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float lo0 = __uint_as_float(w[i] << 16), hi0 = __uint_as_float(w[i] & 0xffff0000u);
+            const float lo1 = __uint_as_float(w[4 + i] << 16), hi1 = __uint_as_float(w[4 + i] & 0xffff0000u);
+            facc[2 * i] = fmaf(lo1, lo1, fmaf(lo0, lo0, facc[2 * i]));
+            facc[2 * i + 1] = fmaf(hi1, hi1, fmaf(hi0, hi0, facc[2 * i + 1]));
+        }
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(st)) : "memory");
+        if ((t & 7) == 7) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { dacc[e] += (double)facc[e]; facc[e] = 0.f; }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) dacc[e] += (double)facc[e];
+    if (!ok) s_ok = 0;
+    __syncthreads();
+    FSTAMP_MAX(1);
+    // A block that ran out of time leaves the ring alone (a copy may still land in it), lets the others through the
+    // grid barrier, gives copies in flight time to land and returns; the status word tells the host.
+    const bool alive = s_ok != 0;
+    // The last tiles of the stream (up to six) are still in the ring and stay there: the gather starts with them.
+    const int resident = n_tiles < kTmaStages ? n_tiles : kTmaStages;
+    if (alive) {
+        // Row lanes in a fixed order: the four lanes of a column group inside a warp by shuffles, then the 32 warps in
+        // order by the column's owner thread.  The sums live next to the ring, which keeps its tiles.
+        double *s_comb = reinterpret_cast<double *>(s_dyn + kTmaStages * kTmaStageBytes);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            dacc[e] += __shfl_xor_sync(0xffffffffu, dacc[e], 8);
+            dacc[e] += __shfl_xor_sync(0xffffffffu, dacc[e], 16);
+        }
+        if (lane < 8) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s_comb[warp * kTmaCols + tx * 8 + e] = dacc[e];
+        }
+        __syncthreads();
+        if (tid < kTmaCols && col0 + tid < a.n) {
+            double colsum = 0.0;
+#pragma unroll 8
+            for (int q = 0; q < kThreads / 32; ++q) colsum += s_comb[q * kTmaCols + tid];
+            a.energy[col0 + tid] = (float)colsum;
+            if (a.scores != nullptr) a.scores[col0 + tid] = (float)sqrt(colsum);
+        }
+        if (tid == 0) {  // every release of the stream has been waited for once the gather starts
+            for (int s2 = 0; s2 < resident && ok; ++s2)
+                if (!wait_empty(s2)) ok = false;
+            if (!ok) s_ok = 0;
+        }
+    }
+
+    // ---- 2. grid-wide barrier: all energies are visible afterwards.  The block's energy stores are ordered before
+    // thread 0's releasing arrival by the block barrier (release is cumulative); the last block to arrive resets the
+    // count for the next launch and publishes a new generation, which the others acquire.
+    FSTAMP_MAX(2);
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned nblocks = gridDim.x;
+        unsigned old;
+        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(old) : "l"(fa.grid_bar) : "memory");
+        if (old == nblocks - 1u) {
+            asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(fa.grid_bar), "r"(0u) : "memory");
+            asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(fa.grid_bar + 1) : "memory");
+        } else if (alive) {
+            unsigned long long t0 = 0;
+            for (uint32_t it = 0;; ++it) {
+                unsigned g;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(g) : "l"(fa.grid_bar + 1) : "memory");
+                if (g != gen0) break;
+                if ((it & 63u) == 63u) {
+                    unsigned long long now;
+                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+                    if (t0 == 0) t0 = now;
+                    if (now - t0 > fa.wait_ns) {
+                        atomicExch(status, (int)RMM_ERR_TIMEOUT);
+                        s_ok = 0;
+                        break;
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (s_ok == 0) {
+        // nothing more is written; copies in flight (if any) get time to land before shared memory is released
+        unsigned long long t0, now;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+        do { __nanosleep(2000); asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now)); } while (now - t0 < 200000ull);
+        return;
+    }
+
+    // ---- 3. selection, in every block
+    FSTAMP_MAX(3);
+    unsigned u[8];
+    const int nvalid = load_keys_blocked<8>(a.energy, (int)a.n, u);
+    const Threshold th = block_threshold<8>(u, nvalid, a.k, s_sel);
+    const unsigned before = block_rank_blocked<8>(u, nvalid, th.tau, s_sel);
+    {
+        unsigned gt_before = before >> 16, eq_before = before & 0xffffu;
+        const bool writer = blockIdx.x == 0;
+        const int j0 = tid * 8;
+        const bool mine = j0 >= col0 && j0 < col0 + kTmaCols;  // eight threads hold this block's columns
+        if (mine && j0 == col0) s_first = (int)(gt_before + min(eq_before, th.need_eq));
+        double sum_kept = 0.0, sum_all = 0.0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (i < nvalid) {
+                const bool gt = u[i] > th.tau, eq = u[i] == th.tau;
+                const bool keep = gt || (eq && eq_before < th.need_eq);
+                const unsigned pos = gt_before + min(eq_before, th.need_eq);
+                if (writer && keep) a.idx[pos] = j0 + i;
+                if (mine) s_pos[j0 + i - col0] = keep ? (int)pos : -1;
+                if (writer && a.retained != nullptr) {
+                    const double f = (double)key_value(u[i]);
+                    sum_all += f;
+                    if (keep) sum_kept += f;
+                }
+                gt_before += gt ? 1u : 0u;
+                eq_before += eq ? 1u : 0u;
+            } else if (mine) {
+                s_pos[j0 + i - col0] = -1;
+            }
+        }
+        if (mine && j0 + 8 == col0 + kTmaCols) s_end = (int)(gt_before + min(eq_before, th.need_eq));
+        if (writer && a.retained != nullptr) {  // block-uniform
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                sum_kept += __shfl_down_sync(0xffffffffu, sum_kept, d);
+                sum_all += __shfl_down_sync(0xffffffffu, sum_all, d);
+            }
+            if (lane == 0) {
+                s_sel.red[warp] = sum_kept;
+                s_sel.red[32 + warp] = sum_all;
+            }
+            __syncthreads();
+            if (tid == 0) {
+                double x = 0.0, y = 0.0;
+                for (int w2 = 0; w2 < 32; ++w2) {
+                    x += s_sel.red[w2];
+                    y += s_sel.red[32 + w2];
+                }
+                *a.retained = (y > 0.0) ? (float)(x / y) : 1.0f;
+            }
+        }
+    }
+    __syncthreads();
+    const int pos0 = s_first, cnt = s_end - s_first;
+    if (tid < kTmaCols && s_pos[tid] >= 0) s_own[s_pos[tid] - pos0] = (unsigned short)tid;
+    __syncthreads();
+    {
+        // the rows of B that this block copies in step 5 are requested into L2 now, so that they arrive from HBM while
+        // the gather of A runs
+        const int lines = (int)((fa.N * 2 + 127) / 128);
+        const char *b0 = reinterpret_cast<const char *>(fa.B) + (int64_t)col0 * fa.b_sr * 2;
+        for (int i = tid; i < cnt * lines; i += kThreads) {
+            const int j = i / lines, c = i - j * lines;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(b0 + (int64_t)s_own[j] * fa.b_sr * 2 + (int64_t)c * 128));
+        }
+    }
+
+    FSTAMP_MAX(4);
+    // ---- 4 and 5 run side by side: warps 0 .. 15 gather the block's kept columns of A, warps 16 .. 31 copy its rows
+    // of B (requested into L2 above).  The ring's `empty` barriers are set up again for 16 releasing warps.
+    constexpr int kGatherWarps = 16;
+    if (tid == 0) {
+        for (int st = 0; st < kTmaStages; ++st) {
+            asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(empty_bar(st)) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_bar(st)), "r"(kGatherWarps) : "memory");
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        empty_par = 0;
+    }
+    __syncthreads();
+    if (warp < kGatherWarps) {
+        // ---- 4. own kept columns of A -> Ap[:, pos0 .. pos0 + cnt).  Lane l builds the output pair l (and, when pos0 is
+        // odd and all 64 columns are kept, lane 0 also pair 32) counted from the even position at or below pos0: one
+        // 4-byte store per row, a 2-byte store where only one member of the pair belongs to this block.  Everything that
+        // does not change from row to row is worked out here: the loop body is two shared-memory loads, a merge, the stores.
+        const int base_even = pos0 & ~1;
+        const int j_lo = base_even + 2 * lane - pos0, j_hi = j_lo + 1;  // positions of the pair inside this block's list
+        const bool has_lo = j_lo >= 0 && j_lo < cnt, has_hi = j_hi < cnt;   // (j_hi >= 0 always)
+        const uint32_t o_lo = has_lo ? (uint32_t)s_own[j_lo] * 2u : 0u, o_hi = has_hi ? (uint32_t)s_own[j_hi] * 2u : 0u;
+        const bool st_pair = has_lo && has_hi, st_lo = has_lo && !has_hi, st_hi = has_hi && !has_lo;
+        const bool extra = lane == 0 && base_even + 64 < pos0 + cnt;          // pair 32 holds the 64th kept column
+        const uint32_t o_extra = extra ? (uint32_t)s_own[cnt - 1] * 2u : 0u;
+        const int64_t row_step = kGatherWarps * fa.ldp;                       // elements between two rows of this warp
+        unsigned short *dwarp = reinterpret_cast<unsigned short *>(fa.Ap) + (int64_t)warp * fa.ldp + base_even + 2 * lane;
+        // Step t < resident works on the tile the stream left in the ring (no copy, nothing to wait for); later steps
+        // work on tiles 0, 1, ... copied again (from L2 when A is small) into the slots in the order they were released,
+        // requested two steps after the release.
+        const int n_reload = n_tiles - resident;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const int tile = t < resident ? n_tiles - resident + t : t - resident;
+            const int st = (n_tiles - resident + t) % kTmaStages;
+            if (tid == 0 && t >= 2 && t - 2 < n_reload) {
+                const int q = t - 2, qs = (n_tiles - resident + q) % kTmaStages;  // the slot step q released
+                if (!wait_empty(qs)) ok = false;
+                if (ok) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    fill(qs, q);
+                }
+            }
+            if (t >= resident && !wait_full(st)) { ok = false; break; }
+            const int64_t left = a.m - (int64_t)tile * kTmaRows - warp;      // rows of this tile at or below the warp's first
+            const int np = left <= 0 ? 0 : (int)min((int64_t)(kTmaRows / kGatherWarps), (left + kGatherWarps - 1) / kGatherWarps);
+            uint32_t row_s = ring + st * kTmaStageBytes + (uint32_t)warp * (kTmaCols * 2);
+            unsigned short *d = dwarp + (int64_t)tile * kTmaRows * fa.ldp;
+#pragma unroll 4
+            for (int p = 0; p < np; ++p) {
+                unsigned short v0, v1;
+                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v0) : "r"(row_s + o_lo));
+                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v1) : "r"(row_s + o_hi));
+                if (st_pair) *reinterpret_cast<unsigned *>(d) = (unsigned)v0 | ((unsigned)v1 << 16);
+                if (st_lo) d[0] = v0;
+                if (st_hi) d[1] = v1;
+                if (extra) {
+                    unsigned short v2;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v2) : "r"(row_s + o_extra));
+                    d[64] = v2;
+                }
+                row_s += kGatherWarps * kTmaCols * 2;
+                d += row_step;
+            }
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(st)) : "memory");
+        }
+    } else {
+        // ---- 5. rows of B of the own kept columns -> Bp[pos0 .. pos0 + cnt, :], 16-byte vectors.  Rows shorter than
+        // these warps are wide are copied several at a time (thread = vector c of row j0, j0 + rows_par, ...).
+        constexpr int kCopyThreads = kThreads - 32 * kGatherWarps;
+        const int ct = tid - 32 * kGatherWarps;
+        const int nvec = (int)(fa.N / 8);
+        const uint4 *src = reinterpret_cast<const uint4 *>(fa.B) + (int64_t)col0 * (fa.b_sr / 8);
+        uint4 *dst = reinterpret_cast<uint4 *>(fa.Bp) + (int64_t)pos0 * nvec;
+        const int s_pitch = (int)(fa.b_sr / 8);
+        const int rows_par = nvec >= kCopyThreads ? 1 : kCopyThreads / nvec;
+        const int c0 = rows_par == 1 ? ct : ct % nvec, j0 = rows_par == 1 ? 0 : ct / nvec;
+        if (j0 < rows_par) {
+            for (int c = c0; c < nvec; c += kCopyThreads) {
+                for (int j = j0; j < cnt; j += 8 * rows_par) {
+                    uint4 q[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (j + i * rows_par < cnt) q[i] = __ldg(src + (int)s_own[j + i * rows_par] * s_pitch + c);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (j + i * rows_par < cnt) dst[(j + i * rows_par) * nvec + c] = q[i];
+                }
+            }
+        }
+    }
+    if (!__syncthreads_and(ok)) {
+        unsigned long long t0, now;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+        do { __nanosleep(2000); asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now)); } while (now - t0 < 200000ull);
+        return;
+    }
+    FSTAMP_MAX(6);
+}
+
 __global__ void __launch_bounds__(1024) select_kernel(const float *keys, int K, int k, int32_t *idx, float *retained,
                                                       int use_cache)
 {
@@ -356,7 +736,7 @@ int plan_score(const rmm_mat_t *A, int axis, ScorePlan *p)
     // thread layout: tx column groups x ty row lanes.  Narrow blocks (down to 8 groups = 128 contiguous bytes per
     // row) are preferred as long as the grid stays within one block per SM, because a block that owns all the rows
     // of its columns needs no cross-block combine; row splits only fill the machine when there are few columns.
-    const int64_t sms = 148;
+    const int64_t sms = sm_count();
     int64_t groups = ceil_div(p->n, p->vec);
     int tx = 32;
     while (tx > 1 && tx / 2 >= groups) tx /= 2;
@@ -459,6 +839,71 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
     return launch_select(a.energy, A->batch, p.n, k, idx, retained, ws, stream);
 }
 
+bool front_eligible(const rmm_mat_t *A, const rmm_mat_t *B, const rmm_mat_t *Y, int64_t k, FrontPlan *plan)
+{
+    TcPlan tc;
+    if (A->batch != 1 || !tc_eligible(A, B, k, Y, &tc) || tc.b_kmajor) return false;
+    if (A->rows <= 256) return false;  // short outputs: the product fetches the kept rows of B itself
+    ScorePlan sp;
+    if (plan_score(A, 1, &sp) != RMM_OK || !sp.use_tma) return false;
+    if (sp.n > kFusedSelectMax || sp.n % 8 != 0) return false;
+    const int col_blocks = (int)ceil_div(sp.n, kTmaCols);
+    // every block owns all the rows of its columns, and the whole grid has to be resident for the grid-wide barrier
+    if (col_blocks > sm_count() || col_blocks < sm_count() / 4) return false;
+    if (plan != nullptr) {
+        plan->col_blocks = col_blocks;
+        plan->ldp = (k + 7) / 8 * 8;
+        size_t off = RMM_WS_HEADER_BYTES;
+        plan->off_energy = off;
+        off += align_up((size_t)sp.n * 4, 256);
+        plan->off_ap = off;
+        off += align_up((size_t)A->rows * plan->ldp * 2, 256);
+        plan->off_bp = off;
+        off += align_up((size_t)k * B->cols * 2, 256);
+        plan->total_bytes = off;
+    }
+    return true;
+}
+
+int launch_front(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, int32_t *idx, float *energy, float *retained,
+                 const FrontPlan &plan, void *ws, cudaStream_t stream)
+{
+    char *w = static_cast<char *>(ws);
+    WsHeader *hdr = reinterpret_cast<WsHeader *>(w);
+    FrontArgs fa = {};
+    ScoreArgs &a = fa.sc;
+    a.A = A->ptr;
+    a.s_batch = 0; a.s_red = A->stride_row; a.s_n = 1;
+    a.n = A->cols; a.m = A->rows; a.rows_per_split = A->rows;
+    a.row_splits = 1; a.col_blocks = plan.col_blocks; a.tx = 8; a.ty = kThreads / 8;
+    a.partials = nullptr; a.counters = nullptr;
+    a.energy = energy != nullptr ? energy : reinterpret_cast<float *>(w + plan.off_energy);
+    a.scores = nullptr;
+    a.do_select = 1; a.k = (int)k; a.idx = idx; a.retained = retained;
+    fa.grid_bar = &hdr->counters[kHeaderCounters - 2];
+    fa.Ap = reinterpret_cast<__nv_bfloat16 *>(w + plan.off_ap);
+    fa.ldp = plan.ldp;
+    fa.B = static_cast<const __nv_bfloat16 *>(B->ptr);
+    fa.b_sr = B->stride_row; fa.N = B->cols;
+    fa.Bp = reinterpret_cast<__nv_bfloat16 *>(w + plan.off_bp);
+    fa.wait_ns = wait_limit_ns();
+    CUtensorMap map;
+    const uint64_t dims[3] = {(uint64_t)a.n, (uint64_t)a.m, 1};
+    const uint64_t st[2] = {(uint64_t)A->stride_row * 2, (uint64_t)A->stride_row * 2 * (uint64_t)a.m};
+    const uint32_t box[3] = {kTmaCols, kTmaRows, 1};
+    int rc = make_map(&map, const_cast<void *>(a.A), 3, dims, st, box, false);
+    if (rc != RMM_OK) return rc;
+    static PerDeviceOnce configured;
+    if (configured.first()) {
+        cudaError_t e = cudaFuncSetAttribute(rmm_front_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFrontSmemBytes);
+        if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "front: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    }
+    prof_begin("rmm_front_kernel", stream);
+    launch_kernel(rmm_front_kernel, dim3((unsigned)plan.col_blocks), dim3(kThreads), kFrontSmemBytes, stream, 1, map, fa,
+                  &hdr->status);
+    return check_launch("rmm_front_kernel", stream);
+}
+
 int launch_select(const float *keys, int64_t batch, int64_t K, int64_t k, int32_t *idx, float *retained, void *ws,
                   cudaStream_t stream)
 {
@@ -559,3 +1004,16 @@ extern "C" int rmm_score_select_static_status(int *device_status)
     if (rc != RMM_OK) return rc;
     return rmm_status_read(ws, device_status);  // blocking 4-byte copy; clears the word if it was set
 }
+
+#ifdef RMM_FRONT_STAMPS
+// Debug build only: copy the front kernel's phase stamps (nanoseconds of %globaltimer) to out[0 .. 15] and re-arm them.
+extern "C" int rmm_debug_front_stamps(unsigned long long *out)
+{
+    unsigned long long init[16];
+    cudaError_t e = cudaMemcpyFromSymbol(out, rmm::g_fstamps, sizeof init);
+    for (int i = 0; i < 16; ++i) init[i] = 0;
+    init[0] = ~0ull;
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(rmm::g_fstamps, init, sizeof init);
+    return e == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
+}
+#endif

@@ -550,3 +550,34 @@ def test_small_batch_product_fetches_rows_of_b_in_the_kernel(oracle, M, K, N, rh
     torch.cuda.synchronize()
     assert rmm.rmm_status_read() == 6          # RMM_ERR_BOUNDS, cleared by the read
     assert rmm.rmm_status_read() == 0
+
+
+@pytest.mark.parametrize("M,K,N,rho", [(2048, 8192, 2048, 0.5), (2048, 8192, 2048, 0.25), (300, 4096, 264, 0.75), (1000, 8000, 512, 0.5),
+                                       (513, 2560, 1024, 0.3), (4096, 8192, 1024, 1.0), (700, 4096, 256, 0.011)])
+def test_whole_product_in_one_front_launch(oracle, M, K, N, rho):
+    """rmm_product on one bf16 product with 2368 .. 8192 columns runs scores, selection and both gathers in a single
+    launch (grid-wide barrier, every block selects and gathers its own columns).  Index set and Y must equal the two-call
+    form bit for bit, the set must match the oracle's, and Y the oracle's product on that set.  Ragged last column block
+    (8000), ragged row tile (300, 513, 1000), odd list positions, k not a multiple of 8."""
+    A, B = synth.mlp_product(M, K, N, seed=M + K)
+    Ad, Bd = dev(A), dev(B)
+    launches0 = rmm.rmm_launch_count()
+    Y, idx, ret = rmm.rmm_product(Ad, Bd, rho=rho, want_retained=True)
+    torch.cuda.synchronize()
+    assert rmm.rmm_launch_count() - launches0 == 2                  # front end + product
+    idx2, _, _, ret2 = rmm.rmm_score_select(Ad, rho=rho, want_retained=True)
+    Y2 = rmm.rmm_reduced_gemm(Ad, Bd, idx2)
+    assert torch.equal(idx, idx2) and torch.equal(ret, ret2) and torch.equal(Y, Y2)
+    e64, _ = oracle.score(A)
+    k = oracle.keep_count(rho, K)
+    check_index_set(idx.cpu().numpy(), e64, k)
+    rows = sorted({0, 127, 128, 255, 256, M // 2, M - 1})
+    idx_np = idx.cpu().numpy()
+    Yc = Y.float().cpu().numpy()
+    for r in rows:
+        want = oracle.reduced_gemm(A, B, idx_np, rows=(r, r + 1))[r]
+        assert rel_fro(Yc[r], want) <= TOL_BF16
+    # run to run identical, and the workspace is left reusable
+    Y3, idx3 = rmm.rmm_product(Ad, Bd, rho=rho)
+    assert torch.equal(idx3, idx) and torch.equal(Y3, Y)
+    assert rmm.rmm_status_read() == 0
