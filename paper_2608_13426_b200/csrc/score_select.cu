@@ -366,7 +366,7 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
     extern __shared__ __align__(128) unsigned char s_dyn[];  // the tile ring, then the per-warp column sums
     __shared__ SelectSmem s_sel;
     __shared__ __align__(8) unsigned long long s_bar[2 * kTmaStages];
-    __shared__ int s_ok, s_first, s_end;
+    __shared__ int s_ok, s_first, s_end, s_next;
     __shared__ int s_pos[kTmaCols];           // position in the index list of each own column, or -1
     __shared__ unsigned short s_own[kTmaCols];  // own kept columns (0 .. 63) in list order
 
@@ -584,9 +584,25 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
             }
         }
     }
+    if (tid == 0) s_next = -1;
     __syncthreads();
     const int pos0 = s_first, cnt = s_end - s_first;
     if (tid < kTmaCols && s_pos[tid] >= 0) s_own[s_pos[tid] - pos0] = (unsigned short)tid;
+    {
+        // the kept column that follows this block's range in the list (position pos0 + cnt), if any: when the range ends
+        // at an odd position its last element shares a 4-byte word of Ap with that column's, and this block writes both
+        unsigned gt_before = before >> 16, eq_before = before & 0xffffu;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (i < nvalid) {
+                const bool gt = u[i] > th.tau, eq = u[i] == th.tau;
+                const bool keep = gt || (eq && eq_before < th.need_eq);
+                if (keep && (int)(gt_before + min(eq_before, th.need_eq)) == pos0 + cnt) s_next = tid * 8 + i;
+                gt_before += gt ? 1u : 0u;
+                eq_before += eq ? 1u : 0u;
+            }
+        }
+    }
     __syncthreads();
     {
         // the rows of B that this block copies in step 5 are requested into L2 now, so that they arrive from HBM while
@@ -613,19 +629,30 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
     }
     __syncthreads();
     if (warp < kGatherWarps) {
-        // ---- 4. own kept columns of A -> Ap[:, pos0 .. pos0 + cnt).  Lane l builds the output pair l (and, when pos0 is
-        // odd and all 64 columns are kept, lane 0 also pair 32) counted from the even position at or below pos0: one
-        // 4-byte store per row, a 2-byte store where only one member of the pair belongs to this block.  Everything that
-        // does not change from row to row is worked out here: the loop body is two shared-memory loads, a merge, the stores.
-        const int base_even = pos0 & ~1;
-        const int j_lo = base_even + 2 * lane - pos0, j_hi = j_lo + 1;  // positions of the pair inside this block's list
-        const bool has_lo = j_lo >= 0 && j_lo < cnt, has_hi = j_hi < cnt;   // (j_hi >= 0 always)
-        const uint32_t o_lo = has_lo ? (uint32_t)s_own[j_lo] * 2u : 0u, o_hi = has_hi ? (uint32_t)s_own[j_hi] * 2u : 0u;
-        const bool st_pair = has_lo && has_hi, st_lo = has_lo && !has_hi, st_hi = has_hi && !has_lo;
-        const bool extra = lane == 0 && base_even + 64 < pos0 + cnt;          // pair 32 holds the 64th kept column
-        const uint32_t o_extra = extra ? (uint32_t)s_own[cnt - 1] * 2u : 0u;
-        const int64_t row_step = kGatherWarps * fa.ldp;                       // elements between two rows of this warp
-        unsigned short *dwarp = reinterpret_cast<unsigned short *>(fa.Ap) + (int64_t)warp * fa.ldp + base_even + 2 * lane;
+        // ---- 4. own kept columns of A -> Ap.  What bounds this step is the number of store requests that reach L2 (about
+        // 64 G requests/s over the whole GPU, however few bytes each carries), so a block issues exactly one per row: lane l
+        // stores the 4-byte word at the even list position e = pos0 rounded up to even, plus 2 l.  If the block's range
+        // starts at an odd position, its first element belongs to the previous block's last word and that block writes
+        // it; if the range ends at an odd position, the last word's upper half is the next kept column of A (outside this
+        // block's tiles): the warp fetches that element for its rows of the next step from A itself (2-byte loads, L2).
+        const int e0 = pos0 + (pos0 & 1);
+        const int j_lo = e0 + 2 * lane - pos0, j_hi = j_lo + 1;               // positions inside this block's list
+        const bool st_pair = j_lo < cnt;                                       // (j_lo >= 0 always)
+        const bool hi_own = j_hi < cnt;
+        const bool has_partner = ((pos0 + cnt) & 1) != 0;                      // the last word's upper half is not this block's
+        const uint32_t o_lo = st_pair ? (uint32_t)s_own[j_lo] * 2u : 0u, o_hi = hi_own ? (uint32_t)s_own[j_hi] * 2u : 0u;
+        const int next_col = s_next;                                           // -1: the list ends here (the half is padding)
+        const int64_t row_step = kGatherWarps * fa.ldp;                        // elements between two rows of this warp
+        unsigned short *dwarp = reinterpret_cast<unsigned short *>(fa.Ap) + (int64_t)warp * fa.ldp + e0 + 2 * lane;
+        const unsigned short *a16 = reinterpret_cast<const unsigned short *>(a.A);
+        // lane p < 16 holds the partner element of the warp's p-th row of the current step
+        auto partner = [&](int tile) -> unsigned short {
+            const int64_t row = (int64_t)tile * kTmaRows + warp + kGatherWarps * lane;
+            return (has_partner && next_col >= 0 && lane < kTmaRows / kGatherWarps && row < a.m) ? __ldg(a16 + row * a.s_red + next_col)
+                                                                                                 : (unsigned short)0;
+        };
+        auto tile_of_step = [&](int t) { return t < resident ? n_tiles - resident + t : t - resident; };
+        unsigned short pv_next = n_tiles > 0 ? partner(tile_of_step(0)) : (unsigned short)0;
         // Step t < resident works on the tile the stream left in the ring (no copy, nothing to wait for); later steps
         // work on tiles 0, 1, ... copied again (from L2 when A is small) into the slots in the order they were released,
         // requested two steps after the release.
@@ -644,23 +671,25 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
             if (t >= resident && !wait_full(st)) { ok = false; break; }
             const int64_t left = a.m - (int64_t)tile * kTmaRows - warp;      // rows of this tile at or below the warp's first
             const int np = left <= 0 ? 0 : (int)min((int64_t)(kTmaRows / kGatherWarps), (left + kGatherWarps - 1) / kGatherWarps);
-            uint32_t row_s = ring + st * kTmaStageBytes + (uint32_t)warp * (kTmaCols * 2);
+            const unsigned pv = pv_next;
+            if (t + 1 < n_tiles) pv_next = partner(tile_of_step(t + 1));     // in flight while this tile is gathered
+            const unsigned char *row_g = s_dyn + st * kTmaStageBytes + warp * (kTmaCols * 2);
+            constexpr int S = kGatherWarps * kTmaCols * 2;                   // bytes between two rows of this warp in the tile
             unsigned short *d = dwarp + (int64_t)tile * kTmaRows * fa.ldp;
-#pragma unroll 4
-            for (int p = 0; p < np; ++p) {
-                unsigned short v0, v1;
-                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v0) : "r"(row_s + o_lo));
-                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v1) : "r"(row_s + o_hi));
-                if (st_pair) *reinterpret_cast<unsigned *>(d) = (unsigned)v0 | ((unsigned)v1 << 16);
-                if (st_lo) d[0] = v0;
-                if (st_hi) d[1] = v1;
-                if (extra) {
-                    unsigned short v2;
-                    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v2) : "r"(row_s + o_extra));
-                    d[64] = v2;
+            for (int p0 = 0; p0 < np; p0 += 4) {                             // four rows at a time: loads first, then stores
+                unsigned w[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int p = p0 + i < np ? p0 + i : np - 1;
+                    const unsigned lo = *reinterpret_cast<const unsigned short *>(row_g + p * S + o_lo);
+                    const unsigned hi_o = *reinterpret_cast<const unsigned short *>(row_g + p * S + o_hi);
+                    const unsigned hi_p = __shfl_sync(0xffffffffu, pv, p);
+                    w[i] = lo | ((hi_own ? hi_o : hi_p) << 16);
                 }
-                row_s += kGatherWarps * kTmaCols * 2;
-                d += row_step;
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (st_pair && p0 + i < np) *reinterpret_cast<unsigned *>(d + i * row_step) = w[i];
+                d += 4 * row_step;
             }
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(st)) : "memory");
