@@ -1,11 +1,12 @@
 #!/usr/bin/env python
 """Benchmark of the RMM hot path on B200.
 
-A step is one pass of the whole hot path over one product: fused score + top-k select on A, then the
-reduced product Y = A[:, I] B[I, :] (gathers included).  Workload at N = 1: the 1B-class MLP down
-projection (A 2048 x 8192 activations with 1 % heavy-tailed channels, B 8192 x 2048 weight, bf16), headline
-retention ratio rho = 0.5; the other ratios are reported in `per_rho`.  With N > 1 every rank runs the
-same workload on its own GPU (independent replicas, no data-path collective).
+A step is one pass of the whole hot path over one product: scores of A, top-k selection, gathers and the
+reduced product Y = A[:, I] B[I, :] (rmm_product).  Workload at N = 1: the 70B-class MLP down projection, the
+largest single-GPU product of the benchmark configurations (A 32768 tokens x 28672 intermediate activations
+with 1 % heavy-tailed channels, B 28672 x 8192 weight, bf16), headline retention ratio rho = 0.5; the other
+ratios, the 1B-class product (2048 x 8192 x 2048) and the other 70B-class products are reported beside it.
+With N > 1 every rank runs the same workload on its own GPU (independent replicas, no data-path collective).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
@@ -16,6 +17,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -28,21 +30,27 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-M, K, N = 2048, 8192, 2048
+M, K, N = 32768, 28672, 8192          # headline product: 70B-class down projection
+M1, K1, N1 = 2048, 8192, 2048         # the 1B-class down projection (reported in `mlp_1b`)
 RHO = 0.5
 RHOS = (0.25, 0.5, 0.75, 1.0)
 METRIC = "reduced-GEMM retained TFLOP/s (whole RMM op: score + select + reduced product)"
 UNIT = "TFLOP/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the GEMM kernel on this workload at rho = 0.5, from the
-# ncu capture summarised in profiles/reduced_gemm_tc_kernel_mlp_2048x8192x2048_rho0.5.md
-GEMM_DRAM_TRAFFIC_BYTES = 33.67e6
-WORKLOAD = "1B-class MLP down-projection: A 2048x8192 bf16 N(0,1) with 1% Student-t(3) channels, B 8192x2048 bf16 N(0,0.02^2)"
+NOMINAL_BF16_TFLOPS = 2250.0          # dense bf16 tensor peak of a B200 as specified (context beside the measured peaks)
+NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the GEMM kernel on the headline workload at rho = 0.5,
+# from the one-pass ncu capture summarised in profiles/reduced_gemm_tc_kernel_down_proj_32768x28672x8192_rho0.5.md
+GEMM_DRAM_TRAFFIC_BYTES = None
+WORKLOAD = ("70B-class MLP down-projection: A 32768x28672 bf16 N(0,1) with 1% Student-t(3) channels, "
+            "B 28672x8192 bf16 N(0,0.02^2)")
 
 
-def retained_flops(rho: float) -> float:
-    import math
-    k = max(1, math.ceil(rho * K - 1e-9))
-    return 2.0 * M * k * N
+def keep(rho: float, k_axis: int) -> int:
+    return max(1, math.ceil(rho * k_axis - 1e-9))
+
+
+def retained_flops(rho: float, m: int = M, k_axis: int = K, n: int = N) -> float:
+    return 2.0 * m * keep(rho, k_axis) * n
 
 
 def measured_peaks():
@@ -144,6 +152,22 @@ def whole_job_value(ms_step: float, world: int, rho: float = RHO) -> float:
     return world * retained_flops(rho) / (ms_step * 1e-3) / 1e12
 
 
+def gemm_roofline(achieved_tflops: float, kernel_ms: float, peaks: dict, clocks: dict, traffic):
+    """Roofline entry of the tensor-core GEMM.  The denominator is the measured cuBLAS bf16 rate that matches the clocks
+    the kernel actually ran at: the sustained figure when the SM clock sampled during the timed region sagged under the
+    power cap (median below 85 % of the maximum), the burst figure otherwise."""
+    sm, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    sagged = bool(sm and mx and sm < 0.85 * mx)
+    peak = peaks["bf16_sustained"] if sagged else peaks["bf16_burst"]
+    return {"bound": "tensor", "kernel": "reduced_gemm_tc_kernel", "achieved": achieved_tflops, "peak": peak, "unit": "TFLOP/s",
+            "frac": achieved_tflops / peak, "traffic": traffic,
+            "peak_source": f"{peaks['source']} cuBLAS bf16, {'sustained (SM clock sagged under load)' if sagged else 'burst (SM clock stayed near maximum)'}",
+            "frac_of_burst_peak": achieved_tflops / peaks["bf16_burst"],
+            "frac_of_sustained_peak": achieved_tflops / peaks["bf16_sustained"],
+            "frac_of_nominal_peak": achieved_tflops / NOMINAL_BF16_TFLOPS,
+            "kernel_ms": kernel_ms, "sm_mhz_x_kernel_ms": (sm * kernel_ms) if sm else None}
+
+
 def time_region(fn, steps: int, world: int) -> float:
     """ms per step over exactly `steps` calls, device-timed, barrier + synchronize on both sides, max over ranks."""
     barrier(world)
@@ -156,57 +180,65 @@ def time_region(fn, steps: int, world: int) -> float:
     return max_over_ranks(e0.elapsed_time(e1), world) / steps
 
 
-def cpu_oracle_sample(A, B, rho: float, target_s: float = 12.0):
-    """Time the oracle as it stands (score + select at full size, product on a sample of rows)."""
+def cpu_oracle_sample(A_rows, B, rho: float, m_total: int, target_s: float = 12.0):
+    """Time the oracle as it stands on a bounded sample of the headline workload: the score pass on `A_rows` (a slice of
+    the activations), the selection at full width, the product on as many of those rows as fit the time target.  The
+    whole-workload figure is an extrapolation to all m_total rows (score and product are row-separable) and says so."""
     import oracle
     oracle.build()
     cores = oracle.num_threads()
+    R, k_axis = A_rows.shape
+    n = B.shape[1]
     t0 = time.perf_counter()
-    e, _ = oracle.score(A)
-    idx, _ = oracle.select(e, oracle.keep_count(rho, A.shape[1]))
+    e, _ = oracle.score(A_rows)
+    t_score = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    idx, _ = oracle.select(e, oracle.keep_count(rho, k_axis))
     t_sel = time.perf_counter() - t0
-    probe = min(M, 4 * cores)
+    probe = min(R, cores)
     t0 = time.perf_counter()
-    oracle.reduced_gemm(A, B, idx, rows=(0, probe))
+    oracle.reduced_gemm(A_rows, B, idx, rows=(0, probe))
     t_probe = time.perf_counter() - t0
-    rows = int(max(probe, min(M, target_s / max(t_probe / probe, 1e-9))))
+    rows = int(max(probe, min(R, target_s / max(t_probe / probe, 1e-9))))
     rows = max(cores, rows // cores * cores)
     t0 = time.perf_counter()
-    oracle.reduced_gemm(A, B, idx, rows=(0, rows))
+    oracle.reduced_gemm(A_rows, B, idx, rows=(0, rows))
     t_rows = time.perf_counter() - t0
-    # whole-op time for the sampled rows: the score/select pass is charged in proportion to the rows kept
-    t = t_rows + t_sel * rows / M
-    flops = 2.0 * rows * len(idx) * N
-    return {"value": flops / t / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"score+select on the full {M}x{K} A ({t_sel:.3f} s, charged pro rata), product on rows 0..{rows - 1} of {M} "
-                      f"at rho={rho} ({t_rows:.2f} s)", "seconds": t_rows + t_sel}
+    # time of the whole workload, extrapolated: score on m_total rows, one selection, product on m_total rows
+    t_full = t_score * m_total / R + t_sel + t_rows * m_total / rows
+    flops = 2.0 * m_total * len(idx) * n
+    return {"value": flops / t_full / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"extrapolated from a sample: score on {R} of {m_total} rows ({t_score:.2f} s), selection over {k_axis} keys "
+                      f"({t_sel:.3f} s), product on {rows} rows at rho={rho} ({t_rows:.2f} s); whole workload would take {t_full:.0f} s",
+            "seconds": t_score + t_sel + t_probe + t_rows}
 
 
 def run_reference(args):
-    """Reference arm: the CPU oracle, timed on this machine's host cores; rank 0 only."""
+    """Reference arm: the CPU oracle, timed on this machine's host cores; rank 0 only.  Every step is a bounded sample of the
+    headline workload: score, selection and product on `cores` rows of activations of the same width."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from paper_2608_13426_b200 import synth
-    A, B = synth.mlp_product(M, K, N, seed=0)
     import oracle
     oracle.build()
     cores = oracle.num_threads()
-    e, _ = oracle.score(A)
-    idx, _ = oracle.select(e, oracle.keep_count(RHO, K))
-    rows = cores                             # bounded sample per step: one row per thread
+    rows = cores                             # one row per thread
+    A = synth.heavy_tailed_activations(rows, K, seed=0)
+    B = synth.weight(K, N, seed=1)
+    k = oracle.keep_count(RHO, K)
     times = []
     for i in range(args.warmup + args.steps):
         t0 = time.perf_counter()
-        e, _ = oracle.score(A[: max(rows, 1)])          # score pass on the same row sample
-        oracle.select(e, len(idx))
+        e, _ = oracle.score(A)
+        idx, _ = oracle.select(e, k)
         oracle.reduced_gemm(A, B, idx, rows=(0, rows))
         dt = time.perf_counter() - t0
         if i >= args.warmup:
             times.append(dt)
     ms = 1e3 * sum(times) / len(times)
-    val = 2.0 * rows * len(idx) * N / (ms / 1e3) / 1e12
-    sample = f"rows 0..{rows - 1} of {M} per step (score, select and product on that sample), rho={RHO}"
+    val = 2.0 * rows * k * N / (ms / 1e3) / 1e12
+    sample = f"{rows} rows of {M} per step (score, selection and product on that sample), rho={RHO}"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -264,15 +296,15 @@ def layer_sweep_70b(rmm, synth, dev, peaks, tokens=32768, hidden=8192, inter=286
             idx = torch.empty(k, dtype=torch.int32, device=dev)
 
             def op(i):
-                rmm.rmm_score_select(A, rho=rho, idx=idx)
-                rmm.rmm_reduced_gemm(A, B, idx, out=Y)
+                rmm.rmm_product(A, B, rho=rho, out=Y, idx=idx)
 
             op(0)
             op(1)
             t = time_region(op, reps, 1)
             fl = 2.0 * m * k * n
             rows.append({"layer": name, "shape": [m, kk, n], "rho": rho, "whole_op_ms": t, "whole_op_tflops": fl / t / 1e9,
-                         "frac_of_sustained_peak": fl / t / 1e9 / peaks["bf16_sustained"]})
+                         "frac_of_sustained_peak": fl / t / 1e9 / peaks["bf16_sustained"],
+                         "frac_of_burst_peak": fl / t / 1e9 / peaks["bf16_burst"]})
         # the dense product is timed before and after the sweep (the clocks sag under sustained tensor load): mean of both
         dense_after = time_region(lambda i: torch.matmul(A, B, out=Y), reps, 1)
         dense = 0.5 * (dense_before + dense_after)
@@ -364,15 +396,66 @@ def run_attention_only(args):
     print(json.dumps({"attention_prefill": res}))
 
 
+def small_product_sweep(rmm, binding, synth, dev, peaks, rank, reps=40, n_sets=5):
+    """The 1B-class down projection (A 2048 x 8192, B 8192 x 2048): whole op per rho through rmm_product (one front-end
+    launch + the product), its kernels, dense cuBLAS at the same shape and cuBLAS on operands gathered beforehand.
+    Five (A, B, Y) sets (377 MB, above L2) are rotated."""
+    sets = []
+    for s_ in range(n_sets):
+        A, B = synth.mlp_product(M1, K1, N1, seed=100 * rank + s_)
+        sets.append((A.to(dev), B.to(dev), torch.empty(M1, N1, dtype=torch.bfloat16, device=dev)))
+    for i in range(5):
+        torch.matmul(sets[i % n_sets][0], sets[i % n_sets][1], out=sets[i % n_sets][2])
+    dense_ms = time_region(lambda i: torch.matmul(sets[i % n_sets][0], sets[i % n_sets][1], out=sets[i % n_sets][2]), reps, 1)
+    out = []
+    for rho in RHOS:
+        kk = rmm.rmm_keep_count(rho, K1)
+        idx_r = torch.empty(kk, dtype=torch.int32, device=dev)
+
+        def step(i):
+            A, B, Y = sets[i % n_sets]
+            rmm.rmm_product(A, B, rho=rho, out=Y, idx=idx_r)
+
+        for i in range(3):
+            step(i)
+        whole = time_region(step, reps, 1)
+        kt = binding.KernelTimer(4 * reps)
+        with kt:
+            for i in range(reps):
+                step(i)
+        parts = {}
+        for name, x in kt.times_ms():
+            parts.setdefault(name, []).append(1e3 * x)
+        parts = {name: sum(v) / reps for name, v in parts.items()}      # us per step, launch gaps included
+        g = parts.get("reduced_gemm_tc_kernel", float("nan")) * 1e-3
+        front = sum(v for name, v in parts.items() if name != "reduced_gemm_tc_kernel") * 1e-3
+        pre = [(a_[:, idx_r.long()].contiguous(), b_[idx_r.long()].contiguous(), y_) for a_, b_, y_ in sets]
+        for i in range(3):
+            torch.matmul(pre[i % n_sets][0], pre[i % n_sets][1], out=pre[i % n_sets][2])
+        ideal = time_region(lambda i: torch.matmul(pre[i % n_sets][0], pre[i % n_sets][1], out=pre[i % n_sets][2]), reps, 1)
+        del pre
+        fl = retained_flops(rho, M1, K1, N1)
+        out.append({"rho": rho, "k": kk, "shape": [M1, K1, N1], "whole_op_ms": whole, "whole_op_tflops": fl / whole / 1e9,
+                    "kernels_us_event_bracketed": parts,
+                    "gemm_kernel_ms": g, "gemm_kernel_tflops": fl / g / 1e9,
+                    "gemm_frac_of_burst_peak": fl / g / 1e9 / peaks["bf16_burst"],
+                    "gemm_frac_of_sustained_peak": fl / g / 1e9 / peaks["bf16_sustained"],
+                    "gemm_frac_of_nominal_peak": fl / g / 1e9 / NOMINAL_BF16_TFLOPS,
+                    "front_end_ms": front, "front_end_gbs": M1 * K1 * 2 / front / 1e6 if front > 0 else None,
+                    "front_end_frac_of_hbm": M1 * K1 * 2 / front / 1e6 / peaks["hbm_gbs"] if front > 0 else None,
+                    "cublas_on_pregathered_ms": ideal, "dense_cublas_ms": dense_ms, "speedup_vs_dense_cublas": dense_ms / whole})
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU oracle timing (quick runs, profiling)")
-    ap.add_argument("--no-sweep", action="store_true", help="skip the per-rho sweep")
-    ap.add_argument("--sets", type=int, default=5, help="independent (A, B, Y) input sets rotated per step (5 = 377 MB, above L2)")
+    ap.add_argument("--no-sweep", action="store_true", help="skip everything but the headline step (quick runs, profiling)")
+    ap.add_argument("--rows", type=int, default=M, help="rows of the headline product (smaller: profiler captures)")
     ap.add_argument("--attention-only", action="store_true",
                     help="run only the reduced-attention case (a few launches: for profiler captures) and print its own JSON line")
     ap.add_argument("--attn-heads", type=int, default=32)
@@ -391,33 +474,28 @@ def main():
     rank, world, local = dist_setup(args.gpus)
     dev = torch.device("cuda", local if world > 1 else 0)
     peaks = measured_peaks()
+    m = args.rows
 
-    # ---- inputs: several independent (A, B, Y) sets, together well above the 126 MB L2, rotated per step
-    n_sets = max(1, args.sets)
-    sets = []
-    for s in range(n_sets):
-        A, B = synth.mlp_product(M, K, N, seed=100 * rank + s)
-        sets.append((A.to(dev), B.to(dev), torch.empty(M, N, dtype=torch.bfloat16, device=dev)))
-    A0_cpu, B0_cpu = synth.mlp_product(M, K, N, seed=0)
-    resident_bytes = n_sets * (M * K + K * N + M * N) * 2
+    # ---- inputs, resident in HBM before the timed region: A 1.88 GB, B 470 MB, Y 537 MB (far above the 126 MB L2)
+    A = synth.heavy_tailed_activations(m, K, seed=100 * rank, device=str(dev))
+    B = synth.weight(K, N, seed=100 * rank + 1, device=str(dev))
+    Y = torch.empty(m, N, dtype=torch.bfloat16, device=dev)
     k = rmm.rmm_keep_count(RHO, K)
     idx_buf = torch.empty(k, dtype=torch.int32, device=dev)
+    resident_bytes = (m * K + K * N + m * N) * 2
 
     def step(i, rho=RHO, idx=idx_buf):
-        A, B, Y = sets[i % n_sets]
-        rmm.rmm_score_select(A, rho=rho, idx=idx)
-        rmm.rmm_reduced_gemm(A, B, idx, out=Y)
+        rmm.rmm_product(A, B, rho=rho, out=Y, idx=idx)
 
     for i in range(args.warmup):
         step(i)
     torch.cuda.synchronize()
     assert rmm.rmm_status_read() == 0
 
-    # ---- timed region: exactly K steps; the GEMM kernel of every step is bracketed by events on the same stream
+    # ---- timed region: exactly K steps; every GEMM launch is bracketed by events on the same stream (a step lasts
+    # milliseconds, so the event records cost nothing measurable)
     sampler = ClockSampler(local if world > 1 else 0)
-    # one GEMM launch in 8 is bracketed by events: event records between kernels cost launch overlap (about 6 us per
-    # step when every launch is bracketed)
-    timer = binding.KernelTimer(min(args.steps, 4096), "reduced_gemm_tc_kernel", every=8)
+    timer = binding.KernelTimer(min(args.steps, 4096), "reduced_gemm_tc_kernel")
     launches0 = rmm.rmm_launch_count()
     sampler.start()
     with timer:
@@ -427,70 +505,94 @@ def main():
     gemm_ms = [t for _, t in timer.times_ms()]
     gemm_ms_avg = sum(gemm_ms) / len(gemm_ms)
     assert rmm.rmm_status_read() == 0
-    value = whole_job_value(ms_step, world)
+    flops_step = retained_flops(RHO, m, K, N)
+    value = world * flops_step / (ms_step * 1e-3) / 1e12
 
     # ---- roofline of the dominant kernel (the tensor-core GEMM): retained FLOPs of one launch / its mean duration
-    achieved = retained_flops(RHO) / (gemm_ms_avg * 1e-3) / 1e12
-    traffic = GEMM_DRAM_TRAFFIC_BYTES
-    roofline = {"bound": "tensor", "kernel": "reduced_gemm_tc_kernel", "achieved": achieved, "peak": peaks["bf16_sustained"],
-                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": traffic,
-                "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step loop)",
-                "frac_of_burst_peak": achieved / peaks["bf16_burst"], "kernel_ms": gemm_ms_avg}
+    achieved = flops_step / (gemm_ms_avg * 1e-3) / 1e12
+    roofline = gemm_roofline(achieved, gemm_ms_avg, peaks, clocks, GEMM_DRAM_TRAFFIC_BYTES if m == M else None)
 
-    # ---- end to end: host buffers in, host buffer out, through the C-ABI host entry point
-    Ah, Bh = A0_cpu.pin_memory(), B0_cpu.pin_memory()
-    Yh = torch.empty(M, N, dtype=torch.bfloat16).pin_memory()
-    ih = torch.empty(K, dtype=torch.int32).pin_memory()
+    # ---- per-kernel breakdown of one step (a separate, untimed pass with every launch bracketed by events)
+    breakdown = {}
+    if rank == 0:
+        nb = 5
+        kt = binding.KernelTimer(nb * 8)
+        with kt:
+            for i in range(nb):
+                step(i)
+        for name, t in kt.times_ms():
+            breakdown.setdefault(name, []).append(t)
+        breakdown = {name: {"launches_per_step": len(v) / nb, "mean_ms": sum(v) / len(v)} for name, v in breakdown.items()}
+        sel_ms = sum(v["mean_ms"] * v["launches_per_step"] for name, v in breakdown.items() if name in ("score_tma_kernel", "select_kernel", "score_select_kernel"))
+        if sel_ms > 0:
+            gbs = m * K * 2 / sel_ms / 1e6
+            breakdown["selection_pass"] = {"ms": sel_ms, "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
+                                           "frac_of_nominal_hbm": gbs / NOMINAL_HBM_GBS}
 
-    def step_e2e(i):
-        rmm.rmm_product_host(Ah, Bh, RHO, Yh, ih)
-        torch.cuda.current_stream().synchronize()      # the caller reads Y_host after every step
-
-    for i in range(3):
-        step_e2e(i)
-    e2e_steps = max(5, min(args.steps, 50))
-    ms_e2e = time_region(step_e2e, e2e_steps, world)
-    e2e = {"value": world * retained_flops(RHO) / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e, "steps": e2e_steps,
-           "h2d_bytes_per_step": (M * K + K * N) * 2, "d2h_bytes_per_step": M * N * 2 + k * 4}
-
-    # ---- per-rho sweep: whole op, its parts, dense cuBLAS at the same shape
+    # ---- per-rho sweep on the headline product: whole op beside dense cuBLAS at the same shape
     per_rho = []
     if not args.no_sweep and rank == 0:
-        reps = 40
-        for i in range(5):
-            torch.matmul(sets[i % n_sets][0], sets[i % n_sets][1], out=sets[i % n_sets][2])
-        dense_ms = time_region(lambda i: torch.matmul(sets[i % n_sets][0], sets[i % n_sets][1], out=sets[i % n_sets][2]), reps, 1)
+        reps = 5
+        for _ in range(2):
+            torch.matmul(A, B, out=Y)
+        dense_before = time_region(lambda i: torch.matmul(A, B, out=Y), reps, 1)
         for rho in RHOS:
             kk = rmm.rmm_keep_count(rho, K)
             idx_r = torch.empty(kk, dtype=torch.int32, device=dev)
-            for i in range(3):
+            for i in range(2):
                 step(i, rho, idx_r)
             whole = time_region(lambda i: step(i, rho, idx_r), reps, 1)
             t = binding.KernelTimer(reps, "reduced_gemm_tc_kernel")
             with t:
                 time_region(lambda i: step(i, rho, idx_r), reps, 1)
             g = sum(x for _, x in t.times_ms()) / reps
-            sel = time_region(lambda i: rmm.rmm_score_select(sets[i % n_sets][0], rho=rho, idx=idx_r), reps, 1)
-            # ceiling: cuBLAS on operands gathered beforehand (the gather is not timed)
-            pre = [(a_[:, idx_r.long()].contiguous(), b_[idx_r.long()].contiguous(), y_) for a_, b_, y_ in sets]
-            for i in range(3):
-                torch.matmul(pre[i % n_sets][0], pre[i % n_sets][1], out=pre[i % n_sets][2])
-            ideal = time_region(lambda i: torch.matmul(pre[i % n_sets][0], pre[i % n_sets][1], out=pre[i % n_sets][2]), reps, 1)
-            del pre
-            fl = retained_flops(rho)
+            fl = retained_flops(rho, m, K, N)
             per_rho.append({"rho": rho, "k": kk, "whole_op_ms": whole, "whole_op_tflops": fl / whole / 1e9,
                             "gemm_kernel_ms": g, "gemm_kernel_tflops": fl / g / 1e9,
                             "gemm_frac_of_sustained_peak": fl / g / 1e9 / peaks["bf16_sustained"],
                             "gemm_frac_of_burst_peak": fl / g / 1e9 / peaks["bf16_burst"],
-                            "score_select_ms": sel, "score_select_gbs": M * K * 2 / sel / 1e6,
-                            "score_select_frac_of_hbm": M * K * 2 / sel / 1e6 / peaks["hbm_gbs"],
-                            "cublas_on_pregathered_ms": ideal,
-                            "dense_cublas_ms": dense_ms, "speedup_vs_dense_cublas": dense_ms / whole})
+                            "gemm_frac_of_nominal_peak": fl / g / 1e9 / NOMINAL_BF16_TFLOPS})
+        dense_after = time_region(lambda i: torch.matmul(A, B, out=Y), reps, 1)
+        dense_ms = 0.5 * (dense_before + dense_after)      # the clocks sag under sustained tensor load: mean of both
+        for r in per_rho:
+            r.update({"dense_cublas_ms": dense_ms, "dense_cublas_ms_before_after": [dense_before, dense_after],
+                      "dense_cublas_tflops": 2.0 * m * K * N / dense_ms / 1e9, "speedup_vs_dense_cublas": dense_ms / r["whole_op_ms"]})
 
-    # ---- the selection pass on a 70B-class activation (32768 tokens x 8192 hidden, 537 MB): the same kernel where it is
-    # bandwidth-bound rather than latency-bound (the benchmark product's 33.6 MB input is too small to show it)
-    selection_large = None
+    # ---- CPU oracle on a bounded sample of the same workload (rank 0, one GPU only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_oracle_sample(A[:1024].cpu(), B.cpu(), RHO, m)
+
+    # ---- end to end: host buffers in, host buffer out, through the C-ABI host entry point (copies inside the timed region)
+    Ah = torch.empty(m, K, dtype=torch.bfloat16).pin_memory()
+    Bh = torch.empty(K, N, dtype=torch.bfloat16).pin_memory()
+    Ah.copy_(A)
+    Bh.copy_(B)
+    Yh = torch.empty(m, N, dtype=torch.bfloat16).pin_memory()
+    ih = torch.empty(K, dtype=torch.int32).pin_memory()
+    del A, B, Y
+    torch.cuda.empty_cache()
+
+    def step_e2e(i):
+        rmm.rmm_product_host(Ah, Bh, RHO, Yh, ih)
+        torch.cuda.current_stream().synchronize()      # the caller reads Y_host after every step
+
+    for i in range(2):
+        step_e2e(i)
+    e2e_steps = max(3, min(args.steps, 5))
+    ms_e2e = time_region(step_e2e, e2e_steps, world)
+    e2e = {"value": world * flops_step / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e, "steps": e2e_steps,
+           "h2d_bytes_per_step": (m * K + K * N) * 2, "d2h_bytes_per_step": m * N * 2 + k * 4}
+    del Ah, Bh, Yh
+    binding._ws_cache.clear()
+    torch.cuda.empty_cache()
+
+    extras = {}
     if not args.no_sweep and rank == 0:
+        # ---- the 1B-class product (where launch and selection latencies matter most)
+        extras["mlp_1b"] = small_product_sweep(rmm, binding, synth, dev, peaks, rank)
+
+        # ---- the selection pass on a 70B-class activation (32768 tokens x 8192 hidden, 537 MB): bandwidth-bound
         Ml, Kl = 32768, 8192
         big = [synth.heavy_tailed_activations(Ml, Kl, seed=50 + i, device=str(dev)) for i in range(2)]
         idx_l = torch.empty(rmm.rmm_keep_count(RHO, Kl), dtype=torch.int32, device=dev)
@@ -498,13 +600,12 @@ def main():
             rmm.rmm_score_select(big[i % 2], rho=RHO, idx=idx_l)
         t = time_region(lambda i: rmm.rmm_score_select(big[i % 2], rho=RHO, idx=idx_l), 20, 1)
         gbs = Ml * Kl * 2 / t / 1e6
-        selection_large = {"shape": [Ml, Kl], "ms": t, "gbs": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
-                           "note": "fused score + top-k select, two alternating 537 MB inputs (above L2)"}
+        extras["selection_pass_large"] = {"shape": [Ml, Kl], "ms": t, "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
+                                          "frac_of_nominal_hbm": gbs / NOMINAL_HBM_GBS,
+                                          "note": "fused score + top-k select, two alternating 537 MB inputs (above L2)"}
         del big
 
-    # ---- decode step (one activation row) on a 70B-class gate/up projection: the gathered GEMV reads only the kept rows
-    decode = None
-    if not args.no_sweep and rank == 0:
+        # ---- decode step (one activation row) on a 70B-class gate/up projection: the gathered GEMV reads only the kept rows
         Kd, Nd = 8192, 28672
         Ws = [synth.weight(Kd, Nd, seed=70 + i, device=str(dev)) for i in range(3)]     # 3 x 470 MB, rotated
         x = synth.heavy_tailed_activations(1, Kd, seed=73, device=str(dev))
@@ -521,8 +622,6 @@ def main():
             gbs = idx_d.numel() * Nd * 2 / t / 1e6
             decode.append({"rho": rho, "shape": [1, Kd, Nd], "reduced_gemv_ms": t, "kept_rows_gbs": gbs,
                            "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "dense_cublas_ms": dense, "speedup_vs_dense": dense / t})
-        # small decode batches (2 .. 128 rows): up to 4 rows the gathered GEMV, above it the tensor-core kernel that
-        # fetches the kept rows of W itself (no packed copy of W); rho = 0.5
         for Mb in (4, 16, 64, 128):
             xb = synth.heavy_tailed_activations(Mb, Kd, seed=74, device=str(dev))
             yb = torch.empty(Mb, Nd, dtype=torch.bfloat16, device=dev)
@@ -536,47 +635,27 @@ def main():
             decode.append({"rho": 0.5, "shape": [Mb, Kd, Nd], "reduced_product_ms": t, "kept_rows_gbs": gbs,
                            "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "dense_cublas_ms": dn, "speedup_vs_dense": dn / t})
         del Ws
+        extras["decode_step"] = decode
 
-    # ---- reduced attention on a 7B-class prefill (32 heads, 4096 tokens, head_dim 128, causal)
-    attention = table5 = framed = None
-    if not args.no_sweep and rank == 0:
-        attention = attention_case(rmm, binding, synth, dev, 32, 4096)
-        table5 = paper_table5_case(rmm, synth, dev)
-        framed = gemm_framed_attention(rmm, synth, dev, peaks)
+        # ---- reduced attention on a 7B-class prefill, the paper's kernel-latency setting, the attention products as GEMMs
+        extras["attention_prefill"] = attention_case(rmm, binding, synth, dev, 32, 4096)
+        extras["attention_paper_setting"] = paper_table5_case(rmm, synth, dev)
+        extras["attention_products_in_memory"] = gemm_framed_attention(rmm, synth, dev, peaks)
 
-    # ---- 70B-class layer (hidden 8192, intermediate 28672, 64 query / 8 kv heads, 32768 prefill tokens): every
-    # projection at every rho beside dense cuBLAS, and the attention of one layer
-    layer70 = None
-    if not args.no_sweep and rank == 0:
-        layer70 = layer_sweep_70b(rmm, synth, dev, peaks)
-
-    # ---- per-kernel breakdown of one step (a separate, untimed pass with every launch bracketed by events)
-    breakdown = {}
-    if rank == 0:
-        nb = 20
-        kt = binding.KernelTimer(nb * 8)
-        with kt:
-            for i in range(nb):
-                step(i)
-        for name, t in kt.times_ms():
-            breakdown.setdefault(name, []).append(t)
-        breakdown = {name: {"launches_per_step": len(v) / nb, "mean_us": 1e3 * sum(v) / len(v)} for name, v in breakdown.items()}
-
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu = cpu_oracle_sample(A0_cpu, B0_cpu, RHO)
+        # ---- the other 70B-class products and the attention of one layer
+        extras["layer_sweep_70b"] = layer_sweep_70b(rmm, synth, dev, peaks)
 
     if rank == 0:
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": {"workload": WORKLOAD, "rho": RHO, "k": k, "M": M, "K": K, "N": N, "parallelism": f"replicas x{world}",
-                       "l2_policy": f"inputs larger than L2: {n_sets} rotating (A, B, Y) sets, {resident_bytes / 1e6:.0f} MB resident"},
+            "config": {"workload": WORKLOAD, "rho": RHO, "k": k, "M": m, "K": K, "N": N, "parallelism": f"replicas x{world}",
+                       "l2_policy": f"inputs larger than L2: {resident_bytes / 1e9:.2f} GB of operands resident per GPU"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
-            "kernel_breakdown": breakdown, "per_rho": per_rho, "selection_pass_large": selection_large, "decode_step": decode,
-            "attention_prefill": attention, "attention_paper_setting": table5, "attention_products_in_memory": framed, "layer_sweep_70b": layer70, "peaks": peaks,
+            "kernel_breakdown": breakdown, "per_rho": per_rho, "peaks": peaks,
         }
+        out.update(extras)
         print(json.dumps(out))
     if world > 1:
         import torch.distributed as dist

@@ -128,6 +128,17 @@ size_t rmm_reduced_gemm_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, 
 int rmm_reduced_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
                      const rmm_mat_t *Y, void *ws, size_t ws_bytes, void *stream);
 
+/* rmm_reduced_gemm that also scores its output: energy_out fp32 [batch, N] receives sum_i Y[b, i, c]^2 of the outputs as
+ * stored (after rounding to bf16 when Y is bf16), i.e. the selection keys of the NEXT product that contracts over Y's
+ * columns, so that rmm_select can run on them without a score pass over Y (the paper's closing section names this joint
+ * treatment of selection and reduced multiplication as the way to cut memory movement).  On the tensor-core path with a
+ * bf16 Y the epilogue accumulates the sums while it holds the rounded tile (exact squares, fp32 chains of 16, 32-row
+ * groups added in fp64 in a fixed order: deterministic, about 1e-7 relative); every other form of the product runs
+ * rmm_score on Y afterwards.  Arguments otherwise as rmm_reduced_gemm. */
+size_t rmm_reduced_gemm_scored_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y);
+int rmm_reduced_gemm_scored(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
+                            const rmm_mat_t *Y, float *energy_out, void *ws, size_t ws_bytes, void *stream);
+
 /* Reduced attention of Sec. 3.3 for B sequences, Hq query heads, Hkv key/value heads (Hq % Hkv == 0,
  * query head h reads kv head h / (Hq/Hkv)).  Per (sequence, query head):
  *   I  = TopK of ||Q[:, j]||_2, |I| = ceil(rho_d Dh);  S~ = Q[:, I] K[:, I]^T / sqrt(Dh)  (full Dh in the scale)
@@ -174,9 +185,22 @@ size_t rmm_product_host_workspace_bytes(int64_t M, int64_t K, int64_t N);
 int rmm_product_host(const void *A_host, const void *B_host, int64_t M, int64_t K, int64_t N, double rho, int copy_B,
                      void *Y_host, int32_t *idx_host, void *ws, size_t ws_bytes, void *stream);
 
-/* Copy the device status word of a workspace to *device_status (an rmm_status_t) and clear it.
- * Synchronous: call it after the stream the workspace was used on has been synchronised. */
+/* Copy the device status word of a workspace to *device_status (an rmm_status_t) and clear it.  If the word was set,
+ * the whole header (the arrival counters too: a kernel that gave up may have left them half way) is zeroed, which
+ * makes the workspace usable again.  Synchronous: call it after the stream the workspace was used on has been
+ * synchronised. */
 int rmm_status_read(void *ws, int *device_status);
+
+/* Testing aid (the paper has no counterpart).  Every wait inside a kernel (on a copy, on another warp, on another block)
+ * is bounded: 2 s by default, RMM_SPIN_LIMIT_MS milliseconds if that environment variable is set when the library is
+ * first used.  rmm_debug_control("wait_limit_ms", x) overrides the bound for later launches (0 = back to the default);
+ * rmm_debug_control("withhold", w) makes block 0 of one kernel family never request its first tile (w = 1 tensor-core
+ * product, 2 score pass, 3 fused attention, 4 one-launch front end of rmm_product, 5 streaming column gather; 0 = off,
+ * -1 = back to the environment variable RMM_TEST_WITHHOLD = gemm | score | attn | front | pack), so that the waits behind
+ * that tile run out: the kernel must then report RMM_ERR_TIMEOUT in the status word, release what it holds and return.
+ * Results of such a call are undefined; rmm_status_read clears the workspace header, after which the workspace is
+ * usable again.  Not thread-safe against concurrent launches. */
+int rmm_debug_control(const char *key, double value);
 
 /* Timing hook for benchmarks (the paper has no counterpart).  After rmm_profile_kernels(start, stop, n, filter, every),
  * launches of library kernels whose name contains `name_filter` (NULL or "" = every kernel) are bracketed by

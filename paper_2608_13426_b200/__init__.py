@@ -8,6 +8,7 @@ from . import synth  # noqa: F401
 from .binding import (  # noqa: F401
     RmmError,
     rmm,
+    rmm_debug_control,
     rmm_keep_count,
     rmm_launch_count,
     rmm_product,

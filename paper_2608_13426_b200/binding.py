@@ -48,9 +48,10 @@ class rmm_attn_desc_t(ctypes.Structure):
 EXPORTS = ["rmm_keep_count", "rmm_score_workspace_bytes", "rmm_score", "rmm_select_workspace_bytes", "rmm_select",
            "rmm_score_select_workspace_bytes", "rmm_score_select", "rmm_score_select_static",
            "rmm_score_select_static_capacity", "rmm_score_select_static_status", "rmm_reduced_gemm_workspace_bytes",
-           "rmm_reduced_gemm", "rmm_reduced_attn_workspace_bytes", "rmm_reduced_attn",
+           "rmm_reduced_gemm", "rmm_reduced_gemm_scored_workspace_bytes", "rmm_reduced_gemm_scored",
+           "rmm_reduced_attn_workspace_bytes", "rmm_reduced_attn",
            "rmm_product_workspace_bytes", "rmm_product", "rmm_product_host_workspace_bytes", "rmm_product_host", "rmm_status_read", "rmm_last_error",
-           "rmm_launch_count", "rmm_profile_kernels", "rmm_profile_count", "rmm_profile_name"]
+           "rmm_launch_count", "rmm_debug_control", "rmm_profile_kernels", "rmm_profile_count", "rmm_profile_name"]
 
 _lib = None
 
@@ -82,6 +83,9 @@ def lib() -> ctypes.CDLL:
     L.rmm_reduced_gemm_workspace_bytes.argtypes = [mp, mp, i64, mp]
     L.rmm_reduced_gemm_workspace_bytes.restype = sz
     L.rmm_reduced_gemm.argtypes = [mp, mp, vp, i64, flt, mp, vp, sz, vp]
+    L.rmm_reduced_gemm_scored_workspace_bytes.argtypes = [mp, mp, i64, mp]
+    L.rmm_reduced_gemm_scored_workspace_bytes.restype = sz
+    L.rmm_reduced_gemm_scored.argtypes = [mp, mp, vp, i64, flt, mp, vp, vp, sz, vp]
     L.rmm_reduced_attn_workspace_bytes.argtypes = [ctypes.POINTER(rmm_attn_desc_t)]
     L.rmm_reduced_attn_workspace_bytes.restype = sz
     L.rmm_reduced_attn.argtypes = [ctypes.POINTER(rmm_attn_desc_t), vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -94,6 +98,7 @@ def lib() -> ctypes.CDLL:
     L.rmm_status_read.argtypes = [vp, ctypes.POINTER(i32)]
     L.rmm_last_error.restype = ctypes.c_char_p
     L.rmm_launch_count.restype = i64
+    L.rmm_debug_control.argtypes = [ctypes.c_char_p, dbl]
     L.rmm_profile_kernels.argtypes = [vp, vp, i32, ctypes.c_char_p, i32]
     L.rmm_profile_name.argtypes = [i32]
     L.rmm_profile_name.restype = ctypes.c_char_p
@@ -173,6 +178,12 @@ def rmm_keep_count(rho: float, K: int) -> int:
     k = ctypes.c_int64(0)
     _check(lib().rmm_keep_count(float(rho), int(K), ctypes.byref(k)))
     return int(k.value)
+
+
+def rmm_debug_control(key: str, value: float) -> None:
+    """Testing aid: "wait_limit_ms" bounds the device-side waits of later launches, "withhold" makes one kernel family's
+    block 0 skip its first tile request (see rmm.h)."""
+    _check(lib().rmm_debug_control(key.encode(), float(value)))
 
 
 def rmm_launch_count() -> int:
@@ -319,9 +330,10 @@ def rmm_score_select_static_status() -> int:
 
 def rmm_reduced_gemm(A: torch.Tensor, B: torch.Tensor, idx: Optional[torch.Tensor], scale: float = 1.0,
                      out: Optional[torch.Tensor] = None, out_dtype: Optional[torch.dtype] = None,
-                     ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+                     ws: Optional[torch.Tensor] = None, want_energy: bool = False):
     """Y = scale * A[:, idx] @ B[idx, :].  A [M,K] or [b,M,K]; B [K,N] or [b,K,N]; idx int32 [k] or [b,k]
-    (None: the unreduced product, k = K, nothing gathered)."""
+    (None: the unreduced product, k = K, nothing gathered).  want_energy: returns (Y, energy) with energy fp32 [N] or
+    [b, N] = column sums of squares of Y as stored (rmm_reduced_gemm_scored)."""
     ma, mb = as_mat(A), as_mat(B)
     if idx is None:
         k = ma.cols
@@ -336,6 +348,14 @@ def rmm_reduced_gemm(A: torch.Tensor, B: torch.Tensor, idx: Optional[torch.Tenso
         shape = (ma.batch, ma.rows, mb.cols) if A.dim() == 3 else (ma.rows, mb.cols)
         out = _out(shape, dt, A.device)
     my = as_mat(out)
+    if want_energy:
+        need = lib().rmm_reduced_gemm_scored_workspace_bytes(ctypes.byref(ma), ctypes.byref(mb), k, ctypes.byref(my))
+        ws = workspace(need, A.device) if ws is None else ws
+        p, nb = _ws_ptr(ws)
+        energy = _out((ma.batch, mb.cols) if A.dim() == 3 else (mb.cols,), torch.float32, A.device)
+        _check(lib().rmm_reduced_gemm_scored(ctypes.byref(ma), ctypes.byref(mb), idx.data_ptr() if idx is not None else None, k,
+                                             float(scale), ctypes.byref(my), energy.data_ptr(), p, nb, _stream()))
+        return out, energy
     need = lib().rmm_reduced_gemm_workspace_bytes(ctypes.byref(ma), ctypes.byref(mb), k, ctypes.byref(my))
     ws = workspace(need, A.device) if ws is None else ws
     p, nb = _ws_ptr(ws)

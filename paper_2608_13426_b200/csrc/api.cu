@@ -64,6 +64,9 @@ int sm_count()
     return n;
 }
 
+static std::atomic<unsigned long long> g_wait_override{0};  // rmm_debug_control("wait_limit_ms", ...): 0 = not set
+static std::atomic<int> g_withhold_override{-1};             // rmm_debug_control("withhold", ...): -1 = not set
+
 unsigned long long wait_limit_ns()
 {
     static const unsigned long long limit = []() -> unsigned long long {
@@ -71,7 +74,25 @@ unsigned long long wait_limit_ns()
         const double ms = e != nullptr ? atof(e) : 0.0;
         return ms > 0.0 ? (unsigned long long)(ms * 1e6) : 2000000000ull;
     }();
-    return limit;
+    const unsigned long long o = g_wait_override.load(std::memory_order_relaxed);
+    return o != 0 ? o : limit;
+}
+
+int debug_withhold()
+{
+    const int o = g_withhold_override.load(std::memory_order_relaxed);
+    if (o >= 0) return o;
+    static const int which = []() {
+        const char *e = getenv("RMM_TEST_WITHHOLD");
+        if (e == nullptr) return 0;
+        if (strcmp(e, "gemm") == 0) return (int)WITHHOLD_GEMM;
+        if (strcmp(e, "score") == 0) return (int)WITHHOLD_SCORE;
+        if (strcmp(e, "attn") == 0) return (int)WITHHOLD_ATTN;
+        if (strcmp(e, "front") == 0) return (int)WITHHOLD_FRONT;
+        if (strcmp(e, "pack") == 0) return (int)WITHHOLD_PACK;
+        return 0;
+    }();
+    return which;
 }
 
 static int check_ws(void *ws, size_t ws_bytes, size_t need, const char *who)
@@ -245,6 +266,47 @@ int rmm_reduced_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx,
     return launch_gemm_simt(A, &b, idx, k, scale, Y, ws, static_cast<cudaStream_t>(stream));
 }
 
+// ---- product that also scores its output ---------------------------------------------------------------
+size_t rmm_reduced_gemm_scored_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y)
+{
+    if (A == nullptr || B == nullptr || Y == nullptr) return 0;
+    rmm_mat_t b = shared_b(A, B);
+    GemvPlan gplan;
+    TcPlan plan;
+    size_t need;
+    if (!gemv_eligible(A, &b, k, Y, &gplan) && tc_eligible(A, &b, k, Y, &plan, true)) {
+        if (plan.epilogue_energy) return plan.total_bytes;
+        need = plan.total_bytes;
+    } else {
+        need = rmm_reduced_gemm_workspace_bytes(A, B, k, Y);
+    }
+    const size_t s = rmm_score_workspace_bytes(Y, 1);  // the output is scored by a pass of its own
+    if (need == 0 || s == 0) return 0;
+    return need > s ? need : s;
+}
+
+int rmm_reduced_gemm_scored(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale, const rmm_mat_t *Y,
+                            float *energy_out, void *ws, size_t ws_bytes, void *stream)
+{
+    if (energy_out == nullptr) return fail(RMM_ERR_INVALID_ARG, "reduced_gemm_scored: energy_out is NULL");
+    int rc = check_gemm(A, B, idx, k, Y);
+    if (rc != RMM_OK) return rc;
+    rmm_mat_t b = shared_b(A, B);
+    GemvPlan gplan;
+    TcPlan plan;
+    if (!gemv_eligible(A, &b, k, Y, &gplan) && tc_eligible(A, &b, k, Y, &plan, true) && plan.epilogue_energy) {
+        rc = check_ws(ws, ws_bytes, plan.total_bytes, "reduced_gemm_scored");
+        if (rc != RMM_OK) return rc;
+        return launch_gemm_tc(A, &b, idx, k, scale, Y, plan, ws, static_cast<cudaStream_t>(stream), energy_out);
+    }
+    // every other form of the product: the output is scored by the ordinary pass once it has been written
+    rc = check_ws(ws, ws_bytes, rmm_reduced_gemm_scored_workspace_bytes(A, B, k, Y), "reduced_gemm_scored");
+    if (rc != RMM_OK) return rc;
+    rc = rmm_reduced_gemm(A, B, idx, k, scale, Y, ws, ws_bytes, stream);
+    if (rc != RMM_OK) return rc;
+    return rmm_score(Y, 1, nullptr, energy_out, ws, ws_bytes, stream);
+}
+
 // ---- whole operation on device operands ------------------------------------------------------------
 struct ProductPlan {
     bool fused;
@@ -255,7 +317,7 @@ struct ProductPlan {
 static int plan_product(const rmm_mat_t *A, const rmm_mat_t *B, const rmm_mat_t *Y, int64_t k, ProductPlan *pp)
 {
     rmm_mat_t b = shared_b(A, B);
-    pp->fused = front_eligible(A, &b, Y, k, &pp->front);
+    pp->fused = k < A->cols && front_eligible(A, &b, Y, k, &pp->front);
     if (pp->fused) {
         pp->total = pp->front.total_bytes;
         return RMM_OK;
@@ -270,14 +332,13 @@ static int plan_product(const rmm_mat_t *A, const rmm_mat_t *B, const rmm_mat_t 
 size_t rmm_product_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, const rmm_mat_t *Y)
 {
     if (A == nullptr || B == nullptr || Y == nullptr || A->cols < 1) return 0;
-    ProductPlan pp;
-    if (plan_product(A, B, Y, A->cols, &pp) != RMM_OK) return 0;  // k = K bounds every k
-    size_t need = pp.total;
-    if (pp.fused) {  // a k for which the fused form does not apply falls back to the two-call form
-        const size_t s1 = rmm_score_select_workspace_bytes(A, 1), s2 = rmm_reduced_gemm_workspace_bytes(A, B, A->cols, Y);
-        if (s1 > need) need = s1;
-        if (s2 > need) need = s2;
-    }
+    // k = K bounds every k, for the two-call form and for the one-launch front end alike
+    const size_t s1 = rmm_score_select_workspace_bytes(A, 1), s2 = rmm_reduced_gemm_workspace_bytes(A, B, A->cols, Y);
+    if (s1 == 0 || s2 == 0) return 0;
+    size_t need = s1 > s2 ? s1 : s2;
+    rmm_mat_t b = shared_b(A, B);
+    FrontPlan fp;
+    if (front_eligible(A, &b, Y, A->cols, &fp) && fp.total_bytes > need) need = fp.total_bytes;
     return need;
 }
 
@@ -297,6 +358,13 @@ int rmm_product(const rmm_mat_t *A, const rmm_mat_t *B, double rho, int64_t k, f
     rc = check_ws(ws, ws_bytes, pp.total, "product");
     if (rc != RMM_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (kk == A->cols) {
+        // every index is kept: the list is 0 .. K-1 (written by the selection, which also gives `retained`), and the product
+        // is the unreduced one, which needs no gather at all
+        rc = rmm_score_select(A, 1, rho, kk, idx, nullptr, nullptr, retained, ws, ws_bytes, stream);
+        if (rc != RMM_OK) return rc;
+        return rmm_reduced_gemm(A, B, nullptr, kk, scale, Y, ws, ws_bytes, stream);
+    }
     if (!pp.fused) {
         rc = rmm_score_select(A, 1, rho, kk, idx, nullptr, nullptr, retained, ws, ws_bytes, stream);
         if (rc != RMM_OK) return rc;
@@ -393,12 +461,29 @@ int rmm_status_read(void *ws, int *device_status)
     cudaError_t e = cudaMemcpy(&v, ws, sizeof v, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "status_read: %s", cudaGetErrorString(e));
     if (v != 0) {
-        int zero = 0;
-        e = cudaMemcpy(ws, &zero, sizeof zero, cudaMemcpyHostToDevice);
+        // a kernel that gave up may have left arrival counters half way: the whole header starts from zero again
+        e = cudaMemset(ws, 0, RMM_WS_HEADER_BYTES);
         if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "status_read: %s", cudaGetErrorString(e));
     }
     *device_status = v;
     return RMM_OK;
+}
+
+int rmm_debug_control(const char *key, double value)
+{
+    if (key == nullptr) return fail(RMM_ERR_INVALID_ARG, "debug_control: NULL key");
+    if (strcmp(key, "wait_limit_ms") == 0) {
+        if (!(value >= 0.0) || value > 60000.0) return fail(RMM_ERR_INVALID_ARG, "debug_control: wait_limit_ms must be in [0, 60000]");
+        g_wait_override.store((unsigned long long)(value * 1e6), std::memory_order_relaxed);
+        return RMM_OK;
+    }
+    if (strcmp(key, "withhold") == 0) {
+        const int w = (int)value;
+        if (w < -1 || w > WITHHOLD_PACK) return fail(RMM_ERR_INVALID_ARG, "debug_control: withhold must be -1 .. %d", (int)WITHHOLD_PACK);
+        g_withhold_override.store(w, std::memory_order_relaxed);
+        return RMM_OK;
+    }
+    return fail(RMM_ERR_INVALID_ARG, "debug_control: unknown key '%s'", key);
 }
 
 int rmm_profile_kernels(void **start_events, void **stop_events, int n, const char *name_filter, int every)

@@ -81,6 +81,8 @@ struct FusedArgs {
     const int32_t *tok;          // GATHERED: [heads, Lc] kept key positions, ascending
     float scale_log2;            // (1 / sqrt(Dh)) * log2(e)
     int *status;
+    unsigned long long wait_ns;  // bound of every device-side wait
+    int withhold;                // test switch: block 0 never requests its first key tile
 };
 
 template <int MODE>
@@ -195,12 +197,16 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------------ producer: Q, then K_0, K_1, V_0, K_2, V_1, ...
         uint32_t ks = 0, kph = 0, n_item = 0;
-        bool ok = true;
+        bool ok = true, first_load = true;
         auto load_kv = [&](const CUtensorMap *map, int chunks, int64_t row, int z) -> bool {
-            if (!mbar_wait_sleepy(kv_empty(ks), kph ^ 1u, abort_flag, a.status)) return false;
+            if (!mbar_wait_sleepy(kv_empty(ks), kph ^ 1u, abort_flag, a.status, a.wait_ns)) return false;
             const uint32_t dst = base + kOffKv + ks * kKvTile;
-            mbar_arrive_expect_tx(kv_full(ks), (uint32_t)chunks * kKvChunk);
-            for (int c = 0; c < chunks; ++c) tma_load_3d(dst + c * kKvChunk, map, c * 64, (int)row, z, kv_full(ks));
+            if (a.withhold && blockIdx.x == 0 && first_load) {
+                first_load = false;  // (test switch) this tile is never requested: its barrier stays incomplete
+            } else {
+                mbar_arrive_expect_tx(kv_full(ks), (uint32_t)chunks * kKvChunk);
+                for (int c = 0; c < chunks; ++c) tma_load_3d(dst + c * kKvChunk, map, c * 64, (int)row, z, kv_full(ks));
+            }
             if (++ks == kKvStages) { ks = 0; kph ^= 1u; }
             return true;
         };
@@ -211,7 +217,7 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             block_range(head, r0, &jb, &je);
             if (je <= jb) continue;
             const int vb = (int)((head + a.v_off) / a.v_div);
-            if (!mbar_wait_sleepy(q_empty, (n_item & 1u) ^ 1u, abort_flag, a.status)) { ok = false; break; }
+            if (!mbar_wait_sleepy(q_empty, (n_item & 1u) ^ 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
             mbar_arrive_expect_tx(q_full, (uint32_t)(kGroups * kq) * kQChunk);
             for (int g = 0; g < kGroups; ++g)
                 for (int c = 0; c < kq; ++c)
@@ -246,11 +252,11 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         ASTAMP_DECL(blockIdx.x == 0 && lane == 0 && g == 0);
         auto step_s = [&](int j) -> bool {  // S~ of tile j (if this group needs it); consumes one ring entry
             ASTAMP(7);
-            if (!mbar_wait(kv_full(ks), kph, abort_flag, a.status)) return false;
+            if (!mbar_wait(kv_full(ks), kph, abort_flag, a.status, a.wait_ns)) return false;
             ASTAMP(0);
             if (j >= gb && j < ge) {
                 // S~ is single-buffered: the softmax warps release it as soon as they hold the tile in registers
-                if (!mbar_wait(s_empty(g, 0), (s_it & 1u) ^ 1u, abort_flag, a.status)) return false;
+                if (!mbar_wait(s_empty(g, 0), (s_it & 1u) ^ 1u, abort_flag, a.status, a.wait_ns)) return false;
                 ASTAMP(1);
                 tc_fence_after();
                 uint32_t ql = q_lo, kl = k_lo + ks * (kKvTile >> 4), acc = 0;
@@ -277,19 +283,19 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             block_range(head, r0, &jb, &je);
             if (je <= jb) continue;
             tile_range(head, r0 + g * FM, &gb, &ge);
-            if (!mbar_wait(q_full, n_item & 1u, abort_flag, a.status)) { ok = false; break; }
+            if (!mbar_wait(q_full, n_item & 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
             ok = step_s(jb);
             for (int j = jb; j < je && ok; ++j) {
                 if (j + 1 < je) ok = step_s(j + 1);                        // S~ of the next tile runs ahead of this P V
                 if (!ok) break;
                 if constexpr (kHasV) {
                     ASTAMP(7);
-                    if (!mbar_wait(kv_full(ks), kph, abort_flag, a.status)) { ok = false; break; }
+                    if (!mbar_wait(kv_full(ks), kph, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                     ASTAMP(3);
                     if (j >= gb && j < ge) {
-                        if (j == gb && !mbar_wait(o_empty(g), (o_it & 1u) ^ 1u, abort_flag, a.status)) { ok = false; break; }
+                        if (j == gb && !mbar_wait(o_empty(g), (o_it & 1u) ^ 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                         ASTAMP(4);
-                        if (!mbar_wait(p_full(g), p_it & 1u, abort_flag, a.status)) { ok = false; break; }
+                        if (!mbar_wait(p_full(g), p_it & 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                         ASTAMP(5);
                         tc_fence_after();
                         const uint32_t vl = v_lo + ks * (kKvTile >> 4);
@@ -445,7 +451,7 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         asm volatile("prefetch.global.L1 [%0];" ::"l"(a.lse + head * a.lse_ld + nxt));
                 }
                 ASTAMP(7);
-                if (!mbar_wait(s_full(g, 0), s_it & 1u, abort_flag, a.status)) { ok = false; break; }
+                if (!mbar_wait(s_full(g, 0), s_it & 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                 ASTAMP(0);
                 tc_fence_after();
                 uint32_t v0[32], v1[32];
@@ -499,7 +505,7 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     const float neg_m = -row_lse;   // +inf normaliser (row sees nothing): p = 0
                     load_chunk(j, 0, v0, v1);
                     emit_chunk(v0, v1, neg_m, w);
-                    if (!mbar_wait(p_empty(g), (p_it & 1u) ^ 1u, abort_flag, a.status)) { ok = false; break; }
+                    if (!mbar_wait(p_empty(g), (p_it & 1u) ^ 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                     store_chunk(0, w);
                     load_chunk(j, 64, v0, v1);
                     release_s();
@@ -515,7 +521,7 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     bool any_grow;
                     const float alpha = follow_max(mc, &any_grow);
                     if (any_grow && j > jb) {  // rows of O already hold sums taken against the old maximum
-                        if (!mbar_wait(p_empty(g), (p_it & 1u) ^ 1u, abort_flag, a.status)) { ok = false; break; }
+                        if (!mbar_wait(p_empty(g), (p_it & 1u) ^ 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                         tc_fence_after();
                         for (int c = 0; c < nv * 64; c += 16) {
                             uint32_t o[16];
@@ -532,7 +538,7 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     emit_chunk(v0, v1, neg_m, w);
                     ASTAMP(3);
                     // (a repeated wait on a completed phase returns at once: the rescale above may have waited already)
-                    if (!mbar_wait(p_empty(g), (p_it & 1u) ^ 1u, abort_flag, a.status)) { ok = false; break; }
+                    if (!mbar_wait(p_empty(g), (p_it & 1u) ^ 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                     ASTAMP(4);
                     store_chunk(1, w);
                     load_chunk(j, 0, v0, v1);
@@ -554,7 +560,7 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 if (i < a.Lr) a.energy[head * a.Lr + i] = l;
             } else {
                 // ---- epilogue: O row (/ l) -> bf16 -> global
-                if (!mbar_wait(o_full(g), o_it & 1u, abort_flag, a.status)) { ok = false; break; }
+                if (!mbar_wait(o_full(g), o_it & 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                 tc_fence_after();
                 const float inv_l = MODE == MODE_GATHERED ? 1.f : (l > 0.f ? 1.f / l : 0.f);
                 for (int c = 0; c < nv * 64; c += 32) {
@@ -670,6 +676,8 @@ int launch_fused_attn(const __nv_bfloat16 *Qp, const __nv_bfloat16 *Kp, int64_t 
     a.lse = const_cast<float *>(lse); a.lse_ld = lse_ld; a.tok = tok;
     a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)Dh));
     a.status = status;
+    a.wait_ns = wait_limit_ns();
+    a.withhold = debug_withhold() == WITHHOLD_ATTN;
     if (tok != nullptr) return launch_mode<MODE_GATHERED>(mq, mk, mv, a, "fused_attn_gathered_kernel", stream);
     return launch_mode<MODE_FULL>(mq, mk, mv, a, "fused_attn_kernel", stream);
 }
@@ -690,6 +698,8 @@ int launch_fused_attn_scores(const __nv_bfloat16 *Qp, const __nv_bfloat16 *Kp, i
     a.lse = lse; a.lse_ld = lse_ld; a.energy = energy;
     a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)Dh));
     a.status = status;
+    a.wait_ns = wait_limit_ns();
+    a.withhold = debug_withhold() == WITHHOLD_ATTN;
     // sweep 1: rows = queries
     if ((rc = packed_map(&mq, Qp, kd, Lq, heads, ldd, FM)) != RMM_OK) return rc;
     if ((rc = packed_map(&mk, Kp, kd, Lk, heads, ldd, FN)) != RMM_OK) return rc;

@@ -70,6 +70,10 @@ struct PerDeviceOnce {
 
 int sm_count();                      // multiprocessors of the current device
 unsigned long long wait_limit_ns();  // bound of every device-side wait: 2 s, or RMM_SPIN_LIMIT_MS from the environment
+// Test switch (environment RMM_TEST_WITHHOLD = gemm | score | attn | front | pack, read once): block 0 of that kernel
+// family never requests its first tile, so the waits behind it run out and the kernel's give-up path runs.  0 = off.
+enum { WITHHOLD_GEMM = 1, WITHHOLD_SCORE = 2, WITHHOLD_ATTN = 3, WITHHOLD_FRONT = 4, WITHHOLD_PACK = 5 };
+int debug_withhold();
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -136,11 +140,13 @@ int launch_gemv(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int6
 struct TcPlan {
     int b_kmajor;       // 0: B rows (contraction slices) contiguous, kept rows copied; 1: B is K-contiguous, packed like A
     int64_t ldp;        // leading dimension of the packed operands (multiple of 8)
-    size_t off_ap, off_bp, total_bytes;
+    size_t off_ap, off_bp, off_colen, total_bytes;
+    bool epilogue_energy;  // the plan reserves the per-group column energies of Y and the epilogue fills them
 };
-bool tc_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y, TcPlan *plan);
+bool tc_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y, TcPlan *plan, bool with_energy = false);
+// energy_out (with a plan made with_energy): also energy_out[b, c] = sum_i Y[b, i, c]^2 of the rounded outputs
 int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
-                   const rmm_mat_t *Y, const TcPlan &plan, void *ws, cudaStream_t stream);
+                   const rmm_mat_t *Y, const TcPlan &plan, void *ws, cudaStream_t stream, float *energy_out = nullptr);
 
 // A tensor-core problem on operands that are already in TMA-loadable form.
 struct TcProblem {
@@ -160,8 +166,13 @@ struct TcProblem {
     int64_t y_sb, y_sr;
     float scale;
     int *status;
+    // bf16 output only: when set, the epilogue also writes, per 32-row group g and column c, the sum of the squares of the
+    // rounded outputs Y[32 g .. 32 g + 31, c] to col_energy[(batch entry * ceil(M / 32) + g) * N + c]
+    float *col_energy;
 };
 int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream);
+// energy[b, c] = sum over the 32-row groups of col_energy (fp64, in group order), rounded to fp32
+int launch_energy_combine(const float *col_energy, int64_t batch, int64_t groups, int64_t N, float *energy, cudaStream_t stream);
 
 // One gather of kept slices (see pack.cu).  Columns: dst[b, r, j] = src[sb, r, idx[b, j]], j < k, dst row pitch
 // ld_dst >= k (columns k .. ld_dst zeroed).  Rows: dst[b, j, 0:n] = src[sb, idx[b, j], 0:n].  NULL idx = 0 .. k-1.

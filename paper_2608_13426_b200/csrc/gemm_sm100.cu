@@ -60,6 +60,9 @@ struct TcArgs {
     int tiles_m, tiles_n;
     int epi_sets;           // 1, or 2: a second set of four epilogue warps takes every other 64-column chunk
     int *status;
+    unsigned long long wait_ns;  // bound of every device-side wait
+    int withhold;                // test switch: the producer skips its very first stage, so that the waits behind it expire
+    float *col_energy;           // [batch, ceil(M / 32), N] or NULL: sum of squares of the rounded outputs per 32-row group
     // B_GATHER: the unpacked B and the kept row numbers
     const __nv_bfloat16 *b_src;
     const int32_t *b_idx;
@@ -160,8 +163,10 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             int64_t bb = (b + a.b_batch_off) / a.b_batch_div;
             if (bb >= a.b_batches) bb = a.b_batches - 1;
             for (int kb = 0; kb < num_kb; ++kb) {
-                if (!mbar_wait_lane(empty_bar(s), ph ^ 1u, abort_flag, a.status)) { ok = false; break; }
-                {
+                if (!mbar_wait_lane(empty_bar(s), ph ^ 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
+                if (a.withhold && blockIdx.x == 0 && tile == tile0 && kb == 0) {
+                    // (test switch) this stage is never requested: its barrier stays incomplete
+                } else {
                     const uint32_t sa = base + s * L::kStageBytes;
                     const uint32_t sb = sa + L::kABytes;
                     const int row_a = tm * (BM * CTAS) + (int)rank * BM, col_b = tn * BN + (int)rank * BNL;
@@ -216,12 +221,12 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         bool ok = true;
         for (int64_t tile = tile0; lane == 0 && tile < num_tiles && ok; tile += tile_step, ++tcount) {
             const uint32_t acc = tcount & 1u, acc_ph = (tcount >> 1) & 1u;
-            if (!mbar_wait_lane(tempty_bar(acc), acc_ph ^ 1u, abort_flag, a.status)) { ok = false; break; }
+            if (!mbar_wait_lane(tempty_bar(acc), acc_ph ^ 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * BN;
             uint32_t accumulate = 0;
             for (int kb = 0; kb < num_kb; ++kb) {
-                if (!mbar_wait_lane(full_bar(stage), phase, abort_flag, a.status)) { ok = false; break; }
+                if (!mbar_wait_lane(full_bar(stage), phase, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                 if constexpr (B_GATHER) fence_proxy_async();  // B arrived through the generic proxy (cp.async)
                 tc_fence_after();
                 if (kb == 0 && tcount == 0) { GSTAMP_MAX(2); }
@@ -281,7 +286,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 #pragma unroll
                 for (int i = 0; i < kRowsPerWarp; ++i) rows[i] = rows_next[i];
                 if (kb + 1 < num_kb) fetch_rows(kb + 1, rows_next);
-                if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status)) { ok = false; break; }
+                if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                 const uint32_t sb = base + s * L::kStageBytes + L::kABytes + lane_off;
 #pragma unroll
                 for (int i = 0; i < kRowsPerWarp; ++i) {
@@ -317,7 +322,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
             tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, tm, tn);
             const uint32_t acc = tcount & 1u, acc_ph = (tcount >> 1) & 1u;
-            if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, a.status)) { ok = false; break; }
+            if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
             tc_fence_after();
             if (lane == 0) { GSTAMP_MAX(4); }
             const int64_t m_warp = (int64_t)tm * (BM * CTAS) + rank * BM + q * 32, m = m_warp + lane;
@@ -356,6 +361,29 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     put(r1, 4);
                     fence_proxy_async();  // generic writes -> visible to the copy engine
                     __syncwarp();
+                    if (a.col_energy != nullptr) {
+                        // Column energies of the output, where it is produced: lane l sums the squares of columns 2 l and
+                        // 2 l + 1 of the slab's 32 rounded rows (two fp32 chains of 16 terms each, exact squares) and stores
+                        // the pair; the 32-row groups are added up in fp64, in order, by a small kernel afterwards.
+                        const uint8_t *col = base_ptr + L::kEpiOffset + slab_id * 4096 + ebuf * 4096 + (lane & 3) * 4;
+                        const int u = lane >> 2;
+                        float e0a = 0.f, e0b = 0.f, e1a = 0.f, e1b = 0.f;
+#pragma unroll
+                        for (int r = 0; r < 32; r += 2) {
+                            const uint32_t wa = *reinterpret_cast<const uint32_t *>(col + r * 128 + ((u ^ (r & 7)) << 4));
+                            const uint32_t wb = *reinterpret_cast<const uint32_t *>(col + (r + 1) * 128 + ((u ^ ((r + 1) & 7)) << 4));
+                            const float a0 = __uint_as_float(wa << 16), a1 = __uint_as_float(wa & 0xffff0000u);
+                            const float b0 = __uint_as_float(wb << 16), b1 = __uint_as_float(wb & 0xffff0000u);
+                            e0a = fmaf(a0, a0, e0a); e1a = fmaf(a1, a1, e1a);
+                            e0b = fmaf(b0, b0, e0b); e1b = fmaf(b1, b1, e1b);
+                        }
+                        const int64_t cn = n + 2 * lane;
+                        if (cn < a.N) {  // N is even for a bf16 tensor-core output
+                            const int64_t groups = (a.M + 31) / 32;
+                            float2 *dst = reinterpret_cast<float2 *>(a.col_energy + (b * groups + m_warp / 32) * a.N + cn);
+                            *dst = make_float2(e0a + e0b, e1a + e1b);
+                        }
+                    }
                     if (lane == 0) {
                         tma_store_3d(&map_y, slab_s + ebuf * 4096, (int)n, (int)m_warp, (int)b);
                         bulk_commit();
@@ -449,7 +477,7 @@ int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorM
 
 }  // namespace
 
-bool tc_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y, TcPlan *plan)
+bool tc_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y, TcPlan *plan, bool with_energy)
 {
     if (A->dtype != RMM_BF16 || B->dtype != RMM_BF16) return false;
     const int64_t M = A->rows, K = A->cols, N = B->cols, batch = A->batch;
@@ -477,6 +505,10 @@ bool tc_eligible(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_ma
         off += align_up((size_t)batch * M * plan->ldp * 2, 256);
         plan->off_bp = off;
         off += align_up(b_kmajor ? (size_t)batch * N * plan->ldp * 2 : (size_t)batch * k * N * 2, 256);
+        // column energies from the epilogue: bf16 output with an even number of columns (the pairs are stored as float2)
+        plan->epilogue_energy = with_energy && Y->dtype == RMM_BF16 && N % 2 == 0;
+        plan->off_colen = off;
+        if (plan->epilogue_energy) off += align_up((size_t)batch * ceil_div(M, 32) * N * 4, 256);
         plan->total_bytes = off;
     }
     return true;
@@ -512,8 +544,13 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     a.tiles_m = (int)ceil_div(p.M, BM * ctas);
     a.tiles_n = (int)ceil_div(p.N, BN);
     a.status = p.status;
-    // products with at most four k-blocks per tile are bound by the epilogue: two sets of epilogue warps
-    a.epi_sets = (p.y_bf16 && p.b_idx == nullptr && ceil_div(p.k, BK) <= 4) ? 2 : 1;
+    a.wait_ns = wait_limit_ns();
+    a.withhold = debug_withhold() == WITHHOLD_GEMM;
+    a.col_energy = p.col_energy;
+    // products with at most four k-blocks per tile are bound by the epilogue, and a block with a single tile has no next
+    // main loop to hide its epilogue behind: two sets of epilogue warps in both cases
+    const int64_t n_tiles = p.batch * ceil_div(p.M, BM * ctas) * ceil_div(p.N, BN);
+    a.epi_sets = (p.y_bf16 && p.b_idx == nullptr && (ceil_div(p.k, BK) <= 4 || n_tiles <= sm_count() / ctas)) ? 2 : 1;
     a.b_src = p.b; a.b_idx = p.b_idx; a.b_ld = p.b_ld; a.b_sb = p.b_batches > 1 ? p.b_sb : 0; a.b_idx_stride = p.b_idx_stride;
     a.b_rows = p.b_rows;
     if (p.b_idx != nullptr) {
@@ -566,8 +603,15 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
 }
 
 int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
-                   const rmm_mat_t *Y, const TcPlan &plan, void *ws, cudaStream_t stream)
+                   const rmm_mat_t *Y, const TcPlan &plan, void *ws, cudaStream_t stream, float *energy_out)
 {
+    if (energy_out != nullptr && plan.epilogue_energy) {
+        // the product writes per-group column energies, a small kernel adds the groups up
+        int rc0 = launch_gemm_tc(A, B, idx, k, scale, Y, plan, ws, stream, nullptr);
+        if (rc0 != RMM_OK) return rc0;
+        return launch_energy_combine(reinterpret_cast<const float *>(static_cast<char *>(ws) + plan.off_colen), A->batch,
+                                     ceil_div(A->rows, 32), B->cols, energy_out, stream);
+    }
     char *w = static_cast<char *>(ws);
     int *status = &reinterpret_cast<WsHeader *>(w)->status;
     const int64_t M = A->rows, K = A->cols, N = B->cols, batch = A->batch;
@@ -579,6 +623,7 @@ int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, i
     p.b_kmajor = plan.b_kmajor;
     p.y = Y->ptr; p.y_bf16 = Y->dtype == RMM_BF16; p.y_sb = Y->stride_batch; p.y_sr = Y->stride_row;
     p.scale = scale; p.status = status;
+    p.col_energy = plan.epilogue_energy ? reinterpret_cast<float *>(w + plan.off_colen) : nullptr;
     p.b_batch_off = 0; p.b_batch_div = 1; p.b_batches = batch;
 
     // the unreduced product (idx NULL, k == K) on TMA-loadable operands needs no gather at all

@@ -261,7 +261,8 @@ __device__ void pack_rows_short(const PackJob &p, int64_t blk, int *status)
 
 // Column gather of long rows: see the file header.  Block b owns the contiguous (batch, row) range
 // [b * per_block, (b + 1) * per_block); rows stream through two buffers filled by cp.async.bulk.
-__global__ void __launch_bounds__(kThreadsLong, 1) pack_long_kernel(const __grid_constant__ PackJob p, int64_t per_block, int *status)
+__global__ void __launch_bounds__(kThreadsLong, 1) pack_long_kernel(const __grid_constant__ PackJob p, int64_t per_block, int *status,
+                                                                    unsigned long long wait_ns, int withhold)
 {
     using namespace ptx;
     extern __shared__ __align__(16) unsigned char smem[];
@@ -292,7 +293,7 @@ __global__ void __launch_bounds__(kThreadsLong, 1) pack_long_kernel(const __grid
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                      ::"r"(dst), "l"(src), "r"((uint32_t)K * 2u), "r"(bar) : "memory");
     };
-    if (tid == 0 && lo < hi) issue(lo, 0);
+    if (tid == 0 && lo < hi && !(withhold && blockIdx.x == 0)) issue(lo, 0);  // (test switch: block 0's first row is never requested)
     uint32_t cb[2 * kLongPairs];   // byte offsets of this thread's source columns inside a staged row
     int64_t cur_batch = -1;
     for (int64_t g = lo; g < hi; ++g) {
@@ -322,7 +323,7 @@ __global__ void __launch_bounds__(kThreadsLong, 1) pack_long_kernel(const __grid
             }
         }
         // every thread comes out of the wait (landed, timed out, or told to abort) and the block decides together
-        const bool landed = mbar_wait(smem_u32(&full[stage]), (uint32_t)(it >> 1) & 1u, &abort_flag, status);
+        const bool landed = mbar_wait(smem_u32(&full[stage]), (uint32_t)(it >> 1) & 1u, &abort_flag, status, wait_ns);
         if (!__syncthreads_and(landed)) break;
         const uint32_t row_s = smem_u32(smem) + (uint32_t)stage * pitch;
         unsigned *d = reinterpret_cast<unsigned *>(p.dst + b * p.rows * p.ld_dst + r * p.ld_dst);
@@ -427,7 +428,7 @@ int launch_pack(const PackSpec *specs, int n, int *status, cudaStream_t stream)
         const int64_t total = p.batch * p.rows, per_block = ceil_div(total, sms);
         prof_begin("pack_long_kernel", stream);
         launch_kernel(pack_long_kernel, dim3((unsigned)ceil_div(total, per_block)), dim3(kThreadsLong), 2 * row_bytes, stream, 1, p,
-                      per_block, status);
+                      per_block, status, wait_limit_ns(), debug_withhold() == WITHHOLD_PACK ? 1 : 0);
         int rc = check_launch("pack_long_kernel", stream);
         if (rc != RMM_OK) return rc;
         blocks -= p.blocks;

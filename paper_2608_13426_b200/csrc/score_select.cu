@@ -45,6 +45,8 @@ struct ScoreArgs {
     int k;
     int32_t *idx;        // [batch, k]
     float *retained;     // [batch] or null
+    unsigned long long wait_ns;  // bound of every device-side wait
+    int withhold;                // test switch: block 0 never requests its first tile
 };
 
 template <int VEC, bool BF16>
@@ -269,8 +271,10 @@ __global__ void __launch_bounds__(kThreads, 1) score_tma_kernel(const __grid_con
     __syncthreads();
     pdl_wait();
 
+    const bool withheld = a.withhold && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0;
     auto issue = [&](int t) {  // thread 0 only: fetch tile t into its ring slot
         const int st = t % kTmaStages;
+        if (withheld && t == 0) return;  // (test switch) never requested: the slot's barrier stays incomplete
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full_bar(st)), "r"(kTmaStageBytes) : "memory");
         asm volatile(
             "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
@@ -293,10 +297,12 @@ __global__ void __launch_bounds__(kThreads, 1) score_tma_kernel(const __grid_con
         if (tid == 0 && t + kAhead < n_tiles) {
             // the slot of tile t + kAhead was last used by tile t - 2: wait until every warp has released it
             const int nt = t + kAhead, ns = nt % kTmaStages;
-            if (nt >= kTmaStages && !score_wait(empty_bar(ns), (uint32_t)(nt / kTmaStages - 1) & 1u, status)) ok = false;
+            if (nt >= kTmaStages && !score_wait(empty_bar(ns), (uint32_t)(nt / kTmaStages - 1) & 1u, status, a.wait_ns)) ok = false;
             if (ok) issue(nt);
         }
-        if (!score_wait(full_bar(st), ph, status)) { ok = false; }
+        if (!score_wait(full_bar(st), ph, status, a.wait_ns)) ok = false;
+        ok = __all_sync(0xffffffffu, ok);  // the warp leaves as a whole (thread 0 also waits on behalf of the producer)
+        if (!ok) break;
         const uint4 *tile = reinterpret_cast<const uint4 *>(s_dyn + st * kTmaStageBytes);
         const uint4 q0 = tile[ty * 8 + tx], q1 = tile[(ty + 128) * 8 + tx];
         const unsigned w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
@@ -316,7 +322,16 @@ __global__ void __launch_bounds__(kThreads, 1) score_tma_kernel(const __grid_con
     }
 #pragma unroll
     for (int e = 0; e < 8; ++e) dacc[e] += (double)facc[e];
-    __syncthreads();  // every tile has landed and been read: the ring can be reused for the partial sums
+    if (!__syncthreads_and(ok)) {
+        // A wait ran out (the status word says so).  The ring is not reused (a copy might still land in it) and nothing
+        // is published; copies in flight get time to land before shared memory is released.  The arrival counters of this
+        // call stay incomplete: rmm_status_read clears them together with the status word.
+        unsigned long long t0, now;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+        do { __nanosleep(2000); asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now)); } while (now - t0 < 200000ull);
+        return;
+    }
+    // every tile has landed and been read: the ring can be reused for the partial sums
     score_finish<8>(a, dacc, s_dyn, s_sel, s_flag);
 }
 
@@ -400,7 +415,12 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
     // have released it.  full_par (every thread) and empty_par (thread 0) hold, per slot, the parity of the next
     // completion to wait for; every completion is waited for exactly once, in order.
     uint32_t full_par = 0, empty_par = 0;
+    bool withheld = a.withhold && blockIdx.x == 0;
     auto fill = [&](int slot, int tile) {  // thread 0 only: rows of `tile` -> slot
+        if (withheld) {  // (test switch) the block's very first request is dropped: the slot's barrier stays incomplete
+            withheld = false;
+            return;
+        }
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full_bar(slot)), "r"(kTmaStageBytes) : "memory");
         asm volatile(
             "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
@@ -434,7 +454,9 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
             if (nt >= kTmaStages && !wait_empty(ns)) ok = false;
             if (ok) fill(ns, nt);
         }
-        if (!wait_full(st)) { ok = false; break; }
+        if (!wait_full(st)) ok = false;
+        ok = __all_sync(0xffffffffu, ok);  // the warp leaves as a whole (thread 0 also waits on behalf of the producer)
+        if (!ok) break;
         const uint4 *tile = reinterpret_cast<const uint4 *>(s_dyn + st * kTmaStageBytes);
         const uint4 q0 = tile[ty * 8 + tx], q1 = tile[(ty + 128) * 8 + tx];
         const unsigned w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
@@ -617,17 +639,8 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
 
     FSTAMP_MAX(4);
     // ---- 4 and 5 run side by side: warps 0 .. 15 gather the block's kept columns of A, warps 16 .. 31 copy its rows
-    // of B (requested into L2 above).  The ring's `empty` barriers are set up again for 16 releasing warps.
+    // of B (requested into L2 above).  A ring slot is still released by 32 arrivals: two lanes of each gathering warp.
     constexpr int kGatherWarps = 16;
-    if (tid == 0) {
-        for (int st = 0; st < kTmaStages; ++st) {
-            asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(empty_bar(st)) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_bar(st)), "r"(kGatherWarps) : "memory");
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        empty_par = 0;
-    }
-    __syncthreads();
     if (warp < kGatherWarps) {
         // ---- 4. own kept columns of A -> Ap.  What bounds this step is the number of store requests that reach L2 (about
         // 64 G requests/s over the whole GPU, however few bytes each carries), so a block issues exactly one per row: lane l
@@ -668,7 +681,11 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
                     fill(qs, q);
                 }
             }
-            if (t >= resident && !wait_full(st)) { ok = false; break; }
+            if (t >= resident && !wait_full(st)) ok = false;
+            // a warp leaves the loop as a whole (the shuffles and warp barriers below involve every lane): lanes may see a
+            // wait expire at slightly different moments, and thread 0 also waits on behalf of the producer
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
             const int64_t left = a.m - (int64_t)tile * kTmaRows - warp;      // rows of this tile at or below the warp's first
             const int np = left <= 0 ? 0 : (int)min((int64_t)(kTmaRows / kGatherWarps), (left + kGatherWarps - 1) / kGatherWarps);
             const unsigned pv = pv_next;
@@ -692,7 +709,7 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
                 d += 4 * row_step;
             }
             __syncwarp();
-            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(st)) : "memory");
+            if (lane < kThreads / 32 / kGatherWarps) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(st)) : "memory");
         }
     } else {
         // ---- 5. rows of B of the own kept columns -> Bp[pos0 .. pos0 + cnt, :], 16-byte vectors.  Rows shorter than
@@ -826,6 +843,8 @@ int launch_score_select(const rmm_mat_t *A, const ScorePlan &p, bool do_select, 
     a.k = (int)k;
     a.idx = idx;
     a.retained = retained;
+    a.wait_ns = wait_limit_ns();
+    a.withhold = debug_withhold() == WITHHOLD_SCORE;
 
     dim3 grid((unsigned)p.col_blocks, (unsigned)p.row_splits, (unsigned)A->batch);
     const bool bf16 = A->dtype == RMM_BF16;
@@ -916,6 +935,8 @@ int launch_front(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, int32_t *idx
     fa.b_sr = B->stride_row; fa.N = B->cols;
     fa.Bp = reinterpret_cast<__nv_bfloat16 *>(w + plan.off_bp);
     fa.wait_ns = wait_limit_ns();
+    a.wait_ns = fa.wait_ns;
+    a.withhold = debug_withhold() == WITHHOLD_FRONT;
     CUtensorMap map;
     const uint64_t dims[3] = {(uint64_t)a.n, (uint64_t)a.m, 1};
     const uint64_t st[2] = {(uint64_t)A->stride_row * 2, (uint64_t)A->stride_row * 2 * (uint64_t)a.m};

@@ -8,7 +8,7 @@
 namespace rmm {
 namespace ptx {
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // every spin gives up after 2 s
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // default bound of every spin: 2 s (the host passes its own, see wait_limit_ns)
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -58,7 +58,8 @@ __device__ __forceinline__ unsigned long long global_ns()
 }
 
 // Bounded wait.  Returns false when the block is aborting (this or another thread ran out of time).
-__device__ __forceinline__ bool mbar_wait_lane(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+__device__ __forceinline__ bool mbar_wait_lane(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          unsigned long long limit_ns = kWaitLimitNs)
 {
     unsigned long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
@@ -67,7 +68,7 @@ __device__ __forceinline__ bool mbar_wait_lane(uint32_t bar, uint32_t parity, vo
             if (*abort_flag) return false;
             unsigned long long now = global_ns();
             if (t0 == 0) t0 = now;
-            if (now - t0 > kWaitLimitNs) {
+            if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicExch(status, (int)RMM_ERR_TIMEOUT);
                 return false;
@@ -77,7 +78,8 @@ __device__ __forceinline__ bool mbar_wait_lane(uint32_t bar, uint32_t parity, vo
 }
 
 // Bounded wait of a single thread that may sleep: for roles whose waits are long (a producer on a full ring).
-__device__ __forceinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+__device__ __forceinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          unsigned long long limit_ns = kWaitLimitNs)
 {
     unsigned long long t0 = 0;
     for (uint32_t it = 0;; ++it) {
@@ -86,7 +88,7 @@ __device__ __forceinline__ bool mbar_wait_sleepy(uint32_t bar, uint32_t parity, 
             if (*abort_flag) return false;
             unsigned long long now = global_ns();
             if (t0 == 0) t0 = now;
-            if (now - t0 > kWaitLimitNs) {
+            if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicExch(status, (int)RMM_ERR_TIMEOUT);
                 return false;
@@ -109,16 +111,18 @@ __device__ __forceinline__ bool elect_one()
 }
 
 // Whole-warp form of the sleeping wait.
-__device__ __forceinline__ bool mbar_wait_sleepy_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+__device__ __forceinline__ bool mbar_wait_sleepy_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          unsigned long long limit_ns = kWaitLimitNs)
 {
-    bool ok = mbar_wait_sleepy(bar, parity, abort_flag, status);
+    bool ok = mbar_wait_sleepy(bar, parity, abort_flag, status, limit_ns);
     return __all_sync(0xffffffffu, ok);
 }
 
 // Whole-warp form: every lane waits, and the warp takes one common decision.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                          unsigned long long limit_ns = kWaitLimitNs)
 {
-    bool ok = mbar_wait_lane(bar, parity, abort_flag, status);
+    bool ok = mbar_wait_lane(bar, parity, abort_flag, status, limit_ns);
     return __all_sync(0xffffffffu, ok);
 }
 

@@ -42,9 +42,25 @@ def test_replica_aggregation_world_size_2():
 def test_retained_flops_and_single_rank():
     import bench
 
-    assert bench.retained_flops(0.5) == 2.0 * 2048 * 4096 * 2048
-    assert bench.retained_flops(1.0) == 2.0 * 2048 * 8192 * 2048
+    assert bench.retained_flops(0.5) == 2.0 * 32768 * 14336 * 8192          # the headline: 70B-class down projection
+    assert bench.retained_flops(1.0) == 2.0 * 32768 * 28672 * 8192
+    assert bench.retained_flops(0.5, 2048, 8192, 2048) == 2.0 * 2048 * 4096 * 2048
     assert bench.max_over_ranks(1.5, 1) == 1.5
+
+
+def test_roofline_denominator_follows_the_sampled_clocks():
+    """The GEMM's roofline fraction is taken against the sustained cuBLAS rate only when the SM clock sampled during
+    the timed region sagged, against the burst rate otherwise; recomputing achieved / peak gives the reported fraction."""
+    import bench
+
+    peaks = {"bf16_burst": 1600.0, "bf16_sustained": 1300.0, "hbm_gbs": 6500.0, "source": "measured"}
+    hot = bench.gemm_roofline(1000.0, 5.0, peaks, {"sm_mhz": 1300.0, "sm_max_mhz": 1965.0}, None)
+    cool = bench.gemm_roofline(1000.0, 0.03, peaks, {"sm_mhz": 1965.0, "sm_max_mhz": 1965.0}, 1e6)
+    assert hot["peak"] == 1300.0 and cool["peak"] == 1600.0
+    for r in (hot, cool):
+        assert r["frac"] == pytest.approx(r["achieved"] / r["peak"])
+        assert r["frac_of_nominal_peak"] == pytest.approx(1000.0 / 2250.0)
+    assert bench.gemm_roofline(1000.0, 1.0, peaks, {"sm_mhz": None, "sm_max_mhz": None}, None)["peak"] == 1600.0
 
 
 def test_clock_sample_parser():

@@ -581,3 +581,52 @@ def test_whole_product_in_one_front_launch(oracle, M, K, N, rho):
     Y3, idx3 = rmm.rmm_product(Ad, Bd, rho=rho)
     assert torch.equal(idx3, idx) and torch.equal(Y3, Y)
     assert rmm.rmm_status_read() == 0
+
+
+# ------------------------------------------------------------------------------------------------
+# column energies of the output, accumulated in the product's epilogue
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("M,K,N,rho,dtype", [
+    (2048, 8192, 2048, 0.5, torch.bfloat16),      # 1B-class down projection: single-CTA tiles, one tile per block
+    (300, 1024, 264, 0.5, torch.bfloat16),        # ragged rows (last 32-row group partly outside) and ragged columns
+    (100, 2048, 1024, 0.25, torch.bfloat16),      # rows of B fetched inside the kernel
+    (4096, 2048, 4864, 1.0, torch.bfloat16),      # CTA pairs, the unreduced product (nothing gathered)
+    (129, 512, 136, 0.75, torch.float32),         # fp32 output: scored by the ordinary pass afterwards
+    (3, 4096, 512, 0.5, torch.bfloat16),          # decode-step GEMV: scored by the ordinary pass afterwards
+])
+def test_product_scores_its_own_output(oracle, M, K, N, rho, dtype):
+    """rmm_reduced_gemm_scored: energy[c] = sum_i Y[i, c]^2 of the outputs as stored, to 3e-7 of the fp64 sum over the
+    GPU's own Y, and Y itself unchanged by the extra work."""
+    A, B = synth.mlp_product(M, K, N, seed=M + 3)
+    Ad, Bd = dev(A), dev(B)
+    idx = None
+    if rho < 1.0:
+        idx, _, _, _ = rmm.rmm_score_select(Ad, rho=rho)
+    Y, e = rmm.rmm_reduced_gemm(Ad, Bd, idx, out_dtype=dtype, want_energy=True)
+    Y0 = rmm.rmm_reduced_gemm(Ad, Bd, idx, out_dtype=dtype)
+    assert torch.equal(Y, Y0)
+    e64, _ = oracle.score(Y.cpu())
+    assert np.allclose(e.cpu().numpy(), e64, rtol=3e-7, atol=0)
+    Y2, e2 = rmm.rmm_reduced_gemm(Ad, Bd, idx, out_dtype=dtype, want_energy=True)
+    assert torch.equal(e, e2) and torch.equal(Y, Y2)              # deterministic
+    assert rmm.rmm_status_read() == 0
+
+
+def test_next_product_selects_from_epilogue_energies(oracle):
+    """Up projection followed by down projection: the down projection's index set is selected from the energies that the
+    up projection's epilogue accumulated, with no score pass over the intermediate activations.  The set must match the
+    oracle's selection on the GPU's own intermediate activations inside the strict tie band."""
+    X, W_up = synth.mlp_product(2048, 2048, 8192, seed=77)
+    W_down = synth.weight(8192, 2048, seed=79)
+    H, e = rmm.rmm_reduced_gemm(dev(X), dev(W_up), None, want_energy=True)       # dense up projection, scored on the way out
+    k = rmm.rmm_keep_count(0.5, 8192)
+    idx = rmm.rmm_select(e, k=k)
+    e64, _ = oracle.score(H.cpu())
+    check_index_set(idx.cpu().numpy(), e64, k)
+    idx_ref, _, _, _ = rmm.rmm_score_select(H, rho=0.5)
+    assert len(np.setxor1d(idx.cpu().numpy(), idx_ref.cpu().numpy())) <= 4        # both inside the band
+    Y = rmm.rmm_reduced_gemm(H, dev(W_down), idx)
+    rows = [0, 1000, 2047]
+    for r in rows:
+        want = oracle.reduced_gemm(H.cpu(), W_down, idx.cpu().numpy(), rows=(r, r + 1))[r]
+        assert rel_fro(Y[r].float().cpu().numpy(), want) <= TOL_BF16
