@@ -386,6 +386,18 @@ def gemm_framed_attention(rmm, synth, dev, peaks, reps=5):
     return out
 
 
+def run_mlp_1b_only(args):
+    """Only the 1B-class product at rho = 0.5 (a few dozen launches: for profiler captures of the one-launch front end
+    and of the single-tile GEMM); prints its own JSON line."""
+    import paper_2608_13426_b200 as rmm
+    from paper_2608_13426_b200 import binding, synth
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    res = small_product_sweep(rmm, binding, synth, dev, measured_peaks(), 0, reps=max(3, args.steps), rhos=(RHO,))
+    assert rmm.rmm_status_read() == 0
+    print(json.dumps({"mlp_1b": res}))
+
+
 def run_attention_only(args):
     import paper_2608_13426_b200 as rmm
     from paper_2608_13426_b200 import binding, synth
@@ -396,7 +408,7 @@ def run_attention_only(args):
     print(json.dumps({"attention_prefill": res}))
 
 
-def small_product_sweep(rmm, binding, synth, dev, peaks, rank, reps=40, n_sets=5):
+def small_product_sweep(rmm, binding, synth, dev, peaks, rank, reps=40, n_sets=5, rhos=RHOS):
     """The 1B-class down projection (A 2048 x 8192, B 8192 x 2048): whole op per rho through rmm_product (one front-end
     launch + the product), its kernels, dense cuBLAS at the same shape and cuBLAS on operands gathered beforehand.
     Five (A, B, Y) sets (377 MB, above L2) are rotated."""
@@ -408,7 +420,7 @@ def small_product_sweep(rmm, binding, synth, dev, peaks, rank, reps=40, n_sets=5
         torch.matmul(sets[i % n_sets][0], sets[i % n_sets][1], out=sets[i % n_sets][2])
     dense_ms = time_region(lambda i: torch.matmul(sets[i % n_sets][0], sets[i % n_sets][1], out=sets[i % n_sets][2]), reps, 1)
     out = []
-    for rho in RHOS:
+    for rho in rhos:
         kk = rmm.rmm_keep_count(rho, K1)
         idx_r = torch.empty(kk, dtype=torch.int32, device=dev)
 
@@ -458,6 +470,8 @@ def main():
     ap.add_argument("--rows", type=int, default=M, help="rows of the headline product (smaller: profiler captures)")
     ap.add_argument("--attention-only", action="store_true",
                     help="run only the reduced-attention case (a few launches: for profiler captures) and print its own JSON line")
+    ap.add_argument("--mlp-1b-only", action="store_true",
+                    help="run only the 1B-class product at rho = 0.5 (for profiler captures) and print its own JSON line")
     ap.add_argument("--attn-heads", type=int, default=32)
     ap.add_argument("--attn-seq", type=int, default=4096)
     args = ap.parse_args()
@@ -465,6 +479,8 @@ def main():
         return run_reference(args)
     if args.attention_only:
         return run_attention_only(args)
+    if args.mlp_1b_only:
+        return run_mlp_1b_only(args)
     if args.warmup < 3:
         args.warmup = 3
 
