@@ -59,6 +59,7 @@ struct TcArgs {
     float scale;
     int tiles_m, tiles_n;
     int epi_sets;           // 1, or 2: a second set of four epilogue warps takes every other 64-column chunk
+    int raster;             // tile columns per raster group (see tile_coords)
     int *status;
     unsigned long long wait_ns;  // bound of every device-side wait
     int withhold;                // test switch: the producer skips its very first stage, so that the waits behind it expire
@@ -84,18 +85,19 @@ struct SmemLayout {
     static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack to align the base to 1024 B
 };
 
-// Tile order within one batch entry: column groups of kRasterGroup tiles, rows within a group, columns fastest.  A
-// wave of blocks then shares kRasterGroup column slices of B (which stay in L2 while A streams past) instead of all of
-// them; on 32768-row outputs the GEMM gained 3 to 23 % over plain row-major order, most where N is largest.  Outputs
-// with up to kRasterGroup tile columns keep the row-major order.
-constexpr int kRasterGroup = 16;
-__device__ __forceinline__ void tile_coords(int64_t t, int tiles_m, int tiles_n, int &tm, int &tn)
+// Tile order within one batch entry: column groups of `group` tiles, rows within a group, columns fastest.  A wave of
+// blocks then shares `group` column slices of B (which stay in L2 while A streams past) instead of all of them; on
+// 32768-row outputs the GEMM gained 3 to 23 % over plain row-major order, most where N is largest.  The host picks the
+// group width so that the slices of B that a group keeps alive (group * BN columns x k rows) fit well inside L2: 16 for
+// short contractions, down to 2 for a 28672-long one.  Outputs with up to `group` tile columns keep the row-major order.
+constexpr int kRasterGroupMax = 16;
+__device__ __forceinline__ void tile_coords(int64_t t, int tiles_m, int tiles_n, int group, int &tm, int &tn)
 {
-    const int64_t per_group = (int64_t)kRasterGroup * tiles_m;
+    const int64_t per_group = (int64_t)group * tiles_m;
     const int grp = (int)(t / per_group);
-    const int width = min(kRasterGroup, tiles_n - grp * kRasterGroup);
+    const int width = min(group, tiles_n - grp * group);
     const int64_t r = t - grp * per_group;
-    tn = grp * kRasterGroup + (int)(r % width);
+    tn = grp * group + (int)(r % width);
     tm = (int)(r / width);
 }
 
@@ -159,7 +161,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         for (int64_t tile = tile0; lane == 0 && tile < num_tiles && ok; tile += tile_step) {
             int tm, tn;
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
-            tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, tm, tn);
+            tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, a.raster, tm, tn);
             int64_t bb = (b + a.b_batch_off) / a.b_batch_div;
             if (bb >= a.b_batches) bb = a.b_batches - 1;
             for (int kb = 0; kb < num_kb; ++kb) {
@@ -265,7 +267,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         for (int64_t tile = tile0; tile < num_tiles && ok; tile += tile_step) {
             int tm, tn;
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
-            tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, tm, tn);
+            tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, a.raster, tm, tn);
             int64_t bb = (b + a.b_batch_off) / a.b_batch_div;
             if (bb >= a.b_batches) bb = a.b_batches - 1;
             const int32_t *ix = a.b_idx + b * a.b_idx_stride;
@@ -320,7 +322,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         for (int64_t tile = tile0; tile < num_tiles && ok; tile += tile_step, ++tcount) {
             int tm, tn;
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
-            tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, tm, tn);
+            tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, a.raster, tm, tn);
             const uint32_t acc = tcount & 1u, acc_ph = (tcount >> 1) & 1u;
             if (!mbar_wait(tfull_bar(acc), acc_ph, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
             tc_fence_after();
@@ -544,6 +546,15 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     a.tiles_m = (int)ceil_div(p.M, BM * ctas);
     a.tiles_n = (int)ceil_div(p.N, BN);
     a.status = p.status;
+    {
+        // column slices of B kept alive by one raster group: group * BN columns x k rows of bf16, held to about 40 MB
+        static const int forced_raster = []() { const char *e = getenv("RMM_GEMM_RASTER"); return e ? atoi(e) : 0; }();
+        const int64_t slice = (int64_t)BN * p.k * 2;
+        int64_t grp = slice > 0 ? (40ll << 20) / slice : kRasterGroupMax;
+        if (grp > kRasterGroupMax) grp = kRasterGroupMax;
+        if (grp < 2) grp = 2;
+        a.raster = forced_raster > 0 ? forced_raster : (int)grp;
+    }
     a.wait_ns = wait_limit_ns();
     a.withhold = debug_withhold() == WITHHOLD_GEMM;
     a.col_energy = p.col_energy;
