@@ -158,6 +158,10 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         // ---------------------------------------------------------------- producer (one thread; the others idle)
         uint32_t s = 0, ph = 0;
         bool ok = true;
+        // L2 priority: within a raster group the column slices of B are what every row of tiles comes back to (a row panel
+        // of A is shared only by the tiles of one wave and keeps the default priority: marked evict-first it was dropped
+        // before its last reader arrived and DRAM traffic went up by two thirds)
+        const uint64_t pol_b = l2_policy_evict_last();
         for (int64_t tile = tile0; lane == 0 && tile < num_tiles && ok; tile += tile_step) {
             int tm, tn;
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
@@ -179,12 +183,12 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                         mbar_arrive_expect_tx(full_bar(s), L::kStageBytes);
                         tma_load_3d(sa, &map_a, kb * BK, row_a, (int)b, full_bar(s));
                         if constexpr (B_KMAJOR) {
-                            tma_load_3d(sb, &map_b, kb * BK, col_b, (int)bb, full_bar(s));
+                            tma_load_3d_hint(sb, &map_b, kb * BK, col_b, (int)bb, full_bar(s), pol_b);
                         } else {
                             // 64 contraction rows x 64 columns per load; rows past k read as zeros
 #pragma unroll
                             for (int c = 0; c < BNL / 64; ++c)
-                                tma_load_3d(sb + c * (BK * 128), &map_b, col_b + c * 64, kb * BK, (int)bb, full_bar(s));
+                                tma_load_3d_hint(sb + c * (BK * 128), &map_b, col_b + c * 64, kb * BK, (int)bb, full_bar(s), pol_b);
                         }
                     } else {
                         // both CTAs report their bytes to the leader's barrier; the leader arms it for the pair
@@ -192,11 +196,11 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                         if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * L::kStageBytes);
                         tma_load_3d_pair(sa, &map_a, kb * BK, row_a, (int)b, lead_full);
                         if constexpr (B_KMAJOR) {
-                            tma_load_3d_pair(sb, &map_b, kb * BK, col_b, (int)bb, lead_full);
+                            tma_load_3d_pair_hint(sb, &map_b, kb * BK, col_b, (int)bb, lead_full, pol_b);
                         } else {
 #pragma unroll
                             for (int c = 0; c < BNL / 64; ++c)
-                                tma_load_3d_pair(sb + c * (BK * 128), &map_b, col_b + c * 64, kb * BK, (int)bb, lead_full);
+                                tma_load_3d_pair_hint(sb + c * (BK * 128), &map_b, col_b + c * 64, kb * BK, (int)bb, lead_full, pol_b);
                         }
                     }
                 }
@@ -547,10 +551,10 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     a.tiles_n = (int)ceil_div(p.N, BN);
     a.status = p.status;
     {
-        // column slices of B kept alive by one raster group: group * BN columns x k rows of bf16, held to about 40 MB
+        // column slices of B kept alive by one raster group: group * BN columns x k rows of bf16, held to about 64 MB (half of L2)
         static const int forced_raster = []() { const char *e = getenv("RMM_GEMM_RASTER"); return e ? atoi(e) : 0; }();
         const int64_t slice = (int64_t)BN * p.k * 2;
-        int64_t grp = slice > 0 ? (40ll << 20) / slice : kRasterGroupMax;
+        int64_t grp = slice > 0 ? (64ll << 20) / slice : kRasterGroupMax;
         if (grp > kRasterGroupMax) grp = kRasterGroupMax;
         if (grp < 2) grp = 2;
         a.raster = forced_raster > 0 ? forced_raster : (int)grp;
