@@ -44,7 +44,7 @@ typedef enum {
     RMM_ERR_BOUNDS = 6       /* device status word: an index outside [0, K) was met and skipped */
 } rmm_status_t;
 
-typedef enum { RMM_BF16 = 0, RMM_F32 = 1 } rmm_dtype_t;
+typedef enum { RMM_BF16 = 0, RMM_F32 = 1, RMM_F8E4M3 = 2 /* one byte: 4 exponent bits (bias 7), 3 mantissa bits, no infinities, largest 448; accepted by rmm_reduced_gemm_q8 only */ } rmm_dtype_t;
 
 /* A batch of matrices in device memory.  Element (b, r, c) lives at
  * ptr + (b*stride_batch + r*stride_row + c*stride_col) elements.  stride_batch may be 0 (one matrix
@@ -138,6 +138,19 @@ int rmm_reduced_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx,
 size_t rmm_reduced_gemm_scored_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y);
 int rmm_reduced_gemm_scored(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, int64_t k, float scale,
                             const rmm_mat_t *Y, float *energy_out, void *ws, size_t ws_bytes, void *stream);
+
+/* The reduced product with 8-bit operands (the paper's appendix "Compatibility with quantization" shows that RMM composes
+ * with INT8 inference and leaves a fused low-bit kernel as future work; this is the e4m3 form on the fp8 tensor cores):
+ *   Y = scale * b_scale * diag(s) * Aq Bq[I, :],  Aq[i, j] = e4m3(A[i, I_j] / s_i),  s_i = max_j |A[i, I_j]| / 448
+ * A bf16 [M, K] (batch 1, contiguous rows 16-byte aligned); the activation rows are quantised on the fly, each with its own
+ * step taken over the KEPT columns (an all-zero row: s_i = 1); every decision that yields a code is taken in fp32 (IEEE
+ * division, round to nearest even, saturating).  B holds e4m3 codes of the weight, dtype RMM_F8E4M3, as a [K, N] matrix
+ * with stride_row == 1 (i.e. stored N x K, contraction axis contiguous; stride_col a multiple of 16, base 16-byte
+ * aligned), with one scale b_scale for the tensor.  Y bf16 or fp32 [M, N]; a_scale fp32 [M] receives the s_i (or NULL).
+ * The index set comes from the bf16 activations as always (rmm_score_select).  Accumulation is exact products in fp32. */
+size_t rmm_reduced_gemm_q8_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y);
+int rmm_reduced_gemm_q8(const rmm_mat_t *A, const rmm_mat_t *B, float b_scale, const int32_t *idx, int64_t k, float scale,
+                        const rmm_mat_t *Y, float *a_scale, void *ws, size_t ws_bytes, void *stream);
 
 /* Reduced attention of Sec. 3.3 for B sequences, Hq query heads, Hkv key/value heads (Hq % Hkv == 0,
  * query head h reads kv head h / (Hq/Hkv)).  Per (sequence, query head):

@@ -217,3 +217,64 @@ def attn(Q, K, V, causal: bool, rho_d: float, rho_t: float, round_p: bool = True
                                O.ctypes.data, out_feat.ctypes.data, ptr(out_tok), ptr(P))
     assert rc == 0
     return O, out_feat, out_tok, P
+
+
+# ------------------------------------------------------------------------------------------------
+# 8-bit operands (the paper's appendix "Compatibility with quantization": RMM composed with low-bit inference; the
+# e4m3 form).  Plain numpy, written from the format's definition; pinned in tests/test_oracle_pins.py against the
+# library's own conversion, hand-made ties, and the exact product of small integer codes.
+# ------------------------------------------------------------------------------------------------
+E4M3_MAX = 448.0
+
+
+def e4m3_grid() -> np.ndarray:
+    """Every finite non-negative value of the format, ascending: 1 sign, 4 exponent bits (bias 7), 3 mantissa bits, no
+    infinities; exponent field 0 holds the subnormals m * 2^-9; the all-ones code is NaN, so the largest value is 448."""
+    vals = []
+    for e in range(16):
+        for m in range(8):
+            if e == 15 and m == 7:
+                continue                                   # NaN
+            vals.append(m * 2.0 ** -9 if e == 0 else (1 + m / 8.0) * 2.0 ** (e - 7))
+    return np.array(vals, dtype=np.float64)
+
+
+def round_e4m3(x) -> np.ndarray:
+    """Nearest value of the format to every element of x (given as float32 numbers), ties to the value with the even
+    mantissa code, magnitudes beyond the largest value saturate to +-448.  Returned as float64."""
+    x = np.asarray(x, dtype=np.float32).astype(np.float64)
+    grid = e4m3_grid()
+    a = np.minimum(np.abs(x), E4M3_MAX)
+    hi = np.searchsorted(grid, a, side="left")             # first grid value >= a
+    hi = np.clip(hi, 0, len(grid) - 1)
+    lo = np.clip(hi - 1, 0, len(grid) - 1)
+    d_lo, d_hi = a - grid[lo], grid[hi] - a
+    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))     # codes ascend with the values: even index = even mantissa bit
+    out = np.where(pick_hi, grid[hi], grid[lo])
+    return np.copysign(out, x)
+
+
+def quantize_rows_e4m3(A_kept):
+    """Per-row dynamic quantisation of already gathered activations A[:, I] (given exactly, as float32-representable
+    numbers): step s_i = fp32(max_j |a_ij|) / fp32(448) (1 for an all-zero row), codes q_ij = e4m3(fp32(a_ij / s_i)).
+    The division and the step are taken in fp32, which is the precision the decision is defined in.
+    Returns (values of the codes as float64 [M, k], steps float32 [M])."""
+    A32 = np.asarray(A_kept, dtype=np.float32)
+    amax = np.abs(A32).max(axis=1)
+    step = np.where(amax > 0, (amax / np.float32(448.0)).astype(np.float32), np.float32(1.0)).astype(np.float32)
+    q = round_e4m3((A32 / step[:, None]).astype(np.float32))
+    return q, step
+
+
+def reduced_gemm_q8(A, Bq_values_nk, b_scale: float, idx, rows: Optional[Tuple[int, int]] = None):
+    """Y = diag(s) Aq Bq[I, :] * b_scale in fp64, with Aq, s = quantize_rows_e4m3(A[:, I]) and Bq_values_nk the VALUES of
+    the weight's codes, stored [N, K].  Returns (Y [M, N] fp64, s)."""
+    A = as_np(A)
+    if A.dtype == np.uint16:
+        A = (A.astype(np.uint32) << 16).view(np.float32)
+    idx = np.asarray(as_np(idx), dtype=np.int64)
+    q, step = quantize_rows_e4m3(A[:, idx])
+    Adeq = q * step.astype(np.float64)[:, None]
+    Bdeq = np.ascontiguousarray(np.asarray(Bq_values_nk, dtype=np.float64)[:, idx].T) * float(np.float32(b_scale))
+    Y = reduced_gemm(Adeq, Bdeq, np.arange(len(idx), dtype=np.int32), rows=rows)
+    return Y, step

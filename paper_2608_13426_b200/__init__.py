@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     rmm_product_host,
     rmm_reduced_attn,
     rmm_reduced_gemm,
+    rmm_reduced_gemm_q8,
     rmm_score,
     rmm_score_select,
     rmm_score_select_static,

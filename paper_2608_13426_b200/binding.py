@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "librmm_b200.so")
 
 RMM_OK, RMM_ERR_INVALID_ARG, RMM_ERR_UNSUPPORTED, RMM_ERR_WORKSPACE, RMM_ERR_CUDA, RMM_ERR_TIMEOUT, RMM_ERR_BOUNDS = range(7)
-RMM_BF16, RMM_F32 = 0, 1
+RMM_BF16, RMM_F32, RMM_F8E4M3 = 0, 1, 2
 RMM_WS_HEADER_BYTES = 4096
 _STATUS_NAMES = ["RMM_OK", "RMM_ERR_INVALID_ARG", "RMM_ERR_UNSUPPORTED", "RMM_ERR_WORKSPACE", "RMM_ERR_CUDA",
                  "RMM_ERR_TIMEOUT", "RMM_ERR_BOUNDS"]
@@ -49,7 +49,7 @@ EXPORTS = ["rmm_keep_count", "rmm_score_workspace_bytes", "rmm_score", "rmm_sele
            "rmm_score_select_workspace_bytes", "rmm_score_select", "rmm_score_select_static",
            "rmm_score_select_static_capacity", "rmm_score_select_static_status", "rmm_reduced_gemm_workspace_bytes",
            "rmm_reduced_gemm", "rmm_reduced_gemm_scored_workspace_bytes", "rmm_reduced_gemm_scored",
-           "rmm_reduced_attn_workspace_bytes", "rmm_reduced_attn",
+           "rmm_reduced_gemm_q8_workspace_bytes", "rmm_reduced_gemm_q8", "rmm_reduced_attn_workspace_bytes", "rmm_reduced_attn",
            "rmm_product_workspace_bytes", "rmm_product", "rmm_product_host_workspace_bytes", "rmm_product_host", "rmm_status_read", "rmm_last_error",
            "rmm_launch_count", "rmm_debug_control", "rmm_profile_kernels", "rmm_profile_count", "rmm_profile_name"]
 
@@ -86,6 +86,9 @@ def lib() -> ctypes.CDLL:
     L.rmm_reduced_gemm_scored_workspace_bytes.argtypes = [mp, mp, i64, mp]
     L.rmm_reduced_gemm_scored_workspace_bytes.restype = sz
     L.rmm_reduced_gemm_scored.argtypes = [mp, mp, vp, i64, flt, mp, vp, vp, sz, vp]
+    L.rmm_reduced_gemm_q8_workspace_bytes.argtypes = [mp, mp, i64, mp]
+    L.rmm_reduced_gemm_q8_workspace_bytes.restype = sz
+    L.rmm_reduced_gemm_q8.argtypes = [mp, mp, flt, vp, i64, flt, mp, vp, vp, sz, vp]
     L.rmm_reduced_attn_workspace_bytes.argtypes = [ctypes.POINTER(rmm_attn_desc_t)]
     L.rmm_reduced_attn_workspace_bytes.restype = sz
     L.rmm_reduced_attn.argtypes = [ctypes.POINTER(rmm_attn_desc_t), vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -116,7 +119,9 @@ def _dtype_code(t: torch.Tensor) -> int:
         return RMM_BF16
     if t.dtype == torch.float32:
         return RMM_F32
-    raise RmmError(RMM_ERR_UNSUPPORTED, f"dtype {t.dtype} (bf16 and fp32 only)")
+    if t.dtype == torch.float8_e4m3fn:
+        return RMM_F8E4M3
+    raise RmmError(RMM_ERR_UNSUPPORTED, f"dtype {t.dtype} (bf16, fp32, and e4m3 codes for the 8-bit product)")
 
 
 def as_mat(t: torch.Tensor) -> rmm_mat_t:
@@ -362,6 +367,32 @@ def rmm_reduced_gemm(A: torch.Tensor, B: torch.Tensor, idx: Optional[torch.Tenso
     _check(lib().rmm_reduced_gemm(ctypes.byref(ma), ctypes.byref(mb), idx.data_ptr() if idx is not None else None, k, float(scale),
                                   ctypes.byref(my), p, nb, _stream()))
     return out
+
+
+def rmm_reduced_gemm_q8(A: torch.Tensor, Bq_nk: torch.Tensor, b_scale: float, idx: torch.Tensor, scale: float = 1.0,
+                        out: Optional[torch.Tensor] = None, out_dtype: Optional[torch.dtype] = None, want_scales: bool = False,
+                        ws: Optional[torch.Tensor] = None):
+    """Reduced product with 8-bit operands.  A bf16 [M, K]; Bq_nk float8_e4m3fn [N, K] (the weight as stored, contraction
+    axis contiguous) with one scale b_scale; idx int32 [k].  Returns Y [M, N] (bf16 unless out_dtype says fp32), or
+    (Y, a_scale) with want_scales: the per-row quantisation steps of the activations."""
+    if Bq_nk.dim() != 2 or Bq_nk.dtype != torch.float8_e4m3fn:
+        raise RmmError(RMM_ERR_UNSUPPORTED, "Bq_nk must be a 2-D float8_e4m3fn tensor [N, K]")
+    if idx.dtype != torch.int32 or not idx.is_cuda or not idx.is_contiguous() or idx.dim() != 1:
+        raise RmmError(RMM_ERR_INVALID_ARG, "idx must be a contiguous 1-D int32 CUDA tensor")
+    ma, mb = as_mat(A), as_mat(Bq_nk.t())          # B as a [K, N] matrix whose rows (contraction slices) have stride 1
+    k = idx.numel()
+    if out is None:
+        out = _out((ma.rows, mb.cols), out_dtype if out_dtype is not None else torch.bfloat16, A.device)
+    my = as_mat(out)
+    need = lib().rmm_reduced_gemm_q8_workspace_bytes(ctypes.byref(ma), ctypes.byref(mb), k, ctypes.byref(my))
+    if need == 0:
+        raise RmmError(RMM_ERR_UNSUPPORTED, lib().rmm_last_error().decode())
+    ws = workspace(need, A.device) if ws is None else ws
+    p, nb = _ws_ptr(ws)
+    a_scale = _out((ma.rows,), torch.float32, A.device) if want_scales else None
+    _check(lib().rmm_reduced_gemm_q8(ctypes.byref(ma), ctypes.byref(mb), float(b_scale), idx.data_ptr(), k, float(scale), ctypes.byref(my),
+                                     a_scale.data_ptr() if want_scales else None, p, nb, _stream()))
+    return (out, a_scale) if want_scales else out
 
 
 def rmm_reduced_attn(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, causal: bool, rho_d: float, rho_t: float = 1.0,

@@ -266,6 +266,73 @@ int rmm_reduced_gemm(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx,
     return launch_gemm_simt(A, &b, idx, k, scale, Y, ws, static_cast<cudaStream_t>(stream));
 }
 
+// ---- 8-bit operands -------------------------------------------------------------------------------------
+struct Q8Plan {
+    int64_t ldq;
+    size_t off_aq, off_bq, off_scale, total;
+};
+
+static int plan_q8(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y, Q8Plan *q)
+{
+    if (A == nullptr || B == nullptr || Y == nullptr || A->ptr == nullptr || B->ptr == nullptr || Y->ptr == nullptr)
+        return fail(RMM_ERR_INVALID_ARG, "reduced_gemm_q8: NULL matrix");
+    if (A->batch != 1 || B->batch != 1 || Y->batch != 1) return fail(RMM_ERR_UNSUPPORTED, "reduced_gemm_q8: one product per call (batch 1)");
+    if (A->rows < 1 || A->cols < 1 || B->cols < 1) return fail(RMM_ERR_INVALID_ARG, "reduced_gemm_q8: non-positive dimension");
+    if (A->dtype != RMM_BF16 || B->dtype != RMM_F8E4M3) return fail(RMM_ERR_UNSUPPORTED, "reduced_gemm_q8: A must be bf16 and B e4m3 codes");
+    if (Y->dtype != RMM_BF16 && Y->dtype != RMM_F32) return fail(RMM_ERR_UNSUPPORTED, "reduced_gemm_q8: Y must be bf16 or fp32");
+    if (A->cols != B->rows || Y->rows != A->rows || Y->cols != B->cols) return fail(RMM_ERR_INVALID_ARG, "reduced_gemm_q8: shapes do not agree");
+    if (k < 1 || k > A->cols) return fail(RMM_ERR_INVALID_ARG, "reduced_gemm_q8: k = %lld is outside [1, K]", (long long)k);
+    auto al16 = [](const void *p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; };
+    const int64_t yq = Y->dtype == RMM_BF16 ? 8 : 4;
+    if (A->stride_col != 1 || A->stride_row % 8 != 0 || !al16(A->ptr) || B->stride_row != 1 || B->stride_col % 16 != 0 || !al16(B->ptr) ||
+        Y->stride_col != 1 || Y->stride_row % yq != 0 || !al16(Y->ptr) || A->rows > INT32_MAX || B->cols > INT32_MAX)
+        return fail(RMM_ERR_UNSUPPORTED, "reduced_gemm_q8: operands must have contiguous, 16-byte aligned contraction rows");
+    q->ldq = (k + 15) / 16 * 16;
+    size_t off = RMM_WS_HEADER_BYTES;
+    q->off_aq = off; off += align_up((size_t)A->rows * q->ldq, 256);
+    q->off_bq = off; off += align_up((size_t)B->cols * q->ldq, 256);
+    q->off_scale = off; off += align_up((size_t)A->rows * 4, 256);
+    q->total = off;
+    return RMM_OK;
+}
+
+size_t rmm_reduced_gemm_q8_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y)
+{
+    Q8Plan q = {};
+    return plan_q8(A, B, k, Y, &q) == RMM_OK ? q.total : 0;
+}
+
+int rmm_reduced_gemm_q8(const rmm_mat_t *A, const rmm_mat_t *B, float b_scale, const int32_t *idx, int64_t k, float scale,
+                        const rmm_mat_t *Y, float *a_scale, void *ws, size_t ws_bytes, void *stream)
+{
+    Q8Plan q = {};
+    int rc = plan_q8(A, B, k, Y, &q);
+    if (rc != RMM_OK) return rc;
+    if (idx == nullptr) return fail(RMM_ERR_INVALID_ARG, "reduced_gemm_q8: idx is NULL");
+    rc = check_ws(ws, ws_bytes, q.total, "reduced_gemm_q8");
+    if (rc != RMM_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *w = static_cast<char *>(ws);
+    int *status = &reinterpret_cast<WsHeader *>(w)->status;
+    uint8_t *Aq = reinterpret_cast<uint8_t *>(w + q.off_aq), *Bq = reinterpret_cast<uint8_t *>(w + q.off_bq);
+    float *row_scale = a_scale != nullptr ? a_scale : reinterpret_cast<float *>(w + q.off_scale);
+    rc = launch_gather_q8(true, A->ptr, A->rows, A->stride_row, A->cols, idx, k, Aq, q.ldq, row_scale, status, st);
+    if (rc != RMM_OK) return rc;
+    rc = launch_gather_q8(false, B->ptr, B->cols, B->stride_col, B->rows, idx, k, Bq, q.ldq, nullptr, status, st);
+    if (rc != RMM_OK) return rc;
+    TcProblem p = {};
+    p.batch = 1; p.M = A->rows; p.N = B->cols; p.k = k;
+    p.fp8 = 1; p.row_scale = row_scale;
+    p.a = reinterpret_cast<const __nv_bfloat16 *>(Aq); p.a_ld = q.ldq; p.a_sb = A->rows * q.ldq;
+    p.b_kmajor = 1;
+    p.b = reinterpret_cast<const __nv_bfloat16 *>(Bq); p.b_ld = q.ldq; p.b_sb = B->cols * q.ldq; p.b_batches = 1;
+    p.b_batch_off = 0; p.b_batch_div = 1;
+    p.y = Y->ptr; p.y_bf16 = Y->dtype == RMM_BF16; p.y_sb = Y->stride_batch; p.y_sr = Y->stride_row;
+    p.scale = scale * b_scale;
+    p.status = status;
+    return launch_gemm_tc_problem(p, st);
+}
+
 // ---- product that also scores its output ---------------------------------------------------------------
 size_t rmm_reduced_gemm_scored_workspace_bytes(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, const rmm_mat_t *Y)
 {

@@ -77,12 +77,12 @@ int debug_withhold();
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
-static inline size_t dtype_size(int dt) { return dt == RMM_BF16 ? 2 : 4; }
+static inline size_t dtype_size(int dt) { return dt == RMM_BF16 ? 2 : (dt == RMM_F8E4M3 ? 1 : 4); }
 
 // ---- TMA tensor map for a bf16 tensor: dims / box innermost first, strides in bytes for dims 1..rank-1; 128-byte
 // swizzle or none.  `map` points to a CUtensorMap (opaque here so that only the users include <cuda.h>).
 int make_map(::CUtensorMap_st *map, void *ptr, int rank, const uint64_t *dims, const uint64_t *strides_bytes,
-             const uint32_t *box, bool swizzle128);
+             const uint32_t *box, bool swizzle128, int elem_bytes = 2);
 
 // ---- workspace header: status word, then self-resetting arrival counters --------------------------
 struct WsHeader {
@@ -166,6 +166,10 @@ struct TcProblem {
     int64_t y_sb, y_sr;
     float scale;
     int *status;
+    // 8-bit operands (e4m3 bytes; a and b then point to bytes, leading dimensions and batch strides count bytes, both
+    // K-major): the product of the codes is multiplied by scale * row_scale[batch entry * M + row]
+    int fp8;
+    const float *row_scale;
     // bf16 output only: when set, the epilogue also writes, per 32-row group g and column c, the sum of the squares of the
     // rounded outputs Y[32 g .. 32 g + 31, c] to col_energy[(batch entry * ceil(M / 32) + g) * N + c]
     float *col_energy;
@@ -204,6 +208,13 @@ static inline PackSpec pack_rows_spec(const __nv_bfloat16 *src, int64_t batch, i
 }
 // One launch for one or two gathers.
 int launch_pack(const PackSpec *specs, int n, int *status, cudaStream_t stream);
+
+// Gather of the kept contraction indices into an 8-bit K-major operand (quant.cu): dst[r, j] = code of src[r, idx[j]],
+// j < k, zero bytes up to ld_dst (a multiple of 16).  quantise: src is bf16 and every row gets its own step
+// row_scale[r] = max_j |src[r, idx[j]]| / 448, codes are e4m3(src / step); otherwise src already holds codes (bytes).
+// s_row: elements between two rows of src; rows must start on 16-byte boundaries.
+int launch_gather_q8(bool quantise, const void *src, int64_t rows, int64_t s_row, int64_t K, const int32_t *idx, int64_t k, uint8_t *dst,
+                     int64_t ld_dst, float *row_scale, int *status, cudaStream_t stream);
 
 // ---- attention helpers --------------------------------------------------------------------------------
 // Row softmax of fp32 logits S [heads, Lq, ld_s] with optional end-aligned causal mask; writes bf16

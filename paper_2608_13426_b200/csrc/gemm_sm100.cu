@@ -64,6 +64,7 @@ struct TcArgs {
     unsigned long long wait_ns;  // bound of every device-side wait
     int withhold;                // test switch: the producer skips its very first stage, so that the waits behind it expire
     float *col_energy;           // [batch, ceil(M / 32), N] or NULL: sum of squares of the rounded outputs per 32-row group
+    const float *row_scale;      // 8-bit operands: [batch, M] factor of every output row, or NULL
     // B_GATHER: the unpacked B and the kept row numbers
     const __nv_bfloat16 *b_src;
     const int32_t *b_idx;
@@ -101,7 +102,10 @@ __device__ __forceinline__ void tile_coords(int64_t t, int tiles_m, int tiles_n,
     tm = (int)(r / width);
 }
 
-template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS, bool B_GATHER>
+// FP8: both operands are e4m3 bytes, K-major (tcgen05.mma kind::f8f6f4, 32 contraction indices per instruction); a
+// pipeline stage is still 128 bytes per row, i.e. 128 indices instead of 64, and the epilogue multiplies every output
+// row by its own scale (the activation row's quantisation step times the weight's).
+template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS, bool B_GATHER, bool FP8>
 __global__ void __launch_bounds__(B_GATHER ? kThreadsTc + 32 * kGatherWarps : kThreadsTc2, 1)
 reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                        const __grid_constant__ CUtensorMap map_y, TcArgs a)
@@ -125,7 +129,10 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     if (threadIdx.x == 0) { GSTAMP_MIN(0); }
     const int64_t num_tiles = a.batch * a.tiles_m * a.tiles_n;  // tiles of (128 * CTAS) x BN
     const int64_t tile0 = blockIdx.x / CTAS, tile_step = gridDim.x / CTAS;
-    const int num_kb = (int)((a.k + BK - 1) / BK);
+    constexpr int BKE = FP8 ? 2 * BK : BK;          // contraction indices per stage (128 bytes per row either way)
+    constexpr int UK = FP8 ? 2 * UMMA_K : UMMA_K;   // contraction indices per MMA instruction (32 bytes per row)
+    static_assert(!FP8 || (B_KMAJOR && !B_GATHER), "8-bit operands: both K-major, packed");
+    const int num_kb = (int)((a.k + BKE - 1) / BKE);
 
     if (threadIdx.x == 32) {  // descriptor fetch overlaps barrier set-up and the TMEM allocation
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
@@ -178,12 +185,12 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     const int row_a = tm * (BM * CTAS) + (int)rank * BM, col_b = tn * BN + (int)rank * BNL;
                     if constexpr (B_GATHER) {
                         mbar_arrive_expect_tx(full_bar(s), L::kABytes);
-                        tma_load_3d(sa, &map_a, kb * BK, row_a, (int)b, full_bar(s));
+                        tma_load_3d(sa, &map_a, kb * BKE, row_a, (int)b, full_bar(s));
                     } else if constexpr (CTAS == 1) {
                         mbar_arrive_expect_tx(full_bar(s), L::kStageBytes);
-                        tma_load_3d(sa, &map_a, kb * BK, row_a, (int)b, full_bar(s));
+                        tma_load_3d(sa, &map_a, kb * BKE, row_a, (int)b, full_bar(s));
                         if constexpr (B_KMAJOR) {
-                            tma_load_3d_hint(sb, &map_b, kb * BK, col_b, (int)bb, full_bar(s), pol_b);
+                            tma_load_3d_hint(sb, &map_b, kb * BKE, col_b, (int)bb, full_bar(s), pol_b);
                         } else {
                             // 64 contraction rows x 64 columns per load; rows past k read as zeros
 #pragma unroll
@@ -194,9 +201,9 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                         // both CTAs report their bytes to the leader's barrier; the leader arms it for the pair
                         const uint32_t lead_full = map_to_cta(full_bar(s), 0);
                         if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * L::kStageBytes);
-                        tma_load_3d_pair(sa, &map_a, kb * BK, row_a, (int)b, lead_full);
+                        tma_load_3d_pair(sa, &map_a, kb * BKE, row_a, (int)b, lead_full);
                         if constexpr (B_KMAJOR) {
-                            tma_load_3d_pair_hint(sb, &map_b, kb * BK, col_b, (int)bb, lead_full, pol_b);
+                            tma_load_3d_pair_hint(sb, &map_b, kb * BKE, col_b, (int)bb, lead_full, pol_b);
                         } else {
 #pragma unroll
                             for (int c = 0; c < BNL / 64; ++c)
@@ -211,7 +218,8 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     } else if (warp == 1 && rank == 0) {
         // ---------------------------------------------------------------- MMA issuer (the pair's leader only)
         // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B K- or MN-major, N = BN, M = 128
-        constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((B_KMAJOR ? 0u : 1u) << 16) |
+        // (operand format fields: 1 = bf16 for kind::f16, 0 = e4m3 for kind::f8f6f4)
+        constexpr uint32_t idesc = (1u << 4) | ((FP8 ? 0u : 1u) << 7) | ((FP8 ? 0u : 1u) << 10) | ((B_KMAJOR ? 0u : 1u) << 16) |
                                    ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CTAS) >> 4) << 24);
         // The issuing thread is the pacemaker of the whole kernel (one thread feeds the tensor cores of one or two
         // SMs), so its loop is kept short: stage and phase are counters, descriptors advance by one add each.
@@ -222,7 +230,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         const uint32_t a_hi = (uint32_t)(da0 >> 32), b_hi = (uint32_t)(db0 >> 32);
         const uint32_t a_lo0 = (uint32_t)da0, b_lo0 = (uint32_t)db0;
         constexpr uint32_t kStageUnits = L::kStageBytes >> 4, kAStep = 32 >> 4, kBStep = (B_KMAJOR ? 32 : 2048) >> 4;
-        const int last_steps = (int)((a.k - (int64_t)(num_kb - 1) * BK + UMMA_K - 1) / UMMA_K);  // MMAs of the last k-block
+        const int last_steps = (int)((a.k - (int64_t)(num_kb - 1) * BKE + UK - 1) / UK);  // MMAs of the last k-block
         uint32_t stage = 0, phase = 0, tcount = 0;
         bool ok = true;
         for (int64_t tile = tile0; lane == 0 && tile < num_tiles && ok; tile += tile_step, ++tcount) {
@@ -240,12 +248,12 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 if (kb + 1 < num_kb || last_steps == BK / UMMA_K) {
 #pragma unroll
                     for (int ks = 0; ks < BK / UMMA_K; ++ks) {
-                        umma_bf16_lohi<CTAS>(d_tmem, a_lo + ks * kAStep, a_hi, b_lo + ks * kBStep, b_hi, idesc, accumulate);
+                        umma_lohi<CTAS, FP8>(d_tmem, a_lo + ks * kAStep, a_hi, b_lo + ks * kBStep, b_hi, idesc, accumulate);
                         accumulate = 1;
                     }
                 } else {
                     for (int ks = 0; ks < last_steps; ++ks) {
-                        umma_bf16_lohi<CTAS>(d_tmem, a_lo + ks * kAStep, a_hi, b_lo + ks * kBStep, b_hi, idesc, accumulate);
+                        umma_lohi<CTAS, FP8>(d_tmem, a_lo + ks * kAStep, a_hi, b_lo + ks * kBStep, b_hi, idesc, accumulate);
                         accumulate = 1;
                     }
                 }
@@ -334,6 +342,10 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
             const int64_t m_warp = (int64_t)tm * (BM * CTAS) + rank * BM + q * 32, m = m_warp + lane;
             const int64_t n0 = (int64_t)tn * BN;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
+            float scale_r = a.scale;  // this thread's output row: the common factor times the row's own (8-bit operands)
+            if constexpr (FP8) {
+                if (a.row_scale != nullptr && m < a.M) scale_r *= __ldg(a.row_scale + b * a.M + m);
+            }
             if constexpr (OUT_BF16) {
                 // 64 columns at a time: two TMEM loads, scale and round, one 32 x 64 slab per warp through a TMA store
 #pragma unroll 1
@@ -356,8 +368,8 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                             uint32_t w[4];
 #pragma unroll
                             for (int p = 0; p < 4; ++p) {
-                                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * v + 2 * p]) * a.scale,
-                                                                         __uint_as_float(r[8 * v + 2 * p + 1]) * a.scale);
+                                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * v + 2 * p]) * scale_r,
+                                                                         __uint_as_float(r[8 * v + 2 * p + 1]) * scale_r);
                                 w[p] = *reinterpret_cast<uint32_t *>(&h);
                             }
                             *reinterpret_cast<uint4 *>(row + (((u0 + v) ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -406,10 +418,10 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 #pragma unroll
                         for (int v = 0; v < 8; ++v)
                             reinterpret_cast<float4 *>(y)[v] =
-                                make_float4(__uint_as_float(r[4 * v]) * a.scale, __uint_as_float(r[4 * v + 1]) * a.scale,
-                                            __uint_as_float(r[4 * v + 2]) * a.scale, __uint_as_float(r[4 * v + 3]) * a.scale);
+                                make_float4(__uint_as_float(r[4 * v]) * scale_r, __uint_as_float(r[4 * v + 1]) * scale_r,
+                                            __uint_as_float(r[4 * v + 2]) * scale_r, __uint_as_float(r[4 * v + 3]) * scale_r);
                     } else {
-                        for (int e = 0; e < 32 && n + e < a.N; ++e) y[e] = __uint_as_float(r[e]) * a.scale;
+                        for (int e = 0; e < 32 && n + e < a.N; ++e) y[e] = __uint_as_float(r[e]) * scale_r;
                     }
                 };
                 // four TMEM loads in flight per wait: the load latency is paid BN / 128 times per tile instead of BN / 32
@@ -461,10 +473,10 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 // ----------------------------------------------------------------------------------------------
 // host side
 // ----------------------------------------------------------------------------------------------
-template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS, bool B_GATHER = false>
+template <int BN, bool B_KMAJOR, bool OUT_BF16, int CTAS, bool B_GATHER = false, bool FP8 = false>
 int launch_variant(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &my, const TcArgs &a, cudaStream_t stream)
 {
-    auto kern = reduced_gemm_tc_kernel<BN, B_KMAJOR, OUT_BF16, CTAS, B_GATHER>;
+    auto kern = reduced_gemm_tc_kernel<BN, B_KMAJOR, OUT_BF16, CTAS, B_GATHER, FP8>;
     using L = SmemLayout<BN, CTAS>;
     static PerDeviceOnce configured;
     if (configured.first()) {
@@ -524,11 +536,15 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
 {
     CUtensorMap ma, mb;
     int rc;
+    const int es = p.fp8 ? 1 : 2;             // bytes per operand element
+    const uint32_t bke = p.fp8 ? 2 * BK : BK;  // contraction indices per 128-byte stage row
+    if (p.fp8 && (!p.b_kmajor || p.b_idx != nullptr))
+        return fail(RMM_ERR_UNSUPPORTED, "reduced_gemm_tc: 8-bit operands must both be K-major and packed");
     {
         uint64_t dims[3] = {(uint64_t)p.k, (uint64_t)p.M, (uint64_t)p.batch};
-        uint64_t st[2] = {(uint64_t)p.a_ld * 2, (uint64_t)p.a_sb * 2};
-        uint32_t box[3] = {BK, BM, 1};
-        rc = make_map(&ma, const_cast<__nv_bfloat16 *>(p.a), 3, dims, st, box, true);
+        uint64_t st[2] = {(uint64_t)p.a_ld * es, (uint64_t)p.a_sb * es};
+        uint32_t box[3] = {bke, BM, 1};
+        rc = make_map(&ma, const_cast<__nv_bfloat16 *>(p.a), 3, dims, st, box, true, es);
         if (rc != RMM_OK) return rc;
     }
     const int BN = p.N <= 128 ? 128 : 256;
@@ -553,7 +569,7 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     {
         // column slices of B kept alive by one raster group: group * BN columns x k rows of bf16, held to about 64 MB (half of L2)
         static const int forced_raster = []() { const char *e = getenv("RMM_GEMM_RASTER"); return e ? atoi(e) : 0; }();
-        const int64_t slice = (int64_t)BN * p.k * 2;
+        const int64_t slice = (int64_t)BN * p.k * es;
         int64_t grp = slice > 0 ? (64ll << 20) / slice : kRasterGroupMax;
         if (grp > kRasterGroupMax) grp = kRasterGroupMax;
         if (grp < 2) grp = 2;
@@ -562,10 +578,11 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     a.wait_ns = wait_limit_ns();
     a.withhold = debug_withhold() == WITHHOLD_GEMM;
     a.col_energy = p.col_energy;
+    a.row_scale = p.row_scale;
     // products with at most four k-blocks per tile are bound by the epilogue, and a block with a single tile has no next
     // main loop to hide its epilogue behind: two sets of epilogue warps in both cases
     const int64_t n_tiles = p.batch * ceil_div(p.M, BM * ctas) * ceil_div(p.N, BN);
-    a.epi_sets = (p.y_bf16 && p.b_idx == nullptr && (ceil_div(p.k, BK) <= 4 || n_tiles <= sm_count() / ctas)) ? 2 : 1;
+    a.epi_sets = (p.y_bf16 && p.b_idx == nullptr && (ceil_div(p.k, (int64_t)bke) <= 4 || n_tiles <= sm_count() / ctas)) ? 2 : 1;
     a.b_src = p.b; a.b_idx = p.b_idx; a.b_ld = p.b_ld; a.b_sb = p.b_batches > 1 ? p.b_sb : 0; a.b_idx_stride = p.b_idx_stride;
     a.b_rows = p.b_rows;
     if (p.b_idx != nullptr) {
@@ -582,12 +599,12 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
         }
         return launch_variant<256, false, false, 1, true>(ma, ma, my_g, a, stream);
     }
-    const uint64_t b_sb = p.b_batches > 1 ? (uint64_t)p.b_sb * 2 : (uint64_t)p.b_ld * 2 * (uint64_t)(p.b_kmajor ? p.N : p.k);
+    const uint64_t b_sb = p.b_batches > 1 ? (uint64_t)p.b_sb * es : (uint64_t)p.b_ld * es * (uint64_t)(p.b_kmajor ? p.N : p.k);
     if (p.b_kmajor) {
         uint64_t dims[3] = {(uint64_t)p.k, (uint64_t)p.N, (uint64_t)p.b_batches};
-        uint64_t st[2] = {(uint64_t)p.b_ld * 2, b_sb};
-        uint32_t box[3] = {BK, (uint32_t)(BN / ctas), 1};
-        rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 3, dims, st, box, true);
+        uint64_t st[2] = {(uint64_t)p.b_ld * es, b_sb};
+        uint32_t box[3] = {bke, (uint32_t)(BN / ctas), 1};
+        rc = make_map(&mb, const_cast<__nv_bfloat16 *>(p.b), 3, dims, st, box, true, es);
     } else {
         uint64_t dims[3] = {(uint64_t)p.N, (uint64_t)p.k, (uint64_t)p.b_batches};
         uint64_t st[2] = {(uint64_t)p.b_ld * 2, b_sb};
@@ -604,6 +621,11 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
         uint32_t box[3] = {64, 32, 1};
         rc = make_map(&my, p.y, 3, dims, st, box, true);
         if (rc != RMM_OK) return rc;
+    }
+    if (p.fp8) {
+        if (ctas == 2) return out_bf16 ? launch_variant<256, true, true, 2, false, true>(ma, mb, my, a, stream) : launch_variant<256, true, false, 2, false, true>(ma, mb, my, a, stream);
+        if (BN == 256) return out_bf16 ? launch_variant<256, true, true, 1, false, true>(ma, mb, my, a, stream) : launch_variant<256, true, false, 1, false, true>(ma, mb, my, a, stream);
+        return out_bf16 ? launch_variant<128, true, true, 1, false, true>(ma, mb, my, a, stream) : launch_variant<128, true, false, 1, false, true>(ma, mb, my, a, stream);
     }
     if (ctas == 2) {
         if (p.b_kmajor) return out_bf16 ? launch_variant<256, true, true, 2>(ma, mb, my, a, stream) : launch_variant<256, true, false, 2>(ma, mb, my, a, stream);

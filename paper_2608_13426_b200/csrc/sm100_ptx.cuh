@@ -291,6 +291,32 @@ __device__ __forceinline__ void umma_bf16_lohi(uint32_t d_tmem, uint32_t a_lo, u
             : "memory");
     }
 }
+// Either operand kind: bf16 (kind::f16) or 8-bit e4m3 / e5m2 (kind::f8f6f4); same operand descriptors, the formats are
+// in the instruction descriptor.
+template <int CTAS, bool FP8>
+__device__ __forceinline__ void umma_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    if constexpr (!FP8) {
+        umma_bf16_lohi<CTAS>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+    } else if constexpr (CTAS == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+            "setp.ne.b32 p, %6, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %5, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+            "setp.ne.b32 p, %6, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %5, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
 // Arrive on an mbarrier once every tcgen05 operation issued so far by this thread has completed.  CTAS == 2: the
 // arrival is delivered to the barrier at this offset in both CTAs of the pair.
 template <int CTAS>

@@ -1,4 +1,4 @@
-// Host helper: TMA tensor maps (cuTensorMapEncodeTiled fetched through the runtime, so the library links against
+// Host helper: TMA tensor maps (bf16 elements, or bytes for 8-bit operands) (cuTensorMapEncodeTiled fetched through the runtime, so the library links against
 // libcudart only).
 #include <cuda.h>
 
@@ -24,7 +24,7 @@ static EncodeTiledFn encode_fn()
 }
 
 int make_map(CUtensorMap *map, void *ptr, int rank, const uint64_t *dims, const uint64_t *strides_bytes,
-             const uint32_t *box, bool swizzle128)
+             const uint32_t *box, bool swizzle128, int elem_bytes)
 {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return fail(RMM_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
@@ -32,7 +32,7 @@ int make_map(CUtensorMap *map, void *ptr, int rank, const uint64_t *dims, const 
     cuuint32_t bx[5], es[5];
     for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
     for (int i = 0; i + 1 < rank; ++i) st[i] = strides_bytes[i];
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, ptr, d, st, bx, es,
+    CUresult r = fn(map, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, ptr, d, st, bx, es,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(RMM_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);

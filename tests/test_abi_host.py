@@ -23,7 +23,7 @@ def L():
 def declared_symbols():
     text = open(os.path.join(ROOT, "include", "rmm.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(rmm_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(rmm_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_header_symbols_are_exported(L):

@@ -630,3 +630,49 @@ def test_next_product_selects_from_epilogue_energies(oracle):
     for r in rows:
         want = oracle.reduced_gemm(H.cpu(), W_down, idx.cpu().numpy(), rows=(r, r + 1))[r]
         assert rel_fro(Y[r].float().cpu().numpy(), want) <= TOL_BF16
+
+
+# ------------------------------------------------------------------------------------------------
+# 8-bit operands (e4m3 codes on the fp8 tensor cores)
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("M,K,N,rho", [(128, 256, 256, 0.5), (300, 1008, 264, 0.75), (2048, 8192, 2048, 0.5), (77, 4096, 128, 0.25),
+                                       (4096, 2048, 4864, 1.0), (513, 528, 1032, 0.3)])
+def test_reduced_product_with_8_bit_operands(oracle, M, K, N, rho):
+    """Activation rows quantised on the fly over the kept columns (per-row step), weight given as e4m3 codes [N, K] with one
+    scale.  The steps must equal the oracle's bit for bit (every decision in fp32); Y is held to the product of the
+    oracle's dequantised operands: 1e-5 with fp32 output (exact products, fp32 accumulation), 1e-2 with bf16 output.
+    Single-CTA and CTA-pair tiles, ragged last stage (k not a multiple of 128 or of 16), ragged rows and columns."""
+    A = synth.heavy_tailed_activations(M, K, seed=M + 5)
+    W = synth.weight(K, N, seed=M + 6, dtype=torch.float32)                       # fp32 weight, to be quantised offline
+    b_scale = float(W.abs().max()) / 448.0
+    Bq = (W.t().contiguous() / b_scale).to(torch.float8_e4m3fn)                   # stored [N, K]
+    Ad, Bqd = dev(A), Bq.cuda()
+    idx, _, _, _ = rmm.rmm_score_select(Ad, rho=rho)
+    idx_np = idx.cpu().numpy()
+    check_index_set(idx_np, oracle.score(A)[0], oracle.keep_count(rho, K))
+    Yf, s = rmm.rmm_reduced_gemm_q8(Ad, Bqd, b_scale, idx, out_dtype=torch.float32, want_scales=True)
+    Yb = rmm.rmm_reduced_gemm_q8(Ad, Bqd, b_scale, idx, scale=0.5)
+    rows = sorted({0, 1, 127, 128, M // 2, M - 1} & set(range(M)))
+    want_rows, want_s = [], None
+    Bv = Bq.to(torch.float64).numpy()
+    for r in rows:
+        Yo, so = oracle.reduced_gemm_q8(A[r:r + 1], Bv, b_scale, idx_np)
+        want_rows.append(Yo[0])
+        assert float(s[r]) == float(so[0]), (r, float(s[r]), float(so[0]))
+    want = np.stack(want_rows)
+    assert rel_fro(Yf[rows].cpu().numpy(), want) <= 1e-5
+    assert rel_fro(Yb[rows].float().cpu().numpy(), 0.5 * want) <= TOL_BF16
+    assert torch.isfinite(Yf).all()
+    # and the quantised product is close to the unquantised one on the same index set (the point of the 8-bit form)
+    Y16 = rmm.rmm_reduced_gemm(Ad, dev(W.to(torch.bfloat16)), idx, out_dtype=torch.float32)
+    assert rel_fro(Yf.cpu().numpy(), Y16.cpu().numpy().astype(np.float64)) <= 0.08
+    assert rmm.rmm_status_read() == 0
+
+
+def test_8_bit_product_refuses_unaligned_weight_rows():
+    A = dev(synth.heavy_tailed_activations(64, 1000, seed=1))
+    Bq = torch.zeros(128, 1000, dtype=torch.float8_e4m3fn, device="cuda")          # rows of 1000 bytes: not 16-byte multiples
+    idx = torch.arange(500, dtype=torch.int32, device="cuda")
+    with pytest.raises(rmm.RmmError) as e:
+        rmm.rmm_reduced_gemm_q8(A, Bq, 1.0, idx)
+    assert e.value.code == 2

@@ -454,3 +454,58 @@ def test_attention_on_sampled_query_rows(oracle, causal):
     assert np.array_equal(Itr, It) and np.array_equal(O5r, O5[:, :, rows])
     with pytest.raises(AssertionError):
         oracle.attn(Q, K, V, causal, 0.5, 0.4, rows=rows)
+
+
+# --------------------------------------------------------------------------------------------
+# 8-bit operands (appendix "Compatibility with quantization"): the e4m3 rounding, the per-row step, the product
+# --------------------------------------------------------------------------------------------
+def test_e4m3_rounding_against_the_library_and_the_definition(oracle):
+    grid = oracle.e4m3_grid()
+    assert len(grid) == 127 and grid[0] == 0.0 and grid[1] == 2.0 ** -9 and grid[-1] == 448.0
+    assert np.all(np.diff(grid) > 0)
+    # every value of the format is a fixed point, in both signs
+    assert np.array_equal(oracle.round_e4m3(grid), grid) and np.array_equal(oracle.round_e4m3(-grid), -grid)
+    # the library's conversion (round to nearest even) on a dense sweep inside the range
+    g = torch.Generator().manual_seed(5)
+    x = torch.cat([torch.randn(200000, generator=g) * 100, torch.randn(50000, generator=g) * 0.01, torch.linspace(-448, 448, 100001)])
+    x = x[x.abs() <= 448].float()
+    want = x.to(torch.float8_e4m3fn).to(torch.float64).numpy()
+    assert np.array_equal(oracle.round_e4m3(x.numpy()), want)
+    # hand-made ties: half way between neighbours goes to the even mantissa code
+    assert oracle.round_e4m3([1.0625])[0] == 1.0          # 1.0 (code ..000) | 1.125 (..001)
+    assert oracle.round_e4m3([1.1875])[0] == 1.25         # 1.125 (..001) | 1.25 (..010)
+    assert oracle.round_e4m3([2.0 ** -10])[0] == 0.0      # 0 | smallest subnormal 2^-9: tie to the even code 0
+    assert oracle.round_e4m3([3 * 2.0 ** -10])[0] == 2.0 ** -8
+    # saturation instead of overflow
+    assert np.array_equal(oracle.round_e4m3([449.0, 1e9, -1e9]), [448.0, 448.0, -448.0])
+
+
+def test_row_quantisation_and_8_bit_product(oracle):
+    # steps: the row maximum maps onto 448 exactly; an all-zero row has step 1 and codes 0
+    A = np.array([[448.0, -224.0, 1.0, 0.0], [0.0, 0.0, 0.0, 0.0], [3.0, -7.0, 0.5, 0.25]], dtype=np.float32)
+    q, s = oracle.quantize_rows_e4m3(A)
+    assert s[0] == 1.0 and np.array_equal(q[0], [448.0, -224.0, 1.0, 0.0])
+    assert s[1] == 1.0 and not q[1].any()
+    assert s[2] == np.float32(7.0) / np.float32(448.0) and q[2, 1] == -448.0 and q[2, 0] == 192.0 and q[2, 2] == 32.0
+    # operands whose codes are exact: entries 0, +-1, +-2, +-4, +-8 with row maximum 8 (step 8 / 448, codes a * 56 are all
+    # values of the format), so the quantised product equals the plain one up to the fp32 rounding of the step
+    rng = np.random.default_rng(0)
+    M, K, N = 5, 24, 7
+    Aint = (rng.choice([0.0, 1.0, 2.0, 4.0, 8.0], size=(M, K)) * rng.choice([-1.0, 1.0], size=(M, K))).astype(np.float32)
+    Aint[:, 0] = 8.0
+    Bq = rng.choice(oracle.e4m3_grid()[:40], size=(N, K)) * rng.choice([-1.0, 1.0], size=(N, K))
+    idx = np.array([0, 5, 2, 23, 11, 7], dtype=np.int32)
+    Y, s = oracle.reduced_gemm_q8(Aint, Bq, 0.5, idx)
+    assert np.all(s == np.float32(8.0) / np.float32(448.0))
+    want = (Aint[:, idx].astype(np.float64) @ Bq[:, idx].T) * 0.5
+    assert np.allclose(Y, want, rtol=1e-7, atol=0)               # (the fp32 step 8/448 is not a power of two: 6e-8 relative)
+    # against the library end to end: torch's own conversion of A / step, dequantised, matmul in fp64
+    A2 = synth.heavy_tailed_activations(33, 64, seed=3)
+    idx2 = np.sort(rng.choice(64, 20, replace=False)).astype(np.int32)
+    Bq2 = (torch.randn(9, 64, generator=torch.Generator().manual_seed(1)) * 0.3).to(torch.float8_e4m3fn)
+    Y2, s2 = oracle.reduced_gemm_q8(A2, Bq2.to(torch.float64).numpy(), 0.02, idx2)
+    Asel = A2.float()[:, idx2.tolist()]
+    st = Asel.abs().amax(dim=1) / 448.0
+    qt = (Asel / st[:, None]).to(torch.float8_e4m3fn).to(torch.float64)
+    want2 = (qt * st.double()[:, None]) @ (Bq2.to(torch.float64)[:, idx2.tolist()].T * float(np.float32(0.02)))
+    assert np.array_equal(s2, st.numpy()) and np.allclose(Y2, want2.numpy(), rtol=1e-12, atol=1e-300)
