@@ -386,6 +386,36 @@ def gemm_framed_attention(rmm, synth, dev, peaks, reps=5):
     return out
 
 
+def low_bit_sweep(rmm, binding, synth, dev, peaks, reps=10):
+    """The reduced product with 8-bit operands (e4m3 activations quantised on the fly, e4m3 weight) beside the bf16 one, on
+    the 1B-class and the 70B-class down projection at rho = 0.5: gathers + product, and the product kernel alone."""
+    out = []
+    for (m, kk, n) in ((M1, K1, N1), (M, K, N)):
+        A = synth.heavy_tailed_activations(m, kk, seed=5, device=str(dev))
+        W = synth.weight(kk, n, seed=6, device=str(dev))
+        b_scale = float(W.abs().max()) / 448.0
+        Bq = (W.t().float() / b_scale).to(torch.float8_e4m3fn).contiguous()
+        Y = torch.empty(m, n, dtype=torch.bfloat16, device=dev)
+        idx, _, _, _ = rmm.rmm_score_select(A, rho=RHO)
+        row = {"shape": [m, kk, n], "rho": RHO, "k": int(idx.numel())}
+        for name, fn in (("bf16", lambda i: rmm.rmm_reduced_gemm(A, W, idx, out=Y)),
+                         ("e4m3", lambda i: rmm.rmm_reduced_gemm_q8(A, Bq, b_scale, idx, out=Y))):
+            for i in range(3):
+                fn(i)
+            t = time_region(fn, reps, 1)
+            kt = binding.KernelTimer(reps, "reduced_gemm_tc_kernel")
+            with kt:
+                time_region(fn, reps, 1)
+            g = sum(x for _, x in kt.times_ms()) / reps
+            fl = 2.0 * m * idx.numel() * n
+            row[name] = {"gathers_and_product_ms": t, "product_kernel_ms": g, "product_kernel_tflops": fl / g / 1e9}
+        row["e4m3_speedup_product_kernel"] = row["bf16"]["product_kernel_ms"] / row["e4m3"]["product_kernel_ms"]
+        row["e4m3_speedup_with_gathers"] = row["bf16"]["gathers_and_product_ms"] / row["e4m3"]["gathers_and_product_ms"]
+        out.append(row)
+        del A, W, Bq, Y
+    return out
+
+
 def run_mlp_1b_only(args):
     """Only the 1B-class product at rho = 0.5 (a few dozen launches: for profiler captures of the one-launch front end
     and of the single-tile GEMM); prints its own JSON line."""
@@ -657,6 +687,9 @@ def main():
         extras["attention_prefill"] = attention_case(rmm, binding, synth, dev, 32, 4096)
         extras["attention_paper_setting"] = paper_table5_case(rmm, synth, dev)
         extras["attention_products_in_memory"] = gemm_framed_attention(rmm, synth, dev, peaks)
+
+        # ---- 8-bit operands beside bf16
+        extras["low_bit_operands"] = low_bit_sweep(rmm, binding, synth, dev, peaks)
 
         # ---- the other 70B-class products and the attention of one layer
         extras["layer_sweep_70b"] = layer_sweep_70b(rmm, synth, dev, peaks)

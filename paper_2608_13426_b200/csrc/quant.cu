@@ -9,6 +9,7 @@
 #include <cuda_fp8.h>
 
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace rmm {
 namespace {
@@ -82,12 +83,156 @@ __global__ void __launch_bounds__(kThreadsQ) gather_q8_kernel(const void *__rest
     }
 }
 
+
+// The same gather as a streaming kernel: one persistent 1024-thread block per SM owns a contiguous range of rows, which
+// arrive through two shared-memory buffers by bulk asynchronous copies (the next row lands while the current one is
+// worked on).  Thread t owns the output words t, t + 1024, ... (four codes each) and keeps the byte offsets of their
+// source columns in registers for all its rows, so the index list is read once per block instead of once per row.
+constexpr int kThreadsS = 1024;
+constexpr int kWordsS = 8;                       // output words per thread: k <= 4 * 8 * 1024
+constexpr int kStreamMaxRowBytes = 110 * 1024;   // two such rows (and their zero pads) fit in shared memory
+
+template <bool QUANT>
+__global__ void __launch_bounds__(kThreadsS, 1) gather_q8_stream_kernel(const void *__restrict__ src, int64_t s_row, int K, const int32_t *__restrict__ idx,
+                                                                         int k, uint8_t *__restrict__ dst, int64_t ld_dst, float *__restrict__ row_scale,
+                                                                         int64_t rows, int64_t per_block, int *status, unsigned long long wait_ns)
+{
+    using namespace ptx;
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ uint64_t full[2];
+    __shared__ int abort_flag;
+    __shared__ float s_red[kThreadsS / 32];
+    constexpr int ES = QUANT ? 2 : 1;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t row_bytes = (uint32_t)K * ES;           // a multiple of 16
+    const uint32_t pitch = row_bytes + 16;                  // 16 zero bytes after each staged row: where missing indices point
+    if (tid == 0) {
+        mbar_init(smem_u32(&full[0]), 1);
+        mbar_init(smem_u32(&full[1]), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (tid < 8) {
+        reinterpret_cast<uint32_t *>(smem + row_bytes)[tid & 3] = 0;
+        reinterpret_cast<uint32_t *>(smem + pitch + row_bytes)[tid & 3] = 0;
+    }
+    __syncthreads();
+    pdl_wait();
+    const int64_t lo = (int64_t)blockIdx.x * per_block, hi = min(rows, lo + per_block);
+    auto issue = [&](int64_t r, int stage) {  // thread 0: one row, global -> shared
+        const unsigned char *g = static_cast<const unsigned char *>(src) + r * s_row * ES;
+        const uint32_t bar = smem_u32(&full[stage]), d = smem_u32(smem) + (uint32_t)stage * pitch;
+        mbar_arrive_expect_tx(bar, row_bytes);
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(d), "l"(g), "r"(row_bytes), "r"(bar) : "memory");
+    };
+    if (tid == 0 && lo < hi) issue(lo, 0);
+    // source columns of this thread's outputs inside a staged row (column K = the zero pad).  bf16 rows hold at most
+    // 55 K columns, so two column numbers share a register; byte rows keep one offset per register.
+    constexpr int kRegs = QUANT ? 2 * kWordsS : 4 * kWordsS;
+    uint32_t cb[kRegs];
+    const int words = (int)(ld_dst / 4);
+#pragma unroll
+    for (int i = 0; i < kWordsS; ++i) {
+        const int w = tid + i * kThreadsS;
+        uint32_t col[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int j = 4 * w + e;
+            col[e] = (uint32_t)K;
+            if (w < words && j < k) {
+                const int c = __ldg(idx + j);
+                if (c < 0 || c >= K) atomicExch(status, (int)RMM_ERR_BOUNDS);
+                else col[e] = (uint32_t)c;
+            }
+        }
+        if constexpr (QUANT) {
+            cb[2 * i] = col[0] | (col[1] << 16);
+            cb[2 * i + 1] = col[2] | (col[3] << 16);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) cb[4 * i + e] = col[e];
+        }
+    }
+    auto offset = [&](int i, int e) -> uint32_t {  // byte offset of output e of word i inside the staged row
+        if constexpr (QUANT) return ((cb[2 * i + (e >> 1)] >> (16 * (e & 1))) & 0xffffu) * 2u;
+        else return cb[4 * i + e];
+    };
+    for (int64_t r = lo; r < hi; ++r) {
+        const int it = (int)(r - lo), stage = it & 1;
+        // the other buffer was last read in the previous iteration, which ended with a block-wide barrier
+        if (tid == 0 && r + 1 < hi) issue(r + 1, stage ^ 1);
+        const bool landed = mbar_wait(smem_u32(&full[stage]), (uint32_t)(it >> 1) & 1u, &abort_flag, status, wait_ns);
+        if (!__syncthreads_and(landed)) break;
+        const unsigned char *row = smem + (size_t)stage * pitch;
+        float step = 1.f;
+        if constexpr (QUANT) {
+            float amax = 0.f;
+#pragma unroll
+            for (int i = 0; i < kWordsS; ++i)
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    amax = fmaxf(amax, fabsf(__uint_as_float((unsigned)*reinterpret_cast<const unsigned short *>(row + offset(i, e)) << 16)));
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+            if (lane == 0) s_red[warp] = amax;
+            __syncthreads();
+            amax = s_red[lane];
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+            step = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+            if (tid == 0) row_scale[r] = step;
+        }
+        uint32_t *drow = reinterpret_cast<uint32_t *>(dst + r * ld_dst);
+#pragma unroll
+        for (int i = 0; i < kWordsS; ++i) {
+            const int w = tid + i * kThreadsS;
+            if (w < words) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    uint32_t code;
+                    if constexpr (QUANT) {
+                        const float x = __uint_as_float((unsigned)*reinterpret_cast<const unsigned short *>(row + offset(i, e)) << 16);
+                        code = __nv_cvt_float_to_fp8(__fdiv_rn(x, step), __NV_SATFINITE, __NV_E4M3);
+                    } else {
+                        code = row[offset(i, e)];
+                    }
+                    word |= code << (8 * e);
+                }
+                drow[w] = word;
+            }
+        }
+        __syncthreads();
+    }
+}
+
 }  // namespace
 
 int launch_gather_q8(bool quantise, const void *src, int64_t rows, int64_t s_row, int64_t K, const int32_t *idx, int64_t k, uint8_t *dst,
                      int64_t ld_dst, float *row_scale, int *status, cudaStream_t stream)
 {
-    const size_t smem = align_up((size_t)K * (quantise ? 2 : 1), 16);
+    const size_t row_bytes = (size_t)K * (quantise ? 2 : 1);
+    if (row_bytes % 16 == 0 && row_bytes <= (size_t)kStreamMaxRowBytes && ld_dst <= 4 * kWordsS * kThreadsS && rows >= 32 * (int64_t)sm_count()) {  // (few rows: one block per row keeps every SM busy)
+        static PerDeviceOnce stream_configured;
+        if (stream_configured.first()) {
+            cudaError_t e = cudaFuncSetAttribute(gather_q8_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * (kStreamMaxRowBytes + 16));
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(gather_q8_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * (kStreamMaxRowBytes + 16));
+            if (e != cudaSuccess) return fail(RMM_ERR_CUDA, "gather_q8: cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+        }
+        const int64_t per_block = ceil_div(rows, sm_count());
+        const unsigned grid = (unsigned)ceil_div(rows, per_block);
+        prof_begin("gather_q8_stream_kernel", stream);
+        if (quantise)
+            launch_kernel(gather_q8_stream_kernel<true>, dim3(grid), dim3(kThreadsS), 2 * (row_bytes + 16), stream, 1, src, s_row, (int)K, idx, (int)k,
+                          dst, ld_dst, row_scale, rows, per_block, status, wait_limit_ns());
+        else
+            launch_kernel(gather_q8_stream_kernel<false>, dim3(grid), dim3(kThreadsS), 2 * (row_bytes + 16), stream, 1, src, s_row, (int)K, idx, (int)k,
+                          dst, ld_dst, row_scale, rows, per_block, status, wait_limit_ns());
+        return check_launch("gather_q8_stream_kernel", stream);
+    }
+    const size_t smem = align_up(row_bytes, 16);
     if (smem > 200 * 1024 || K > INT32_MAX / 4 || rows > INT32_MAX) return fail(RMM_ERR_UNSUPPORTED, "gather_q8: row too long");
     static PerDeviceOnce configured;
     if (configured.first()) {
