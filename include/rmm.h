@@ -178,9 +178,11 @@ int rmm_reduced_attn(const rmm_attn_desc_t *desc, const void *Q, const void *K, 
                      int32_t *idx_feat, int32_t *idx_tok, void *ws, size_t ws_bytes, void *stream);
 
 /* The whole operation of Sec. 3.2 on device operands: I = TopK of the column norms of A with |I| = k (k == 0:
- * ceil(rho K)), Y = scale * A[:, I] B[I, :].  The result is that of rmm_score_select followed by rmm_reduced_gemm, bit
- * for bit; idx [batch, k] and retained [batch] (or NULL) as there.  For one bf16 product (batch 1) whose A has 2048 to
- * 8192 columns and more than 256 rows, and whose operands meet the tensor-core layout rules, the scores, the selection
+ * ceil(rho K)), Y = scale * A[:, I] B[I, :].  The result is that of rmm_score_select followed by rmm_reduced_gemm
+ * (in the one-launch form below the column energies are summed in a different fixed order, which can move a key by one
+ * fp64 rounding before it is rounded to fp32); idx [batch, k] and retained [batch] (or NULL) as there.  For one small bf16 product (batch 1, A with 2368 to
+ * 8192 columns and 257 to 8192 rows, B with at most 4096 columns) whose operands meet the tensor-core layout rules (the
+ * regime where launch and hand-off latencies weigh most), the scores, the selection
  * and both gathers run in ONE launch (every block owns 64 columns of A, a grid-wide barrier makes all column energies
  * visible, every block then selects and gathers its own kept columns and the matching rows of B), followed by the
  * tensor-core product; this form expects the GPU to itself (all of its blocks must be resident at once; if they are

@@ -373,6 +373,11 @@ struct FrontArgs {
     unsigned long long wait_ns;
 };
 
+// Tall or wide products gather faster through the separate gather launches (whole rows of A per block with full-line
+// stores; rows of B spread over every SM) than through this kernel's 64-byte pieces per row and its 16 copying warps
+// per block.  Measured at 8192 columns of A, rho = 0.5: ahead by 4 to 6 us up to 8192 rows when B has 2048 columns,
+// level at 16384 rows, behind by 15 % at 32768; behind at every row count when B has 8192 columns.
+constexpr int64_t kFrontMaxRows = 8192, kFrontMaxCols = 4096;
 constexpr int kFrontCombBytes = (kThreads / 32) * kTmaCols * 8;              // per-warp column sums (fp64)
 constexpr int kFrontSmemBytes = kTmaStages * kTmaStageBytes + kFrontCombBytes;
 
@@ -892,6 +897,10 @@ bool front_eligible(const rmm_mat_t *A, const rmm_mat_t *B, const rmm_mat_t *Y, 
     TcPlan tc;
     if (A->batch != 1 || !tc_eligible(A, B, k, Y, &tc) || tc.b_kmajor) return false;
     if (A->rows <= 256) return false;  // short outputs: the product fetches the kept rows of B itself
+    // RMM_PRODUCT_FUSED=0 / 1 (measurement switch) forces the two-call form / lifts the row limit below
+    static const int forced = []() { const char *e = getenv("RMM_PRODUCT_FUSED"); return e ? atoi(e) : -1; }();
+    if (forced == 0) return false;
+    if (forced != 1 && (A->rows > kFrontMaxRows || B->cols > kFrontMaxCols)) return false;
     ScorePlan sp;
     if (plan_score(A, 1, &sp) != RMM_OK || !sp.use_tma) return false;
     if (sp.n > kFusedSelectMax || sp.n % 8 != 0) return false;

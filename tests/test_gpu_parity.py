@@ -636,12 +636,13 @@ def test_next_product_selects_from_epilogue_energies(oracle):
 # 8-bit operands (e4m3 codes on the fp8 tensor cores)
 # ------------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("M,K,N,rho", [(128, 256, 256, 0.5), (300, 1008, 264, 0.75), (2048, 8192, 2048, 0.5), (77, 4096, 128, 0.25),
-                                       (4096, 2048, 4864, 1.0), (513, 528, 1032, 0.3)])
+                                       (4096, 2048, 4864, 1.0), (513, 528, 1032, 0.3), (5000, 1040, 4880, 0.4)])
 def test_reduced_product_with_8_bit_operands(oracle, M, K, N, rho):
     """Activation rows quantised on the fly over the kept columns (per-row step), weight given as e4m3 codes [N, K] with one
     scale.  The steps must equal the oracle's bit for bit (every decision in fp32); Y is held to the product of the
     oracle's dequantised operands: 1e-5 with fp32 output (exact products, fp32 accumulation), 1e-2 with bf16 output.
-    Single-CTA and CTA-pair tiles, ragged last stage (k not a multiple of 128 or of 16), ragged rows and columns."""
+    Single-CTA and CTA-pair tiles, ragged last stage (k not a multiple of 128 or of 16), ragged rows and columns; the last
+    case has enough rows on both sides for the streaming form of the quantising gather."""
     A = synth.heavy_tailed_activations(M, K, seed=M + 5)
     W = synth.weight(K, N, seed=M + 6, dtype=torch.float32)                       # fp32 weight, to be quantised offline
     b_scale = float(W.abs().max()) / 448.0
@@ -676,3 +677,24 @@ def test_8_bit_product_refuses_unaligned_weight_rows():
     with pytest.raises(rmm.RmmError) as e:
         rmm.rmm_reduced_gemm_q8(A, Bq, 1.0, idx)
     assert e.value.code == 2
+
+
+def test_one_launch_front_end_on_a_tall_product(oracle):
+    """The one-launch front end is chosen for small products only; forced onto a tall one (12288 rows: 48 row tiles, the
+    ring reloads 42 of them during the gather) it must still give the two-call form's index set and output."""
+    import os, subprocess, sys
+    code = (
+        "import torch, paper_2608_13426_b200 as rmm\n"
+        "from paper_2608_13426_b200 import synth, binding\n"
+        "binding.poison_outputs(True)\n"
+        "A = synth.heavy_tailed_activations(12288, 4096, seed=3, device='cuda'); B = synth.weight(4096, 1024, seed=4, device='cuda')\n"
+        "n0 = rmm.rmm_launch_count()\n"
+        "Y, idx = rmm.rmm_product(A, B, rho=0.5)\n"
+        "assert rmm.rmm_launch_count() - n0 == 2\n"
+        "idx2, _, _, _ = rmm.rmm_score_select(A, rho=0.5)\n"
+        "Y2 = rmm.rmm_reduced_gemm(A, B, idx2)\n"
+        "assert torch.equal(idx, idx2) and torch.equal(Y, Y2) and rmm.rmm_status_read() == 0\n")
+    env = dict(os.environ, RMM_PRODUCT_FUSED="1")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", code], env=env, cwd=root, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-3000:]
