@@ -344,9 +344,9 @@ __global__ void __launch_bounds__(kThreads, 1) score_tma_kernel(const __grid_con
 //   3. EVERY block runs the selection on all n energies (redundantly: a block-wide select costs the same whether one
 //      block or all of them run it, and nobody then waits for a second barrier), so each knows the threshold, the kept
 //      columns among its own 64 and their positions in the index list; block 0 writes the list itself;
-//   4. (warps 0-15) its kept columns of A go to Ap[:, pos0 .. pos0 + cnt): the last six tiles of the stream are still in
-//      the ring and are gathered from there, the earlier ones are copied again (from L2 when A is small); a warp copies
-//      2-byte elements from shared memory to 4-byte stores;
+//   4. (warps 0-15) the kept columns of A go to Ap for the block's share of the ROWS (all kept columns of those rows):
+//      chunks of whole rows arrive in the ring by bulk copies (from L2 when A is small; the first chunks are requested
+//      before the barrier), a thread builds four consecutive outputs and stores 8 bytes, so Ap is written in full lines;
 //   5. (warps 16-31, at the same time) the rows of B that belong to its kept columns, requested into L2 right after the
 //      selection, go to Bp[pos0 .. pos0 + cnt, :] as 16-byte vectors.
 // The reduced product then reads Ap and Bp with TMA tile loads.  Against separate score, select and gather launches
@@ -371,6 +371,7 @@ struct FrontArgs {
     int64_t b_sr, N;
     __nv_bfloat16 *Bp;        // [k, N]
     unsigned long long wait_ns;
+    int rows_per_chunk;       // rows of A per chunk of the gather: 64 KB / (2 n)
 };
 
 // Tall or wide products gather faster through the separate gather launches (whole rows of A per block with full-line
@@ -378,6 +379,9 @@ struct FrontArgs {
 // per block.  Measured at 8192 columns of A, rho = 0.5: ahead by 4 to 6 us up to 8192 rows when B has 2048 columns,
 // level at 16384 rows, behind by 15 % at 32768; behind at every row count when B has 8192 columns.
 constexpr int64_t kFrontMaxRows = 8192, kFrontMaxCols = 4096;
+constexpr int kChunkSlots = 3;                         // row chunks in the ring
+constexpr int kChunkBytes = 2 * kTmaStageBytes;        // 64 KB: rows_per_chunk = 64 KB / row bytes
+constexpr int kGroupsPerThread = 4;                    // 8-byte output groups per gathering thread and row: k <= 4 * 4 * 512
 constexpr int kFrontCombBytes = (kThreads / 32) * kTmaCols * 8;              // per-warp column sums (fp64)
 constexpr int kFrontSmemBytes = kTmaStages * kTmaStageBytes + kFrontCombBytes;
 
@@ -386,7 +390,7 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
     extern __shared__ __align__(128) unsigned char s_dyn[];  // the tile ring, then the per-warp column sums
     __shared__ SelectSmem s_sel;
     __shared__ __align__(8) unsigned long long s_bar[2 * kTmaStages];
-    __shared__ int s_ok, s_first, s_end, s_next;
+    __shared__ int s_ok, s_first, s_end;
     __shared__ int s_pos[kTmaCols];           // position in the index list of each own column, or -1
     __shared__ unsigned short s_own[kTmaCols];  // own kept columns (0 .. 63) in list order
 
@@ -487,11 +491,28 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
     // A block that ran out of time leaves the ring alone (a copy may still land in it), lets the others through the
     // grid barrier, gives copies in flight time to land and returns; the status word tells the host.
     const bool alive = s_ok != 0;
-    // The last tiles of the stream (up to six) are still in the ring and stay there: the gather starts with them.
-    const int resident = n_tiles < kTmaStages ? n_tiles : kTmaStages;
+    // The gather (step 4) works on ROW chunks of A: this block's rows [row_lo, row_hi), rb rows at a time, every chunk
+    // whole (a chunk fills up to a third of the ring).
+    const int used_slots = n_tiles < kTmaStages ? n_tiles : kTmaStages;
+    const int rows_per_block = (int)((a.m + gridDim.x - 1) / gridDim.x);
+    const int64_t row_lo = (int64_t)blockIdx.x * rows_per_block, row_hi = min(a.m, row_lo + rows_per_block);
+    const int rb = fa.rows_per_chunk;                                                 // rows per chunk
+    const int n_chunks = row_hi > row_lo ? (int)((row_hi - row_lo + rb - 1) / rb) : 0;
+    const uint32_t row_bytes = (uint32_t)a.n * 2u;                                    // a multiple of 16
+    auto fill_chunk = [&](int c) {  // thread 0: chunk c of the block's rows -> chunk slot c % 3 (two ring slots wide)
+        const int cs = c % kChunkSlots;
+        const int64_t r0 = row_lo + (int64_t)c * rb;
+        const int nr = (int)min((int64_t)rb, row_hi - r0);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full_bar(cs)), "r"((uint32_t)nr * row_bytes) : "memory");
+        const unsigned short *g = reinterpret_cast<const unsigned short *>(a.A) + r0 * a.s_red;
+        for (int r = 0; r < nr; ++r)  // a row of A is contiguous: one bulk copy per row
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(ring + cs * kChunkBytes + (uint32_t)r * row_bytes), "l"(g + (int64_t)r * a.s_red), "r"(row_bytes), "r"(full_bar(cs))
+                         : "memory");
+    };
     if (alive) {
         // Row lanes in a fixed order: the four lanes of a column group inside a warp by shuffles, then the 32 warps in
-        // order by the column's owner thread.  The sums live next to the ring, which keeps its tiles.
+        // order by the column's owner thread.
         double *s_comb = reinterpret_cast<double *>(s_dyn + kTmaStages * kTmaStageBytes);
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
@@ -510,9 +531,15 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
             a.energy[col0 + tid] = (float)colsum;
             if (a.scores != nullptr) a.scores[col0 + tid] = (float)sqrt(colsum);
         }
-        if (tid == 0) {  // every release of the stream has been waited for once the gather starts
-            for (int s2 = 0; s2 < resident && ok; ++s2)
+        if (tid == 0) {
+            // every release of the stream is waited for (the ring is free), then the gather's first chunks are requested:
+            // they arrive (from L2 when A is small) while the barrier and the selection run
+            for (int s2 = 0; s2 < used_slots && ok; ++s2)
                 if (!wait_empty(s2)) ok = false;
+            if (ok) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                for (int c = 0; c < kChunkSlots && c < n_chunks; ++c) fill_chunk(c);
+            }
             if (!ok) s_ok = 0;
         }
     }
@@ -557,25 +584,30 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
         return;
     }
 
-    // ---- 3. selection, in every block
+    // ---- 3. selection, in every block, 8 keys per thread.  (Run by eight warps with 32 keys per thread instead it was
+    // slower, 47.6 against 39 us for the kernel at n = 8192: the serial work per thread grows faster than the
+    // barriers get cheaper.)
     FSTAMP_MAX(3);
-    unsigned u[8];
-    const int nvalid = load_keys_blocked<8>(a.energy, (int)a.n, u);
-    const Threshold th = block_threshold<8>(u, nvalid, a.k, s_sel);
-    const unsigned before = block_rank_blocked<8>(u, nvalid, th.tau, s_sel);
-    {
+    constexpr int kSelThreads = kThreads, kSelItems = kFusedSelectMax / kSelThreads;
+    unsigned short *s_list = reinterpret_cast<unsigned short *>(s_dyn + kTmaStages * kTmaStageBytes);  // position -> column
+    if (tid < kSelThreads) {
+        unsigned u[kSelItems];
+        const int nvalid = load_keys_blocked<kSelItems>(a.energy, (int)a.n, u);
+        const Threshold th = block_threshold<kSelItems, kSelThreads>(u, nvalid, a.k, s_sel);
+        const unsigned before = block_rank_blocked<kSelItems, kSelThreads>(u, nvalid, th.tau, s_sel);
         unsigned gt_before = before >> 16, eq_before = before & 0xffffu;
         const bool writer = blockIdx.x == 0;
-        const int j0 = tid * 8;
-        const bool mine = j0 >= col0 && j0 < col0 + kTmaCols;  // eight threads hold this block's columns
+        const int j0 = tid * kSelItems;
+        const bool mine = j0 >= col0 && j0 < col0 + kTmaCols;  // the threads that hold this block's columns
         if (mine && j0 == col0) s_first = (int)(gt_before + min(eq_before, th.need_eq));
         double sum_kept = 0.0, sum_all = 0.0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < kSelItems; ++i) {
             if (i < nvalid) {
                 const bool gt = u[i] > th.tau, eq = u[i] == th.tau;
                 const bool keep = gt || (eq && eq_before < th.need_eq);
                 const unsigned pos = gt_before + min(eq_before, th.need_eq);
+                if (keep) s_list[pos] = (unsigned short)(j0 + i);     // the whole list: the gather of A needs every kept column
                 if (writer && keep) a.idx[pos] = j0 + i;
                 if (mine) s_pos[j0 + i - col0] = keep ? (int)pos : -1;
                 if (writer && a.retained != nullptr) {
@@ -589,8 +621,8 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
                 s_pos[j0 + i - col0] = -1;
             }
         }
-        if (mine && j0 + 8 == col0 + kTmaCols) s_end = (int)(gt_before + min(eq_before, th.need_eq));
-        if (writer && a.retained != nullptr) {  // block-uniform
+        if (mine && j0 + kSelItems == col0 + kTmaCols) s_end = (int)(gt_before + min(eq_before, th.need_eq));
+        if (writer && a.retained != nullptr) {  // uniform over the selecting warps
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) {
                 sum_kept += __shfl_down_sync(0xffffffffu, sum_kept, d);
@@ -600,10 +632,10 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
                 s_sel.red[warp] = sum_kept;
                 s_sel.red[32 + warp] = sum_all;
             }
-            __syncthreads();
+            group_sync<kSelThreads>();
             if (tid == 0) {
                 double x = 0.0, y = 0.0;
-                for (int w2 = 0; w2 < 32; ++w2) {
+                for (int w2 = 0; w2 < kSelThreads / 32; ++w2) {
                     x += s_sel.red[w2];
                     y += s_sel.red[32 + w2];
                 }
@@ -611,25 +643,9 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
             }
         }
     }
-    if (tid == 0) s_next = -1;
     __syncthreads();
     const int pos0 = s_first, cnt = s_end - s_first;
     if (tid < kTmaCols && s_pos[tid] >= 0) s_own[s_pos[tid] - pos0] = (unsigned short)tid;
-    {
-        // the kept column that follows this block's range in the list (position pos0 + cnt), if any: when the range ends
-        // at an odd position its last element shares a 4-byte word of Ap with that column's, and this block writes both
-        unsigned gt_before = before >> 16, eq_before = before & 0xffffu;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            if (i < nvalid) {
-                const bool gt = u[i] > th.tau, eq = u[i] == th.tau;
-                const bool keep = gt || (eq && eq_before < th.need_eq);
-                if (keep && (int)(gt_before + min(eq_before, th.need_eq)) == pos0 + cnt) s_next = tid * 8 + i;
-                gt_before += gt ? 1u : 0u;
-                eq_before += eq ? 1u : 0u;
-            }
-        }
-    }
     __syncthreads();
     {
         // the rows of B that this block copies in step 5 are requested into L2 now, so that they arrive from HBM while
@@ -647,74 +663,56 @@ __global__ void __launch_bounds__(kThreads, 1) rmm_front_kernel(const __grid_con
     // of B (requested into L2 above).  A ring slot is still released by 32 arrivals: two lanes of each gathering warp.
     constexpr int kGatherWarps = 16;
     if (warp < kGatherWarps) {
-        // ---- 4. own kept columns of A -> Ap.  What bounds this step is the number of store requests that reach L2 (about
-        // 64 G requests/s over the whole GPU, however few bytes each carries), so a block issues exactly one per row: lane l
-        // stores the 4-byte word at the even list position e = pos0 rounded up to even, plus 2 l.  If the block's range
-        // starts at an odd position, its first element belongs to the previous block's last word and that block writes
-        // it; if the range ends at an odd position, the last word's upper half is the next kept column of A (outside this
-        // block's tiles): the warp fetches that element for its rows of the next step from A itself (2-byte loads, L2).
-        const int e0 = pos0 + (pos0 & 1);
-        const int j_lo = e0 + 2 * lane - pos0, j_hi = j_lo + 1;               // positions inside this block's list
-        const bool st_pair = j_lo < cnt;                                       // (j_lo >= 0 always)
-        const bool hi_own = j_hi < cnt;
-        const bool has_partner = ((pos0 + cnt) & 1) != 0;                      // the last word's upper half is not this block's
-        const uint32_t o_lo = st_pair ? (uint32_t)s_own[j_lo] * 2u : 0u, o_hi = hi_own ? (uint32_t)s_own[j_hi] * 2u : 0u;
-        const int next_col = s_next;                                           // -1: the list ends here (the half is padding)
-        const int64_t row_step = kGatherWarps * fa.ldp;                        // elements between two rows of this warp
-        unsigned short *dwarp = reinterpret_cast<unsigned short *>(fa.Ap) + (int64_t)warp * fa.ldp + e0 + 2 * lane;
-        const unsigned short *a16 = reinterpret_cast<const unsigned short *>(a.A);
-        // lane p < 16 holds the partner element of the warp's p-th row of the current step
-        auto partner = [&](int tile) -> unsigned short {
-            const int64_t row = (int64_t)tile * kTmaRows + warp + kGatherWarps * lane;
-            return (has_partner && next_col >= 0 && lane < kTmaRows / kGatherWarps && row < a.m) ? __ldg(a16 + row * a.s_red + next_col)
-                                                                                                 : (unsigned short)0;
-        };
-        auto tile_of_step = [&](int t) { return t < resident ? n_tiles - resident + t : t - resident; };
-        unsigned short pv_next = n_tiles > 0 ? partner(tile_of_step(0)) : (unsigned short)0;
-        // Step t < resident works on the tile the stream left in the ring (no copy, nothing to wait for); later steps
-        // work on tiles 0, 1, ... copied again (from L2 when A is small) into the slots in the order they were released,
-        // requested two steps after the release.
-        const int n_reload = n_tiles - resident;
-        for (int t = 0; t < n_tiles && ok; ++t) {
-            const int tile = t < resident ? n_tiles - resident + t : t - resident;
-            const int st = (n_tiles - resident + t) % kTmaStages;
-            if (tid == 0 && t >= 2 && t - 2 < n_reload) {
-                const int q = t - 2, qs = (n_tiles - resident + q) % kTmaStages;  // the slot step q released
-                if (!wait_empty(qs)) ok = false;
+        // ---- 4. kept columns of A -> Ap for this block's ROWS.  What bounds a gather of 2-byte elements is the number of
+        // store requests that reach L2 (about 64 G requests/s over the whole GPU, however few bytes each carries: 64-byte
+        // pieces per row and column block took 10 us here).  So a block owns whole rows: thread t builds the output
+        // groups t, t + 512, ... of four consecutive list positions from four 2-byte shared-memory loads and stores them
+        // as one 8-byte word, a warp store is 256 contiguous bytes, and every line of Ap is written once, in full.
+        const int gt = tid;                                    // 0 .. 511
+        const int n_groups = (int)(fa.ldp / 4);                // groups of four positions per output row
+        uint32_t off[kGroupsPerThread][4];                     // byte offset of the source column inside a staged row, or ~0
+#pragma unroll
+        for (int g = 0; g < kGroupsPerThread; ++g)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int j = 4 * (gt + g * 32 * kGatherWarps) + e;
+                uint32_t o = 0xffffffffu;
+                if (j < a.k) o = (uint32_t)s_list[j] * 2u;
+                off[g][e] = o;
+            }
+        for (int c = 0; c < n_chunks && ok; ++c) {
+            const int cs = c % kChunkSlots;
+            if (tid == 0 && c >= 1 && c - 1 + kChunkSlots < n_chunks) {
+                // the slot that chunk c - 1 used is free once all gathering warps have released it
+                if (!wait_empty((c - 1) % kChunkSlots)) ok = false;
                 if (ok) {
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    fill(qs, q);
+                    fill_chunk(c - 1 + kChunkSlots);
                 }
             }
-            if (t >= resident && !wait_full(st)) ok = false;
-            // a warp leaves the loop as a whole (the shuffles and warp barriers below involve every lane): lanes may see a
-            // wait expire at slightly different moments, and thread 0 also waits on behalf of the producer
-            ok = __all_sync(0xffffffffu, ok);
+            if (!wait_full(cs)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);  // a warp leaves the loop as a whole
             if (!ok) break;
-            const int64_t left = a.m - (int64_t)tile * kTmaRows - warp;      // rows of this tile at or below the warp's first
-            const int np = left <= 0 ? 0 : (int)min((int64_t)(kTmaRows / kGatherWarps), (left + kGatherWarps - 1) / kGatherWarps);
-            const unsigned pv = pv_next;
-            if (t + 1 < n_tiles) pv_next = partner(tile_of_step(t + 1));     // in flight while this tile is gathered
-            const unsigned char *row_g = s_dyn + st * kTmaStageBytes + warp * (kTmaCols * 2);
-            constexpr int S = kGatherWarps * kTmaCols * 2;                   // bytes between two rows of this warp in the tile
-            unsigned short *d = dwarp + (int64_t)tile * kTmaRows * fa.ldp;
-            for (int p0 = 0; p0 < np; p0 += 4) {                             // four rows at a time: loads first, then stores
-                unsigned w[4];
+            const unsigned char *chunk = s_dyn + cs * kChunkBytes;
+            const int64_t r0 = row_lo + (int64_t)c * rb;
+            const int nr = (int)min((int64_t)rb, row_hi - r0);
+            for (int r = 0; r < nr; ++r) {
+                const unsigned char *srow = chunk + (uint32_t)r * row_bytes;
+                uint2 *drow = reinterpret_cast<uint2 *>(fa.Ap + (r0 + r) * fa.ldp);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int p = p0 + i < np ? p0 + i : np - 1;
-                    const unsigned lo = *reinterpret_cast<const unsigned short *>(row_g + p * S + o_lo);
-                    const unsigned hi_o = *reinterpret_cast<const unsigned short *>(row_g + p * S + o_hi);
-                    const unsigned hi_p = __shfl_sync(0xffffffffu, pv, p);
-                    w[i] = lo | ((hi_own ? hi_o : hi_p) << 16);
+                for (int g = 0; g < kGroupsPerThread; ++g) {
+                    const int grp = gt + g * 32 * kGatherWarps;
+                    if (grp < n_groups) {
+                        unsigned v[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            v[e] = off[g][e] != 0xffffffffu ? (unsigned)*reinterpret_cast<const unsigned short *>(srow + off[g][e]) : 0u;
+                        drow[grp] = make_uint2(v[0] | (v[1] << 16), v[2] | (v[3] << 16));
+                    }
                 }
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    if (st_pair && p0 + i < np) *reinterpret_cast<unsigned *>(d + i * row_step) = w[i];
-                d += 4 * row_step;
             }
             __syncwarp();
-            if (lane < kThreads / 32 / kGatherWarps) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(st)) : "memory");
+            if (lane < kThreads / 32 / kGatherWarps) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(cs)) : "memory");
         }
     } else {
         // ---- 5. rows of B of the own kept columns -> Bp[pos0 .. pos0 + cnt, :], 16-byte vectors.  Rows shorter than
@@ -952,6 +950,9 @@ int launch_front(const rmm_mat_t *A, const rmm_mat_t *B, int64_t k, int32_t *idx
     const uint32_t box[3] = {kTmaCols, kTmaRows, 1};
     int rc = make_map(&map, const_cast<void *>(a.A), 3, dims, st, box, false);
     if (rc != RMM_OK) return rc;
+    // row chunks of the gather: whole rows of A (one bulk copy each), as many as fit 64 KB of the ring
+    fa.rows_per_chunk = (int)(kChunkBytes / (a.n * 2));
+    if (fa.rows_per_chunk < 1) return fail(RMM_ERR_UNSUPPORTED, "front: row too long");
     static PerDeviceOnce configured;
     if (configured.first()) {
         cudaError_t e = cudaFuncSetAttribute(rmm_front_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFrontSmemBytes);

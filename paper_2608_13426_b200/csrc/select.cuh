@@ -255,6 +255,15 @@ __device__ void block_select(const float *__restrict__ keys, int K, int k, int32
 // Thread t of a 1024-thread block holds the ITEMS consecutive keys [t * ITEMS, (t + 1) * ITEMS): the index order is
 // the (thread, item) order, so the ordered emission needs one block-wide scan of per-thread counts and every thread
 // writes its kept indices next to each other.  Digits after the first are up to 11 bits wide as well.
+// The blocked form runs on a group of NTHR threads: the whole block (1024, ordinary block barrier) or its first eight
+// warps (256, named barrier 2) while the other warps of the block do something else or wait.
+template <int NTHR>
+__device__ __forceinline__ void group_sync()
+{
+    if constexpr (NTHR == 1024) __syncthreads();
+    else asm volatile("bar.sync 2, %0;" ::"n"(NTHR) : "memory");
+}
+
 struct Threshold {
     unsigned tau;      // image of the k-th largest key
     unsigned need_eq;  // how many keys equal to tau are kept (lowest indices first)
@@ -286,6 +295,7 @@ __device__ __forceinline__ int load_keys_blocked(const float *__restrict__ keys,
 // nbins / 256 warps work: a thread owns eight consecutive bins (two 16-byte loads, no bank conflicts), warps scan
 // with shuffles, and with eight warps a named barrier among them exchanges the warp totals.  With 32 warps sharing four
 // schedulers, instructions issued by every warp are what a block-wide step costs; this keeps them to a few warps.
+template <int NTHR>
 __device__ __forceinline__ void find_bin8(SelectSmem &sm, int nbins, unsigned remaining)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -331,7 +341,7 @@ __device__ __forceinline__ void find_bin8(SelectSmem &sm, int nbins, unsigned re
             }
         }
     }
-    __syncthreads();
+    group_sync<NTHR>();
 }
 
 // Image of the k-th largest key and the number of keys equal to it that are kept.  Items 0 .. nvalid-1 of every thread
@@ -340,10 +350,11 @@ __device__ __forceinline__ void find_bin8(SelectSmem &sm, int nbins, unsigned re
 // the keys that share the prefix found so far count (a per-thread bit mask of those keys is carried along, and warps
 // without any skip the pass).  With 32 warps on four schedulers every instruction that all warps execute costs eight
 // issue clocks, so the code paths below are kept short rather than general.
-template <int ITEMS>
+template <int ITEMS, int NTHR = 1024>
 __device__ __forceinline__ Threshold block_threshold(const unsigned (&u)[ITEMS], int nvalid, int k, SelectSmem &sm)
 {
-    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int nthr = NTHR, nwarp = NTHR / 32;
     unsigned lo = 0xffffffffu, hi = 0u;
     if (nvalid == ITEMS) {
 #pragma unroll
@@ -368,9 +379,9 @@ __device__ __forceinline__ Threshold block_threshold(const unsigned (&u)[ITEMS],
     }
     {
         uint4 *h4 = reinterpret_cast<uint4 *>(sm.hist);
-        if (tid < kBins / 4) h4[tid] = make_uint4(0, 0, 0, 0);
+        for (int i = tid; i < kBins / 4; i += nthr) h4[i] = make_uint4(0, 0, 0, 0);
     }
-    __syncthreads();
+    group_sync<NTHR>();
     SEL_STAMP(0);
     {
         const unsigned l = lane < nwarp ? sm.warp_lo[lane] : 0xffffffffu, h = lane < nwarp ? sm.warp_hi[lane] : 0u;
@@ -398,9 +409,9 @@ __device__ __forceinline__ Threshold block_threshold(const unsigned (&u)[ITEMS],
         for (int i = 0; i < ITEMS; ++i)
             if (i < nvalid) atomicAdd(&sm.hist[(u[i] >> shift) & m], 1u);
     }
-    __syncthreads();
+    group_sync<NTHR>();
     SEL_STAMP(1);
-    find_bin8(sm, d > 8 ? 2048 : 256, remaining);  // bins beyond 1 << d are zero
+    find_bin8<NTHR>(sm, d > 8 ? 2048 : 256, remaining);  // bins beyond 1 << d are zero
     SEL_STAMP(2);
     prefix |= sm.bin << shift;
     mask |= m << shift;
@@ -417,15 +428,15 @@ __device__ __forceinline__ Threshold block_threshold(const unsigned (&u)[ITEMS],
         shift -= d;
         m = (1u << d) - 1u;
         if (tid < 64) reinterpret_cast<uint4 *>(sm.hist)[tid] = make_uint4(0, 0, 0, 0);
-        __syncthreads();
+        group_sync<NTHR>();
         if (__any_sync(0xffffffffu, live != 0u)) {
 #pragma unroll
             for (int i = 0; i < ITEMS; ++i)
                 if (live & (1u << i)) atomicAdd(&sm.hist[(u[i] >> shift) & m], 1u);
         }
-        __syncthreads();
+        group_sync<NTHR>();
         SEL_STAMP(1 + 2 * pass);
-        find_bin8(sm, 256, remaining);
+        find_bin8<NTHR>(sm, 256, remaining);
         SEL_STAMP(2 + 2 * pass);
         ++pass;
         prefix |= sm.bin << shift;
@@ -447,7 +458,7 @@ __device__ __forceinline__ Threshold block_threshold(const unsigned (&u)[ITEMS],
             if (live & (1u << i)) mn = min(mn, u[i]);
         mn = __reduce_min_sync(0xffffffffu, mn);
         if (lane == 0) sm.warp_lo[warp] = mn;
-        __syncthreads();
+        group_sync<NTHR>();
         mn = __reduce_min_sync(0xffffffffu, lane < nwarp ? sm.warp_lo[lane] : 0xffffffffu);
         unsigned c = 0;
 #pragma unroll
@@ -455,7 +466,7 @@ __device__ __forceinline__ Threshold block_threshold(const unsigned (&u)[ITEMS],
             if ((live & (1u << i)) && u[i] == mn) ++c;
         c = __reduce_add_sync(0xffffffffu, c);
         if (lane == 0) sm.warp_hi[warp] = c;
-        __syncthreads();
+        group_sync<NTHR>();
         t.tau = mn;
         t.need_eq = __reduce_add_sync(0xffffffffu, lane < nwarp ? sm.warp_hi[lane] : 0u);
         return t;
@@ -468,7 +479,7 @@ __device__ __forceinline__ Threshold block_threshold(const unsigned (&u)[ITEMS],
 // Exclusive block-wide scan of this thread's (keys greater than tau, keys equal to tau) counts, packed as
 // (greater << 16 | equal): the number of such keys at lower indices.  Whole block (1024 threads), K <= 65535.
 // One barrier: every warp scans the 32 warp totals itself.
-template <int ITEMS>
+template <int ITEMS, int NTHR = 1024>
 __device__ __forceinline__ unsigned block_rank_blocked(const unsigned (&u)[ITEMS], int nvalid, unsigned tau, SelectSmem &sm)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -483,8 +494,8 @@ __device__ __forceinline__ unsigned block_rank_blocked(const unsigned (&u)[ITEMS
         if (lane >= d) incl += v;
     }
     if (lane == 31) sm.warp_a[warp] = incl;
-    __syncthreads();
-    const unsigned w = sm.warp_a[lane];
+    group_sync<NTHR>();
+    const unsigned w = lane < NTHR / 32 ? sm.warp_a[lane] : 0u;
     unsigned wi = w;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
