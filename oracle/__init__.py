@@ -61,7 +61,7 @@ def _load():
                            i32, dbl, dbl, i32, vp, vp, vp, vp]
     L.orc_attn_sets.restype = i32
     L.orc_attn_sets.argtypes = [vp, vp, vp, i32, i64, i64, i64, i64, i64, i64, vp, vp, vp,
-                                i32, dbl, dbl, i32, vp, vp, vp, i64, vp, vp, vp, vp]
+                                i32, dbl, dbl, i32, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp]
     _lib = L
     return L
 
@@ -174,12 +174,14 @@ def rmm(A, B, rho: float):
 
 
 def attn(Q, K, V, causal: bool, rho_d: float, rho_t: float, round_p: bool = True, want_p: bool = False,
-         idx_feat=None, idx_tok=None, rows=None):
+         idx_feat=None, idx_tok=None, rows=None, mask=None):
     """Reduced attention of Sec. 3.3.  Q [B,Hq,Lq,Dh]; K, V [B,Hkv,Lk,Dh] (same dtype).
 
     idx_feat [B,Hq,kd] / idx_tok [B,Hq,kt] (int32), if given, replace the TopK choice of the feature / token set
     (the formulas for S~ and O~ hold for any set); rows (a list of query rows), if given, restricts the evaluation
     to those rows (with rho_t < 1 the token set must then be given, because token scores need every row).
+
+    mask, if given, is the additive M of P = softmax(S~ + M): an array broadcastable to [B,Hq,Lq,Lk] (-inf hides a key).
 
     Returns (O [B,Hq,Lq or len(rows),Dh] fp64, idx_feat [B,Hq,kd], idx_tok [B,Hq,kt] or None, P or None):
     the sets are the ones that were used.
@@ -211,9 +213,18 @@ def attn(Q, K, V, causal: bool, rho_d: float, rho_t: float, round_p: bool = True
     P = np.zeros((B, Hq, nq, Lk), np.float64) if want_p else None
     s3 = [(ctypes.c_int64 * 4)(*_estr(x)) for x in (Q, K, V)]
     ptr = lambda a: a.ctypes.data if a is not None else None
+    mask_in = sm = None
+    if mask is not None:
+        m = np.asarray(as_np(mask), dtype=np.float64)
+        while m.ndim < 4:
+            m = m[None]
+        assert m.shape[3] == Lk and all(m.shape[a] in (1, n) for a, n in enumerate((B, Hq, Lq)))
+        mask_in = np.ascontiguousarray(m)
+        full = (mask_in.shape[1] * mask_in.shape[2] * Lk, mask_in.shape[2] * Lk, Lk)
+        sm = (ctypes.c_int64 * 3)(*[0 if mask_in.shape[a] == 1 else full[a] for a in range(3)])
     rc = _load().orc_attn_sets(Q.ctypes.data, K.ctypes.data, V.ctypes.data, _dt(Q), B, Hq, Hkv, Lq, Lk, Dh,
                                s3[0], s3[1], s3[2], int(bool(causal)), float(rho_d), float(rho_t),
-                               int(bool(round_p)), ptr(feat_in), ptr(tok_in), ptr(rows_in), nq,
+                               int(bool(round_p)), ptr(feat_in), ptr(tok_in), ptr(rows_in), nq, ptr(mask_in), sm,
                                O.ctypes.data, out_feat.ctypes.data, ptr(out_tok), ptr(P))
     assert rc == 0
     return O, out_feat, out_tok, P

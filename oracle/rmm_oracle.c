@@ -256,7 +256,7 @@ double orc_round_bf16(double x)
  * Per (b, h):
  *   1. s_j = ||Q_h[:, j]||_2,  I = TopK(s, ceil(rho_d Dh))               -> idx_feat[b,h,:]
  *   2. S~[i,t] = (sum_{j in I} Q[i,j] K_g[t,j]) / sqrt(Dh), g = h / (Hq/Hkv)
- *   3. causal: t > i + (Lk - Lq) masked out;  P = softmax over t (fp64)
+ *   3. causal: t > i + (Lk - Lq) masked out;  P = softmax over t (fp64) of S~ + M
  *   4. if round_p: P <- bf16(P)
  *   5. if rho_t < 1: a_t = ||P[:, t]||_2, T = TopK(a, ceil(rho_t Lk))     -> idx_tok[b,h,:]
  *      O~ = P[:, T] V_g[T, :]  (no renormalisation); else O~ = P V_g
@@ -272,6 +272,9 @@ double orc_round_bf16(double x)
  * row, so nothing else changes); O is then [B, Hq, n_rows, Dh] and P_out [B, Hq, n_rows, Lk].  Token scores need
  * every row, so with rows given and rho_t < 1 the token set must be handed in; otherwise -1 is returned and
  * nothing is written.  Returns 0 on success.
+ * mask non-NULL: the additive mask M of "P = softmax(S~ + M)" (Sec. 3.3), doubles, entry (b, h, i, t) at
+ * mask[b sm[0] + h sm[1] + i sm[2] + t] (a stride of 0 shares the mask along that axis); -inf hides a key, and a
+ * row whose keys are all hidden gives zeros, as under the causal mask.  It applies on top of `causal`.
  * O [B, Hq, Lq (or n_rows), Dh] contiguous doubles.
  * P_out, if non-NULL, receives P for every (b,h) as [B,Hq,Lq (or n_rows),Lk] doubles (small cases only).
  */
@@ -281,6 +284,7 @@ int orc_attn_sets(const void *Q, const void *Kt, const void *V, int dtype,
                   int causal, double rho_d, double rho_t, int round_p,
                   const int32_t *idx_feat_in, const int32_t *idx_tok_in,
                   const int64_t *rows, int64_t n_rows,
+                  const double *mask, const int64_t *sm,
                   double *O, int32_t *idx_feat, int32_t *idx_tok, double *P_out)
 {
     int64_t kd = orc_keep_count(rho_d, Dh);
@@ -334,12 +338,14 @@ int orc_attn_sets(const void *Q, const void *Kt, const void *V, int dtype,
                                orc_load(Kt, dtype, k0 + t * sk[2] + j * sk[3]);
                     }
                     row[t] = acc * scale;
+                    if (mask != NULL) /* S~ + M: an additive mask entry, -inf hides the key */
+                        row[t] += mask[b * sm[0] + h * sm[1] + i * sm[2] + t];
                     if (row[t] > mx)
                         mx = row[t];
                 }
                 double den = 0.0;
                 for (int64_t t = 0; t < Lk; ++t) {
-                    row[t] = (t > last) ? 0.0 : exp(row[t] - mx);
+                    row[t] = (t > last || mx == -INFINITY) ? 0.0 : exp(row[t] - mx);
                     den += row[t];
                 }
                 for (int64_t t = 0; t < Lk; ++t) {
@@ -394,5 +400,5 @@ void orc_attn(const void *Q, const void *Kt, const void *V, int dtype,
               double *O, int32_t *idx_feat, int32_t *idx_tok, double *P_out)
 {
     (void)orc_attn_sets(Q, Kt, V, dtype, B, Hq, Hkv, Lq, Lk, Dh, sq, sk, sv, causal, rho_d, rho_t, round_p,
-                        NULL, NULL, NULL, 0, O, idx_feat, idx_tok, P_out);
+                        NULL, NULL, NULL, 0, NULL, NULL, O, idx_feat, idx_tok, P_out);
 }

@@ -441,6 +441,30 @@ def test_fused_attention_feature_reduction_only(oracle, shape):
     assert rmm.rmm_status_read() == 0
 
 
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("rho_d", [1.0, 0.5])
+def test_fused_attention_logits_that_outgrow_the_running_maximum(oracle, causal, rho_d):
+    """Keys whose logits lie far (more than 2^40 in weight) above everything before them, placed in the second half
+    of the second tile, the first half of the third and the second half of the fourth: the kernel takes weights
+    against the maximum it already has and must notice, from the row sums, that it no longer holds, then rescale
+    its sums, its O rows and the half tile of P already written."""
+    B, H, L, Dh = 1, 2, 640, 128
+    Q, K, V = synth.attention_qkv(B, H, H, L, L, Dh, seed=48, n_outlier=0)
+    Q = (Q.float() * 0.125 + 1.0).to(torch.bfloat16)
+    K = (K.float() * 0.125).to(torch.bfloat16)
+    for t, c in ((200, 8.0), (300, 16.0), (450, 32.0)):
+        K[:, :, t, :] = c
+    O, idx_feat, _ = rmm.rmm_reduced_attn(dev(Q), dev(K), dev(V), causal, rho_d, 1.0, want_idx=True)
+    assert rmm.rmm_status_read() == 0
+    Oo, _, _, _ = oracle.attn(Q, K, V, causal, rho_d, 1.0, round_p=True, idx_feat=idx_feat.cpu().numpy())
+    Og = O.float().cpu().numpy()
+    assert np.isfinite(Og).all()
+    for h in range(H):
+        assert rel_fro(Og[0, h], Oo[0, h]) <= TOL_BF16, h
+        for lo, hi in ((0, 200), (200, 300), (300, 450), (450, L)):      # the rows that see 0, 1, 2, 3 of the keys (causal)
+            assert rel_fro(Og[0, h, lo:hi], Oo[0, h, lo:hi]) <= TOL_BF16, (h, lo)
+
+
 def test_fused_attention_rows_without_keys_are_zero():
     B, Hq, Hkv, Lq, Lk, Dh = 1, 2, 2, 300, 100, 64
     Q, K, V = synth.attention_qkv(B, Hq, Hkv, Lq, Lk, Dh, seed=47)

@@ -437,6 +437,53 @@ def test_attention_on_given_sets(oracle):
     assert not np.allclose(Ot, O)
 
 
+def test_attention_with_an_additive_mask(oracle):
+    """Sec. 3.3: P = softmax(S~ + M) with M the optional causal or attention mask.  (i) The causal mask written out as
+    an additive 0 / -inf matrix reproduces causal = True exactly; (ii) a finite additive bias with some keys hidden
+    equals the library's attention with that float mask, per head and broadcast over heads; (iii) a mask entry moves
+    the logit it belongs to: hiding one key of one head zeroes that column of P and nothing in other heads; (iv) rows
+    whose keys are all hidden give zeros; (v) token scores are taken on the masked P."""
+    B, Hq, Hkv, Lq, Lk, Dh = 2, 4, 2, 9, 13, 16
+    Q, K, V = synth.attention_qkv(B, Hq, Hkv, Lq, Lk, Dh, seed=26, n_outlier=2)
+    tri = np.where(np.tril(np.ones((Lq, Lk), bool), k=Lk - Lq), 0.0, -np.inf)
+    for rho_d, rho_t in ((1.0, 1.0), (0.5, 0.5)):
+        want = oracle.attn(Q, K, V, True, rho_d, rho_t, want_p=True)
+        got = oracle.attn(Q, K, V, False, rho_d, rho_t, want_p=True, mask=tri)
+        assert np.array_equal(got[0], want[0]) and np.array_equal(got[3], want[3]) and np.array_equal(got[1], want[1])
+        both = oracle.attn(Q, K, V, True, rho_d, rho_t, mask=tri)                      # the two masks compose
+        assert np.array_equal(both[0], want[0])
+    # (ii) a float mask against the library, unrounded P, no reduction
+    rng = np.random.default_rng(5)
+    M4 = rng.normal(0.0, 2.0, (B, Hq, Lq, Lk))
+    M4[rng.random(M4.shape) < 0.2] = -np.inf
+    M4[..., 0] = 0.5                                                                   # every row keeps a key
+    for M in (M4, M4[0, 0], M4[:, :1], M4[:1]):                                        # full, [Lq,Lk], per batch, per head
+        O, _, _, _ = oracle.attn(Q, K, V, False, 1.0, 1.0, round_p=False, mask=M)
+        Mt = torch.from_numpy(np.broadcast_to(M, (B, Hq, Lq, Lk)).copy())
+        Kr, Vr = K.double().repeat_interleave(Hq // Hkv, 1), V.double().repeat_interleave(Hq // Hkv, 1)
+        want = torch.nn.functional.scaled_dot_product_attention(Q.double(), Kr, Vr, attn_mask=Mt).numpy()
+        assert np.allclose(O, want, rtol=1e-11, atol=1e-12)
+    # (iii) one hidden key of one head
+    M = np.zeros((B, Hq, Lq, Lk))
+    M[1, 2, :, 5] = -np.inf
+    base = oracle.attn(Q, K, V, False, 0.5, 1.0, want_p=True)
+    got = oracle.attn(Q, K, V, False, 0.5, 1.0, want_p=True, mask=M)
+    assert np.all(got[3][1, 2][:, 5] == 0.0) and np.all(base[3][1, 2][:, 5] > 0.0)
+    keep = np.ones((B, Hq), bool)
+    keep[1, 2] = False
+    assert np.array_equal(got[3][keep], base[3][keep]) and not np.array_equal(got[0][1, 2], base[0][1, 2])
+    # (iv) rows with every key hidden
+    M = np.zeros((Lq, Lk))
+    M[3] = -np.inf
+    O, _, _, P = oracle.attn(Q, K, V, False, 1.0, 1.0, want_p=True, mask=M)
+    assert np.all(O[:, :, 3] == 0.0) and np.all(P[:, :, 3] == 0.0) and np.isfinite(O).all()
+    # (v) hidden keys have zero score and are never kept while visible ones remain
+    M = np.zeros((Lq, Lk))
+    M[:, [1, 4, 7]] = -np.inf
+    _, _, It, P = oracle.attn(Q, K, V, False, 1.0, 0.5, want_p=True, mask=M)
+    assert not np.isin(It, [1, 4, 7]).any() and np.all(P[..., [1, 4, 7]] == 0.0)
+
+
 @pytest.mark.parametrize("causal", [False, True])
 def test_attention_on_sampled_query_rows(oracle, causal):
     """Steps 2-4 of Sec. 3.3 and the final product are row by row: evaluating a subset of the query rows gives
