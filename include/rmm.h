@@ -155,7 +155,8 @@ int rmm_reduced_gemm_q8(const rmm_mat_t *A, const rmm_mat_t *B, float b_scale, c
 /* Reduced attention of Sec. 3.3 for B sequences, Hq query heads, Hkv key/value heads (Hq % Hkv == 0,
  * query head h reads kv head h / (Hq/Hkv)).  Per (sequence, query head):
  *   I  = TopK of ||Q[:, j]||_2, |I| = ceil(rho_d Dh);  S~ = Q[:, I] K[:, I]^T / sqrt(Dh)  (full Dh in the scale)
- *   P  = softmax(S~ + M), M = causal mask aligned to the end (query i sees keys t <= i + Lk - Lq) or none;
+ *   P  = softmax(S~ + M), M = causal mask aligned to the end (query i sees keys t <= i + Lk - Lq), and / or an
+ *        additive mask given by the caller (`mask`), or none;
  *        P is rounded once to bf16 and that rounded P is what is scored and multiplied
  *   rho_t < 1:  T = TopK of ||P[:, t]||_2, |T| = ceil(rho_t Lk);  O = P[:, T] V[T, :]  (no renormalisation)
  *   rho_t == 1: O = P V
@@ -165,13 +166,19 @@ int rmm_reduced_gemm_q8(const rmm_mat_t *A, const rmm_mat_t *B, float b_scale, c
  * for rho_t == 1; row normalisers, token scores and a gathered P V pass for rho_t < 1, where the normalised P is
  * what is rounded, scored and multiplied; for rho_t == 1 the bf16 rounding is applied to P times a per-row factor,
  * which changes O by rounding noise only).  Wider heads materialise S~ and P in the workspace one group of heads at a
- * time.  An evenly strided batch is processed as B * Hq heads in one pass of launches. */
+ * time.  An evenly strided batch is processed as B * Hq heads in one pass of launches.
+ * mask (device, fp32, or NULL): the additive M of Sec. 3.3, entry (b, h, i, t) at mask[b ms[0] + h ms[1] + i ms[2] + t]
+ * with ms = mask_stride in elements (0 shares the mask along that axis; rows contiguous); -inf hides a key; a row with
+ * every key hidden gives zeros.  It composes with `causal`.  With a mask the composed form runs (S~ and P in the
+ * workspace) whatever the head dimension: the fused kernels take the causal mask only. */
 typedef struct {
     int64_t B, Hq, Hkv, Lq, Lk, Dh;
     int32_t causal;
     double rho_d; /* feature retention of Q K^T */
     double rho_t; /* token retention of P V; 1.0 switches token reduction off */
     int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3]; /* batch, head, row (elements); last dim contiguous */
+    const float *mask;                                          /* optional additive mask (device) or NULL */
+    int64_t mask_stride[3];                                     /* batch, head, query row (elements) */
 } rmm_attn_desc_t;
 size_t rmm_reduced_attn_workspace_bytes(const rmm_attn_desc_t *desc);
 int rmm_reduced_attn(const rmm_attn_desc_t *desc, const void *Q, const void *K, const void *V, void *O,

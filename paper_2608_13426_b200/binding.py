@@ -42,7 +42,8 @@ class rmm_attn_desc_t(ctypes.Structure):
                 ("Lk", ctypes.c_int64), ("Dh", ctypes.c_int64), ("causal", ctypes.c_int32),
                 ("rho_d", ctypes.c_double), ("rho_t", ctypes.c_double),
                 ("q_stride", ctypes.c_int64 * 3), ("k_stride", ctypes.c_int64 * 3),
-                ("v_stride", ctypes.c_int64 * 3), ("o_stride", ctypes.c_int64 * 3)]
+                ("v_stride", ctypes.c_int64 * 3), ("o_stride", ctypes.c_int64 * 3),
+                ("mask", ctypes.c_void_p), ("mask_stride", ctypes.c_int64 * 3)]
 
 
 EXPORTS = ["rmm_keep_count", "rmm_score_workspace_bytes", "rmm_score", "rmm_select_workspace_bytes", "rmm_select",
@@ -396,8 +397,9 @@ def rmm_reduced_gemm_q8(A: torch.Tensor, Bq_nk: torch.Tensor, b_scale: float, id
 
 
 def rmm_reduced_attn(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, causal: bool, rho_d: float, rho_t: float = 1.0,
-                     want_idx: bool = False, ws: Optional[torch.Tensor] = None):
-    """Reduced attention.  Q [B,Hq,Lq,Dh], K,V [B,Hkv,Lk,Dh] bf16 with contiguous last dim.
+                     want_idx: bool = False, ws: Optional[torch.Tensor] = None, mask: Optional[torch.Tensor] = None):
+    """Reduced attention.  Q [B,Hq,Lq,Dh], K,V [B,Hkv,Lk,Dh] bf16 with contiguous last dim; mask (optional): additive
+    fp32 CUDA tensor [.., Lq, Lk] with up to four dims, size-1 batch / head / row dims shared, contiguous last dim.
     Returns O [B,Hq,Lq,Dh] bf16, or (O, idx_feat, idx_tok) with want_idx (idx_tok None when rho_t == 1)."""
     for t in (Q, K, V):
         if t.dim() != 4 or t.dtype != torch.bfloat16 or not t.is_cuda or t.stride(3) != 1:
@@ -407,7 +409,17 @@ def rmm_reduced_attn(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, causal: 
     O = _out((B, Hq, Lq, Dh), torch.bfloat16, Q.device)
     d = rmm_attn_desc_t(B, Hq, Hkv, Lq, Lk, Dh, int(bool(causal)), float(rho_d), float(rho_t),
                         (ctypes.c_int64 * 3)(*Q.stride()[:3]), (ctypes.c_int64 * 3)(*K.stride()[:3]),
-                        (ctypes.c_int64 * 3)(*V.stride()[:3]), (ctypes.c_int64 * 3)(*O.stride()[:3]))
+                        (ctypes.c_int64 * 3)(*V.stride()[:3]), (ctypes.c_int64 * 3)(*O.stride()[:3]),
+                        None, (ctypes.c_int64 * 3)(0, 0, 0))
+    if mask is not None:
+        m = mask
+        while m.dim() < 4:
+            m = m.unsqueeze(0)
+        if (m.dim() != 4 or m.dtype != torch.float32 or not m.is_cuda or m.shape[3] != Lk or (Lk > 1 and m.stride(3) != 1)
+                or any(m.shape[a] not in (1, n) for a, n in enumerate((B, Hq, Lq)))):
+            raise RmmError(RMM_ERR_INVALID_ARG, "mask must be an fp32 CUDA tensor broadcastable to [B,Hq,Lq,Lk], last dim contiguous")
+        d.mask = m.data_ptr()
+        d.mask_stride = (ctypes.c_int64 * 3)(*[0 if m.shape[a] == 1 else m.stride(a) for a in range(3)])
     need = lib().rmm_reduced_attn_workspace_bytes(ctypes.byref(d))
     if need == 0:
         raise RmmError(RMM_ERR_INVALID_ARG, "reduced_attn: invalid description (check shapes and retention ratios)")

@@ -48,29 +48,35 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float *sh)
 }
 
 // One block per row: max, sum of exp, normalise, round to bf16 (RNE).  Keys t > i + (Lk - Lq) are masked
-// when causal; a row with no visible key is all zeros.
+// when causal; `mask` (or NULL) is the additive M of P = softmax(S~ + M), row (h, i) at mask + h m_sh + i m_sr; a row
+// with no visible key is all zeros.
 __global__ void __launch_bounds__(kSoftmaxThreads) softmax_rows_kernel(const float *__restrict__ S, int64_t ld_s,
                                                                        int64_t Lq, int64_t Lk, int causal,
-                                                                       __nv_bfloat16 *__restrict__ P, int64_t ld_p)
+                                                                       const float *__restrict__ mask, int64_t m_sh,
+                                                                       int64_t m_sr, __nv_bfloat16 *__restrict__ P,
+                                                                       int64_t ld_p)
 {
     __shared__ float sh[32];
     pdl_wait();
     const int64_t i = blockIdx.x, h = blockIdx.y;
     const float *s = S + (h * Lq + i) * ld_s;
+    const float *m = mask != nullptr ? mask + h * m_sh + i * m_sr : nullptr;
     __nv_bfloat16 *p = P + (h * Lq + i) * ld_p;
     int64_t visible = causal ? i + (Lk - Lq) + 1 : Lk;
     if (visible > Lk) visible = Lk;
     if (visible < 0) visible = 0;
+    auto logit = [&](int64_t t) { return m != nullptr ? s[t] + m[t] : s[t]; };
 
     float mx = -INFINITY;
-    for (int64_t t = threadIdx.x; t < visible; t += kSoftmaxThreads) mx = fmaxf(mx, s[t]);
+    for (int64_t t = threadIdx.x; t < visible; t += kSoftmaxThreads) mx = fmaxf(mx, logit(t));
     mx = block_reduce(mx, true, sh);
+    if (!(mx > -INFINITY)) visible = 0;  // every key hidden
     float sum = 0.f;
-    for (int64_t t = threadIdx.x; t < visible; t += kSoftmaxThreads) sum += expf(s[t] - mx);
+    for (int64_t t = threadIdx.x; t < visible; t += kSoftmaxThreads) sum += expf(logit(t) - mx);
     sum = block_reduce(sum, false, sh);
     const float inv = sum > 0.f ? 1.0f / sum : 0.f;
     for (int64_t t = threadIdx.x; t < ld_p; t += kSoftmaxThreads) {
-        float v = t < visible ? expf(s[t] - mx) * inv : 0.f;
+        float v = t < visible ? expf(logit(t) - mx) * inv : 0.f;
         p[t] = __float2bfloat16_rn(v);
     }
 }
@@ -99,7 +105,8 @@ rmm_attn_desc_t fold_batch(const rmm_attn_desc_t &d)
     rmm_attn_desc_t f = d;
     const bool even = d.B > 1 && d.Hkv >= 1 && d.Hq % d.Hkv == 0 && d.B * d.Hq <= 65535 &&
                       d.q_stride[0] == d.Hq * d.q_stride[1] && d.k_stride[0] == d.Hkv * d.k_stride[1] &&
-                      d.v_stride[0] == d.Hkv * d.v_stride[1] && d.o_stride[0] == d.Hq * d.o_stride[1];
+                      d.v_stride[0] == d.Hkv * d.v_stride[1] && d.o_stride[0] == d.Hq * d.o_stride[1] &&
+                      (d.mask == nullptr || d.mask_stride[0] == d.Hq * d.mask_stride[1]);
     if (even) {
         f.B = 1;
         f.Hq = d.B * d.Hq;
@@ -108,6 +115,7 @@ rmm_attn_desc_t fold_batch(const rmm_attn_desc_t &d)
         f.k_stride[0] = f.Hkv * d.k_stride[1];
         f.v_stride[0] = f.Hkv * d.v_stride[1];
         f.o_stride[0] = f.Hq * d.o_stride[1];
+        f.mask_stride[0] = f.Hq * d.mask_stride[1];
     }
     return f;
 }
@@ -125,6 +133,8 @@ int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
     for (int i = 0; i < 3; ++i)
         if (d->q_stride[i] % 8 || d->k_stride[i] % 8 || d->v_stride[i] % 8 || d->o_stride[i] % 8)
             return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: strides must be multiples of 8 elements");
+    if (d->mask != nullptr && (d->mask_stride[0] < 0 || d->mask_stride[1] < 0 || d->mask_stride[2] < 0))
+        return fail(RMM_ERR_INVALID_ARG, "reduced_attn: negative mask stride");
     // V's (batch, head) pairs must form one batch axis of the tensor map used when V is read in place
     if (d->v_stride[2] < d->Dh || d->v_stride[0] != d->Hkv * d->v_stride[1])
         return fail(RMM_ERR_UNSUPPORTED, "reduced_attn: V needs batch stride = Hkv * head stride");
@@ -136,7 +146,7 @@ int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
     const double per_head = (double)d->Lq * ((double)p->ld_s * 4 + (double)p->ld_p * 2 + (double)p->ldt * 2);
     int64_t hg = (int64_t)(6.0 * 1073741824.0 / per_head);
     if (hg < 1) hg = 1;
-    p->fused = use_fused(d, p->kd);
+    p->fused = d->mask == nullptr && use_fused(d, p->kd);  // the fused kernels take the causal mask only
     if (hg > d->Hq || p->fused) hg = d->Hq;  // the fused form materialises neither S~ nor P: all heads at once
     p->hg = hg;
 
@@ -171,12 +181,13 @@ int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
 
 }  // namespace
 
-int launch_softmax_rows(const float *S, int64_t ld_s, int64_t heads, int64_t Lq, int64_t Lk, int causal,
-                        __nv_bfloat16 *P, int64_t ld_p, cudaStream_t stream)
+int launch_softmax_rows(const float *S, int64_t ld_s, int64_t heads, int64_t Lq, int64_t Lk, int causal, const float *mask,
+                        int64_t m_sh, int64_t m_sr, __nv_bfloat16 *P, int64_t ld_p, cudaStream_t stream)
 {
     dim3 grid((unsigned)Lq, (unsigned)heads);
     prof_begin("softmax_rows_kernel", stream);
-    launch_kernel(softmax_rows_kernel, grid, dim3(kSoftmaxThreads), 0, stream, 1, S, ld_s, Lq, Lk, causal, P, ld_p);
+    launch_kernel(softmax_rows_kernel, grid, dim3(kSoftmaxThreads), 0, stream, 1, S, ld_s, Lq, Lk, causal, mask, m_sh, m_sr, P,
+                  ld_p);
     return check_launch("softmax_rows_kernel", stream);
 }
 
@@ -283,7 +294,10 @@ int rmm_reduced_attn(const rmm_attn_desc_t *desc, const void *Q, const void *K, 
             g1.scale = scale; g1.status = status;
             if ((rc = launch_gemm_tc_problem(g1, st)) != RMM_OK) return rc;
 
-            if ((rc = launch_softmax_rows(S, p.ld_s, hg, d->Lq, d->Lk, d->causal, P, p.ld_p, st)) != RMM_OK) return rc;
+            const float *mask = d->mask != nullptr ? d->mask + b * d->mask_stride[0] + h0 * d->mask_stride[1] : nullptr;
+            if ((rc = launch_softmax_rows(S, p.ld_s, hg, d->Lq, d->Lk, d->causal, mask, d->mask_stride[1], d->mask_stride[2], P,
+                                          p.ld_p, st)) != RMM_OK)
+                return rc;
 
             TcProblem g2 = {};
             g2.batch = hg; g2.M = d->Lq; g2.N = d->Dh;

@@ -217,10 +217,10 @@ int launch_gather_q8(bool quantise, const void *src, int64_t rows, int64_t s_row
                      int64_t ld_dst, float *row_scale, int *status, cudaStream_t stream);
 
 // ---- attention helpers --------------------------------------------------------------------------------
-// Row softmax of fp32 logits S [heads, Lq, ld_s] with optional end-aligned causal mask; writes bf16
-// P [heads, Lq, ld_p] (columns Lk .. ld_p zeroed).
-int launch_softmax_rows(const float *S, int64_t ld_s, int64_t heads, int64_t Lq, int64_t Lk, int causal,
-                        __nv_bfloat16 *P, int64_t ld_p, cudaStream_t stream);
+// Row softmax of fp32 logits S [heads, Lq, ld_s] with optional end-aligned causal mask and optional additive mask
+// (row (h, i) at mask + h m_sh + i m_sr, fp32); writes bf16 P [heads, Lq, ld_p] (columns Lk .. ld_p zeroed).
+int launch_softmax_rows(const float *S, int64_t ld_s, int64_t heads, int64_t Lq, int64_t Lk, int causal, const float *mask,
+                        int64_t m_sh, int64_t m_sr, __nv_bfloat16 *P, int64_t ld_p, cudaStream_t stream);
 // Fused forms (S~ and P stay on the SM; head_dim and kept features up to 128) on packed Qp [heads, Lq, ldd],
 // Kp [heads, Lk, ldd] (kd valid columns) and V [v_batches, Lk, Dh] (row pitch v_ld, batch pitch v_sb; head h uses
 // batch entry (h + v_off) / v_div).

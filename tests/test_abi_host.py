@@ -36,7 +36,7 @@ def test_header_symbols_are_exported(L):
 
 def test_struct_layouts_match_header(L):
     assert ctypes.sizeof(binding.rmm_mat_t) == 64
-    assert ctypes.sizeof(binding.rmm_attn_desc_t) == 6 * 8 + 8 + 16 + 12 * 8
+    assert ctypes.sizeof(binding.rmm_attn_desc_t) == 6 * 8 + 8 + 16 + 12 * 8 + 8 + 3 * 8
 
 
 def test_keep_count_host(L):

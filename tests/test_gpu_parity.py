@@ -371,13 +371,15 @@ def test_host_buffer_entry_point(oracle):
 # ------------------------------------------------------------------------------------------------
 # attention
 # ------------------------------------------------------------------------------------------------
-def check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t, seed, n_outlier=4, tok_band=1e-4):
+def check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t, seed, n_outlier=4, tok_band=1e-4, mask=None):
     """Feature sets: strict 1e-6 band against the oracle's TopK on Q.  Everything after that is judged on the GPU's
     OWN sets: the oracle is evaluated on the GPU's feature sets (its P and its TopK token sets are then the
     reference for the token sets) and on the GPU's token sets (its O is the reference for O).  No comparison is
     conditional on the sets coinciding.  Returns whether the feature sets coincided with the oracle's."""
     Q, K, V = synth.attention_qkv(B, Hq, Hkv, Lq, Lk, Dh, seed=seed, n_outlier=n_outlier)
-    O, idx_feat, idx_tok = rmm.rmm_reduced_attn(dev(Q), dev(K), dev(V), causal, rho_d, rho_t, want_idx=True)
+    mask_np = None if mask is None else mask.numpy().astype(np.float64)      # fp32 values, exact in fp64
+    O, idx_feat, idx_tok = rmm.rmm_reduced_attn(dev(Q), dev(K), dev(V), causal, rho_d, rho_t, want_idx=True,
+                                                mask=None if mask is None else dev(mask))
     kd = oracle.keep_count(rho_d, Dh)
     feat = idx_feat.cpu().numpy()
     same_feat = True
@@ -390,7 +392,7 @@ def check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t, seed, 
         kt = oracle.keep_count(rho_t, Lk)
         tok = idx_tok.cpu().numpy()
         assert tok.shape == (B, Hq, kt)
-        _, _, It, P = oracle.attn(Q, K, V, causal, rho_d, rho_t, round_p=True, want_p=True, idx_feat=feat)
+        _, _, It, P = oracle.attn(Q, K, V, causal, rho_d, rho_t, round_p=True, want_p=True, idx_feat=feat, mask=mask_np)
         for b in range(B):
             for h in range(Hq):
                 # token scores come from an fp32 softmax on the GPU: judge the criterion (Theorem 1) --
@@ -403,7 +405,7 @@ def check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, causal, rho_d, rho_t, seed, 
                 tau = np.sort(s)[::-1][kt - 1]
                 diff = np.setxor1d(tok[b, h], It[b, h])
                 assert np.all(np.abs(s[diff] - tau) <= tok_band * s.max())
-    Oo, _, _, _ = oracle.attn(Q, K, V, causal, rho_d, rho_t, round_p=True, idx_feat=feat, idx_tok=tok)
+    Oo, _, _, _ = oracle.attn(Q, K, V, causal, rho_d, rho_t, round_p=True, idx_feat=feat, idx_tok=tok, mask=mask_np)
     Og = O.float().cpu().numpy()
     assert np.isfinite(Og).all()
     for b in range(B):
@@ -463,6 +465,30 @@ def test_fused_attention_logits_that_outgrow_the_running_maximum(oracle, causal,
         assert rel_fro(Og[0, h], Oo[0, h]) <= TOL_BF16, h
         for lo, hi in ((0, 200), (200, 300), (300, 450), (450, L)):      # the rows that see 0, 1, 2, 3 of the keys (causal)
             assert rel_fro(Og[0, h, lo:hi], Oo[0, h, lo:hi]) <= TOL_BF16, (h, lo)
+
+
+@pytest.mark.parametrize("rho_d,rho_t", [(0.5, 1.0), (0.5, 0.5), (1.0, 0.25)])
+def test_reduced_attention_with_an_additive_mask(oracle, rho_d, rho_t):
+    """P = softmax(S~ + M) of Sec. 3.3 with a caller-given M: a finite bias with hidden entries per (sequence, head); a
+    sliding window shared by all heads on top of the causal mask (some rows lose every key to neither); a per-head
+    bias shared across the batch; a mask that hides whole rows."""
+    g = torch.Generator().manual_seed(70)
+    B, Hq, Hkv, Lq, Lk, Dh = 2, 4, 2, 150, 173, 64
+    M = torch.randn(B, Hq, Lq, Lk, generator=g) * 2.0
+    M[torch.rand(B, Hq, Lq, Lk, generator=g) < 0.2] = -float("inf")
+    M[..., 0] = 0.25
+    assert check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, False, rho_d, rho_t, seed=71, mask=M)
+    L = 300
+    i, t = torch.arange(L)[:, None], torch.arange(L)[None, :]
+    window = torch.where((i - t).abs() <= 40, 0.0, -float("inf"))
+    assert check_attention(oracle, 1, 4, 2, L, L, 128, True, rho_d, rho_t, seed=72, mask=window)
+    bias = torch.randn(1, 4, 1, L, generator=g)                     # per head and key, shared by rows and sequences
+    assert check_attention(oracle, 2, 4, 4, L, L, 128, False, rho_d, rho_t, seed=73, mask=bias)
+    rows_off = torch.zeros(L, L)
+    rows_off[17] = -float("inf")
+    rows_off[200:230] = -float("inf")
+    assert check_attention(oracle, 1, 2, 1, L, L, 64, False, rho_d, rho_t, seed=74, mask=rows_off)
+    assert rmm.rmm_status_read() == 0
 
 
 def test_fused_attention_rows_without_keys_are_zero():
