@@ -428,6 +428,70 @@ def run_mlp_1b_only(args):
     print(json.dumps({"mlp_1b": res}))
 
 
+def run_phase_stamps(args):
+    """Per-phase timelines from a library built with the debug time stamps
+    (RMM_NVCC_EXTRA="-DRMM_GEMM_STAMPS -DRMM_FRONT_STAMPS -DRMM_ATTN_STAMPS" python -m paper_2608_13426_b200.build):
+    the one-launch front end and the GEMM of the 1B-class product (microseconds from the first block's start; maxima over
+    blocks), and the clocks per phase of the fused attention kernel's MMA-issuing thread and of one softmax warp.  The
+    shipped library has no stamps; rebuild without the flags afterwards."""
+    import ctypes
+    import paper_2608_13426_b200 as rmm
+    from paper_2608_13426_b200 import binding, synth
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    L = binding.lib()
+    have = {n: hasattr(L, n) for n in ("rmm_debug_front_stamps", "rmm_debug_gemm_stamps", "rmm_debug_attn_stamps")}
+    if not any(have.values()):
+        print(json.dumps({"phase_stamps": None, "why": "the library was built without -DRMM_*_STAMPS"}))
+        return
+    buf = (ctypes.c_ulonglong * 16)()
+    out = {}
+    A, B = synth.mlp_product(M1, K1, N1, seed=0)
+    A, B = A.to(dev), B.to(dev)
+    front_names = ["stream_end", "energies_published", "barrier_passed", "selected", None, "a_gathered_b_copied"]
+    gemm_names = ["setup_done", "first_mma", "last_main_loop_issued", "last_accumulator_complete", "last_epilogue_done", "last_thread_out"]
+    reps = max(5, args.steps)
+    for rho in (0.25, 0.5):
+        for _ in range(3):
+            rmm.rmm_product(A, B, rho=rho)
+        torch.cuda.synchronize()
+        for n in ("rmm_debug_front_stamps", "rmm_debug_gemm_stamps"):
+            if have[n]:
+                getattr(L, n)(buf)
+        acc_f, acc_g = [0.0] * 6, [0.0] * 6
+        for _ in range(reps):
+            rmm.rmm_product(A, B, rho=rho)
+            torch.cuda.synchronize()
+            if have["rmm_debug_front_stamps"]:
+                L.rmm_debug_front_stamps(buf)
+                for j in range(6):
+                    acc_f[j] += (buf[j + 1] - buf[0]) / 1e3
+            if have["rmm_debug_gemm_stamps"]:
+                L.rmm_debug_gemm_stamps(buf)
+                for j in range(6):
+                    acc_g[j] += (buf[j + 1] - buf[0]) / 1e3
+        e = {}
+        if have["rmm_debug_front_stamps"]:
+            e["front_us_from_start"] = {n: round(v / reps, 2) for n, v in zip(front_names, acc_f) if n}
+        if have["rmm_debug_gemm_stamps"]:
+            e["gemm_us_from_start"] = {n: round(v / reps, 2) for n, v in zip(gemm_names, acc_g)}
+        out[f"mlp_1b_rho{rho}"] = e
+    if have["rmm_debug_attn_stamps"]:
+        Q, Kk, V = synth.attention_qkv(1, args.attn_heads, args.attn_heads, args.attn_seq, args.attn_seq, 128, seed=0, device=str(dev))
+        mma = ["wait_k", "wait_s_empty", "issue_s", "wait_v", "wait_o_empty", "wait_p_full", "issue_pv", "other"]
+        smx = ["wait_s_full", "unused", "max_and_rescale", "weights_chunk_1", "wait_p_empty", "store_reload_weights_chunk_0", "epilogue", "loop_top"]
+        for causal in (True, False):
+            for _ in range(2):
+                rmm.rmm_reduced_attn(Q, Kk, V, causal, 0.5, 1.0)
+            L.rmm_debug_attn_stamps(buf)
+            rmm.rmm_reduced_attn(Q, Kk, V, causal, 0.5, 1.0)
+            L.rmm_debug_attn_stamps(buf)
+            v = list(buf)
+            out[f"fused_attn_clocks_block0_causal{int(causal)}"] = {"mma_thread": dict(zip(mma, v[:8])), "softmax_warp": dict(zip(smx, v[8:]))}
+    assert rmm.rmm_status_read() == 0
+    print(json.dumps({"phase_stamps": out}))
+
+
 def run_attention_only(args):
     import paper_2608_13426_b200 as rmm
     from paper_2608_13426_b200 import binding, synth
@@ -502,6 +566,8 @@ def main():
                     help="run only the reduced-attention case (a few launches: for profiler captures) and print its own JSON line")
     ap.add_argument("--mlp-1b-only", action="store_true",
                     help="run only the 1B-class product at rho = 0.5 (for profiler captures) and print its own JSON line")
+    ap.add_argument("--phase-stamps", action="store_true",
+                    help="print per-phase timelines; needs a library built with -DRMM_GEMM_STAMPS -DRMM_FRONT_STAMPS -DRMM_ATTN_STAMPS")
     ap.add_argument("--attn-heads", type=int, default=32)
     ap.add_argument("--attn-seq", type=int, default=4096)
     args = ap.parse_args()
@@ -511,6 +577,8 @@ def main():
         return run_attention_only(args)
     if args.mlp_1b_only:
         return run_mlp_1b_only(args)
+    if args.phase_stamps:
+        return run_phase_stamps(args)
     if args.warmup < 3:
         args.warmup = 3
 

@@ -703,3 +703,18 @@ int launch_gemm_tc(const rmm_mat_t *A, const rmm_mat_t *B, const int32_t *idx, i
 }
 
 }  // namespace rmm
+
+#ifdef RMM_GEMM_STAMPS
+// Debug build only: copy the GEMM kernel's phase stamps (nanoseconds of %globaltimer; slot 0 the first block's start, a
+// minimum; 1 set-up done, 2 first tensor-core instruction, 3 last main loop issued, 4 last accumulator complete, 5 last
+// epilogue done, 6 last thread out: maxima over blocks) to out[0 .. 15] and re-arm them.
+extern "C" int rmm_debug_gemm_stamps(unsigned long long *out)
+{
+    unsigned long long init[16];
+    cudaError_t e = cudaMemcpyFromSymbol(out, rmm::g_gstamps, sizeof init);
+    for (int i = 0; i < 16; ++i) init[i] = 0;
+    init[0] = ~0ull;
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(rmm::g_gstamps, init, sizeof init);
+    return e == cudaSuccess ? RMM_OK : RMM_ERR_CUDA;
+}
+#endif
