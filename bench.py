@@ -39,8 +39,8 @@ UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0          # dense bf16 tensor peak of a B200 as specified (context beside the measured peaks)
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the GEMM kernel on the headline workload at rho = 0.5,
-# from the one-pass ncu capture summarised in profiles/reduced_gemm_tc_kernel_down_proj_32768x28672x8192_rho0.5.md
-GEMM_DRAM_TRAFFIC_BYTES = None
+# from the one-pass ncu capture summarised in profiles/reduced_gemm_tc_kernel_down_proj_28672x8192_rho0.5.md
+GEMM_DRAM_TRAFFIC_BYTES = 14246983168 + 536363008
 WORKLOAD = ("70B-class MLP down-projection: A 32768x28672 bf16 N(0,1) with 1% Student-t(3) channels, "
             "B 28672x8192 bf16 N(0,0.02^2)")
 
@@ -324,6 +324,65 @@ def layer_sweep_70b(rmm, synth, dev, peaks, tokens=32768, hidden=8192, inter=286
         out.append({"layer": "attention", "shape": [64, 8, tokens, 128], "rho_d": rho_d, "rho_t": rho_t, "ms": t,
                     "dense_sdpa_ms": dense, "speedup_vs_dense_sdpa": dense / t})
     return out
+
+
+def chained_mlp_70b(rmm, synth, dev, tokens=32768, hidden=8192, inter=28672, rho=RHO, reps=5):
+    """Up projection followed by the reduced down projection of a 70B-class MLP.  The up projection's epilogue leaves
+    the column energies of the activations it writes, so the down projection selects its index set from them and needs
+    no pass over the 1.9 GB of activations: times with and without that pass, and what the epilogue sums cost."""
+    X = synth.heavy_tailed_activations(tokens, hidden, seed=11, device=str(dev))
+    W_up = synth.weight(hidden, inter, seed=12, device=str(dev))
+    W_down = synth.weight(inter, hidden, seed=13, device=str(dev))
+    H = torch.empty(tokens, inter, dtype=torch.bfloat16, device=dev)
+    Y = torch.empty(tokens, hidden, dtype=torch.bfloat16, device=dev)
+    k = rmm.rmm_keep_count(rho, inter)
+    idx = torch.empty(k, dtype=torch.int32, device=dev)
+    keep = {}
+
+    def up_plain(i):
+        rmm.rmm_reduced_gemm(X, W_up, None, out=H)
+
+    def up_scored(i):
+        keep["e"] = rmm.rmm_reduced_gemm(X, W_up, None, out=H, want_energy=True)[1]
+
+    def down_from_energies(i):
+        sel = rmm.rmm_select(keep["e"], k=k)
+        rmm.rmm_reduced_gemm(H, W_down, sel, out=Y)
+
+    def down_with_score_pass(i):
+        rmm.rmm_product(H, W_down, rho=rho, out=Y, idx=idx)
+
+    def dense_block(i):
+        torch.matmul(X, W_up, out=H)
+        torch.matmul(H, W_down, out=Y)
+
+    # The SM clock under the power cap drifts by a quarter over a few seconds of tensor-core load, so the variants are
+    # interleaved call by call (each call bracketed by its own events) instead of being timed one after the other.
+    names = ["up_ms", "up_with_epilogue_energies_ms", "down_selected_from_epilogue_energies_ms", "down_with_score_pass_ms",
+             "block_ms_dense_cublas"]
+    fns = [up_plain, up_scored, down_from_energies, down_with_score_pass, dense_block]
+    for fn in fns:
+        fn(0)
+    total = [0.0] * len(fns)
+    for r in range(reps):
+        for j in range(len(fns)):
+            jj = (j + r) % len(fns)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if jj in (2, 3):
+                up_scored(r)          # the down projection under test reads H and its energies fresh
+            e0.record()
+            fns[jj](r)
+            e1.record()
+            e1.synchronize()
+            total[jj] += e0.elapsed_time(e1)
+    res = {"shape_up": [tokens, hidden, inter], "shape_down": [tokens, inter, hidden], "rho_down": rho,
+           "timing": "variants interleaved call by call"}
+    for n, t in zip(names, total):
+        res[n] = t / reps
+    res["block_ms_epilogue_energies"] = res["up_with_epilogue_energies_ms"] + res["down_selected_from_epilogue_energies_ms"]
+    res["block_ms_score_pass"] = res["up_ms"] + res["down_with_score_pass_ms"]
+    del X, W_up, W_down, H, Y
+    return res
 
 
 def paper_table5_case(rmm, synth, dev, reps=10):
@@ -761,6 +820,9 @@ def main():
 
         # ---- the other 70B-class products and the attention of one layer
         extras["layer_sweep_70b"] = layer_sweep_70b(rmm, synth, dev, peaks)
+
+        # ---- up projection -> reduced down projection, the index set taken from the up projection's epilogue energies
+        extras["mlp_block_70b"] = chained_mlp_70b(rmm, synth, dev)
 
     if rank == 0:
         out = {

@@ -108,6 +108,25 @@ def test_70b_class_down_projection_index_set(oracle):
         assert rel_fro(Y[r].float().cpu().numpy(), want) <= TOL_BF16
 
 
+def test_70b_class_down_projection_selected_from_the_up_projection_epilogue(oracle):
+    """70B-class MLP at full size: the up projection (32768 x 8192 x 28672, CTA pairs) accumulates the column energies
+    of the activations it writes in its epilogue; the down projection's index set, selected from them with no pass over
+    the 1.9 GB of activations, must lie inside the strict tie band of the oracle's scores of those activations."""
+    M, K, N = 32768, 8192, 28672
+    X = synth.heavy_tailed_activations(M, K, seed=21, device="cuda")
+    W = synth.weight(K, N, seed=22, device="cuda")
+    H, e = rmm.rmm_reduced_gemm(X, W, None, want_energy=True)
+    k = rmm.rmm_keep_count(0.5, N)
+    idx = rmm.rmm_select(e, k=k)
+    assert rmm.rmm_status_read() == 0
+    e64, _ = oracle.score(H.cpu())
+    check_index_set(idx.cpu().numpy(), e64, k)
+    assert np.allclose(e.cpu().numpy(), e64, rtol=3e-6)
+    for r in sample_rows(M, 2, seed=5):                                # and the activations themselves, on sampled rows
+        want = oracle.reduced_gemm(X.cpu(), W.cpu(), np.arange(K, dtype=np.int32), rows=(r, r + 1))[r]
+        assert rel_fro(H[r].float().cpu().numpy(), want) <= TOL_BF16
+
+
 def check_token_sets(oracle, tok, It, P, band=1e-4):
     """Token sets of the fused sweeps against the oracle's P (evaluated on the GPU's feature sets): Theorem 1's
     criterion (retained energy within 1e-6 of the optimum) and equality outside a 1e-4 band."""
