@@ -63,6 +63,8 @@ struct TcArgs {
     int *status;
     unsigned long long wait_ns;  // bound of every device-side wait
     int withhold;                // test switch: the producer skips its very first stage, so that the waits behind it expire
+    int sync_kb;                 // the producers also meet every sync_kb k-blocks inside a tile (0: at tile starts only)
+    unsigned *wave_ctr;          // [2] in the workspace header (arrivals, exits) or NULL: keeps the blocks of a wave in step
     float *col_energy;           // [batch, ceil(M / 32), N] or NULL: sum of squares of the rounded outputs per 32-row group
     const float *row_scale;      // 8-bit operands: [batch, M] factor of every output row, or NULL
     // B_GATHER: the unpacked B and the kept row numbers
@@ -169,13 +171,33 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         // of A is shared only by the tiles of one wave and keeps the default priority: marked evict-first it was dropped
         // before its last reader arrived and DRAM traffic went up by two thirds)
         const uint64_t pol_b = l2_policy_evict_last();
-        for (int64_t tile = tile0; lane == 0 && tile < num_tiles && ok; tile += tile_step) {
+        // Blocks start a tile when they finish the last one, so without help the tiles of a wave drift apart along k
+        // and a k-slice fetched for one tile of a row or column is gone from L2 when its neighbours ask for it.  The
+        // producers therefore meet before every wave: each adds one to a counter and waits, for at most 20 us and
+        // without any consequence if the time runs out, until every block with a tile in this wave has done so.
+        unsigned wave_target = 0;
+        int64_t wave_first = 0;  // first tile of the current wave
+        for (int64_t tile = tile0; lane == 0 && tile < num_tiles && ok; tile += tile_step, wave_first += tile_step) {
+            const int64_t in_wave = num_tiles - wave_first < tile_step ? num_tiles - wave_first : tile_step;
+            auto meet = [&]() {
+                wave_target += (unsigned)(in_wave * CTAS);
+                unsigned seen;
+                asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(seen) : "l"(a.wave_ctr) : "memory");
+                ++seen;
+                const unsigned long long t0 = global_ns();
+                while (seen < wave_target && global_ns() - t0 < 20000ull) {
+                    __nanosleep(64);
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.wave_ctr) : "memory");
+                }
+            };
+            if (a.wave_ctr != nullptr) meet();
             int tm, tn;
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
             tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, a.raster, tm, tn);
             int64_t bb = (b + a.b_batch_off) / a.b_batch_div;
             if (bb >= a.b_batches) bb = a.b_batches - 1;
             for (int kb = 0; kb < num_kb; ++kb) {
+                if (a.wave_ctr != nullptr && a.sync_kb > 0 && kb > 0 && kb % a.sync_kb == 0) meet();
                 if (!mbar_wait_lane(empty_bar(s), ph ^ 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                 if (a.withhold && blockIdx.x == 0 && tile == tile0 && kb == 0) {
                     // (test switch) this stage is never requested: its barrier stays incomplete
@@ -212,6 +234,14 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                     }
                 }
                 if (++s == kStages) { s = 0; ph ^= 1u; }
+            }
+        }
+        if (lane == 0 && a.wave_ctr != nullptr) {  // the last block out re-arms the counters for the next launch
+            unsigned out;
+            asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(out) : "l"(a.wave_ctr + 1) : "memory");
+            if (out == gridDim.x - 1) {
+                asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(a.wave_ctr), "r"(0u) : "memory");
+                asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(a.wave_ctr + 1), "r"(0u) : "memory");
             }
         }
         __syncwarp();
@@ -577,6 +607,17 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     }
     a.wait_ns = wait_limit_ns();
     a.withhold = debug_withhold() == WITHHOLD_GEMM;
+    {
+        // wave synchronisation: products with several waves of long tiles (measurement switch RMM_GEMM_WAVE_SYNC=0|1)
+        static const int forced_sync = []() { const char *e = getenv("RMM_GEMM_WAVE_SYNC"); return e ? atoi(e) : -1; }();
+        const int64_t tiles = (int64_t)a.batch * a.tiles_m * a.tiles_n, per_wave = sm_count() / ctas;
+        const bool want = forced_sync >= 0 ? forced_sync != 0 : (tiles > per_wave && p.k * es >= 8192);
+        static const int sync_kb = []() { const char *e = getenv("RMM_GEMM_SYNC_KB"); return e ? atoi(e) : 128; }();
+        a.sync_kb = sync_kb;
+        a.wave_ctr = (want && p.status != nullptr)
+                         ? &reinterpret_cast<WsHeader *>(reinterpret_cast<char *>(p.status) - offsetof(WsHeader, status))->counters[kHeaderCounters - 4]
+                         : nullptr;
+    }
     a.col_energy = p.col_energy;
     a.row_scale = p.row_scale;
     // products with at most four k-blocks per tile are bound by the epilogue, and a block with a single tile has no next
