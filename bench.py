@@ -40,7 +40,7 @@ NOMINAL_BF16_TFLOPS = 2250.0          # dense bf16 tensor peak of a B200 as spec
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the GEMM kernel on the headline workload at rho = 0.5,
 # from the one-pass ncu capture summarised in profiles/reduced_gemm_tc_kernel_down_proj_28672x8192_rho0.5.md
-GEMM_DRAM_TRAFFIC_BYTES = 14246983168 + 536363008
+GEMM_DRAM_TRAFFIC_BYTES = 7609957888 + 536464128
 WORKLOAD = ("70B-class MLP down-projection: A 32768x28672 bf16 N(0,1) with 1% Student-t(3) channels, "
             "B 28672x8192 bf16 N(0,0.02^2)")
 
@@ -180,6 +180,39 @@ def time_region(fn, steps: int, world: int) -> float:
     return max_over_ranks(e0.elapsed_time(e1), world) / steps
 
 
+def interleaved_rho_sweep(rmm, binding, A, B, Y, rhos, rounds: int = 6):
+    """Whole reduced product per rho and the dense cuBLAS product of the same shape, timed call by call in rotation
+    (each call bracketed by its own events): under the power cap the SM clock drifts by a quarter over seconds of
+    tensor-core load, so variants timed one after the other are not comparable, variants that take turns are.
+    Returns ({rho: (whole_op_ms, gemm_kernel_ms)}, dense_ms)."""
+    Kx = A.shape[-1]
+    idx = {rho: torch.empty(rmm.rmm_keep_count(rho, Kx), dtype=torch.int32, device=A.device) for rho in rhos}
+    calls = [lambda: torch.matmul(A, B, out=Y)] + [(lambda rho=rho: rmm.rmm_product(A, B, rho=rho, out=Y, idx=idx[rho])) for rho in rhos]
+    for c in calls:
+        c()
+        c()
+    nv = len(calls)
+    total, gemm, order = [0.0] * nv, [0.0] * nv, []
+    kt = binding.KernelTimer(rounds * nv, "reduced_gemm_tc_kernel")
+    with kt:
+        for r in range(rounds):
+            for j in range(nv):
+                jj = (j + r) % nv
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                calls[jj]()
+                e1.record()
+                e1.synchronize()
+                total[jj] += e0.elapsed_time(e1)
+                if jj > 0:
+                    order.append(jj)
+    times = [t for _, t in kt.times_ms()]
+    assert len(times) == len(order)
+    for jj, t in zip(order, times):
+        gemm[jj] += t
+    return {rho: (total[j + 1] / rounds, gemm[j + 1] / rounds) for j, rho in enumerate(rhos)}, total[0] / rounds
+
+
 def cpu_oracle_sample(A_rows, B, rho: float, m_total: int, target_s: float = 12.0):
     """Time the oracle as it stands on a bounded sample of the headline workload: the score pass on `A_rows` (a slice of
     the activations), the selection at full width, the product on as many of those rows as fit the time target.  The
@@ -276,7 +309,7 @@ def attention_case(rmm, binding, synth, dev, heads, seq, head_dim=128, reps=10):
     return out
 
 
-def layer_sweep_70b(rmm, synth, dev, peaks, tokens=32768, hidden=8192, inter=28672, reps=5):
+def layer_sweep_70b(rmm, binding, synth, dev, peaks, tokens=32768, hidden=8192, inter=28672, reps=5):
     """Whole reduced product (score + select + gathers + GEMM) per projection shape and rho, dense cuBLAS beside it."""
     # (Q, K and V read the same activations, hence the same index set: fused into one product they share the selection
     # and the gather of A, which the narrow K/V projection alone cannot repay)
@@ -287,30 +320,16 @@ def layer_sweep_70b(rmm, synth, dev, peaks, tokens=32768, hidden=8192, inter=286
         A = synth.heavy_tailed_activations(m, kk, seed=7, device=str(dev))
         B = synth.weight(kk, n, seed=8, device=str(dev))
         Y = torch.empty(m, n, dtype=torch.bfloat16, device=dev)
-        for _ in range(2):
-            torch.matmul(A, B, out=Y)
-        dense_before = time_region(lambda i: torch.matmul(A, B, out=Y), reps, 1)
+        res, dense = interleaved_rho_sweep(rmm, binding, A, B, Y, RHOS, rounds=reps)
         rows = []
         for rho in RHOS:
-            k = rmm.rmm_keep_count(rho, kk)
-            idx = torch.empty(k, dtype=torch.int32, device=dev)
-
-            def op(i):
-                rmm.rmm_product(A, B, rho=rho, out=Y, idx=idx)
-
-            op(0)
-            op(1)
-            t = time_region(op, reps, 1)
-            fl = 2.0 * m * k * n
+            t = res[rho][0]
+            fl = 2.0 * m * rmm.rmm_keep_count(rho, kk) * n
             rows.append({"layer": name, "shape": [m, kk, n], "rho": rho, "whole_op_ms": t, "whole_op_tflops": fl / t / 1e9,
                          "frac_of_sustained_peak": fl / t / 1e9 / peaks["bf16_sustained"],
-                         "frac_of_burst_peak": fl / t / 1e9 / peaks["bf16_burst"]})
-        # the dense product is timed before and after the sweep (the clocks sag under sustained tensor load): mean of both
-        dense_after = time_region(lambda i: torch.matmul(A, B, out=Y), reps, 1)
-        dense = 0.5 * (dense_before + dense_after)
-        for r in rows:
-            r.update({"dense_cublas_ms": dense, "dense_cublas_ms_before_after": [dense_before, dense_after],
-                      "dense_cublas_tflops": 2.0 * m * kk * n / dense / 1e9, "speedup_vs_dense_cublas": dense / r["whole_op_ms"]})
+                         "frac_of_burst_peak": fl / t / 1e9 / peaks["bf16_burst"],
+                         "dense_cublas_ms": dense, "dense_cublas_tflops": 2.0 * m * kk * n / dense / 1e9,
+                         "speedup_vs_dense_cublas": dense / t, "timing": "variants interleaved call by call"})
         out += rows
         del A, B, Y
     # attention of one layer: 64 query heads on 8 kv heads, causal
@@ -705,31 +724,17 @@ def main():
     # ---- per-rho sweep on the headline product: whole op beside dense cuBLAS at the same shape
     per_rho = []
     if not args.no_sweep and rank == 0:
-        reps = 5
-        for _ in range(2):
-            torch.matmul(A, B, out=Y)
-        dense_before = time_region(lambda i: torch.matmul(A, B, out=Y), reps, 1)
+        res, dense_ms = interleaved_rho_sweep(rmm, binding, A, B, Y, RHOS)
         for rho in RHOS:
-            kk = rmm.rmm_keep_count(rho, K)
-            idx_r = torch.empty(kk, dtype=torch.int32, device=dev)
-            for i in range(2):
-                step(i, rho, idx_r)
-            whole = time_region(lambda i: step(i, rho, idx_r), reps, 1)
-            t = binding.KernelTimer(reps, "reduced_gemm_tc_kernel")
-            with t:
-                time_region(lambda i: step(i, rho, idx_r), reps, 1)
-            g = sum(x for _, x in t.times_ms()) / reps
+            whole, g = res[rho]
             fl = retained_flops(rho, m, K, N)
-            per_rho.append({"rho": rho, "k": kk, "whole_op_ms": whole, "whole_op_tflops": fl / whole / 1e9,
+            per_rho.append({"rho": rho, "k": rmm.rmm_keep_count(rho, K), "whole_op_ms": whole, "whole_op_tflops": fl / whole / 1e9,
                             "gemm_kernel_ms": g, "gemm_kernel_tflops": fl / g / 1e9,
                             "gemm_frac_of_sustained_peak": fl / g / 1e9 / peaks["bf16_sustained"],
                             "gemm_frac_of_burst_peak": fl / g / 1e9 / peaks["bf16_burst"],
-                            "gemm_frac_of_nominal_peak": fl / g / 1e9 / NOMINAL_BF16_TFLOPS})
-        dense_after = time_region(lambda i: torch.matmul(A, B, out=Y), reps, 1)
-        dense_ms = 0.5 * (dense_before + dense_after)      # the clocks sag under sustained tensor load: mean of both
-        for r in per_rho:
-            r.update({"dense_cublas_ms": dense_ms, "dense_cublas_ms_before_after": [dense_before, dense_after],
-                      "dense_cublas_tflops": 2.0 * m * K * N / dense_ms / 1e9, "speedup_vs_dense_cublas": dense_ms / r["whole_op_ms"]})
+                            "gemm_frac_of_nominal_peak": fl / g / 1e9 / NOMINAL_BF16_TFLOPS,
+                            "dense_cublas_ms": dense_ms, "dense_cublas_tflops": 2.0 * m * K * N / dense_ms / 1e9,
+                            "speedup_vs_dense_cublas": dense_ms / whole, "timing": "variants interleaved call by call"})
 
     # ---- CPU oracle on a bounded sample of the same workload (rank 0, one GPU only)
     cpu = None
@@ -819,7 +824,7 @@ def main():
         extras["low_bit_operands"] = low_bit_sweep(rmm, binding, synth, dev, peaks)
 
         # ---- the other 70B-class products and the attention of one layer
-        extras["layer_sweep_70b"] = layer_sweep_70b(rmm, synth, dev, peaks)
+        extras["layer_sweep_70b"] = layer_sweep_70b(rmm, binding, synth, dev, peaks)
 
         # ---- up projection -> reduced down projection, the index set taken from the up projection's epilogue energies
         extras["mlp_block_70b"] = chained_mlp_70b(rmm, synth, dev)
