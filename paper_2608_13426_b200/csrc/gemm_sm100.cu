@@ -176,6 +176,7 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         // producers therefore meet before every wave: each adds one to a counter and waits, for at most 20 us and
         // without any consequence if the time runs out, until every block with a tile in this wave has done so.
         unsigned wave_target = 0;
+        bool meeting = a.wave_ctr != nullptr;
         int64_t wave_first = 0;  // first tile of the current wave
         for (int64_t tile = tile0; lane == 0 && tile < num_tiles && ok; tile += tile_step, wave_first += tile_step) {
             const int64_t in_wave = num_tiles - wave_first < tile_step ? num_tiles - wave_first : tile_step;
@@ -185,19 +186,23 @@ reduced_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
                 asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(seen) : "l"(a.wave_ctr) : "memory");
                 ++seen;
                 const unsigned long long t0 = global_ns();
-                while (seen < wave_target && global_ns() - t0 < 20000ull) {
+                while (seen < wave_target) {
+                    if (global_ns() - t0 >= 20000ull) {  // somebody is missing (a GPU shared with other work): this block
+                        meeting = false;                 // stops meeting, and so in turn will those that wait for it
+                        break;
+                    }
                     __nanosleep(64);
                     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.wave_ctr) : "memory");
                 }
             };
-            if (a.wave_ctr != nullptr) meet();
+            if (meeting) meet();
             int tm, tn;
             const int64_t b = tile / ((int64_t)a.tiles_n * a.tiles_m);
             tile_coords(tile - b * ((int64_t)a.tiles_n * a.tiles_m), a.tiles_m, a.tiles_n, a.raster, tm, tn);
             int64_t bb = (b + a.b_batch_off) / a.b_batch_div;
             if (bb >= a.b_batches) bb = a.b_batches - 1;
             for (int kb = 0; kb < num_kb; ++kb) {
-                if (a.wave_ctr != nullptr && a.sync_kb > 0 && kb > 0 && kb % a.sync_kb == 0) meet();
+                if (meeting && a.sync_kb > 0 && kb > 0 && kb % a.sync_kb == 0) meet();
                 if (!mbar_wait_lane(empty_bar(s), ph ^ 1u, abort_flag, a.status, a.wait_ns)) { ok = false; break; }
                 if (a.withhold && blockIdx.x == 0 && tile == tile0 && kb == 0) {
                     // (test switch) this stage is never requested: its barrier stays incomplete
