@@ -127,6 +127,28 @@ def test_70b_class_down_projection_selected_from_the_up_projection_epilogue(orac
         assert rel_fro(H[r].float().cpu().numpy(), want) <= TOL_BF16
 
 
+def test_70b_class_down_projection_with_8_bit_operands(oracle):
+    """The 8-bit form at the size and in the launch configuration the benchmark times (32768 x 28672 x 8192, rho = 0.5: the
+    streaming quantising gather and CTA-pair tiles on the fp8 tensor cores): row steps bit for bit and outputs on sampled
+    rows against the oracle's product of the dequantised operands."""
+    M, K, N = 32768, 28672, 8192
+    A = synth.heavy_tailed_activations(M, K, seed=31, device="cuda")
+    W = synth.weight(K, N, seed=32, dtype=torch.float32, device="cuda")
+    b_scale = float(W.abs().max()) / 448.0
+    Bq = (W.t().contiguous() / b_scale).to(torch.float8_e4m3fn)                   # stored [N, K]
+    del W
+    idx, _, _, _ = rmm.rmm_score_select(A, rho=0.5)
+    Y, s = rmm.rmm_reduced_gemm_q8(A, Bq, b_scale, idx, want_scales=True)
+    assert rmm.rmm_status_read() == 0
+    idx_np = idx.cpu().numpy()
+    Bv = Bq.cpu().to(torch.float64).numpy()
+    for r in sample_rows(M, 3, seed=6):
+        Yo, so = oracle.reduced_gemm_q8(A[r:r + 1].cpu(), Bv, b_scale, idx_np)
+        assert float(s[r]) == float(so[0]), r
+        assert rel_fro(Y[r].float().cpu().numpy(), Yo[0]) <= TOL_BF16, r
+    assert torch.isfinite(Y.float()).all()
+
+
 def check_token_sets(oracle, tok, It, P, band=1e-4):
     """Token sets of the fused sweeps against the oracle's P (evaluated on the GPU's feature sets): Theorem 1's
     criterion (retained energy within 1e-6 of the optimum) and equality outside a 1e-4 band."""
