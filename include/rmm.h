@@ -169,8 +169,9 @@ int rmm_reduced_gemm_q8(const rmm_mat_t *A, const rmm_mat_t *B, float b_scale, c
  * time.  An evenly strided batch is processed as B * Hq heads in one pass of launches.
  * mask (device, fp32, or NULL): the additive M of Sec. 3.3, entry (b, h, i, t) at mask[b ms[0] + h ms[1] + i ms[2] + t]
  * with ms = mask_stride in elements (0 shares the mask along that axis; rows contiguous); -inf hides a key; a row with
- * every key hidden gives zeros.  It composes with `causal`.  With a mask the composed form runs (S~ and P in the
- * workspace) whatever the head dimension: the fused kernels take the causal mask only. */
+ * every key hidden gives zeros.  It composes with `causal`.  With rho_t == 1, head_dim <= 128 and mask rows that are
+ * 16-byte aligned (base pointer and all three strides multiples of 4 elements) the one-pass fused kernel adds the mask
+ * itself; otherwise a call with a mask runs the composed form (S~ and P in the workspace). */
 typedef struct {
     int64_t B, Hq, Hkv, Lq, Lk, Dh;
     int32_t causal;

@@ -167,8 +167,8 @@ int rmm_score(const rmm_mat_t *A, int axis, float *scores, float *energy, void *
 
 size_t rmm_select_workspace_bytes(int64_t batch, int64_t K)
 {
-    (void)batch;
-    (void)K;
+    // the select keeps its keys in registers or shared memory (or re-reads them): only the header with the status word
+    if (batch < 1 || K < 1 || K > (int64_t(1) << 30)) return 0;
     return RMM_WS_HEADER_BYTES;
 }
 

@@ -146,7 +146,12 @@ int plan_attn(const rmm_attn_desc_t *d, AttnPlan *p)
     const double per_head = (double)d->Lq * ((double)p->ld_s * 4 + (double)p->ld_p * 2 + (double)p->ldt * 2);
     int64_t hg = (int64_t)(6.0 * 1073741824.0 / per_head);
     if (hg < 1) hg = 1;
-    p->fused = d->mask == nullptr && use_fused(d, p->kd);  // the fused kernels take the causal mask only
+    // the one-pass fused kernel also takes the caller's additive mask (rows 16-byte aligned); the three sweeps of the
+    // token reduction take the causal mask only (their second sweep walks the mask by columns)
+    const bool mask_ok = d->mask == nullptr ||
+                         (d->rho_t >= 1.0 && reinterpret_cast<uintptr_t>(d->mask) % 16 == 0 && d->mask_stride[0] % 4 == 0 &&
+                          d->mask_stride[1] % 4 == 0 && d->mask_stride[2] % 4 == 0);
+    p->fused = mask_ok && use_fused(d, p->kd);
     if (hg > d->Hq || p->fused) hg = d->Hq;  // the fused form materialises neither S~ nor P: all heads at once
     p->hg = hg;
 
@@ -261,7 +266,9 @@ int rmm_reduced_attn(const rmm_attn_desc_t *desc, const void *Q, const void *K, 
                 if (!tok) {
                     rc = launch_fused_attn(Qp, Kp, p.ldd, p.kd, v, d->v_stride[2], d->v_stride[1], d->B * d->Hkv, b * d->Hq + h0, group,
                                            og, d->o_stride[1], d->o_stride[2], hg, d->Lq, d->Lk, d->Dh, d->causal, d->Lk - d->Lq,
-                                           nullptr, 0, nullptr, status, st);
+                                           nullptr, 0, nullptr,
+                                           d->mask != nullptr ? d->mask + b * d->mask_stride[0] + h0 * d->mask_stride[1] : nullptr,
+                                           d->mask_stride[1], d->mask_stride[2], status, st);
                     if (rc != RMM_OK) return rc;
                     continue;
                 }
@@ -279,7 +286,7 @@ int rmm_reduced_attn(const rmm_attn_desc_t *desc, const void *Q, const void *K, 
                 if ((rc = launch_pack(kv, 2, status, st)) != RMM_OK) return rc;
                 // sweep 3: O = P[:, T] V[T, :] against the full-row normalisers
                 rc = launch_fused_attn(Qp, KpT, p.ldd, p.kd, Vp, d->Dh, p.kt * d->Dh, hg, 0, 1, og, d->o_stride[1], d->o_stride[2], hg,
-                                       d->Lq, p.kt, d->Dh, d->causal, d->Lk - d->Lq, lse, p.lse_ld, It, status, st);
+                                       d->Lq, p.kt, d->Dh, d->causal, d->Lk - d->Lq, lse, p.lse_ld, It, nullptr, 0, 0, status, st);
                 if (rc != RMM_OK) return rc;
                 continue;
             }

@@ -80,12 +80,15 @@ struct FusedArgs {
     float *energy;               // ENERGY: [heads, Lr] squared token scores
     const int32_t *tok;          // GATHERED: [heads, Lc] kept key positions, ascending
     float scale_log2;            // (1 / sqrt(Dh)) * log2(e)
+    const float *mask;           // MASK: additive mask M of softmax(S~ + M), fp32, row (head, i) at mask + head m_sh + i m_sr
+    int64_t m_sh, m_sr;
+    float mask_gain;             // sqrt(Dh): M is added to the unscaled S~ tile as M * sqrt(Dh)
     int *status;
     unsigned long long wait_ns;  // bound of every device-side wait
     int withhold;                // test switch: block 0 never requests its first key tile
 };
 
-template <int MODE>
+template <int MODE, bool MASK>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, FusedArgs a)
@@ -382,6 +385,34 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         if (e + 32 > hi || e + 32 < lo) v1[e] = 0xff800000u;
                     }
                 }
+                if constexpr (MASK) {
+                    // the caller's additive mask for this row's 64 columns (-inf hides a key); rows past the end and
+                    // columns past the last key read nothing
+                    if (i < a.Lr) {
+                        const float *mrow = a.mask + head * a.m_sh + i * a.m_sr + c0;
+                        const float gain = a.mask_gain;
+                        auto add4 = [&](uint32_t (&v)[32], int e, int col) {
+                            float4 m4;
+                            if (c0 + col + 3 < a.Lc) {
+                                m4 = __ldg(reinterpret_cast<const float4 *>(mrow + col));
+                            } else {
+                                m4.x = c0 + col < a.Lc ? __ldg(mrow + col) : 0.f;
+                                m4.y = c0 + col + 1 < a.Lc ? __ldg(mrow + col + 1) : 0.f;
+                                m4.z = c0 + col + 2 < a.Lc ? __ldg(mrow + col + 2) : 0.f;
+                                m4.w = 0.f;
+                            }
+                            v[e] = __float_as_uint(fmaf(m4.x, gain, __uint_as_float(v[e])));
+                            v[e + 1] = __float_as_uint(fmaf(m4.y, gain, __uint_as_float(v[e + 1])));
+                            v[e + 2] = __float_as_uint(fmaf(m4.z, gain, __uint_as_float(v[e + 2])));
+                            v[e + 3] = __float_as_uint(fmaf(m4.w, gain, __uint_as_float(v[e + 3])));
+                        };
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4) {
+                            add4(v0, e, e);
+                            add4(v1, e, e + 32);
+                        }
+                    }
+                }
             };
             auto release_s = [&]() {  // this warp holds what it needs of the S~ tile
                 tc_fence_before();
@@ -602,11 +633,11 @@ fused_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (warp == 1) tmem_dealloc<1>(tmem_base, kTmemCols);
 }
 
-template <int MODE>
+template <int MODE, bool MASK = false>
 int launch_mode(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, const FusedArgs &a, const char *name,
                 cudaStream_t stream)
 {
-    auto kern = fused_attn_kernel<MODE>;
+    auto kern = fused_attn_kernel<MODE, MASK>;
     static PerDeviceOnce configured;
     if (configured.first()) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmem);
@@ -649,14 +680,16 @@ bool fused_attn_eligible(const rmm_attn_desc_t *d, int64_t kd)
     return d->Dh % 8 == 0 && d->Dh <= 128 && kd <= 128 && d->Lq <= INT32_MAX && d->Lk <= INT32_MAX;
 }
 
-// FULL (lse NULL, tok NULL): O = softmax(Qp Kp^T / sqrt(Dh) + mask) V.
+// FULL (lse NULL, tok NULL): O = softmax(Qp Kp^T / sqrt(Dh) + mask) V; `mask` (or NULL) is the caller's additive fp32 mask on
+// top of the causal one, row (head, i) at mask + head m_sh + i m_sr (16-byte aligned rows).
 // GATHERED (lse and tok given): Kp and V hold the kept keys only (Lk = their count, tok their positions); O = P V with
 // P = bf16(2^(x - lse)), no renormalisation.  `diag` = Lk - Lq of the unpacked problem.
 // Qp [heads, Lq, ldd], Kp [heads, Lk, ldd] packed; V [v_batches, Lk, Dh] with row pitch v_ld and batch pitch v_sb.
 int launch_fused_attn(const __nv_bfloat16 *Qp, const __nv_bfloat16 *Kp, int64_t ldd, int64_t kd, const __nv_bfloat16 *V,
                       int64_t v_ld, int64_t v_sb, int64_t v_batches, int64_t v_off, int64_t v_div, __nv_bfloat16 *O,
                       int64_t o_sh, int64_t o_sr, int64_t heads, int64_t Lq, int64_t Lk, int64_t Dh, int causal, int64_t diag,
-                      const float *lse, int64_t lse_ld, const int32_t *tok, int *status, cudaStream_t stream)
+                      const float *lse, int64_t lse_ld, const int32_t *tok, const float *mask, int64_t m_sh, int64_t m_sr,
+                      int *status, cudaStream_t stream)
 {
     CUtensorMap mq, mk, mv;
     int rc;
@@ -679,6 +712,11 @@ int launch_fused_attn(const __nv_bfloat16 *Qp, const __nv_bfloat16 *Kp, int64_t 
     a.wait_ns = wait_limit_ns();
     a.withhold = debug_withhold() == WITHHOLD_ATTN;
     if (tok != nullptr) return launch_mode<MODE_GATHERED>(mq, mk, mv, a, "fused_attn_gathered_kernel", stream);
+    if (mask != nullptr) {
+        a.mask = mask; a.m_sh = m_sh; a.m_sr = m_sr;
+        a.mask_gain = (float)sqrt((double)Dh);
+        return launch_mode<MODE_FULL, true>(mq, mk, mv, a, "fused_attn_masked_kernel", stream);
+    }
     return launch_mode<MODE_FULL>(mq, mk, mv, a, "fused_attn_kernel", stream);
 }
 

@@ -231,7 +231,7 @@ bool fused_attn_eligible(const rmm_attn_desc_t *d, int64_t kd);
 int launch_fused_attn(const __nv_bfloat16 *Qp, const __nv_bfloat16 *Kp, int64_t ldd, int64_t kd, const __nv_bfloat16 *V,
                       int64_t v_ld, int64_t v_sb, int64_t v_batches, int64_t v_off, int64_t v_div, __nv_bfloat16 *O,
                       int64_t o_sh, int64_t o_sr, int64_t heads, int64_t Lq, int64_t Lk, int64_t Dh, int causal, int64_t diag,
-                      const float *lse, int64_t lse_ld, const int32_t *tok, int *status, cudaStream_t stream);
+                      const float *lse, int64_t lse_ld, const int32_t *tok, const float *mask, int64_t m_sh, int64_t m_sr, int *status, cudaStream_t stream);
 // Two sweeps: lse [heads, lse_ld] (lse_ld a multiple of 64, >= Lq) = log2-domain row normalisers of softmax(S~ + mask);
 // energy [heads, Lk] = squared token scores sum_i bf16(P_it)^2.
 int launch_fused_attn_scores(const __nv_bfloat16 *Qp, const __nv_bfloat16 *Kp, int64_t ldd, int64_t kd, int64_t heads,

@@ -488,6 +488,13 @@ def test_reduced_attention_with_an_additive_mask(oracle, rho_d, rho_t):
     rows_off[17] = -float("inf")
     rows_off[200:230] = -float("inf")
     assert check_attention(oracle, 1, 2, 1, L, L, 64, False, rho_d, rho_t, seed=74, mask=rows_off)
+    # rows of the mask 16-byte aligned: with rho_t = 1 the one-pass fused kernel adds the mask itself (several key tiles,
+    # a ragged last one, holes and a bias per (sequence, head), on top of the causal mask)
+    B, Hq, Hkv, Lq, Lk, Dh = 2, 4, 2, 520, 648, 128
+    M = torch.randn(B, Hq, Lq, Lk, generator=g)
+    M[torch.rand(B, Hq, Lq, Lk, generator=g) < 0.3] = -float("inf")
+    M[..., 3] = -0.5
+    assert check_attention(oracle, B, Hq, Hkv, Lq, Lk, Dh, True, rho_d, rho_t, seed=75, mask=M)
     assert rmm.rmm_status_read() == 0
 
 
