@@ -755,3 +755,58 @@ def test_one_launch_front_end_on_a_tall_product(oracle):
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-c", code], env=env, cwd=root, capture_output=True, text=True, timeout=300)
     assert r.returncode == 0, r.stderr[-3000:]
+
+
+def test_products_with_and_without_the_wave_meetings_agree(oracle):
+    """Products with several waves of tiles keep their blocks in step along the contraction axis (the producers meet
+    before every tile).  The meetings change timing only: the output with them switched off is the same bit for bit,
+    single-CTA and CTA-pair tiles, batched, and a second product on the same workspace finds the counters re-armed."""
+    import os, subprocess, sys
+    code = (
+        "import torch, hashlib, paper_2608_13426_b200 as rmm\n"
+        "from paper_2608_13426_b200 import synth, binding\n"
+        "binding.poison_outputs(True)\n"
+        "out = []\n"
+        "for (b, M, K, N, rho) in ((1, 8192, 8192, 4096, 0.5), (1, 8192, 8192, 4096, 0.5), (3, 4000, 4104, 1000, 1.0), (1, 20000, 4096, 264, 1.0)):\n"
+        "    A = synth.heavy_tailed_activations(b * M, K, seed=5, device='cuda').view(b, M, K); B = synth.weight(K, N, seed=6, device='cuda')\n"
+        "    idx = rmm.rmm_score_select(A, rho=rho)[0] if rho < 1 else None\n"
+        "    Y = rmm.rmm_reduced_gemm(A, B, idx)\n"
+        "    out.append(hashlib.sha256(Y.cpu().view(torch.int16).numpy().tobytes()).hexdigest())\n"
+        "assert rmm.rmm_status_read() == 0\n"
+        "print(' '.join(out))\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    digests = []
+    for sync in ("1", "0"):
+        env = dict(os.environ, RMM_GEMM_WAVE_SYNC=sync)
+        r = subprocess.run([sys.executable, "-c", code], env=env, cwd=root, capture_output=True, text=True, timeout=300)
+        assert r.returncode == 0, r.stderr[-3000:]
+        digests.append(r.stdout.strip().splitlines()[-1].split())
+    assert digests[0] == digests[1] and len(digests[0]) == 4 and digests[0][0] == digests[0][1]
+
+
+def test_captured_graph_replays_the_product(oracle):
+    """The library neither allocates nor synchronises, so a product (one-launch front end + GEMM, and the two-call form
+    with its grid-wide counters) can be captured into a CUDA graph; replays give the eager result bit for bit."""
+    for (M, K, N, rho) in ((2048, 8192, 2048, 0.5), (9000, 4096, 1032, 0.25)):
+        A, B = synth.mlp_product(M, K, N, seed=11)
+        A, B = dev(A), dev(B)
+        k = rmm.rmm_keep_count(rho, K)
+        Y = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+        idx = torch.empty(k, dtype=torch.int32, device="cuda")
+        rmm.rmm_product(A, B, rho=rho, out=Y, idx=idx)                    # eager: also sizes the default workspace
+        Y0, idx0 = Y.clone(), idx.clone()
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            rmm.rmm_product(A, B, rho=rho, out=Y, idx=idx)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                rmm.rmm_product(A, B, rho=rho, out=Y, idx=idx)
+        torch.cuda.current_stream().wait_stream(s)
+        for _ in range(3):
+            Y.fill_(float("nan"))
+            idx.fill_(-1)
+            g.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(Y, Y0) and torch.equal(idx, idx0)
+        assert rmm.rmm_status_read() == 0
