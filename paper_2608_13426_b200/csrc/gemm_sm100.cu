@@ -602,12 +602,14 @@ int launch_gemm_tc_problem(const TcProblem &p, cudaStream_t stream)
     a.tiles_n = (int)ceil_div(p.N, BN);
     a.status = p.status;
     {
-        // column slices of B kept alive by one raster group: group * BN columns x k rows of bf16, held to about 64 MB (half of L2)
+        // column slices of B kept alive by one raster group: group * BN columns x k rows of bf16, held to about 64 MB (half of
+        // L2) so that they survive from one wave to the next; where not even eight slices fit, eight all the same: a wave
+        // of 74 tiles then reads the fewest bytes when it is about as wide as it is tall
         static const int forced_raster = []() { const char *e = getenv("RMM_GEMM_RASTER"); return e ? atoi(e) : 0; }();
         const int64_t slice = (int64_t)BN * p.k * es;
         int64_t grp = slice > 0 ? (64ll << 20) / slice : kRasterGroupMax;
         if (grp > kRasterGroupMax) grp = kRasterGroupMax;
-        if (grp < 2) grp = 2;
+        if (grp < 8) grp = 8;
         a.raster = forced_raster > 0 ? forced_raster : (int)grp;
     }
     a.wait_ns = wait_limit_ns();
