@@ -723,7 +723,7 @@ def main():
 
     # ---- per-rho sweep on the headline product: whole op beside dense cuBLAS at the same shape
     per_rho = []
-    if not args.no_sweep and rank == 0:
+    if not args.no_sweep and rank == 0 and world == 1:  # (replicas: the headline only)
         res, dense_ms = interleaved_rho_sweep(rmm, binding, A, B, Y, RHOS)
         for rho in RHOS:
             whole, g = res[rho]
@@ -766,7 +766,7 @@ def main():
     torch.cuda.empty_cache()
 
     extras = {}
-    if not args.no_sweep and rank == 0:
+    if not args.no_sweep and rank == 0 and world == 1:  # (replicas: the headline only)
         # ---- the 1B-class product (where launch and selection latencies matter most)
         extras["mlp_1b"] = small_product_sweep(rmm, binding, synth, dev, peaks, rank)
 
