@@ -281,7 +281,7 @@ def run_reference(args):
     }))
 
 
-def attention_case(rmm, binding, synth, dev, heads, seq, head_dim=128, reps=10):
+def attention_case(rmm, binding, synth, dev, heads, seq, head_dim=128, reps=10, ratios=((0.5, 1.0), (0.75, 1.0), (0.5, 0.5), (0.5, 0.25))):
     """Reduced attention on a prefill shape (heads x seq x head_dim, causal): feature reduction only (one fused pass) and
     feature + token reduction (three fused sweeps: row normalisers, token scores, gathered P V); S~ and P stay on the SM
     in both.  torch's dense scaled_dot_product_attention at the same shape is context, not a target."""
@@ -290,7 +290,7 @@ def attention_case(rmm, binding, synth, dev, heads, seq, head_dim=128, reps=10):
         torch.nn.functional.scaled_dot_product_attention(Qa, Ka, Va, is_causal=True)
     dense = time_region(lambda i: torch.nn.functional.scaled_dot_product_attention(Qa, Ka, Va, is_causal=True), reps, 1)
     out = []
-    for rho_d, rho_t in ((0.5, 1.0), (0.75, 1.0), (0.5, 0.5), (0.5, 0.25)):
+    for rho_d, rho_t in ratios:
         for _ in range(2):
             rmm.rmm_reduced_attn(Qa, Ka, Va, True, rho_d, rho_t)
         t = time_region(lambda i: rmm.rmm_reduced_attn(Qa, Ka, Va, True, rho_d, rho_t), reps, 1)
@@ -305,7 +305,10 @@ def attention_case(rmm, binding, synth, dev, heads, seq, head_dim=128, reps=10):
         fl = 2.0 * heads * (seq * (seq + 1) / 2) * (kd + head_dim * rho_t)
         out.append({"rho_d": rho_d, "rho_t": rho_t, "shape": [heads, seq, head_dim], "causal": True, "ms": t,
                     "retained_tflops": fl / t / 1e9, "kernels_us": parts, "dense_sdpa_ms": dense,
-                    "path": "fused, one pass" if rho_t >= 1.0 else "fused, three sweeps"})
+                    "speedup_vs_dense_sdpa": dense / t,
+                    "path": ("composed (S~ and P in memory)" if kd > 128 else "fused, ") +
+                            ("" if kd > 128 else ("one pass" if rho_t >= 1.0 else "three sweeps")) +
+                            ("" if kd > 128 or head_dim <= 128 else ", two passes over the columns of V")})
     return out
 
 
@@ -817,6 +820,8 @@ def main():
 
         # ---- reduced attention on a 7B-class prefill, the paper's kernel-latency setting, the attention products as GEMMs
         extras["attention_prefill"] = attention_case(rmm, binding, synth, dev, 32, 4096)
+        extras["attention_wide_heads"] = attention_case(rmm, binding, synth, dev, 16, 4096, head_dim=256, reps=5,
+                                                        ratios=((0.5, 1.0), (0.25, 1.0), (0.5, 0.5), (0.75, 1.0)))
         extras["attention_paper_setting"] = paper_table5_case(rmm, synth, dev)
         extras["attention_products_in_memory"] = gemm_framed_attention(rmm, synth, dev, peaks)
 

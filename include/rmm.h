@@ -162,14 +162,15 @@ int rmm_reduced_gemm_q8(const rmm_mat_t *A, const rmm_mat_t *B, float b_scale, c
  *   rho_t == 1: O = P V
  * Q [B,Hq,Lq,Dh], K,V [B,Hkv,Lk,Dh], O [B,Hq,Lq,Dh] are bf16 with explicit element strides
  * (batch, head, row, 1).  idx_feat int32 [B,Hq,kd] and idx_tok int32 [B,Hq,kt] receive the index sets
- * (either may be NULL).  With head_dim and kept features up to 128, S~ and P stay on the SM (fused kernel: one pass
+ * (either may be NULL).  With at most 128 kept features and a head_dim of at most 256, S~ and P stay on the SM (heads wider
+ * than 128 columns in two passes over the columns of V; fused kernel: one pass
  * for rho_t == 1; row normalisers, token scores and a gathered P V pass for rho_t < 1, where the normalised P is
  * what is rounded, scored and multiplied; for rho_t == 1 the bf16 rounding is applied to P times a per-row factor,
  * which changes O by rounding noise only).  Wider heads materialise S~ and P in the workspace one group of heads at a
  * time.  An evenly strided batch is processed as B * Hq heads in one pass of launches.
  * mask (device, fp32, or NULL): the additive M of Sec. 3.3, entry (b, h, i, t) at mask[b ms[0] + h ms[1] + i ms[2] + t]
  * with ms = mask_stride in elements (0 shares the mask along that axis; rows contiguous); -inf hides a key; a row with
- * every key hidden gives zeros.  It composes with `causal`.  With rho_t == 1, head_dim <= 128 and mask rows that are
+ * every key hidden gives zeros.  It composes with `causal`.  With rho_t == 1, a fused-eligible shape and mask rows that are
  * 16-byte aligned (base pointer and all three strides multiples of 4 elements) the one-pass fused kernel adds the mask
  * itself; otherwise a call with a mask runs the composed form (S~ and P in the workspace). */
 typedef struct {

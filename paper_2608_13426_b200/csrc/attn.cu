@@ -8,7 +8,7 @@
 //   rho_t = 1: O = P V_g (same kernel, P and V loaded in place)
 // S~ and P live in the workspace (materialised), so this form is bound by HBM traffic, not by the tensor cores.
 //
-// With head_dim and kept features up to 128 the steps after the packing run fused instead (attn_fused.cu), S~ and P
+// With up to 128 kept features and a head_dim of up to 256 the steps after the packing run fused instead (attn_fused.cu), S~ and P
 // staying on the SM:
 //   rho_t = 1: one pass, O = softmax(S~ + mask) V;
 //   rho_t < 1: row normalisers (sweep 1), token scores of the bf16-rounded P (sweep 2), select T, pack K[T] and V[T],
@@ -87,7 +87,7 @@ struct AttnPlan {
     size_t inner_bytes, off_idxf, off_idxt, off_qp, off_kp, off_s, off_p, off_pp, off_vp, off_lse, off_energy, off_kpt, total;
 };
 
-// head_dim and kept features up to 128 run fused (RMM_ATTN_FUSED=0 keeps the composed form, for comparison).
+// up to 128 kept features of heads up to 256 wide run fused (RMM_ATTN_FUSED=0 keeps the composed form, for comparison).
 bool use_fused(const rmm_attn_desc_t *d, int64_t kd)
 {
     static const bool enabled = [] {

@@ -677,7 +677,8 @@ extern "C" void rmm_debug_attn_stamps(unsigned long long *out)
 
 bool fused_attn_eligible(const rmm_attn_desc_t *d, int64_t kd)
 {
-    return d->Dh % 8 == 0 && d->Dh <= 128 && kd <= 128 && d->Lq <= INT32_MAX && d->Lk <= INT32_MAX;
+    // heads of up to 256 columns run as two passes over 128 columns of V and O each (S~ and the weights are taken again)
+    return d->Dh % 8 == 0 && d->Dh <= 256 && kd <= 128 && d->Lq <= INT32_MAX && d->Lk <= INT32_MAX;
 }
 
 // FULL (lse NULL, tok NULL): O = softmax(Qp Kp^T / sqrt(Dh) + mask) V; `mask` (or NULL) is the caller's additive fp32 mask on
@@ -695,29 +696,38 @@ int launch_fused_attn(const __nv_bfloat16 *Qp, const __nv_bfloat16 *Kp, int64_t 
     int rc;
     if ((rc = packed_map(&mq, Qp, kd, Lq, heads, ldd, FM)) != RMM_OK) return rc;
     if ((rc = packed_map(&mk, Kp, kd, Lk, heads, ldd, FN)) != RMM_OK) return rc;
-    {
-        uint64_t dims[3] = {(uint64_t)Dh, (uint64_t)Lk, (uint64_t)v_batches};
-        uint64_t st[2] = {(uint64_t)v_ld * 2, v_batches > 1 ? (uint64_t)v_sb * 2 : (uint64_t)v_ld * 2 * (uint64_t)Lk};
-        const uint32_t box[3] = {64, FN, 1};
-        if ((rc = make_map(&mv, const_cast<__nv_bfloat16 *>(V), 3, dims, st, box, true)) != RMM_OK) return rc;
+    // The O accumulators of a block hold 128 columns per query group: a wider head (up to 256 columns) is produced in
+    // two passes, each over its own 128 columns of V and of O; the softmax scale keeps the full head dimension.
+    for (int64_t c0 = 0; c0 < Dh; c0 += 128) {
+        const int64_t dh = Dh - c0 < 128 ? Dh - c0 : 128;
+        {
+            uint64_t dims[3] = {(uint64_t)dh, (uint64_t)Lk, (uint64_t)v_batches};
+            uint64_t st[2] = {(uint64_t)v_ld * 2, v_batches > 1 ? (uint64_t)v_sb * 2 : (uint64_t)v_ld * 2 * (uint64_t)Lk};
+            const uint32_t box[3] = {64, FN, 1};
+            if ((rc = make_map(&mv, const_cast<__nv_bfloat16 *>(V + c0), 3, dims, st, box, true)) != RMM_OK) return rc;
+        }
+        FusedArgs a = {};
+        a.heads = heads; a.Lr = Lq; a.Lc = Lk; a.diag = diag;
+        a.kd = (int)kd; a.Dh = (int)dh; a.causal = causal;
+        a.v_off = v_off; a.v_div = v_div > 0 ? v_div : 1;
+        a.O = O + c0; a.o_sh = o_sh; a.o_sr = o_sr;
+        a.lse = const_cast<float *>(lse); a.lse_ld = lse_ld; a.tok = tok;
+        a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)Dh));
+        a.status = status;
+        a.wait_ns = wait_limit_ns();
+        a.withhold = debug_withhold() == WITHHOLD_ATTN;
+        if (tok != nullptr) {
+            rc = launch_mode<MODE_GATHERED>(mq, mk, mv, a, "fused_attn_gathered_kernel", stream);
+        } else if (mask != nullptr) {
+            a.mask = mask; a.m_sh = m_sh; a.m_sr = m_sr;
+            a.mask_gain = (float)sqrt((double)Dh);
+            rc = launch_mode<MODE_FULL, true>(mq, mk, mv, a, "fused_attn_masked_kernel", stream);
+        } else {
+            rc = launch_mode<MODE_FULL>(mq, mk, mv, a, "fused_attn_kernel", stream);
+        }
+        if (rc != RMM_OK) return rc;
     }
-    FusedArgs a = {};
-    a.heads = heads; a.Lr = Lq; a.Lc = Lk; a.diag = diag;
-    a.kd = (int)kd; a.Dh = (int)Dh; a.causal = causal;
-    a.v_off = v_off; a.v_div = v_div > 0 ? v_div : 1;
-    a.O = O; a.o_sh = o_sh; a.o_sr = o_sr;
-    a.lse = const_cast<float *>(lse); a.lse_ld = lse_ld; a.tok = tok;
-    a.scale_log2 = (float)(1.4426950408889634 / sqrt((double)Dh));
-    a.status = status;
-    a.wait_ns = wait_limit_ns();
-    a.withhold = debug_withhold() == WITHHOLD_ATTN;
-    if (tok != nullptr) return launch_mode<MODE_GATHERED>(mq, mk, mv, a, "fused_attn_gathered_kernel", stream);
-    if (mask != nullptr) {
-        a.mask = mask; a.m_sh = m_sh; a.m_sr = m_sr;
-        a.mask_gain = (float)sqrt((double)Dh);
-        return launch_mode<MODE_FULL, true>(mq, mk, mv, a, "fused_attn_masked_kernel", stream);
-    }
-    return launch_mode<MODE_FULL>(mq, mk, mv, a, "fused_attn_kernel", stream);
+    return RMM_OK;
 }
 
 // Sweeps 1 and 2 of the token reduction on packed Qp [heads, Lq, ldd], Kp [heads, Lk, ldd]:

@@ -553,9 +553,21 @@ def test_fused_and_composed_attention_agree(oracle, monkeypatch):
 
 
 def test_composed_attention_for_wide_heads(oracle):
-    """head_dim above 128 runs the composed form (S~ and P in the workspace); both reductions."""
-    assert check_attention(oracle, 1, 2, 1, 130, 200, 256, True, 0.5, 0.5, seed=81)
+    """More than 128 kept features run the composed form (S~ and P in the workspace); both reductions."""
+    assert check_attention(oracle, 1, 2, 1, 130, 200, 256, True, 0.75, 0.5, seed=81)
     assert check_attention(oracle, 1, 2, 2, 96, 96, 256, False, 0.75, 1.0, seed=82)
+
+
+@pytest.mark.parametrize("Dh,rho_d,rho_t", [(256, 0.5, 1.0), (256, 0.25, 0.5), (192, 0.5, 1.0), (192, 0.5, 0.3), (136, 0.5, 1.0)])
+def test_fused_attention_for_heads_of_up_to_256_columns(oracle, Dh, rho_d, rho_t):
+    """Heads wider than 128 columns whose kept features still fit 128 stay fused: two passes over 128 (or fewer) columns
+    of V and O each, the softmax scale keeping the full head dimension."""
+    n0 = rmm.rmm_launch_count()
+    assert check_attention(oracle, 1, 4, 2, 300, 391, Dh, True, rho_d, rho_t, seed=83)
+    launched = rmm.rmm_launch_count() - n0
+    assert launched == (4 if rho_t == 1.0 else 8), launched          # score+select, pack, 2 x one-pass | 2 sweeps, select, pack, 2 x gathered instead
+    assert check_attention(oracle, 2, 2, 2, 130, 130, Dh, False, rho_d, rho_t, seed=84)
+    assert rmm.rmm_status_read() == 0
 
 
 def test_attention_batch_folding_and_uneven_batch_stride(oracle):
