@@ -567,6 +567,12 @@ def test_fused_attention_for_heads_of_up_to_256_columns(oracle, Dh, rho_d, rho_t
     launched = rmm.rmm_launch_count() - n0
     assert launched == (4 if rho_t == 1.0 else 8), launched          # score+select, pack, 2 x one-pass | 2 sweeps, select, pack, 2 x gathered instead
     assert check_attention(oracle, 2, 2, 2, 130, 130, Dh, False, rho_d, rho_t, seed=84)
+    if rho_t == 1.0:                                                  # and with an additive mask in both column passes
+        g = torch.Generator().manual_seed(85)
+        M = torch.randn(2, 1, 200, 392, generator=g)
+        M[torch.rand(2, 1, 200, 392, generator=g) < 0.3] = -float("inf")
+        M[..., 0] = 0.0
+        assert check_attention(oracle, 2, 2, 1, 200, 392, Dh, True, rho_d, rho_t, seed=86, mask=M)
     assert rmm.rmm_status_read() == 0
 
 
